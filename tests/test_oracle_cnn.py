@@ -1,0 +1,150 @@
+"""Pins for the oracle's CNN forward/backward (model endnote of the paper).
+
+The oracle is checked against things other than itself: torch's CPU autograd in
+float64 on the same graph (library routines conv2d / max_pool2d / linear /
+cross_entropy), central finite differences, and closed forms.
+"""
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+from oracle import cnn
+from paper_2406_05546_b200 import synth
+
+
+def _torch_grad(theta, x, y, keep, p):
+    t = torch.tensor(theta, dtype=torch.float64, requires_grad=True)
+    def seg(name):
+        off, shape = cnn.TENSORS[name]
+        n = int(np.prod(shape))
+        return t[off:off + n].reshape(shape)
+    xb = torch.tensor(x, dtype=torch.float64).reshape(-1, 1, 28, 28)
+    a = F.max_pool2d(F.relu(F.conv2d(xb, seg("conv1.w"), seg("conv1.b"), padding=1)), 2)
+    a = F.max_pool2d(F.relu(F.conv2d(a, seg("conv2.w"), seg("conv2.b"), padding=1)), 2)
+    h = F.relu(F.linear(a.flatten(1), seg("fc1.w"), seg("fc1.b")))
+    if keep is not None:
+        h = h * torch.tensor(keep, dtype=torch.float64) / (1.0 - p)
+    z = F.linear(h, seg("fc2.w"), seg("fc2.b"))
+    loss = F.cross_entropy(z, torch.tensor(y, dtype=torch.long), reduction="mean")
+    loss.backward()
+    return t.grad.numpy(), float(loss.detach()), z.detach().numpy()
+
+
+def _case(b, seed):
+    rng = np.random.default_rng(seed)
+    theta = synth.init_params(seed=seed + 1, bias_scale=0.1).astype(np.float64)
+    x = rng.random((b, 28, 28))
+    y = rng.integers(0, 10, b).astype(np.int32)
+    keep = (rng.random((b, 512)) >= 0.25).astype(np.uint8)
+    return theta, x, y, keep
+
+
+def test_parameter_count_closed_form():
+    total = 16 * 1 * 9 + 16 + 32 * 16 * 9 + 32 + 512 * (32 * 7 * 7) + 512 + 10 * 512 + 10
+    assert total == cnn.P == 813258
+    end = 0
+    for name, (off, shape) in cnn.TENSORS.items():
+        assert off == end
+        end = off + int(np.prod(shape))
+    assert end == cnn.P
+    assert [(n, o, s) for n, (o, s) in cnn.TENSORS.items()] == synth.layout()
+
+
+@pytest.mark.parametrize("b,seed", [(1, 0), (3, 5), (8, 9)])
+def test_matches_torch_autograd_f64(b, seed):
+    theta, x, y, keep = _case(b, seed)
+    g, loss, am, logits = cnn.grad_step_f64(theta, x, y, keep, 0.25)
+    gt, lt, zt = _torch_grad(theta, x, y, keep, 0.25)
+    assert abs(loss - lt) < 1e-12
+    np.testing.assert_allclose(logits, zt, rtol=0, atol=1e-12)
+    assert (am == zt.argmax(1)).all()
+    for name, (off, shape) in cnn.TENSORS.items():
+        n = int(np.prod(shape))
+        ref = gt[off:off + n]
+        assert np.abs(ref).max() > 0, name
+        assert np.abs(g[off:off + n] - ref).max() <= 1e-11 * max(1.0, np.abs(ref).max()), name
+
+
+def test_no_dropout_path_matches_torch():
+    theta, x, y, _ = _case(2, 3)
+    g, loss, _, _ = cnn.grad_step_f64(theta, x, y, None, 0.25)
+    gt, lt, _ = _torch_grad(theta, x, y, None, 0.25)
+    assert abs(loss - lt) < 1e-12
+    assert np.abs(g - gt).max() < 1e-11
+
+
+def test_central_finite_differences():
+    theta, x, y, keep = _case(2, 21)
+    g, _, _, _ = cnn.grad_step_f64(theta, x, y, keep, 0.25)
+    rng = np.random.default_rng(0)
+    eps = 1e-6
+    checked = 0
+    for name, (off, shape) in cnn.TENSORS.items():
+        n = int(np.prod(shape))
+        for j in rng.choice(n, size=min(n, 6), replace=False):
+            tp, tm = theta.copy(), theta.copy()
+            tp[off + j] += eps
+            tm[off + j] -= eps
+            lp = cnn.grad_step_f64(tp, x, y, keep, 0.25)[1]
+            lm = cnn.grad_step_f64(tm, x, y, keep, 0.25)[1]
+            fd = (lp - lm) / (2 * eps)
+            assert abs(fd - g[off + j]) <= 1e-6 * max(1e-3, abs(fd)) + 1e-9, (name, j, fd, g[off + j])
+            checked += 1
+    assert checked >= 40
+
+
+def test_closed_forms_zero_weights():
+    # all-zero parameters: logits are 0, loss = ln 10, argmax = class 0 (lowest index of a tie),
+    # d loss / d fc2.b = 1/10 - [fraction of samples with that label]
+    b = 5
+    x = np.random.default_rng(1).random((b, 28, 28))
+    y = np.array([3, 3, 7, 0, 9], dtype=np.int32)
+    g, loss, am, logits = cnn.grad_step_f64(np.zeros(cnn.P), x, y, None, 0.25)
+    assert abs(loss - np.log(10.0)) < 1e-15
+    assert (am == 0).all() and (logits == 0).all()
+    off = cnn.TENSORS["fc2.b"][0]
+    expect = np.full(10, 0.1) - np.bincount(y, minlength=10) / b
+    np.testing.assert_allclose(g[off:off + 10], expect, atol=1e-15)
+    assert np.abs(np.delete(g, np.arange(off, off + 10))).max() == 0.0
+
+
+def test_output_bias_gradient_sums_to_zero_and_mean_scaling():
+    theta, x, y, keep = _case(4, 8)
+    g, loss, _, _ = cnn.grad_step_f64(theta, x, y, keep, 0.25)
+    off = cnn.TENSORS["fc2.b"][0]
+    assert abs(g[off:off + 10].sum()) < 1e-14
+    # mean loss: the batch gradient is the mean of the single-sample gradients
+    acc = np.zeros_like(g)
+    losses = []
+    for i in range(4):
+        gi, li, _, _ = cnn.grad_step_f64(theta, x[i:i + 1], y[i:i + 1], keep[i:i + 1], 0.25)
+        acc += gi
+        losses.append(li)
+    assert np.abs(acc / 4 - g).max() < 1e-13
+    assert abs(np.mean(losses) - loss) < 1e-13
+
+
+def test_dead_upper_layers_block_conv_gradients():
+    # only a centred-delta conv1 filter is non-zero: nothing reaches the logits (later layers are
+    # zero), so the loss stays ln 10 and no gradient flows back into the convolutions.
+    theta = np.zeros(cnn.P)
+    theta[0 * 9 + 4] = 1.0
+    x = np.random.default_rng(2).random((1, 28, 28))
+    g, loss, _, _ = cnn.grad_step_f64(theta, x, np.array([1], dtype=np.int32), None, 0.25)
+    assert abs(loss - np.log(10.0)) < 1e-15
+    assert np.abs(g[:4800]).max() == 0.0
+
+
+def test_workers_entry_uses_philox_mask_and_fp32_inputs():
+    rng = np.random.default_rng(4)
+    W, b = 3, 4
+    thetas = [synth.init_params(seed=s, bias_scale=0.05) for s in (1, 2, 1)]
+    x = rng.random((W, b, 28, 28), dtype=np.float32)
+    y = rng.integers(0, 10, (W, b)).astype(np.int32)
+    ids = [7, 2, 5]
+    grads, loss, am, logits = cnn.workers_grad_step(thetas, ids, x, y, seed=0x5EED, step=12, drop_p=0.25)
+    for w in range(W):
+        keep = cnn.dropout_keep(0x5EED, ids[w], 12, b, 0.25)
+        g, l, a, z = cnn.grad_step_f64(thetas[w].astype(np.float64), x[w].astype(np.float64), y[w], keep, 0.25)
+        assert (g == grads[w]).all() and l == loss[w] and (a == am[w]).all() and (z == logits[w]).all()
