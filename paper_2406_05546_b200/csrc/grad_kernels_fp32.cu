@@ -1,0 +1,581 @@
+// Worker-side gradient step on the FP32 CUDA cores: the paper's small CNN (model endnote),
+// forward and backward, for W workers that may hold different weight snapshots.
+//
+// Rows of every activation buffer are (sorted worker s, sample i) -> s*b + i, where the sorted
+// order places workers that share a snapshot next to each other, so that a group's samples form
+// one contiguous row range and the dense layers can run one tiled product per group.
+//
+// Every reduction is taken in a fixed order (no floating-point atomics), so that two runs on the
+// same inputs give the same bits.
+#include "kernels.h"
+
+namespace psk {
+
+namespace {
+
+// ---- Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplications; the high
+// halves are xored with the neighbouring counter words and the key; the key advances by two Weyl
+// constants per round.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0 = __umulhi(M0, c.x), lo0 = M0 * c.x;
+    uint32_t hi1 = __umulhi(M1, c.z), lo1 = M1 * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+    k.x += W0; k.y += W1;
+  }
+  return c;
+}
+
+__device__ __forceinline__ const float* group_theta(const WorkerTable& wt, const GroupTable& gt, int s) {
+  return gt.theta[wt.group[s]];
+}
+
+// ---- conv1 (1->16, 3x3, pad 1) + ReLU + 2x2 max pool.  One sample per block.
+__global__ void __launch_bounds__(256) conv1_fwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+  __shared__ float xs[30][31];
+  __shared__ float w[160];
+  const int s = blockIdx.y, i = blockIdx.x, tid = threadIdx.x;
+  const int64_t row = (int64_t)s * a.b + i;
+  const float* theta = group_theta(wt, gt, s);
+  const float* x = a.x + ((int64_t)wt.src[s] * a.b + i) * (IMG * IMG);
+  for (int t = tid; t < 30 * 30; t += 256) {
+    int yy = t / 30, xx = t % 30;
+    bool in = yy >= 1 && yy <= IMG && xx >= 1 && xx <= IMG;
+    xs[yy][xx] = in ? x[(yy - 1) * IMG + (xx - 1)] : 0.f;
+  }
+  if (tid < 160) w[tid] = theta[OFF_C1W + tid];
+  __syncthreads();
+  for (int o = tid; o < P1_ELEMS; o += 256) {
+    int ch = o / 196, pp = o % 196, py = pp / 14, px = pp % 14;
+    float wv[9];
+#pragma unroll
+    for (int k = 0; k < 9; ++k) wv[k] = w[ch * 9 + k];
+    float bias = w[144 + ch];
+    float best = 0.f;
+    int bi = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int yy = 2 * py + (j >> 1), xx = 2 * px + (j & 1);
+      float v = bias;
+#pragma unroll
+      for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+        for (int kx = 0; kx < 3; ++kx) v = fmaf(wv[ky * 3 + kx], xs[yy + ky][xx + kx], v);
+      float r = fmaxf(v, 0.f);
+      if (j == 0 || r > best) { best = r; bi = j; }
+    }
+    ws.p1[row * P1_ELEMS + o] = best;
+    ws.code1[row * P1_ELEMS + o] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
+  }
+}
+
+// ---- conv2 (16->32, 3x3, pad 1) + ReLU + 2x2 max pool.  A block handles up to CONV_SPB samples of
+// one worker; the filter bank stays in shared memory.  Thread = (pooled position, group of 8 output
+// channels): it accumulates the 2x2 pre-pool window of its 8 channels from a 4x4 input patch.
+__global__ void __launch_bounds__(256) conv2_fwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+  __shared__ float w[4608 + 32];
+  __shared__ float in[16][16][17];
+  const int s = blockIdx.y, tid = threadIdx.x;
+  const float* theta = group_theta(wt, gt, s);
+  for (int t = tid; t < 4640; t += 256) w[t] = theta[OFF_C2W + t];
+  for (int t = tid; t < 16 * 16 * 17; t += 256) (&in[0][0][0])[t] = 0.f;
+  const int i0 = blockIdx.x * CONV_SPB;
+  const int i1 = min(i0 + CONV_SPB, a.b);
+  for (int i = i0; i < i1; ++i) {
+    const int64_t row = (int64_t)s * a.b + i;
+    __syncthreads();
+    for (int t = tid; t < P1_ELEMS; t += 256) {
+      int ic = t / 196, pp = t % 196;
+      in[ic][pp / 14 + 1][pp % 14 + 1] = ws.p1[row * P1_ELEMS + t];
+    }
+    __syncthreads();
+    if (tid < 196) {
+      const int pos = tid % 49, og = tid / 49;
+      const int py = pos / 7, px = pos % 7;
+      float acc[8][4];
+#pragma unroll
+      for (int o = 0; o < 8; ++o) {
+        float bias = w[4608 + og * 8 + o];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[o][j] = bias;
+      }
+      for (int ic = 0; ic < 16; ++ic) {
+        float patch[4][4];
+#pragma unroll
+        for (int yy = 0; yy < 4; ++yy)
+#pragma unroll
+          for (int xx = 0; xx < 4; ++xx) patch[yy][xx] = in[ic][2 * py + yy][2 * px + xx];
+#pragma unroll
+        for (int o = 0; o < 8; ++o) {
+          const float* wk = &w[((og * 8 + o) * 16 + ic) * 9];
+#pragma unroll
+          for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+            for (int kx = 0; kx < 3; ++kx) {
+              float wv = wk[ky * 3 + kx];
+              acc[o][0] = fmaf(wv, patch[ky][kx], acc[o][0]);
+              acc[o][1] = fmaf(wv, patch[ky][kx + 1], acc[o][1]);
+              acc[o][2] = fmaf(wv, patch[ky + 1][kx], acc[o][2]);
+              acc[o][3] = fmaf(wv, patch[ky + 1][kx + 1], acc[o][3]);
+            }
+        }
+      }
+#pragma unroll
+      for (int o = 0; o < 8; ++o) {
+        float best = 0.f;
+        int bi = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float r = fmaxf(acc[o][j], 0.f);
+          if (j == 0 || r > best) { best = r; bi = j; }
+        }
+        int idx = (og * 8 + o) * 49 + pos;
+        ws.p2[row * FLAT + idx] = best;
+        ws.code2[row * FLAT + idx] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
+      }
+    }
+  }
+}
+
+// ---- 64x64x16 tiled FP32 product, 256 threads, 4x4 outputs per thread.
+// A(m,k) = A[m*lda + k] (A_KC) or A[k*lda + m]; B(k,n) = B[n*ldb + k] (B_KC) or B[k*ldb + n].
+// All leading dimensions and tile origins are multiples of 4, so float4 loads stay aligned.
+template <bool A_KC, bool B_KC>
+__device__ __forceinline__ void gemm_tile_64(const float* __restrict__ A, int lda, const float* __restrict__ B,
+                                             int ldb, int M, int N, int K, int m0, int n0,
+                                             float (&acc)[4][4]) {
+  __shared__ __align__(16) float As[16][68];
+  __shared__ __align__(16) float Bs[16][68];
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+#pragma unroll
+  for (int r = 0; r < 4; ++r)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) acc[r][c] = 0.f;
+  for (int k0 = 0; k0 < K; k0 += 16) {
+    {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (A_KC) {
+        int m = tid >> 2, k = (tid & 3) * 4;
+        if (m0 + m < M && k0 + k < K) v = *reinterpret_cast<const float4*>(A + (int64_t)(m0 + m) * lda + k0 + k);
+        As[k][m] = v.x; As[k + 1][m] = v.y; As[k + 2][m] = v.z; As[k + 3][m] = v.w;
+      } else {
+        int k = tid >> 4, m = (tid & 15) * 4;
+        if (k0 + k < K && m0 + m < M) v = *reinterpret_cast<const float4*>(A + (int64_t)(k0 + k) * lda + m0 + m);
+        *reinterpret_cast<float4*>(&As[k][m]) = v;
+      }
+    }
+    {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (B_KC) {
+        int n = tid >> 2, k = (tid & 3) * 4;
+        if (n0 + n < N && k0 + k < K) v = *reinterpret_cast<const float4*>(B + (int64_t)(n0 + n) * ldb + k0 + k);
+        Bs[k][n] = v.x; Bs[k + 1][n] = v.y; Bs[k + 2][n] = v.z; Bs[k + 3][n] = v.w;
+      } else {
+        int k = tid >> 4, n = (tid & 15) * 4;
+        if (k0 + k < K && n0 + n < N) v = *reinterpret_cast<const float4*>(B + (int64_t)(k0 + k) * ldb + n0 + n);
+        *reinterpret_cast<float4*>(&Bs[k][n]) = v;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      float4 av = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+      float4 bv = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+      float ar[4] = {av.x, av.y, av.z, av.w}, br[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(ar[r], br[c], acc[r][c]);
+    }
+    __syncthreads();
+  }
+}
+
+// Maps blockIdx.y to (group, first row of the tile, end row of the group) for 64-row tiles.
+__device__ __forceinline__ bool locate_tile(const GroupTable& gt, int b, int tile, int& g, int& m0, int& m_end) {
+  for (g = 0; g < gt.n_groups; ++g) {
+    int rows = (gt.first[g + 1] - gt.first[g]) * b;
+    int tiles = (rows + 63) >> 6;
+    if (tile < tiles) {
+      m0 = gt.first[g] * b + tile * 64;
+      m_end = gt.first[g + 1] * b;
+      return true;
+    }
+    tile -= tiles;
+  }
+  return false;
+}
+
+// ---- fc1 forward: d = dropout(ReLU(p2 * W1^T + b1)), one product per weight group.
+__global__ void __launch_bounds__(256) fc1_fwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+  int g, m0, m_end;
+  if (!locate_tile(gt, a.b, blockIdx.y, g, m0, m_end)) return;
+  const float* theta = gt.theta[g];
+  const int n0 = blockIdx.x * 64;
+  float acc[4][4];
+  gemm_tile_64<true, true>(ws.p2, FLAT, theta + OFF_F1W, FLAT, m_end, HID, FLAT, m0, n0, acc);
+  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+  const int n = n0 + tx * 4;
+  const float4 bias = *reinterpret_cast<const float4*>(theta + OFF_F1B + n);
+  const float scale = 1.0f / (1.0f - a.drop_p);
+  const uint2 key = make_uint2((uint32_t)a.seed, (uint32_t)(a.seed >> 32));
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    int m = m0 + ty * 4 + r;
+    if (m >= m_end) continue;
+    int s = m / a.b, i = m - s * a.b;
+    uint32_t q = (uint32_t)((i * HID + n) >> 2);
+    uint4 rnd = philox4x32_10(make_uint4(q, (uint32_t)wt.wid[s], (uint32_t)a.step, (uint32_t)(a.step >> 32)), key);
+    float4 o;
+    o.x = rnd.x >= a.drop_thresh ? fmaxf(acc[r][0] + bias.x, 0.f) * scale : 0.f;
+    o.y = rnd.y >= a.drop_thresh ? fmaxf(acc[r][1] + bias.y, 0.f) * scale : 0.f;
+    o.z = rnd.z >= a.drop_thresh ? fmaxf(acc[r][2] + bias.z, 0.f) * scale : 0.f;
+    o.w = rnd.w >= a.drop_thresh ? fmaxf(acc[r][3] + bias.w, 0.f) * scale : 0.f;
+    *reinterpret_cast<float4*>(ws.d + (int64_t)m * HID + n) = o;
+  }
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ---- fc2 forward, softmax cross-entropy, argmax, and the backward pass down to the gradient with
+// respect to fc1's pre-activation; then the worker's fc2 weight/bias and fc1 bias gradients.
+// One block per worker, one warp per sample at a time.
+__global__ void __launch_bounds__(256) fc2_fwd_bwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+  __shared__ float w2[NCLS][HID];
+  __shared__ float b2[NCLS];
+  __shared__ float warp_loss[8];
+  const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* theta = group_theta(wt, gt, s);
+  const int src = wt.src[s];
+  for (int t = tid; t < NCLS * HID; t += 256) (&w2[0][0])[t] = theta[OFF_F2W + t];
+  if (tid < NCLS) b2[tid] = theta[OFF_F2B + tid];
+  __syncthreads();
+  const float scale = 1.0f / (1.0f - a.drop_p);
+  const float inv_b = 1.0f / (float)a.b;
+  float loss_acc = 0.f;
+  for (int i = warp; i < a.b; i += 8) {
+    const int64_t row = (int64_t)s * a.b + i;
+    float dv[16];
+#pragma unroll
+    for (int t = 0; t < 16; ++t) dv[t] = ws.d[row * HID + lane + 32 * t];
+    float z[NCLS];
+#pragma unroll
+    for (int c = 0; c < NCLS; ++c) {
+      float p = 0.f;
+#pragma unroll
+      for (int t = 0; t < 16; ++t) p = fmaf(w2[c][lane + 32 * t], dv[t], p);
+      z[c] = warp_sum(p) + b2[c];
+    }
+    float zmax = z[0];
+    int am = 0;
+#pragma unroll
+    for (int c = 1; c < NCLS; ++c)
+      if (z[c] > zmax) { zmax = z[c]; am = c; }
+    float se = 0.f;
+#pragma unroll
+    for (int c = 0; c < NCLS; ++c) se += expf(z[c] - zmax);
+    const float lse = zmax + logf(se);
+    int label = a.y[(int64_t)src * a.b + i];
+    if (label < 0 || label >= NCLS) {
+      if (lane == 0) atomicOr(ws.status, STATUS_BAD_LABEL);
+      label = 0;
+    }
+    float zy = 0.f, dz[NCLS];
+#pragma unroll
+    for (int c = 0; c < NCLS; ++c) {
+      if (c == label) zy = z[c];
+      dz[c] = (expf(z[c] - lse) - (c == label ? 1.f : 0.f)) * inv_b;
+    }
+    loss_acc += lse - zy;
+    if (lane == 0) a.argmax[(int64_t)src * a.b + i] = am;
+    if (lane < DZ_STRIDE) {
+      float v = 0.f;
+#pragma unroll
+      for (int c = 0; c < NCLS; ++c)
+        if (lane == c) v = dz[c];
+      ws.dz[row * DZ_STRIDE + lane] = v;
+    }
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      int j = lane + 32 * t;
+      float dd = 0.f;
+#pragma unroll
+      for (int c = 0; c < NCLS; ++c) dd = fmaf(w2[c][j], dz[c], dd);
+      ws.da1[row * HID + j] = dv[t] > 0.f ? dd * scale : 0.f;
+    }
+  }
+  if (lane == 0) warp_loss[warp] = loss_acc;
+  __syncthreads();   // also makes this block's dz / da1 stores visible to all of its threads
+  if (tid == 0) {
+    float t = 0.f;
+    for (int w = 0; w < 8; ++w) t += warp_loss[w];
+    a.loss[src] = t * inv_b;
+  }
+  float* grad = wt.grad[s];
+  float gw[2][NCLS], gb1[2] = {0.f, 0.f};
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+#pragma unroll
+    for (int c = 0; c < NCLS; ++c) gw[h][c] = 0.f;
+  float gb2 = 0.f;
+  for (int i = 0; i < a.b; ++i) {
+    const int64_t row = (int64_t)s * a.b + i;
+    float dzv[NCLS];
+#pragma unroll
+    for (int c = 0; c < NCLS; ++c) dzv[c] = ws.dz[row * DZ_STRIDE + c];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float dval = ws.d[row * HID + tid + 256 * h];
+#pragma unroll
+      for (int c = 0; c < NCLS; ++c) gw[h][c] = fmaf(dzv[c], dval, gw[h][c]);
+      gb1[h] += ws.da1[row * HID + tid + 256 * h];
+    }
+    if (tid < NCLS) gb2 += ws.dz[row * DZ_STRIDE + tid];
+  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+#pragma unroll
+    for (int c = 0; c < NCLS; ++c) grad[OFF_F2W + c * HID + tid + 256 * h] = gw[h][c];
+    grad[OFF_F1B + tid + 256 * h] = gb1[h];
+  }
+  if (tid < NCLS) grad[OFF_F2B + tid] = gb2;
+}
+
+// ---- fc1 weight gradient of one worker: dW1 [512][1568] = da1^T [512 x b] * p2 [b x 1568].
+__global__ void __launch_bounds__(256) fc1_dw(GradStepArgs a, WorkerTable wt, Workspace ws) {
+  const int s = blockIdx.z, m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const float* A = ws.da1 + (int64_t)s * a.b * HID;
+  const float* B = ws.p2 + (int64_t)s * a.b * FLAT;
+  float acc[4][4];
+  gemm_tile_64<false, false>(A, HID, B, FLAT, HID, FLAT, a.b, m0, n0, acc);
+  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+  const int n = n0 + tx * 4;
+  if (n >= FLAT) return;
+  float* out = wt.grad[s] + OFF_F1W;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    int m = m0 + ty * 4 + r;
+    *reinterpret_cast<float4*>(out + (int64_t)m * FLAT + n) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+  }
+}
+
+// ---- gradient with respect to p2: dp2 [rows][1568] = da1 [rows][512] * W1 [512][1568], per group.
+__global__ void __launch_bounds__(256) fc1_dx(GradStepArgs a, GroupTable gt, Workspace ws) {
+  int g, m0, m_end;
+  if (!locate_tile(gt, a.b, blockIdx.y, g, m0, m_end)) return;
+  const int n0 = blockIdx.x * 64;
+  float acc[4][4];
+  gemm_tile_64<true, false>(ws.da1, HID, gt.theta[g] + OFF_F1W, FLAT, m_end, FLAT, HID, m0, n0, acc);
+  const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+  const int n = n0 + tx * 4;
+  if (n >= FLAT) return;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    int m = m0 + ty * 4 + r;
+    if (m >= m_end) continue;
+    *reinterpret_cast<float4*>(ws.dp2 + (int64_t)m * FLAT + n) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+  }
+}
+
+// ---- backward through pool2, ReLU and conv2 for up to CONV_SPB samples of one worker:
+// writes dp1 per sample and the block's partial filter / bias gradients.
+constexpr int C2B_SMEM_FLOATS = 4608 + 32 * 16 * 17 + 16 * 16 * 17;
+__global__ void __launch_bounds__(256) conv2_bwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws, int n_chunks) {
+  extern __shared__ float smem[];
+  float* w = smem;                                                        // [32][16][9]
+  float (*g2)[16][17] = reinterpret_cast<float (*)[16][17]>(smem + 4608); // [32] padded gradient at conv2 output
+  float (*in)[16][17] = reinterpret_cast<float (*)[16][17]>(smem + 4608 + 32 * 16 * 17);  // [16] padded p1
+  const int s = blockIdx.y, tid = threadIdx.x;
+  const float* theta = group_theta(wt, gt, s);
+  for (int t = tid; t < 4608; t += 256) w[t] = theta[OFF_C2W + t];
+  for (int t = tid; t < 16 * 16 * 17; t += 256) (&in[0][0][0])[t] = 0.f;
+  const int oc_w = tid >> 3, ic_w = (tid & 7) * 2;   // filter-gradient ownership: (oc, two input channels)
+  float gw[2][9], gb = 0.f;
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+#pragma unroll
+    for (int k = 0; k < 9; ++k) gw[h][k] = 0.f;
+  const int i0 = blockIdx.x * CONV_SPB;
+  const int i1 = min(i0 + CONV_SPB, a.b);
+  for (int i = i0; i < i1; ++i) {
+    const int64_t row = (int64_t)s * a.b + i;
+    __syncthreads();
+    for (int t = tid; t < 32 * 16 * 17; t += 256) (&g2[0][0][0])[t] = 0.f;
+    for (int t = tid; t < P1_ELEMS; t += 256) {
+      int ic = t / 196, pp = t % 196;
+      in[ic][pp / 14 + 1][pp % 14 + 1] = ws.p1[row * P1_ELEMS + t];
+    }
+    __syncthreads();
+    for (int t = tid; t < FLAT; t += 256) {
+      int code = ws.code2[row * FLAT + t];
+      if (code < 4) {
+        int oc = t / 49, pp = t % 49;
+        int y = 2 * (pp / 7) + (code >> 1), x = 2 * (pp % 7) + (code & 1);
+        g2[oc][y + 1][x + 1] = ws.dp2[row * FLAT + t];
+      }
+    }
+    __syncthreads();
+    // gradient with respect to the conv2 input (p1)
+    if (tid < 196) {
+      const int y = tid / 14, x = tid % 14;
+      float acc[16];
+#pragma unroll
+      for (int ic = 0; ic < 16; ++ic) acc[ic] = 0.f;
+      for (int oc = 0; oc < 32; ++oc) {
+#pragma unroll
+        for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+          for (int kx = 0; kx < 3; ++kx) {
+            float g = g2[oc][y - ky + 2][x - kx + 2];
+            if (g != 0.f) {
+#pragma unroll
+              for (int ic = 0; ic < 16; ++ic) acc[ic] = fmaf(g, w[(oc * 16 + ic) * 9 + ky * 3 + kx], acc[ic]);
+            }
+          }
+      }
+#pragma unroll
+      for (int ic = 0; ic < 16; ++ic) ws.dp1[row * P1_ELEMS + ic * 196 + tid] = acc[ic];
+    }
+    // filter and bias gradients
+    for (int y = 0; y < 14; ++y)
+      for (int x = 0; x < 14; ++x) {
+        float g = g2[oc_w][y + 1][x + 1];
+        if (g != 0.f) {
+          if ((tid & 7) == 0) gb += g;
+#pragma unroll
+          for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+              for (int kx = 0; kx < 3; ++kx) gw[h][ky * 3 + kx] = fmaf(g, in[ic_w + h][y + ky][x + kx], gw[h][ky * 3 + kx]);
+        }
+      }
+  }
+  float* part = ws.part2 + ((int64_t)s * n_chunks + blockIdx.x) * C2_GRAD;
+#pragma unroll
+  for (int h = 0; h < 2; ++h)
+#pragma unroll
+    for (int k = 0; k < 9; ++k) part[(oc_w * 16 + ic_w + h) * 9 + k] = gw[h][k];
+  if ((tid & 7) == 0) part[4608 + oc_w] = gb;
+}
+
+// ---- backward through pool1, ReLU and conv1 (filter / bias gradients only: the input needs none).
+__global__ void __launch_bounds__(256) conv1_bwd(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
+  __shared__ float xs[30][31];
+  const int s = blockIdx.y, tid = threadIdx.x;
+  const int oc = tid >> 4, l = tid & 15;
+  float gw[9], gb = 0.f;
+#pragma unroll
+  for (int k = 0; k < 9; ++k) gw[k] = 0.f;
+  const int i0 = blockIdx.x * CONV_SPB;
+  const int i1 = min(i0 + CONV_SPB, a.b);
+  for (int i = i0; i < i1; ++i) {
+    const int64_t row = (int64_t)s * a.b + i;
+    const float* x = a.x + ((int64_t)wt.src[s] * a.b + i) * (IMG * IMG);
+    __syncthreads();
+    for (int t = tid; t < 30 * 30; t += 256) {
+      int yy = t / 30, xx = t % 30;
+      bool in = yy >= 1 && yy <= IMG && xx >= 1 && xx <= IMG;
+      xs[yy][xx] = in ? x[(yy - 1) * IMG + (xx - 1)] : 0.f;
+    }
+    __syncthreads();
+    for (int pp = l; pp < 196; pp += 16) {
+      int code = ws.code1[row * P1_ELEMS + oc * 196 + pp];
+      if (code < 4) {
+        float g = ws.dp1[row * P1_ELEMS + oc * 196 + pp];
+        int y = 2 * (pp / 14) + (code >> 1), xq = 2 * (pp % 14) + (code & 1);
+        gb += g;
+#pragma unroll
+        for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+          for (int kx = 0; kx < 3; ++kx) gw[ky * 3 + kx] = fmaf(g, xs[y + ky][xq + kx], gw[ky * 3 + kx]);
+      }
+    }
+  }
+  // fixed-order reduction over the 16 lanes that share an output channel
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) {
+    gb += __shfl_xor_sync(0xffffffffu, gb, o);
+#pragma unroll
+    for (int k = 0; k < 9; ++k) gw[k] += __shfl_xor_sync(0xffffffffu, gw[k], o);
+  }
+  if (l == 0) {
+    float* part = ws.part1 + ((int64_t)s * n_chunks + blockIdx.x) * C1_GRAD;
+#pragma unroll
+    for (int k = 0; k < 9; ++k) part[oc * 9 + k] = gw[k];
+    part[144 + oc] = gb;
+  }
+}
+
+// ---- sums the per-block partial convolution gradients in block order and zeroes the padding.
+__global__ void __launch_bounds__(256) conv_grad_reduce(WorkerTable wt, Workspace ws, int n_chunks) {
+  const int s = blockIdx.x, tid = threadIdx.x;
+  float* grad = wt.grad[s];
+  for (int o = tid; o < C2_GRAD; o += 256) {
+    float t = 0.f;
+    for (int c = 0; c < n_chunks; ++c) t += ws.part2[((int64_t)s * n_chunks + c) * C2_GRAD + o];
+    grad[OFF_C2W + o] = t;
+  }
+  for (int o = tid; o < C1_GRAD; o += 256) {
+    float t = 0.f;
+    for (int c = 0; c < n_chunks; ++c) t += ws.part1[((int64_t)s * n_chunks + c) * C1_GRAD + o];
+    grad[OFF_C1W + o] = t;
+  }
+  for (int o = P + tid; o < P_PAD; o += 256) grad[o] = 0.f;
+}
+
+// ---- the keep mask on its own: thread e/4 draws the four words of elements 4*(e/4) .. +3.
+__global__ void __launch_bounds__(256) dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int n_quads,
+                                                    uint32_t thresh, uchar4* __restrict__ keep) {
+  int q = blockIdx.x * 256 + threadIdx.x;
+  if (q >= n_quads) return;
+  uint4 r = philox4x32_10(make_uint4((uint32_t)q, worker, (uint32_t)step, (uint32_t)(step >> 32)),
+                          make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)));
+  keep[q] = make_uchar4(r.x >= thresh, r.y >= thresh, r.z >= thresh, r.w >= thresh);
+}
+
+int tiles_64(const GroupTable& gt, int b) {
+  int t = 0;
+  for (int g = 0; g < gt.n_groups; ++g) t += ((gt.first[g + 1] - gt.first[g]) * b + 63) / 64;
+  return t;
+}
+
+}  // namespace
+
+int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, uint32_t thresh,
+                        uint8_t* keep, cudaStream_t st) {
+  int n_quads = b * HID / 4;
+  dropout_mask<<<(n_quads + 255) / 256, 256, 0, st>>>(seed, worker, step, n_quads, thresh,
+                                                      reinterpret_cast<uchar4*>(keep));
+  return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int configure_grad_kernels() {
+  cudaError_t e = cudaFuncSetAttribute(conv2_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)(C2B_SMEM_FLOATS * sizeof(float)));
+  return e == cudaSuccess ? 0 : -1;
+}
+
+int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt,
+                          const Workspace& ws, cudaStream_t st) {
+  const int n_chunks = (a.b + CONV_SPB - 1) / CONV_SPB;
+  const int mt = tiles_64(gt, a.b);
+  conv1_fwd<<<dim3(a.b, a.W), 256, 0, st>>>(a, wt, gt, ws);
+  conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws);
+  fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws);
+  fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws);
+  fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws);
+  fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws);
+  conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks);
+  conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks);
+  conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks);
+  return cudaGetLastError() == cudaSuccess ? 9 : -1;
+}
+
+}  // namespace psk

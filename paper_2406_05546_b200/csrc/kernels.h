@@ -1,0 +1,109 @@
+// Internal launch interface between the host state machine and the sm_100a kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace psk {
+
+constexpr int P = 813258;
+constexpr int P_PAD = 813312;          // floats per stored parameter / gradient vector
+constexpr int P_VEC4 = P_PAD / 4;      // 203,328 float4 columns
+constexpr int MAX_WORKERS = 256;
+constexpr int MAX_RING = 16;
+constexpr int MAX_GROUPS = 16;
+
+constexpr int OFF_C1W = 0, OFF_C1B = 144, OFF_C2W = 160, OFF_C2B = 4768;
+constexpr int OFF_F1W = 4800, OFF_F1B = 807616, OFF_F2W = 808128, OFF_F2B = 813248;
+
+constexpr int IMG = 28, C1 = 16, H1 = 14, C2 = 32, H2 = 7;
+constexpr int P1_ELEMS = C1 * H1 * H1;   // 3136
+constexpr int FLAT = C2 * H2 * H2;       // 1568
+constexpr int HID = 512, NCLS = 10;
+constexpr int DZ_STRIDE = 16;            // logits gradient row, padded
+constexpr int CONV_SPB = 4;              // samples per block in the conv backward kernels
+constexpr int C2_GRAD = 4608 + 32, C1_GRAD = 144 + 16;
+
+constexpr uint32_t STATUS_BAD_LABEL = 1u;
+
+// Per-call tables passed by value as kernel parameters.
+// Workers are processed in "sorted" order: workers sharing a weight snapshot are adjacent, so
+// that a group's samples form one contiguous block of activation rows.
+struct WorkerTable {
+  float* grad[MAX_WORKERS];     // destination gradient vector (P_PAD floats) of sorted worker s
+  int32_t wid[MAX_WORKERS];     // logical worker id (dropout key)
+  int32_t src[MAX_WORKERS];     // index of the worker in the caller's arrays (x, y, loss, argmax)
+  int16_t group[MAX_WORKERS];   // group of sorted worker s
+};
+
+struct GroupTable {
+  const float* theta[MAX_GROUPS];  // weight snapshot of the group
+  int32_t first[MAX_GROUPS + 1];   // first sorted worker of the group; first[n_groups] = W
+  int32_t n_groups;
+};
+
+// Activation workspace carved from the arena (rows = sorted worker * b + sample).
+struct Workspace {
+  float* p1;       // [rows][16][14][14]  conv1 -> ReLU -> pool
+  uint8_t* code1;  // [rows][3136]        pool-1 argmax 0..3, 4 = no gradient (max <= 0)
+  float* p2;       // [rows][1568]        conv2 -> ReLU -> pool, channel-major flatten
+  uint8_t* code2;  // [rows][1568]
+  float* d;        // [rows][512]         fc1 -> ReLU -> dropout (scaled)
+  float* da1;      // [rows][512]         gradient w.r.t. fc1 pre-activation
+  float* dz;       // [rows][16]          gradient w.r.t. logits (10 used)
+  float* dp2;      // [rows][1568]        gradient w.r.t. p2
+  float* dp1;      // [rows][3136]        gradient w.r.t. p1
+  float* part2;    // [W][chunks][4640]   per-block partial conv2 weight/bias gradients
+  float* part1;    // [W][chunks][160]    per-block partial conv1 weight/bias gradients
+  uint32_t* status;
+};
+
+struct GradStepArgs {
+  int W, b;
+  const float* x;      // [W][b][784] caller order
+  const int32_t* y;    // [W][b]
+  float* loss;         // [W]
+  int32_t* argmax;     // [W][b]
+  uint64_t seed, step;
+  float drop_p;
+  uint32_t drop_thresh;   // keep iff word >= thresh
+};
+
+// Part A, FP32 CUDA-core path. Returns the number of kernels launched, or -1 on a launch error.
+int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt,
+                          const Workspace& ws, cudaStream_t st);
+int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, uint32_t thresh,
+                        uint8_t* keep, cudaStream_t st);
+int configure_grad_kernels();   // one-time function attributes (dynamic shared memory sizes)
+
+// Part B.
+struct SumApplyArgs {
+  const float* queue;       // slot 0 of the gradient queue; slot k at queue + k*P_PAD
+  int64_t K;                // gradients to sum (slots 0..K-1)
+  const float* theta_in;    // current head
+  float* theta_out;         // new head (may equal theta_in)
+  float* replica;           // mirror target or nullptr
+  float coef;               // lr*scale/divisor
+  float* partial;           // [max_split][P_PAD] scratch
+  int max_split;
+};
+int launch_sum_apply(const SumApplyArgs& a, cudaStream_t st);
+
+constexpr int ASYNC_SEG = 256;   // gradients per ordered-apply launch
+struct AsyncOrder { int32_t slot[ASYNC_SEG]; };
+struct AsyncApplyArgs {
+  const float* queue;
+  int K;                    // 1..ASYNC_SEG gradients in this segment
+  const float* theta_in;    // version v0
+  float* ring[MAX_RING];    // ring slot buffers
+  int ring_depth;
+  uint64_t v0;              // version of theta_in; version v0+k+1 is stored in ring[(v0+k+1) % depth]
+  int first_stored;         // only k >= first_stored are stored (the last ring_depth versions)
+  int mirror_k;             // k whose result is also written to replica, or -1
+  float* replica;
+  float coef;               // lr*scale
+};
+int launch_async_apply(const AsyncApplyArgs& a, const AsyncOrder& ord, cudaStream_t st);
+
+int launch_copy_rows(float* dst, const float* src, int64_t rows, cudaStream_t st);
+
+}  // namespace psk

@@ -1,0 +1,44 @@
+"""Comparison helpers shared by the GPU parity tests (no method arithmetic)."""
+import numpy as np
+
+from paper_2406_05546_b200 import synth
+
+TOL_FP32 = 1e-4     # max error relative to the tensor's max-abs, FP32 path (stated target)
+TOL_TENSOR = 2e-2   # same, tensor-core path
+
+
+def tensor_rel_errors(got, ref):
+    """Per parameter tensor: max|got-ref| / max|ref| (both flat [P] arrays)."""
+    out = {}
+    for name, off, shape in synth.layout():
+        n = int(np.prod(shape))
+        r = np.asarray(ref[off:off + n], dtype=np.float64)
+        g = np.asarray(got[off:off + n], dtype=np.float64)
+        denom = np.abs(r).max()
+        err = np.abs(g - r).max()
+        out[name] = err / denom if denom > 0 else err
+    return out
+
+
+def assert_params_close(got, ref, tol, what=""):
+    errs = tensor_rel_errors(got, ref)
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, f"{what}: relative error above {tol}: {bad} (all: {errs})"
+    return errs
+
+
+def assert_argmax_valid(got, ref_logits, tol):
+    """Labels must equal the oracle's wherever its top-2 margin exceeds tol*max|logit|; elsewhere
+    the chosen class must be one of the near-maximal ones.  Returns the number of ambiguous rows."""
+    z = np.asarray(ref_logits, dtype=np.float64).reshape(-1, 10)
+    got = np.asarray(got).reshape(-1)
+    top = np.sort(z, axis=1)
+    margin = top[:, -1] - top[:, -2]
+    slack = tol * np.abs(z).max(axis=1)
+    clear = margin > slack
+    ref = z.argmax(axis=1)
+    assert (got[clear] == ref[clear]).all(), "argmax differs where the oracle's margin is clear"
+    amb = np.where(~clear)[0]
+    for r in amb:
+        assert z[r, got[r]] >= top[r, -1] - slack[r]
+    return int(amb.size)

@@ -1,0 +1,151 @@
+"""GPU parity: the worker gradient step against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from paper_2406_05546_b200 import synth
+from tests.parity import TOL_FP32, assert_argmax_valid, assert_params_close
+
+pytestmark = pytest.mark.gpu
+
+SEED = 0x5EED
+
+
+def _setup(W, b, n_versions=1, drop_p=0.25):
+    import torch
+    from paper_2406_05546_b200 import ps
+    theta0 = synth.init_params(seed=1, bias_scale=0.05)
+    srv = ps.ParameterServer(theta0, max_workers=W, max_batch=b, ring_depth=max(1, n_versions),
+                             queue_slots=max(W, n_versions), dropout_p=drop_p)
+    return torch, ps, srv, theta0
+
+
+def _run_and_compare(W, b, lags=None, n_versions=1, step=3, drop_p=0.25, worker_ids=None, in_slots=False):
+    from oracle import cnn
+    torch, ps, srv, theta0 = _setup(W, b, n_versions, drop_p)
+    versions = {0: theta0}
+    # produce older/newer versions with async applies of random "gradients" so that snapshots differ
+    for v in range(1, n_versions):
+        g = np.zeros((1, ps.P_PAD), dtype=np.float32)
+        g[0, :ps.P] = synth.random_gradients(1, seed=50 + v, scale=2.0)[0]
+        srv.ps_enqueue([0], [v - 1], 0, grads_dev=torch.from_numpy(g).cuda())
+        srv.ps_apply(ps.ASYNC, 0.01)
+        versions[v], ver = srv.ps_export_params(0)
+        assert ver == v
+    rng = np.random.default_rng(7)
+    x = rng.random((W, b, 28, 28), dtype=np.float32)
+    y = rng.integers(0, 10, (W, b)).astype(np.int32)
+    lags = [0] * W if lags is None else lags
+    ids = list(range(W)) if worker_ids is None else worker_ids
+    snaps = [srv.ps_pull_snapshot(w, lags[w]) for w in range(W)]
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    if in_slots:
+        slots = srv.ps_queue_reserve(W)
+        loss, am = srv.workers_grad_step(snaps, ids, xd, yd, SEED, step, slot_ids=slots)
+        grads = torch.stack([srv.slot_tensor(s) for s in slots]).cpu().numpy()
+    else:
+        gd = torch.full((W, ps.P_PAD), float("nan"), device="cuda")
+        loss, am = srv.workers_grad_step(snaps, ids, xd, yd, SEED, step, grads_dev=gd)
+        grads = gd.cpu().numpy()
+    srv.ps_stats()
+    thetas = [versions[s.version] for s in snaps]
+    og, ol, oa, oz = cnn.workers_grad_step(thetas, ids, x, y, SEED, step, drop_p)
+    for w in range(W):
+        assert_params_close(grads[w, :ps.P], og[w], TOL_FP32, f"gradient of worker {w}")
+        assert (grads[w, ps.P:] == 0).all()
+    np.testing.assert_allclose(loss.cpu().numpy(), ol, rtol=1e-5, atol=1e-6)
+    assert_argmax_valid(am.cpu().numpy(), oz, TOL_FP32)
+    srv.close()
+    return grads
+
+
+def test_config1_shape_two_workers_batch8():
+    _run_and_compare(2, 8, in_slots=True)
+
+
+def test_ragged_batch_and_worker_ids():
+    _run_and_compare(3, 5, worker_ids=[11, 4, 200], step=(1 << 33) + 5)
+
+
+def test_batch_spanning_several_tiles_with_tail():
+    _run_and_compare(2, 70)
+
+
+def test_stale_snapshots_grouped_over_three_versions():
+    # five workers over three distinct weight versions, interleaved so that grouping must reorder
+    _run_and_compare(5, 6, lags=[2, 0, 1, 2, 0], n_versions=3)
+
+
+def test_no_dropout():
+    _run_and_compare(2, 4, drop_p=0.0)
+
+
+def test_single_sample_single_worker():
+    _run_and_compare(1, 1)
+
+
+def test_repeatable_bit_for_bit():
+    a = _run_and_compare(3, 9)
+    b = _run_and_compare(3, 9)
+    assert (a == b).all()
+
+
+def test_dropout_mask_bit_exact():
+    from oracle import cnn
+    torch, ps, srv, _ = _setup(1, 1)
+    for seed, worker, step, b in [(SEED, 0, 0, 1), (SEED, 3, 7, 64), (0xDEADBEEFCAFEF00D, 255, (5 << 32) | 9, 129)]:
+        got = srv.ps_dropout_mask(seed, worker, step, b).cpu().numpy()
+        assert (got == cnn.dropout_keep(seed, worker, step, b, 0.25)).all()
+    srv.close()
+
+
+def test_grad_step_uses_that_mask():
+    # fc1 weights zero and bias one: the hidden layer is 1 before dropout, so with one sample the
+    # fc2 weight gradient is dz[c] * keep[j] / (1-p): its zero pattern is exactly the mask.
+    from oracle import cnn
+    import torch
+    from paper_2406_05546_b200 import ps
+    theta = synth.init_params(seed=1)
+    theta[4800:807616] = 0
+    theta[807616:808128] = 1
+    srv = ps.ParameterServer(theta, max_workers=4, max_batch=1, queue_slots=4)
+    x = np.random.default_rng(0).random((4, 1, 28, 28), dtype=np.float32)
+    y = np.array([[1], [2], [3], [4]], dtype=np.int32)
+    ids = [9, 0, 77, 3]
+    snaps = [srv.ps_pull_snapshot(w) for w in range(4)]
+    gd = torch.zeros((4, ps.P_PAD), device="cuda")
+    srv.workers_grad_step(snaps, ids, torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(), SEED, 21, grads_dev=gd)
+    g = gd.cpu().numpy()
+    for w in range(4):
+        keep = cnn.dropout_keep(SEED, ids[w], 21, 1, 0.25)[0]
+        gw2 = g[w, 808128:813248].reshape(10, 512)
+        assert ((gw2 != 0).all(axis=0) == (keep == 1)).all()
+        assert ((gw2 == 0).all(axis=0) == (keep == 0)).all()
+    srv.close()
+
+
+def test_bad_label_is_reported_not_trapped():
+    torch, ps, srv, _ = _setup(1, 2)
+    x = torch.zeros((1, 2, 28, 28), device="cuda")
+    y = torch.tensor([[3, 12]], dtype=torch.int32, device="cuda")
+    gd = torch.zeros((1, ps.P_PAD), device="cuda")
+    srv.workers_grad_step([srv.ps_pull_snapshot(0)], [0], x, y, SEED, 0, grads_dev=gd)
+    with pytest.raises(ps.PSError) as e:
+        srv.ps_stats()
+    assert e.value.name == "PS_ERR_DEVICE_STATUS"
+    srv.close()
+
+
+def test_argument_errors():
+    torch, ps, srv, _ = _setup(2, 4)
+    x = torch.zeros((3, 4, 28, 28), device="cuda")
+    y = torch.zeros((3, 4), dtype=torch.int32, device="cuda")
+    snaps = [srv.ps_pull_snapshot(0)] * 3
+    with pytest.raises(ps.PSError) as e:
+        srv.workers_grad_step(snaps, [0, 1, 2], x, y, SEED, 0, grads_dev=torch.zeros((3, ps.P_PAD), device="cuda"))
+    assert e.value.name == "PS_ERR_BAD_ARG"
+    with pytest.raises(ps.PSError):
+        srv.workers_grad_step(snaps[:2], [0, 1], x[:2], y[:2], SEED, 0, slot_ids=[0, 1])   # not reserved
+    with pytest.raises(ps.PSError) as e:
+        srv.ps_pull_snapshot(0, lag=1)
+    assert e.value.name == "PS_ERR_VERSION_EVICTED"
+    srv.close()
