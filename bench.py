@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the parameter-server hot path on B200.
+
+Workload: the largest configuration ("scale"): W = 128 logical workers, batch 128 each, stateless
+server.  A step is one tick of the whole path: every worker pulls its snapshot, the grad step
+writes 128 gradients into reserved queue slots, they are enqueued, and the server applies them
+(the stateless server's step).  `value` is worker-samples/s with inputs resident in HBM; `e2e` is
+the same tick through ps_tick_host with pinned host inputs copied in and losses copied out every
+step.  The deferred replay of a 200-tick outage (25,600 gradients, 83 GB) is timed separately and
+reported as GB/s under "replay".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+W_WORKERS, BATCH = 128, 128
+DOWN_TICKS = 200
+LR = 0.01
+DROP_SEED = 0x5EED
+FLOP_PER_SAMPLE = 10_718_208            # 2 x (1,824,000 forward + 3,535,104 backward multiply-adds)
+GRAD_BYTES = 813258 * 4                 # algorithmic bytes per queued gradient
+N_BATCH_BUFFERS = 8
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                "sm_max_mhz": d.get("sm_max_mhz", 1965.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [l for t, l in self.lines if (t0 is None or t >= t0) and (t1 is None or t <= t1 + 0.1)] or \
+               [l for _, l in self.lines]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            f = [v.strip() for v in l.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_baseline(budget_s=12.0):
+    """The oracle, as it stands, on the host cores: one tick's grad step on a bounded sample of workers."""
+    from oracle import cnn
+    from paper_2406_05546_b200 import synth
+    cores = cnn.num_threads()
+    theta = synth.init_params(1)
+    px, py = synth.image_pool(4096, seed=0)
+    done, t_used = 0, 0.0
+    chunk = max(cores, 1)
+    w0 = 0
+    while t_used < budget_s and w0 < W_WORKERS:
+        n = min(chunk, W_WORKERS - w0)
+        rows = (np.arange(n)[:, None] * BATCH + np.arange(BATCH)[None, :] + w0 * BATCH) % px.shape[0]
+        x, y = px[rows], py[rows]
+        t = time.perf_counter()
+        cnn.workers_grad_step([theta] * n, list(range(w0, w0 + n)), x, y, DROP_SEED, 0, 0.25)
+        t_used += time.perf_counter() - t
+        done += n
+        w0 += n
+    return {"value": done * BATCH / t_used, "unit": "worker-samples/s", "cores": cores, "kind": "oracle",
+            "sample": f"grad step of {done} of the {W_WORKERS} workers of one tick (batch {BATCH}), {t_used:.1f} s"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on a bounded sample of the same workload, per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import cnn, ps as ops
+    from paper_2406_05546_b200 import synth
+    cores = cnn.num_threads()
+    n = min(W_WORKERS, max(cores, 1))                # workers per step in the sample
+    px, py = synth.image_pool(8192, seed=0)
+    srv = ops.OraclePS(synth.init_params(1), external_store=True)
+    times = []
+    for step in range(args.warmup + args.steps):
+        rows = synth.batch_rows(step, n, BATCH, px.shape[0])
+        x, y = px[rows], py[rows]
+        t = time.perf_counter()
+        v, theta = srv.pull_snapshot(0)
+        g, loss, am, _ = cnn.workers_grad_step([theta] * n, list(range(n)), x, y, DROP_SEED, step, 0.25)
+        srv.enqueue(g.astype(np.float32), range(n), [v] * n, step)
+        srv.apply(ops.REPLAY, LR)
+        dt = time.perf_counter() - t
+        if step >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = n * BATCH * args.steps / total
+    sample = f"{n} of the {W_WORKERS} workers per tick (batch {BATCH}): snapshot, grad step, enqueue, apply"
+    print(json.dumps({
+        "impl": "reference", "metric": "worker-samples/s", "value": value, "unit": "worker-samples/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config 5 (scale): W=128 workers x batch 128, stateless server", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "worker-samples/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "worker-samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2406_05546_b200 import ps, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    peaks = measured_peaks()
+    # the CPU leg (OpenMP threads of the oracle) runs before the first GPU call
+    cpu = None
+    if rank == 0 and world == 1:
+        cpu = cpu_baseline()
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v):
+        if dist is None:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    W, b = W_WORKERS, BATCH
+    K_replay = DOWN_TICKS * W
+    do_replay = True
+    srv = ps.ParameterServer(synth.init_params(1), max_workers=W, max_batch=b, ring_depth=1,
+                             queue_slots=(K_replay if do_replay else 0) + W, external_store=True, dropout_p=0.25)
+    # synthetic stand-in for the 60,000-image training pool, resident in HBM; every rank its own rows
+    px, py = synth.image_pool(synth.POOL_IMAGES, seed=0)
+    pool_x, pool_y = torch.from_numpy(px).cuda(), torch.from_numpy(py).cuda()
+    bufs = []
+    for t in range(N_BATCH_BUFFERS):
+        rows = torch.from_numpy(synth.batch_rows(t + rank * 1000, W, b, px.shape[0])).cuda()
+        bufs.append((pool_x[rows].contiguous(), pool_y[rows].contiguous()))
+    loss_dev = torch.empty(W, dtype=torch.float32, device="cuda")
+    am_dev = torch.empty((W, b), dtype=torch.int32, device="cuda")
+    ids = list(range(W))
+    tick_no = [0]
+
+    def tick(apply=True):
+        t = tick_no[0]
+        x, y = bufs[t % N_BATCH_BUFFERS]
+        snaps = [srv.ps_pull_snapshot(w) for w in range(W)]
+        slots = srv.ps_queue_reserve(W)
+        srv.workers_grad_step(snaps, ids, x, y, DROP_SEED, t, slot_ids=slots, loss_dev=loss_dev, argmax_dev=am_dev)
+        srv.ps_enqueue(ids, [s.version for s in snaps], t, slot_ids=slots)
+        if apply:
+            srv.ps_apply(ps.REPLAY, LR)
+        tick_no[0] += 1
+
+    for _ in range(args.warmup):
+        tick()
+    # ---- timed region: K whole ticks, inputs resident, CUDA events on the library's stream
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = srv.ps_stats()["kernel_launches"]
+    barrier()
+    t_wall0 = time.time()
+    ev0.record(srv.stream)
+    for _ in range(args.steps):
+        tick()
+    ev1.record(srv.stream)
+    barrier()
+    t_wall1 = time.time()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    launches = srv.ps_stats()["kernel_launches"] - l0
+
+    # ---- second pass with per-kernel events: which kernel dominates, and its roofline
+    srv.ps_profile(True)
+    for _ in range(args.steps):
+        tick()
+    prof = srv.ps_profile_read()
+    srv.ps_profile(False)
+    clocks = sampler.stop(t_wall0, time.time())
+
+    # ---- end to end: pinned host inputs in, losses out, through ps_tick_host
+    hx = [torch.from_numpy(px[synth.batch_rows(t, W, b, px.shape[0])]).pin_memory() for t in range(2)]
+    hy = [torch.from_numpy(py[synth.batch_rows(t, W, b, px.shape[0])]).pin_memory() for t in range(2)]
+    loss_host = torch.empty(W, dtype=torch.float32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for t in range(3):
+        srv.ps_tick_host(hx[t % 2], hy[t % 2], DROP_SEED, 10_000 + t, ps.REPLAY, LR, loss_host=loss_host)
+    barrier()
+    t0 = time.perf_counter()
+    for t in range(e2e_steps):
+        srv.ps_tick_host(hx[t % 2], hy[t % 2], DROP_SEED, 20_000 + t, ps.REPLAY, LR, loss_host=loss_host)
+    barrier()
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
+    h2d = W * b * 784 * 4 + W * b * 4
+    d2h = W * 4
+
+    # ---- deferred replay of a DOWN_TICKS outage (83 GB of buffered gradients)
+    replay = None
+    if do_replay:
+        reps = []
+        for rep in range(2):
+            srv.ps_kill()
+            for _ in range(DOWN_TICKS):
+                tick(apply=False)
+            srv.ps_restore()
+            assert srv.ps_stats()["queue_len"] == K_replay
+            r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            barrier()
+            r0.record(srv.stream)
+            res = srv.ps_apply(ps.REPLAY, LR, scale=1.0 / DOWN_TICKS)
+            r1.record(srv.stream)
+            barrier()
+            assert res["applied"] == K_replay
+            reps.append(r0.elapsed_time(r1))
+        ms = max_over_ranks(min(reps))
+        bytes_alg = (K_replay + 2) * GRAD_BYTES
+        gbs = bytes_alg / (ms * 1e-3) / 1e9
+        replay = {"queue_gradients": K_replay, "bytes": bytes_alg, "ms": ms, "gb_per_s": gbs * world,
+                  "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+                  "all_ms": reps}
+    stats = srv.ps_stats()
+
+    if rank == 0:
+        samples = W * b * args.steps * world
+        value = samples / (ms_total * 1e-3)
+        total_prof = sum(ms for ms, _ in prof.values()) or 1.0
+        kernels = {k: {"ms_per_launch": ms / n, "launches": n, "share": ms / total_prof}
+                   for k, (ms, n) in prof.items() if n}
+        top = max(kernels, key=lambda k: kernels[k]["share"])
+        roof = kernel_roofline(top, kernels[top]["ms_per_launch"], W, b, peaks)
+        out = {
+            "metric": "worker-samples/s", "value": value, "unit": "worker-samples/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": "config 5 (scale): W=128 workers x batch 128, stateless server, one tick = "
+                                   "pull + grad step + enqueue + apply",
+                       "W": W, "b": b, "l2": "inputs larger than L2: each tick writes 416 MB of gradients and "
+                                             "cycles 8 distinct 51 MB input batches",
+                       "replicas": "independent replica per GPU, no collective" if world > 1 else "single GPU"},
+            "e2e": {"value": W * b * e2e_steps * world / (e2e_ms * 1e-3), "unit": "worker-samples/s",
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": roof,
+            "kernels": kernels,
+            "replay": replay,
+            "cpu_baseline": cpu,
+            "final_version": stats["version"],
+        }
+        print(json.dumps(out))
+    srv.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def kernel_roofline(name, ms_per_launch, W, b, peaks):
+    """Algorithmic work of one launch of the named kernel at (W, b) against the roofline that bounds it."""
+    n = W * b
+    sec = ms_per_launch * 1e-3
+    sm_clock_ghz = peaks["sm_max_mhz"] / 1e3
+    fp32_peak_tflops = 148 * 128 * 2 * sm_clock_ghz / 1e3        # 148 SMs x 128 FP32 lanes x FMA
+    flops = {
+        "conv1_fwd": 2 * 112_896 * n, "conv2_fwd": 2 * 903_168 * n, "fc1_fwd": 2 * 802_816 * n,
+        "fc1_dw": 2 * 802_816 * n, "fc1_dx": 2 * 802_816 * n, "conv2_bwd": 2 * 2 * 903_168 * n,
+        "conv1_bwd": 2 * 112_896 * n, "fc2_fwd_bwd": 2 * 3 * 5_120 * n,
+    }
+    if name in flops:
+        ach = flops[name] / sec / 1e12
+        return {"kernel": name, "bound": "alu", "achieved": ach, "peak": fp32_peak_tflops, "unit": "TFLOP/s",
+                "frac": ach / fp32_peak_tflops, "traffic": None,
+                "peak_source": "148 SMs x 128 FP32 lanes x 2 x max SM clock"}
+    bytes_ = {"sum_apply_direct": (W + 2) * GRAD_BYTES, "conv_grad_reduce": 0}.get(name, 0)
+    ach = bytes_ / sec / 1e9
+    return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}
+
+
+if __name__ == "__main__":
+    main()

@@ -228,6 +228,14 @@ int32_t ps_tick_host(ps_ctx* ctx, int32_t W, int32_t b, const int32_t* lags, con
                      float lr, float scale, const int32_t* order, float* loss_host,
                      int32_t* argmax_host, ps_apply_result* out);
 
+/* Per-kernel timing for measurement (no counterpart in the paper's method; it serves the roofline
+ * report).  ps_profile(ctx, 1) clears the totals and from then on brackets every kernel launch with
+ * two CUDA events on the context's stream; ps_profile(ctx, 0) stops.  ps_profile_read() synchronises
+ * the stream and returns, for kernel index 0..n-1, its name (static string), summed device time in
+ * milliseconds and launch count; an index past the last kernel returns PS_ERR_BAD_ARG. */
+int32_t ps_profile(ps_ctx* ctx, int32_t enable);
+int32_t ps_profile_read(ps_ctx* ctx, int32_t kernel, const char** name, double* total_ms, int64_t* launches);
+
 const char* ps_last_error(ps_ctx* ctx);
 
 #ifdef __cplusplus

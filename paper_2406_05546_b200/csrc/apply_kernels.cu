@@ -127,7 +127,17 @@ __global__ void __launch_bounds__(TPB) copy_rows(float4* __restrict__ dst, const
 
 }  // namespace
 
-int launch_sum_apply(const SumApplyArgs& a, cudaStream_t st) {
+#define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
+
+const char* kernel_name(int id) {
+  static const char* names[K_COUNT] = {
+      "conv1_fwd", "conv2_fwd", "fc1_fwd", "fc2_fwd_bwd", "fc1_dw", "fc1_dx", "conv2_bwd", "conv1_bwd",
+      "conv_grad_reduce", "sum_apply_direct", "sum_partial", "sum_finish", "async_apply", "copy_rows",
+      "dropout_mask"};
+  return id >= 0 && id < K_COUNT ? names[id] : "?";
+}
+
+int launch_sum_apply(const SumApplyArgs& a, cudaStream_t st, Profiler* prof) {
   const float4* q = reinterpret_cast<const float4*>(a.queue);
   const float4* tin = reinterpret_cast<const float4*>(a.theta_in);
   float4* tout = reinterpret_cast<float4*>(a.theta_out);
@@ -139,28 +149,28 @@ int launch_sum_apply(const SumApplyArgs& a, cudaStream_t st) {
   }
   int launches = 0;
   if (n_split <= 1) {
-    sum_apply_direct<<<COL_BLOCKS, TPB, 0, st>>>(q, a.K, tin, tout, rep, a.coef);
+    TIMED(K_SUM_APPLY_DIRECT, (sum_apply_direct<<<COL_BLOCKS, TPB, 0, st>>>(q, a.K, tin, tout, rep, a.coef)));
     launches = 1;
   } else {
     float4* part = reinterpret_cast<float4*>(a.partial);
-    sum_partial<<<dim3(COL_BLOCKS, n_split), TPB, 0, st>>>(q, a.K, n_split, part);
-    sum_finish<<<COL_BLOCKS, TPB, 0, st>>>(part, n_split, tin, tout, rep, a.coef);
+    TIMED(K_SUM_PARTIAL, (sum_partial<<<dim3(COL_BLOCKS, n_split), TPB, 0, st>>>(q, a.K, n_split, part)));
+    TIMED(K_SUM_FINISH, (sum_finish<<<COL_BLOCKS, TPB, 0, st>>>(part, n_split, tin, tout, rep, a.coef)));
     launches = 2;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
-int launch_async_apply(const AsyncApplyArgs& a, const AsyncOrder& ord, cudaStream_t st) {
-  async_apply<<<COL_BLOCKS, TPB, 0, st>>>(a, ord);
+int launch_async_apply(const AsyncApplyArgs& a, const AsyncOrder& ord, cudaStream_t st, Profiler* prof) {
+  TIMED(K_ASYNC_APPLY, (async_apply<<<COL_BLOCKS, TPB, 0, st>>>(a, ord)));
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
-int launch_copy_rows(float* dst, const float* src, int64_t rows, cudaStream_t st) {
+int launch_copy_rows(float* dst, const float* src, int64_t rows, cudaStream_t st, Profiler* prof) {
   int64_t n_vec = rows * P_VEC4;
   int64_t blocks = (n_vec + TPB - 1) / TPB;
   if (blocks > 148 * 16) blocks = 148 * 16;
-  copy_rows<<<(int)blocks, TPB, 0, st>>>(reinterpret_cast<float4*>(dst),
-                                         reinterpret_cast<const float4*>(src), n_vec);
+  TIMED(K_COPY_ROWS, (copy_rows<<<(int)blocks, TPB, 0, st>>>(reinterpret_cast<float4*>(dst),
+                                                            reinterpret_cast<const float4*>(src), n_vec)));
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

@@ -548,11 +548,13 @@ int tiles_64(const GroupTable& gt, int b) {
 
 }  // namespace
 
+#define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
+
 int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, uint32_t thresh,
-                        uint8_t* keep, cudaStream_t st) {
+                        uint8_t* keep, cudaStream_t st, Profiler* prof) {
   int n_quads = b * HID / 4;
-  dropout_mask<<<(n_quads + 255) / 256, 256, 0, st>>>(seed, worker, step, n_quads, thresh,
-                                                      reinterpret_cast<uchar4*>(keep));
+  TIMED(K_DROPOUT_MASK, (dropout_mask<<<(n_quads + 255) / 256, 256, 0, st>>>(seed, worker, step, n_quads, thresh,
+                                                                            reinterpret_cast<uchar4*>(keep))));
   return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
@@ -563,18 +565,18 @@ int configure_grad_kernels() {
 }
 
 int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt,
-                          const Workspace& ws, cudaStream_t st) {
+                          const Workspace& ws, cudaStream_t st, Profiler* prof) {
   const int n_chunks = (a.b + CONV_SPB - 1) / CONV_SPB;
   const int mt = tiles_64(gt, a.b);
-  conv1_fwd<<<dim3(a.b, a.W), 256, 0, st>>>(a, wt, gt, ws);
-  conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws);
-  fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws);
-  fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws);
-  fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws);
-  fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws);
-  conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks);
-  conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks);
-  conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks);
+  TIMED(K_CONV1_FWD, (conv1_fwd<<<dim3(a.b, a.W), 256, 0, st>>>(a, wt, gt, ws)));
+  TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
+  TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
+  TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
+  TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
+  TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
+  TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
+  TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
+  TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks)));
   return cudaGetLastError() == cudaSuccess ? 9 : -1;
 }
 

@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 namespace psk {
 
 constexpr int P = 813258;
@@ -24,6 +26,52 @@ constexpr int CONV_SPB = 4;              // samples per block in the conv backwa
 constexpr int C2_GRAD = 4608 + 32, C1_GRAD = 144 + 16;
 
 constexpr uint32_t STATUS_BAD_LABEL = 1u;
+
+// Optional per-kernel timing: when switched on, every launch is bracketed by two CUDA events on
+// the launching stream; totals per kernel are read back after a synchronisation.
+enum KernelId {
+  K_CONV1_FWD = 0, K_CONV2_FWD, K_FC1_FWD, K_FC2_FWD_BWD, K_FC1_DW, K_FC1_DX, K_CONV2_BWD, K_CONV1_BWD,
+  K_CONV_GRAD_REDUCE, K_SUM_APPLY_DIRECT, K_SUM_PARTIAL, K_SUM_FINISH, K_ASYNC_APPLY, K_COPY_ROWS,
+  K_DROPOUT_MASK, K_COUNT
+};
+const char* kernel_name(int id);
+
+struct Profiler {
+  bool on = false;
+  struct Rec { int id; cudaEvent_t a, b; };
+  std::vector<Rec> recs;
+  std::vector<cudaEvent_t> free_events;
+  cudaEvent_t get() {
+    if (!free_events.empty()) { cudaEvent_t e = free_events.back(); free_events.pop_back(); return e; }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+  }
+  void begin(int id, cudaStream_t st) {
+    if (!on) return;
+    Rec r{id, get(), get()};
+    cudaEventRecord(r.a, st);
+    recs.push_back(r);
+  }
+  void end(cudaStream_t st) {
+    if (!on) return;
+    cudaEventRecord(recs.back().b, st);
+  }
+  // Caller has synchronised the stream.  Adds elapsed times into ms[K_COUNT] / n[K_COUNT] and recycles events.
+  void collect(double* ms, int64_t* n) {
+    for (auto& r : recs) {
+      float t = 0.f;
+      if (cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) { ms[r.id] += t; n[r.id] += 1; }
+      free_events.push_back(r.a);
+      free_events.push_back(r.b);
+    }
+    recs.clear();
+  }
+  ~Profiler() {
+    for (auto& r : recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (auto e : free_events) cudaEventDestroy(e);
+  }
+};
 
 // Per-call tables passed by value as kernel parameters.
 // Workers are processed in "sorted" order: workers sharing a weight snapshot are adjacent, so
@@ -70,9 +118,9 @@ struct GradStepArgs {
 
 // Part A, FP32 CUDA-core path. Returns the number of kernels launched, or -1 on a launch error.
 int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt,
-                          const Workspace& ws, cudaStream_t st);
+                          const Workspace& ws, cudaStream_t st, Profiler* prof);
 int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, uint32_t thresh,
-                        uint8_t* keep, cudaStream_t st);
+                        uint8_t* keep, cudaStream_t st, Profiler* prof);
 int configure_grad_kernels();   // one-time function attributes (dynamic shared memory sizes)
 
 // Part B.
@@ -86,7 +134,7 @@ struct SumApplyArgs {
   float* partial;           // [max_split][P_PAD] scratch
   int max_split;
 };
-int launch_sum_apply(const SumApplyArgs& a, cudaStream_t st);
+int launch_sum_apply(const SumApplyArgs& a, cudaStream_t st, Profiler* prof);
 
 constexpr int ASYNC_SEG = 256;   // gradients per ordered-apply launch
 struct AsyncOrder { int32_t slot[ASYNC_SEG]; };
@@ -102,8 +150,8 @@ struct AsyncApplyArgs {
   float* replica;
   float coef;               // lr*scale
 };
-int launch_async_apply(const AsyncApplyArgs& a, const AsyncOrder& ord, cudaStream_t st);
+int launch_async_apply(const AsyncApplyArgs& a, const AsyncOrder& ord, cudaStream_t st, Profiler* prof);
 
-int launch_copy_rows(float* dst, const float* src, int64_t rows, cudaStream_t st);
+int launch_copy_rows(float* dst, const float* src, int64_t rows, cudaStream_t st, Profiler* prof);
 
 }  // namespace psk

@@ -72,6 +72,9 @@ struct ps_ctx {
   int32_t w_tick = 0;
   std::vector<QueueMeta> meta;
   uint32_t drop_thresh = 0;
+  psk::Profiler prof;
+  double prof_ms[psk::K_COUNT] = {0};
+  int64_t prof_n[psk::K_COUNT] = {0};
 };
 
 namespace {
@@ -311,7 +314,7 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
   psk::GradStepArgs a;
   a.W = W; a.b = b; a.x = x_dev; a.y = y_dev; a.loss = loss_dev; a.argmax = argmax_dev;
   a.seed = seed; a.step = step; a.drop_p = x->cfg.dropout_p; a.drop_thresh = x->drop_thresh;
-  int n = psk::launch_grad_step_fp32(a, wt, gt, x->ws, x->st);
+  int n = psk::launch_grad_step_fp32(a, wt, gt, x->ws, x->st, &x->prof);
   if (n < 0) return cuda_fail(cudaGetLastError(), "grad step launch");
   x->launches += n;
   return PS_OK;
@@ -320,7 +323,7 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
 int32_t ps_dropout_mask(ps_ctx* x, uint64_t seed, int32_t worker_id, uint64_t step, int32_t b, uint8_t* keep_dev) {
   if (!x || !keep_dev || b < 1 || b > 4096) return fail(PS_ERR_BAD_ARG, "bad argument");
   if (((uint64_t)keep_dev & 3) != 0) return fail(PS_ERR_BAD_ARG, "keep_dev must be 4-byte aligned");
-  int n = psk::launch_dropout_mask(seed, (uint32_t)worker_id, step, b, x->drop_thresh, keep_dev, x->st);
+  int n = psk::launch_dropout_mask(seed, (uint32_t)worker_id, step, b, x->drop_thresh, keep_dev, x->st, &x->prof);
   if (n < 0) return cuda_fail(cudaGetLastError(), "dropout mask launch");
   x->launches += n;
   return PS_OK;
@@ -338,7 +341,7 @@ int32_t ps_enqueue(ps_ctx* x, int32_t n, const int64_t* slot_ids, const float* g
     for (int i = 0; i < n; ++i)
       if (slot_ids[i] != x->queue_len + i) return fail(PS_ERR_BAD_ARG, "slot_ids must be the reserved slots in order");
   } else {
-    int r = psk::launch_copy_rows(x->queue + x->queue_len * (int64_t)psk::P_PAD, grads_dev, n, x->st);
+    int r = psk::launch_copy_rows(x->queue + x->queue_len * (int64_t)psk::P_PAD, grads_dev, n, x->st, &x->prof);
     if (r < 0) return cuda_fail(cudaGetLastError(), "enqueue copy");
     x->launches += r;
   }
@@ -395,7 +398,7 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
     a.replica = mirror ? rep->buf : nullptr;
     a.coef = lr * scale / (float)(mode == PS_SYNC ? K : (int64_t)x->w_tick);
     a.partial = x->partial; a.max_split = MAX_SPLIT;
-    int n = psk::launch_sum_apply(a, x->st);
+    int n = psk::launch_sum_apply(a, x->st, &x->prof);
     if (n < 0) return cuda_fail(cudaGetLastError(), "apply launch");
     x->launches += n;
     x->version += 1;
@@ -433,7 +436,7 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
         }
       }
       for (int64_t u = 0; u < seg; ++u) ord.slot[u] = order ? order[pos + u] : (int32_t)(pos + u);
-      int n = psk::launch_async_apply(a, ord, x->st);
+      int n = psk::launch_async_apply(a, ord, x->st, &x->prof);
       if (n < 0) return cuda_fail(cudaGetLastError(), "async apply launch");
       x->launches += n;
       x->version += (uint64_t)seg;
@@ -570,6 +573,26 @@ int32_t ps_stats(ps_ctx* x, ps_stats_t* out) {
   out->last_ckpt_version = x->ckpt_order.empty() ? 0 : x->ckpt_version[x->ckpt_order.back()];
   out->kernel_launches = x->launches;
   if (out->device_status != 0) return fail(PS_ERR_DEVICE_STATUS, "device status 0x%x (bit 0: label outside 0..9)", out->device_status);
+  return PS_OK;
+}
+
+int32_t ps_profile(ps_ctx* x, int32_t enable) {
+  if (!x) return fail(PS_ERR_BAD_ARG, "ctx is NULL");
+  CUDA_TRY(cudaStreamSynchronize(x->st));
+  x->prof.collect(x->prof_ms, x->prof_n);
+  x->prof.on = enable != 0;
+  if (enable) for (int i = 0; i < psk::K_COUNT; ++i) { x->prof_ms[i] = 0; x->prof_n[i] = 0; }
+  return PS_OK;
+}
+
+int32_t ps_profile_read(ps_ctx* x, int32_t kernel, const char** name, double* total_ms, int64_t* launches) {
+  if (!x || kernel < 0) return fail(PS_ERR_BAD_ARG, "bad argument");
+  if (kernel >= psk::K_COUNT) return fail(PS_ERR_BAD_ARG, "no kernel %d", kernel);
+  CUDA_TRY(cudaStreamSynchronize(x->st));
+  x->prof.collect(x->prof_ms, x->prof_n);
+  if (name) *name = psk::kernel_name(kernel);
+  if (total_ms) *total_ms = x->prof_ms[kernel];
+  if (launches) *launches = x->prof_n[kernel];
   return PS_OK;
 }
 

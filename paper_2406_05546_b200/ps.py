@@ -23,7 +23,7 @@ ERRORS = {-1: "PS_ERR_BAD_ARG", -2: "PS_ERR_DOWN", -3: "PS_ERR_QUEUE_FULL", -4: 
 EXPORTS = ["ps_query_bytes", "ps_create", "ps_destroy", "ps_pull_snapshot", "ps_queue_reserve", "ps_slot_ptr",
            "workers_grad_step", "ps_dropout_mask", "ps_enqueue", "ps_apply", "ps_checkpoint", "ps_restore", "ps_replicate",
            "ps_kill", "ps_failover", "ps_import_params", "ps_export_params", "ps_stats", "ps_tick_host",
-           "ps_last_error"]
+           "ps_profile", "ps_profile_read", "ps_last_error"]
 
 
 class PSError(RuntimeError):
@@ -89,6 +89,8 @@ def load(path=None):
         "ps_stats": [vp, C.POINTER(Stats)],
         "ps_tick_host": [vp, i32, i32, vp, vp, vp, u64, u64, i32, f32, f32, vp, vp, vp, C.POINTER(ApplyResult)],
     }
+    sig["ps_profile"] = [vp, i32]
+    sig["ps_profile_read"] = [vp, i32, C.POINTER(C.c_char_p), C.POINTER(C.c_double), C.POINTER(i64)]
     for name, args in sig.items():
         fn = getattr(L, name)
         fn.argtypes = args
@@ -268,6 +270,21 @@ class ParameterServer:
                                           ptr(argmax_host) if argmax_host is not None else None, C.byref(res)))
         return loss_host, {"applied": res.applied, "new_version": res.new_version,
                            "checkpointed": res.checkpointed, "replicated": res.replicated}
+
+    def ps_profile(self, enable):
+        self._check(self.lib.ps_profile(self.ctx, int(bool(enable))))
+
+    def ps_profile_read(self):
+        """{kernel name: (total ms, launches)} since profiling was switched on."""
+        out = {}
+        k = 0
+        while True:
+            name, ms, n = C.c_char_p(), C.c_double(), C.c_int64()
+            if self.lib.ps_profile_read(self.ctx, k, C.byref(name), C.byref(ms), C.byref(n)) != 0:
+                break
+            out[name.value.decode()] = (ms.value, n.value)
+            k += 1
+        return out
 
     # -- helpers for tests (plain copies through torch, no arithmetic) ----------
     def slot_tensor(self, slot):
