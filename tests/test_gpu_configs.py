@@ -1,0 +1,163 @@
+"""GPU parity on the five workload schedules: reduced sizes followed tick by tick by the oracle,
+and the full sizes checked on sampled workers / sampled parameter columns."""
+import numpy as np
+import pytest
+
+from paper_2406_05546_b200 import schedules, synth
+from tests import oracle_driver
+from tests.parity import TOL_FP32, assert_argmax_valid, assert_params_close
+
+pytestmark = pytest.mark.gpu
+
+LOCK_FROM = 20
+
+
+def _follow(n, pool=2048):
+    """Runs reduced config n on the GPU and on the oracle, tick by tick.
+
+    Integers (versions, queue lengths, events, apply counters) are compared exactly at every tick.
+    Floats: the two sides run freely for the first LOCK_FROM ticks; after that the trajectories of a
+    ReLU/max-pool network separate whenever rounding flips one unit's sign, so from then on the GPU
+    head is loaded with the oracle's before each tick (step-locked) and each tick is compared on
+    its own."""
+    from paper_2406_05546_b200 import harness
+    s = schedules.reduced(n)
+    px, py = synth.image_pool(pool, seed=0)
+    theta = synth.init_params(1)
+    srv = harness.make_server(s, theta)
+    o = oracle_driver.make_oracle(s, theta)
+    glog, olog = [], []
+    for t in range(s.ticks):
+        if t >= LOCK_FROM and o.ring and srv.ps_stats()["up"]:
+            srv.ps_import_params(o.head())
+        g = harness.run(s, srv, px, py, first_tick=t, last_tick=t + 1)[0]
+        r = oracle_driver.run(s, o, px, py, first_tick=t, last_tick=t + 1)[0]
+        glog.append(g); olog.append(r)
+        assert g["version"] == r["version"], t
+        assert g["queue_len"] == r["queue_len"], t
+        assert g["events"] == r["events"], t
+        assert g["apply"] == r["apply"], t
+        assert (g["loss"] is None) == (r["loss"] is None)
+        if g["loss"] is not None:
+            np.testing.assert_allclose(g["loss"][0], r["loss"][0], rtol=2e-4, atol=1e-5, err_msg=f"tick {t}")
+            assert_argmax_valid(g["loss"][1], r["loss"][2], 10 * TOL_FP32)
+        if o.ring and g["stats"]["up"]:
+            assert_params_close(srv.ps_export_params()[0], o.head(), TOL_FP32, f"config {n} tick {t}")
+    return s, srv, o, glog, olog
+
+
+def test_config1_sync_ten_steps():
+    s, srv, o, glog, _ = _follow(1)
+    assert glog[-1]["version"] == 10
+    srv.close()
+
+
+def test_config2_checkpoint_rollback():
+    s, srv, o, glog, _ = _follow(2)
+    assert glog[80]["events"] == [("restore", 50)] and glog[-1]["version"] == 170
+    st = srv.ps_stats()
+    assert st["last_ckpt_version"] == 150 and st["checkpoints"] == 6      # 25, 50, then 75..150 after the rollback
+    assert [v for v, _ in o.ckpts] == [25, 50, 75, 100, 125, 150]
+    for j, (v_o, th_o) in enumerate(reversed(o.ckpts)):
+        th_g, v_g = srv.ps_export_params(1000 + j)
+        assert v_g == v_o
+        assert_params_close(th_g, th_o, TOL_FP32, f"checkpoint {v_o}")
+    srv.close()
+
+
+def test_config3_stateless_replay():
+    s, srv, o, glog, _ = _follow(3)
+    assert glog[20]["apply"]["applied"] == 44 and glog[19]["queue_len"] == 40
+    srv.close()
+
+
+def test_config4_async_chain_failover():
+    s, srv, o, glog, _ = _follow(4)
+    assert glog[30]["events"] == [("failover", 240)] and glog[-1]["version"] == 320
+    assert glog[-1]["stats"]["live_replicas"] == 0
+    srv.close()
+
+
+def test_config5_stateless_scale_reduced():
+    s, srv, o, glog, _ = _follow(5)
+    assert glog[30]["apply"]["applied"] == 8 * 11
+    srv.close()
+
+
+def test_full_size_config5_tick_on_sampled_workers():
+    """W=128 x b=128 in the launch configuration the benchmark times; the oracle recomputes three workers."""
+    import torch
+    from oracle import cnn
+    from oracle import ps as ops
+    from paper_2406_05546_b200 import harness, ps
+    s = schedules.config(5)
+    px, py = synth.image_pool(synth.POOL_IMAGES, seed=0)
+    theta = synth.init_params(1)
+    srv = harness.make_server(s, theta, queue_slots=s.W)
+    t = 3
+    x, y = synth.tick_batch(px, py, t, s.W, s.b)
+    snaps = [srv.ps_pull_snapshot(w) for w in range(s.W)]
+    slots = srv.ps_queue_reserve(s.W)
+    loss, am = srv.workers_grad_step(snaps, list(range(s.W)), torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(),
+                                     s.seed, t, slot_ids=slots)
+    loss, am = loss.cpu().numpy(), am.cpu().numpy()
+    sample = [0, 77, 127]
+    og, ol, oa, oz = cnn.workers_grad_step([theta] * 3, sample, x[sample], y[sample], s.seed, t, 0.25)
+    for j, w in enumerate(sample):
+        g = srv.slot_tensor(slots[w]).cpu().numpy()
+        assert_params_close(g[:ps.P], og[j], TOL_FP32, f"worker {w}")
+        assert (g[ps.P:] == 0).all()
+        assert abs(loss[w] - ol[j]) <= 1e-5 * abs(ol[j])
+        assert_argmax_valid(am[w], oz[j], TOL_FP32)
+    for w in range(s.W):      # every worker wrote a finite, non-trivial gradient
+        g = srv.slot_tensor(slots[w])
+        assert bool(torch.isfinite(g).all()) and float(g.abs().max()) > 0
+    # the tick's apply over all 128 gradients, every column against the definition
+    srv.ps_enqueue(list(range(s.W)), [0] * s.W, t, slot_ids=slots)
+    allg = torch.stack([srv.slot_tensor(sl) for sl in slots]).cpu().numpy()[:, :ps.P]
+    o = ops.OraclePS(theta, external_store=True)
+    o.enqueue(allg, range(s.W), [0] * s.W, t)
+    assert o.apply(ops.REPLAY, s.lr) == srv.ps_apply(ps.REPLAY, s.lr)
+    assert_params_close(srv.ps_export_params()[0], o.head(), 1e-6, "tick apply")
+    srv.close()
+
+
+def test_full_size_replay_of_25600_gradients_on_sampled_columns():
+    """The 83 GB replay in the benchmark's launch configuration: the queue is filled with synthetic
+    gradients and the oracle replays a sample of parameter columns."""
+    import torch
+    from oracle import ps as ops
+    from paper_2406_05546_b200 import harness, ps
+    free, total = torch.cuda.mem_get_info()
+    s = schedules.config(5)
+    K = s.W * (s.recover_at - s.kill_at)
+    need = (K + s.W + 64) * ps.P_PAD * 4
+    if free < need + (4 << 30):
+        pytest.skip("not enough free device memory for the 83 GB queue")
+    theta = synth.init_params(1)
+    srv = harness.make_server(s, theta)
+    srv.ps_kill()
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    cols = np.sort(np.random.default_rng(1).choice(ps.P, size=384, replace=False))
+    cols_d = torch.from_numpy(cols).cuda()
+    o = ops.OraclePS(theta[cols], external_store=True)
+    o.kill()
+    block = torch.empty((s.W, ps.P_PAD), device="cuda")
+    for t in range(s.recover_at - s.kill_at):
+        block.normal_(0.0, 0.01, generator=gen)
+        block[:, ps.P:] = 0
+        srv.ps_enqueue(list(range(s.W)), [0] * s.W, t, grads_dev=block)
+        o.enqueue(block[:, cols_d].cpu().numpy(), range(s.W), [0] * s.W, t)
+    assert srv.ps_stats()["queue_len"] == K == 25600
+    srv.ps_restore(); o.restore()
+    rg = srv.ps_apply(ps.REPLAY, s.lr, scale=0.25)
+    ro = o.apply(ops.REPLAY, s.lr, scale=0.25)
+    assert rg == ro and rg["applied"] == K
+    th = srv.ps_export_params()[0]
+    step_g = th[cols].astype(np.float64) - theta[cols]
+    step_o = o.head().astype(np.float64) - theta[cols]
+    assert np.abs(step_o).max() > 1e-4
+    assert np.abs(th[cols] - o.head()).max() <= 1e-6 * np.abs(theta).max()
+    assert np.abs(step_g - step_o).max() <= 2e-3 * np.abs(step_o).max()
+    assert (th != theta).mean() > 0.99      # the whole vector moved, not only the sampled columns
+    srv.close()
