@@ -150,8 +150,8 @@ def test_full_size_replay_of_25600_gradients_on_sampled_columns():
         o.enqueue(block[:, cols_d].cpu().numpy(), range(s.W), [0] * s.W, t)
     assert srv.ps_stats()["queue_len"] == K == 25600
     srv.ps_restore(); o.restore()
-    rg = srv.ps_apply(ps.REPLAY, s.lr, scale=0.25)
-    ro = o.apply(ops.REPLAY, s.lr, scale=0.25)
+    rg = srv.ps_apply(ps.REPLAY, s.lr, scale=4.0)
+    ro = o.apply(ops.REPLAY, s.lr, scale=4.0)
     assert rg == ro and rg["applied"] == K
     th = srv.ps_export_params()[0]
     step_g = th[cols].astype(np.float64) - theta[cols]
