@@ -236,6 +236,33 @@ int32_t ps_tick_host(ps_ctx* ctx, int32_t W, int32_t b, const int32_t* lags, con
 int32_t ps_profile(ps_ctx* ctx, int32_t enable);
 int32_t ps_profile_read(ps_ctx* ctx, int32_t kernel, const char** name, double* total_ms, int64_t* launches);
 
+/* Reduce-and-apply without a context and without any allocation.  The paper has no counterpart:
+ * this exists for callers that cannot obtain device memory at the time of the call, for example
+ * code embedded in an application whose own pool already owns all of the GPU's memory, or a loop
+ * that must not stall on the device-wide synchronisation an allocation implies.
+ *
+ *   theta_out = theta_in - coef * (queue[0] + ... + queue[K-1])
+ *
+ * queue_dev: K gradients, row stride PS_PARAM_STRIDE floats; theta_in_dev / theta_out_dev:
+ * PS_PARAM_STRIDE floats each (may be the same buffer); all dev, 16-byte aligned, caller-owned.
+ * 1 <= K <= PS_STATIC_REPLAY_MAX_GRADIENTS, otherwise PS_ERR_BAD_ARG and nothing is launched
+ * (apply a longer queue in several calls, feeding theta_out back in as theta_in).  The work is
+ * enqueued on `stream` (a cudaStream_t, NULL = legacy default stream) of the current device.
+ *
+ * The partial sums are kept in a fixed array inside the library image: PS_STATIC_REPLAY_SPLITS
+ * vectors of PS_PARAM_STRIDE floats, about 13 MB, resident on every GPU that loads the library
+ * for as long as the process lives.  The entry point calls no allocator, CUDA's or anyone
+ * else's.  The first call on each device looks up that array's device address; make that first
+ * call before starting any stream capture.  All calls on a device share the one array and it is
+ * not cleared between calls (each call overwrites every element it later reads), so two calls
+ * whose kernels may overlap on the GPU, e.g. on different streams, race: serialise them.
+ * ps_replay_sum_static_error() returns the text of the calling thread's last failure here. */
+#define PS_STATIC_REPLAY_SPLITS 4
+#define PS_STATIC_REPLAY_MAX_GRADIENTS 65536
+int32_t ps_replay_sum_static(const float* queue_dev, int64_t K, const float* theta_in_dev,
+                             float* theta_out_dev, float coef, void* stream);
+const char* ps_replay_sum_static_error(void);
+
 const char* ps_last_error(ps_ctx* ctx);
 
 #ifdef __cplusplus

@@ -23,7 +23,7 @@ ERRORS = {-1: "PS_ERR_BAD_ARG", -2: "PS_ERR_DOWN", -3: "PS_ERR_QUEUE_FULL", -4: 
 EXPORTS = ["ps_query_bytes", "ps_create", "ps_destroy", "ps_pull_snapshot", "ps_queue_reserve", "ps_slot_ptr",
            "workers_grad_step", "ps_dropout_mask", "ps_enqueue", "ps_apply", "ps_checkpoint", "ps_restore", "ps_replicate",
            "ps_kill", "ps_failover", "ps_import_params", "ps_export_params", "ps_stats", "ps_tick_host",
-           "ps_profile", "ps_profile_read", "ps_last_error"]
+           "ps_profile", "ps_profile_read", "ps_last_error", "ps_replay_sum_static", "ps_replay_sum_static_error"]
 
 
 class PSError(RuntimeError):
@@ -95,11 +95,33 @@ def load(path=None):
         fn = getattr(L, name)
         fn.argtypes = args
         fn.restype = i32
+    L.ps_replay_sum_static.argtypes = [vp, i64, vp, vp, f32, vp]
+    L.ps_replay_sum_static.restype = i32
+    L.ps_replay_sum_static_error.argtypes = []
+    L.ps_replay_sum_static_error.restype = C.c_char_p
     L.ps_last_error.argtypes = [vp]
     L.ps_last_error.restype = C.c_char_p
     if path is None:
         _lib = L
     return L
+
+
+def ps_replay_sum_static(queue_dev, theta_in_dev, theta_out_dev, coef, stream=None):
+    """theta_out = theta_in - coef * sum of the rows of queue_dev, for callers that may not allocate
+    (the scratch is a fixed array inside the library).  queue_dev: float32 cuda tensor [K, P_PAD];
+    theta_in_dev / theta_out_dev: float32 cuda tensors [P_PAD].  Runs on `stream` (torch stream) or
+    torch's current stream.  Marshalling only: nothing is allocated here either."""
+    import torch
+    L = load()
+    K = int(queue_dev.shape[0])
+    for t in (queue_dev, theta_in_dev, theta_out_dev):
+        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+    assert queue_dev.shape[1] == P_PAD and theta_in_dev.numel() == P_PAD and theta_out_dev.numel() == P_PAD
+    st = (stream or torch.cuda.current_stream()).cuda_stream
+    rc = L.ps_replay_sum_static(queue_dev.data_ptr(), K, theta_in_dev.data_ptr(), theta_out_dev.data_ptr(),
+                                float(coef), st)
+    if rc != 0:
+        raise PSError(rc, L.ps_replay_sum_static_error().decode())
 
 
 def _np_ptr(a):
