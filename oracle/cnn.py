@@ -35,13 +35,15 @@ def lib():
         L.oracle_dropout_keep.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_int32, C.c_double, C.c_void_p]
         L.oracle_dropout_keep.restype = None
         L.oracle_grad_step_f64.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
-                                           C.c_double, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+                                           C.c_double, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.oracle_grad_step_f64.restype = C.c_int32
         L.oracle_workers_grad_step.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
-                                               C.c_void_p, C.c_uint64, C.c_uint64, C.c_double,
+                                               C.c_void_p, C.c_uint64, C.c_uint64, C.c_double, C.c_int32,
                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.oracle_workers_grad_step.restype = C.c_int32
         L.oracle_num_threads.restype = C.c_int32
+        L.oracle_round_operand.argtypes = [C.c_double, C.c_int32]
+        L.oracle_round_operand.restype = C.c_double
         assert L.oracle_param_count() == P
         _lib = L
     return _lib
@@ -65,8 +67,9 @@ def dropout_keep(seed, worker, step, b, p):
     return keep.reshape(b, HID)
 
 
-def grad_step_f64(theta, x, y, keep=None, drop_p=0.25):
-    """One worker, everything double.  Returns (grad[P], loss, argmax[b], logits[b,10])."""
+def grad_step_f64(theta, x, y, keep=None, drop_p=0.25, precision=0):
+    """One worker, everything double.  Returns (grad[P], loss, argmax[b], logits[b,10]).
+    precision 1: ReLU/pooling decisions are taken on a TF32-operand forward pass (values stay exact)."""
     theta = np.ascontiguousarray(theta, dtype=np.float64)
     x = np.ascontiguousarray(x, dtype=np.float64)
     y = np.ascontiguousarray(y, dtype=np.int32)
@@ -79,14 +82,14 @@ def grad_step_f64(theta, x, y, keep=None, drop_p=0.25):
     loss = np.zeros(1, dtype=np.float64)
     am = np.zeros(b, dtype=np.int32)
     logits = np.zeros((b, NCLS), dtype=np.float64)
-    rc = lib().oracle_grad_step_f64(_ptr(theta), _ptr(x), _ptr(y), b, _ptr(keep), float(drop_p),
+    rc = lib().oracle_grad_step_f64(_ptr(theta), _ptr(x), _ptr(y), b, _ptr(keep), float(drop_p), int(precision),
                                     _ptr(grad), _ptr(loss), _ptr(am), _ptr(logits))
     if rc != 0:
         raise ValueError("oracle_grad_step_f64: bad argument")
     return grad, float(loss[0]), am, logits
 
 
-def workers_grad_step(thetas, worker_ids, x, y, seed, step, drop_p=0.25):
+def workers_grad_step(thetas, worker_ids, x, y, seed, step, drop_p=0.25, precision=0):
     """W workers with fp32 snapshots.  thetas: list of W float32 arrays [P] (may repeat).
     x [W,b,28,28] float32, y [W,b] int32.  Returns (grads[W,P] f64, loss[W] f64,
     argmax[W,b] i32, logits[W,b,10] f64)."""
@@ -105,11 +108,15 @@ def workers_grad_step(thetas, worker_ids, x, y, seed, step, drop_p=0.25):
     am = np.zeros((W, b), dtype=np.int32)
     logits = np.zeros((W, b, NCLS), dtype=np.float64)
     rc = lib().oracle_workers_grad_step(W, b, C.cast(ptrs, C.c_void_p), _ptr(wid), _ptr(x), _ptr(y),
-                                        int(seed), int(step), float(drop_p), _ptr(grads), _ptr(loss),
+                                        int(seed), int(step), float(drop_p), int(precision), _ptr(grads), _ptr(loss),
                                         _ptr(am), _ptr(logits))
     if rc != 0:
         raise ValueError("oracle_workers_grad_step: bad argument")
     return grads, loss, am, logits
+
+
+def round_operand(v, precision):
+    return float(lib().oracle_round_operand(float(v), int(precision)))
 
 
 def num_threads():

@@ -120,9 +120,10 @@ static void conv3x3(const double* in, int cin, int hw, const double* w, const do
             }
 }
 
-/* ReLU then 2x2/stride-2 max pooling.  `arg` receives, per pooled element, the
- * index 0..3 (row-major inside the window) of the first maximum (strict >). */
-static void relu_pool(const double* a, int c, int hw, double* pooled, int* arg) {
+/* Decisions of "ReLU then 2x2/stride-2 max pooling" on pre-activations a: per pooled element the
+ * index 0..3 (row-major inside the window) of the first maximum of the rectified values (strict >),
+ * or 4 when that maximum is not positive (then no gradient flows through the element). */
+static void pool_decide(const double* a, int c, int hw, int* code) {
     int ho = hw / 2;
     for (int ch = 0; ch < c; ++ch)
         for (int y = 0; y < ho; ++y)
@@ -134,24 +135,63 @@ static void relu_pool(const double* a, int c, int hw, double* pooled, int* arg) 
                     double r = v > 0.0 ? v : 0.0;
                     if (j == 0 || r > best) { best = r; bi = j; }
                 }
-                pooled[(ch * ho + y) * ho + x] = best;
-                arg[(ch * ho + y) * ho + x] = bi;
+                code[(ch * ho + y) * ho + x] = best > 0.0 ? bi : 4;
             }
 }
 
-/* Backward of relu_pool: the pooled gradient goes to the recorded position and
- * passes the ReLU only where the pre-activation was strictly positive. */
-static void relu_pool_bwd(const double* dpooled, const int* arg, const double* a, int c, int hw,
-                          double* da) {
+/* ReLU + max pooling with the decisions given: the pooled value is the pre-activation at the
+ * chosen position, or 0 for a dead element. */
+static void pool_apply(const double* a, const int* code, int c, int hw, double* pooled) {
+    int ho = hw / 2;
+    for (int ch = 0; ch < c; ++ch)
+        for (int y = 0; y < ho; ++y)
+            for (int x = 0; x < ho; ++x) {
+                int j = code[(ch * ho + y) * ho + x];
+                pooled[(ch * ho + y) * ho + x] =
+                    j < 4 ? a[(ch * hw + 2 * y + j / 2) * hw + 2 * x + j % 2] : 0.0;
+            }
+}
+
+/* Backward of pool_apply: the pooled gradient goes to the chosen position of a live element. */
+static void pool_bwd(const double* dpooled, const int* code, int c, int hw, double* da) {
     int ho = hw / 2;
     memset(da, 0, sizeof(double) * (size_t)c * hw * hw);
     for (int ch = 0; ch < c; ++ch)
         for (int y = 0; y < ho; ++y)
             for (int x = 0; x < ho; ++x) {
-                int j = arg[(ch * ho + y) * ho + x];
-                int idx = (ch * hw + 2 * y + j / 2) * hw + 2 * x + j % 2;
-                if (a[idx] > 0.0) da[idx] = dpooled[(ch * ho + y) * ho + x];
+                int j = code[(ch * ho + y) * ho + x];
+                if (j < 4) da[(ch * hw + 2 * y + j / 2) * hw + 2 * x + j % 2] = dpooled[(ch * ho + y) * ho + x];
             }
+}
+
+/* ---- operand rounding of a reduced-precision contraction ----------------------------------
+ * A tensor-core path rounds the operands of its dense contractions (second convolution, 512-unit
+ * layer) to a short mantissa and accumulates exactly enough that the products dominate the error.
+ * ReLU signs and pooling winners are integer decisions taken on those rounded results, so the
+ * oracle must be able to take them in the same precision: precision 1 rounds an fp32 value to
+ * TF32 (10 explicit mantissa bits, round to nearest, ties away from zero). */
+static double round_operand(double v, int precision) {
+    if (precision == 0) return v;
+    float f = (float)v;
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    u = (u + 0x1000u) & 0xFFFFE000u;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
+double oracle_round_operand(double v, int32_t precision) { return round_operand(v, precision); }
+
+/* conv3x3 with both operands rounded (precision 0 = plain conv3x3). */
+static void conv3x3_rounded(const double* in, int cin, int hw, const double* w, const double* bias,
+                            int cout, int precision, double* out) {
+    size_t nin = (size_t)cin * hw * hw, nw = (size_t)cout * cin * 9;
+    double* inr = malloc(sizeof(double) * nin);
+    double* wr = malloc(sizeof(double) * nw);
+    for (size_t i = 0; i < nin; ++i) inr[i] = round_operand(in[i], precision);
+    for (size_t i = 0; i < nw; ++i) wr[i] = round_operand(w[i], precision);
+    conv3x3(inr, cin, hw, wr, bias, cout, out);
+    free(inr); free(wr);
 }
 
 /* Gradient of conv3x3 with respect to weights and bias (accumulated). */
@@ -202,6 +242,11 @@ static void conv3x3_bwd_x(const double* dout, int cout, int hw, const double* w,
  *   y      [b]          labels 0..9
  *   keep   [b][512]     dropout keep mask (1 = keep), or NULL for no dropout
  *   drop_p              dropout rate; kept activations are scaled by 1/(1-p)
+ *   precision           0: every decision (ReLU signs, pooling winners) is taken on the exact
+ *                       double-precision values.  1: the decisions are taken the way a TF32
+ *                       tensor-core path takes them, on a second forward pass whose second
+ *                       convolution and 512-unit layer use TF32-rounded operands (and fp32-stored
+ *                       activations); all VALUES are still the exact double-precision ones.
  * Outputs (any may be NULL except grad):
  *   grad   [P]          d(mean loss)/d(theta)
  *   loss                mean over the batch of logsumexp(z) - z[y]
@@ -210,8 +255,8 @@ static void conv3x3_bwd_x(const double* dout, int cout, int hw, const double* w,
  * Returns 0, or -1 on a bad argument (label out of range, b <= 0).
  */
 int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t* y, int32_t b,
-                             const uint8_t* keep, double drop_p, double* grad, double* loss,
-                             int32_t* argmax, double* logits) {
+                             const uint8_t* keep, double drop_p, int32_t precision, double* grad,
+                             double* loss, int32_t* argmax, double* logits) {
     if (b <= 0 || !theta || !x || !y || !grad) return -1;
     for (int i = 0; i < b; ++i)
         if (y[i] < 0 || y[i] >= NCLS) return -1;
@@ -228,7 +273,10 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
     double* a2 = malloc(sizeof(double) * na2); double* da2 = malloc(sizeof(double) * na2);
     double* p2 = malloc(sizeof(double) * np2); double* dp2 = malloc(sizeof(double) * np2);
     int* i1 = malloc(sizeof(int) * np1); int* i2 = malloc(sizeof(int) * np2);
+    double* p1q = malloc(sizeof(double) * np1); double* a2q = malloc(sizeof(double) * na2);
+    double* p2q = malloc(sizeof(double) * np2);
     double u[HID], d[HID], du[HID], z[NCLS], dz[NCLS];
+    int on[HID];
 
     memset(grad, 0, sizeof(double) * P_TOTAL);
     double loss_sum = 0.0;
@@ -236,14 +284,32 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
         const double* xi = x + (size_t)i * IMG * IMG;
         /* forward */
         conv3x3(xi, 1, IMG, c1w, c1b, C1, a1);
-        relu_pool(a1, C1, IMG, p1, i1);
+        pool_decide(a1, C1, IMG, i1);            /* the first convolution is exact in every path */
+        pool_apply(a1, i1, C1, IMG, p1);
         conv3x3(p1, C1, H1, c2w, c2b, C2, a2);
-        relu_pool(a2, C2, H1, p2, i2); /* p2 is already the channel-major flatten */
+        if (precision == 0) {
+            pool_decide(a2, C2, H1, i2);
+        } else {
+            /* decision pass in the kernel's precision: activations are stored as fp32 there */
+            for (size_t k = 0; k < np1; ++k) p1q[k] = (double)(float)p1[k];
+            conv3x3_rounded(p1q, C1, H1, c2w, c2b, C2, precision, a2q);
+            pool_decide(a2q, C2, H1, i2);
+            pool_apply(a2q, i2, C2, H1, p2q);
+            for (size_t k = 0; k < np2; ++k) p2q[k] = round_operand((double)(float)p2q[k], precision);
+        }
+        pool_apply(a2, i2, C2, H1, p2); /* p2 is already the channel-major flatten */
         for (int j = 0; j < HID; ++j) {
             double s = f1b[j];
             for (int k = 0; k < FLAT; ++k) s += f1w[(size_t)j * FLAT + k] * p2[k];
             u[j] = s;
-            double h = s > 0.0 ? s : 0.0;
+            if (precision == 0) {
+                on[j] = s > 0.0;
+            } else {
+                double sq = f1b[j];
+                for (int k = 0; k < FLAT; ++k) sq += round_operand(f1w[(size_t)j * FLAT + k], precision) * p2q[k];
+                on[j] = sq > 0.0;
+            }
+            double h = on[j] ? s : 0.0;
             int kept = keep ? keep[(size_t)i * HID + j] : 1;
             d[j] = kept ? h * scale : 0.0;
         }
@@ -272,7 +338,7 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
             for (int c = 0; c < NCLS; ++c) s += f2w[c * HID + j] * dz[c];
             int kept = keep ? keep[(size_t)i * HID + j] : 1;
             double dh = kept ? s * scale : 0.0;
-            du[j] = u[j] > 0.0 ? dh : 0.0;
+            du[j] = on[j] ? dh : 0.0;
         }
         memset(dp2, 0, sizeof(double) * np2);
         for (int j = 0; j < HID; ++j) {
@@ -284,15 +350,15 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
                 dp2[k] += g * f1w[(size_t)j * FLAT + k];
             }
         }
-        relu_pool_bwd(dp2, i2, a2, C2, H1, da2);
+        pool_bwd(dp2, i2, C2, H1, da2);
         conv3x3_bwd_w(p1, C1, H1, da2, C2, grad + OFF_C2W, grad + OFF_C2B);
         conv3x3_bwd_x(da2, C2, H1, c2w, C1, dp1);
-        relu_pool_bwd(dp1, i1, a1, C1, IMG, da1);
+        pool_bwd(dp1, i1, C1, IMG, da1);
         conv3x3_bwd_w(xi, 1, IMG, da1, C1, grad + OFF_C1W, grad + OFF_C1B);
     }
     if (loss) *loss = loss_sum / b;
     free(a1); free(da1); free(p1); free(dp1); free(a2); free(da2); free(p2); free(dp2);
-    free(i1); free(i2);
+    free(i1); free(i2); free(p1q); free(a2q); free(p2q);
     return 0;
 }
 
@@ -309,8 +375,8 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
  */
 int32_t oracle_workers_grad_step(int32_t W, int32_t b, const float* const* thetas,
                                  const int32_t* worker_ids, const float* x, const int32_t* y,
-                                 uint64_t seed, uint64_t step, double drop_p, double* grads,
-                                 double* loss, int32_t* argmax, double* logits) {
+                                 uint64_t seed, uint64_t step, double drop_p, int32_t precision,
+                                 double* grads, double* loss, int32_t* argmax, double* logits) {
     if (W <= 0 || b <= 0) return -1;
     int32_t rc = 0;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -325,7 +391,7 @@ int32_t oracle_workers_grad_step(int32_t W, int32_t b, const float* const* theta
             oracle_dropout_keep(seed, (uint32_t)worker_ids[w], step, b, drop_p, keep);
             kp = keep;
         }
-        int32_t r = oracle_grad_step_f64(th, xd, y + (size_t)w * b, b, kp, drop_p,
+        int32_t r = oracle_grad_step_f64(th, xd, y + (size_t)w * b, b, kp, drop_p, precision,
                                          grads + (size_t)w * P_TOTAL, loss ? loss + w : NULL,
                                          argmax ? argmax + (size_t)w * b : NULL,
                                          logits ? logits + (size_t)w * b * NCLS : NULL);

@@ -1,0 +1,50 @@
+// Device helpers shared by the grad-step kernel files.
+#pragma once
+#include "kernels.h"
+
+namespace psk {
+
+// ---- Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplications; the high
+// halves are xored with the neighbouring counter words and the key; the key advances by two Weyl
+// constants per round.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    uint32_t hi0 = __umulhi(M0, c.x), lo0 = M0 * c.x;
+    uint32_t hi1 = __umulhi(M1, c.z), lo1 = M1 * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+    k.x += W0; k.y += W1;
+  }
+  return c;
+}
+
+__device__ __forceinline__ const float* group_theta(const WorkerTable& wt, const GroupTable& gt, int s) {
+  return gt.theta[wt.group[s]];
+}
+
+
+// Maps a tile index to (group, first row of the tile, end row of the group) for TM-row tiles laid
+// out group after group.
+template <int TM>
+__device__ __forceinline__ bool locate_group_tile(const GroupTable& gt, int b, int tile, int& g, int& m0, int& m_end) {
+  for (g = 0; g < gt.n_groups; ++g) {
+    int rows = (gt.first[g + 1] - gt.first[g]) * b;
+    int tiles = (rows + TM - 1) / TM;
+    if (tile < tiles) {
+      m0 = gt.first[g] * b + tile * TM;
+      m_end = gt.first[g + 1] * b;
+      return true;
+    }
+    tile -= tiles;
+  }
+  return false;
+}
+
+inline int group_tiles(const GroupTable& gt, int b, int tm) {
+  int t = 0;
+  for (int g = 0; g < gt.n_groups; ++g) t += ((gt.first[g + 1] - gt.first[g]) * b + tm - 1) / tm;
+  return t;
+}
+
+}  // namespace psk

@@ -8,29 +8,11 @@
 // Every reduction is taken in a fixed order (no floating-point atomics), so that two runs on the
 // same inputs give the same bits.
 #include "kernels.h"
+#include "device_common.cuh"
 
 namespace psk {
 
 namespace {
-
-// ---- Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplications; the high
-// halves are xored with the neighbouring counter words and the key; the key advances by two Weyl
-// constants per round.
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
-  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    uint32_t hi0 = __umulhi(M0, c.x), lo0 = M0 * c.x;
-    uint32_t hi1 = __umulhi(M1, c.z), lo1 = M1 * c.z;
-    c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
-    k.x += W0; k.y += W1;
-  }
-  return c;
-}
-
-__device__ __forceinline__ const float* group_theta(const WorkerTable& wt, const GroupTable& gt, int s) {
-  return gt.theta[wt.group[s]];
-}
 
 // ---- conv1 (1->16, 3x3, pad 1) + ReLU + 2x2 max pool.  One sample per block.
 __global__ void __launch_bounds__(256) conv1_fwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
@@ -193,25 +175,10 @@ __device__ __forceinline__ void gemm_tile_64(const float* __restrict__ A, int ld
   }
 }
 
-// Maps blockIdx.y to (group, first row of the tile, end row of the group) for 64-row tiles.
-__device__ __forceinline__ bool locate_tile(const GroupTable& gt, int b, int tile, int& g, int& m0, int& m_end) {
-  for (g = 0; g < gt.n_groups; ++g) {
-    int rows = (gt.first[g + 1] - gt.first[g]) * b;
-    int tiles = (rows + 63) >> 6;
-    if (tile < tiles) {
-      m0 = gt.first[g] * b + tile * 64;
-      m_end = gt.first[g + 1] * b;
-      return true;
-    }
-    tile -= tiles;
-  }
-  return false;
-}
-
 // ---- fc1 forward: d = dropout(ReLU(p2 * W1^T + b1)), one product per weight group.
 __global__ void __launch_bounds__(256) fc1_fwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   int g, m0, m_end;
-  if (!locate_tile(gt, a.b, blockIdx.y, g, m0, m_end)) return;
+  if (!locate_group_tile<64>(gt, a.b, blockIdx.y, g, m0, m_end)) return;
   const float* theta = gt.theta[g];
   const int n0 = blockIdx.x * 64;
   float acc[4][4];
@@ -368,7 +335,7 @@ __global__ void __launch_bounds__(256) fc1_dw(GradStepArgs a, WorkerTable wt, Wo
 // ---- gradient with respect to p2: dp2 [rows][1568] = da1 [rows][512] * W1 [512][1568], per group.
 __global__ void __launch_bounds__(256) fc1_dx(GradStepArgs a, GroupTable gt, Workspace ws) {
   int g, m0, m_end;
-  if (!locate_tile(gt, a.b, blockIdx.y, g, m0, m_end)) return;
+  if (!locate_group_tile<64>(gt, a.b, blockIdx.y, g, m0, m_end)) return;
   const int n0 = blockIdx.x * 64;
   float acc[4][4];
   gemm_tile_64<true, false>(ws.da1, HID, gt.theta[g] + OFF_F1W, FLAT, m_end, FLAT, HID, m0, n0, acc);
@@ -540,12 +507,6 @@ __global__ void __launch_bounds__(256) dropout_mask(uint64_t seed, uint32_t work
   keep[q] = make_uchar4(r.x >= thresh, r.y >= thresh, r.z >= thresh, r.w >= thresh);
 }
 
-int tiles_64(const GroupTable& gt, int b) {
-  int t = 0;
-  for (int g = 0; g < gt.n_groups; ++g) t += ((gt.first[g + 1] - gt.first[g]) * b + 63) / 64;
-  return t;
-}
-
 }  // namespace
 
 #define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
@@ -567,13 +528,20 @@ int configure_grad_kernels() {
 int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt,
                           const Workspace& ws, cudaStream_t st, Profiler* prof) {
   const int n_chunks = (a.b + CONV_SPB - 1) / CONV_SPB;
-  const int mt = tiles_64(gt, a.b);
+  const int mt = group_tiles(gt, a.b, 64);
   TIMED(K_CONV1_FWD, (conv1_fwd<<<dim3(a.b, a.W), 256, 0, st>>>(a, wt, gt, ws)));
   TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
-  TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
+  const bool tc = a.precision != 0;
+  if (tc) launch_fc1_fwd_tc(a, wt, gt, ws, st, prof);
+  else TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
   TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
-  TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
-  TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
+  if (tc) {
+    launch_fc1_dw_tc(a, wt, ws, st, prof);
+    launch_fc1_dx_tc(a, gt, ws, st, prof);
+  } else {
+    TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
+    TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
+  }
   TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
   TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
   TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks)));

@@ -114,6 +114,7 @@ struct GradStepArgs {
   uint64_t seed, step;
   float drop_p;
   uint32_t drop_thresh;   // keep iff word >= thresh
+  int precision;          // 0 = FP32 CUDA cores, 1 = TF32 tensor cores for the dense contractions
 };
 
 // Part A, FP32 CUDA-core path. Returns the number of kernels launched, or -1 on a launch error.
@@ -121,7 +122,14 @@ int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const Gr
                           const Workspace& ws, cudaStream_t st, Profiler* prof);
 int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, uint32_t thresh,
                         uint8_t* keep, cudaStream_t st, Profiler* prof);
-int configure_grad_kernels();   // one-time function attributes (dynamic shared memory sizes)
+int configure_grad_kernels();
+int configure_tc_kernels();
+void launch_fc1_fwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                       cudaStream_t st, Profiler* prof);
+void launch_fc1_dx_tc(const GradStepArgs& a, const GroupTable& gt, const Workspace& ws, cudaStream_t st,
+                      Profiler* prof);
+void launch_fc1_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st,
+                      Profiler* prof);   // one-time function attributes (dynamic shared memory sizes)
 
 // Part B.
 struct SumApplyArgs {

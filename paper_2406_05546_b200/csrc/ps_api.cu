@@ -108,7 +108,7 @@ int32_t check_cfg(const ps_config* c) {
   if (c->chain_len < 1 || c->chain_len > 8) return fail(PS_ERR_BAD_ARG, "chain_len must be 1..8");
   if (c->replicate_every < 1) return fail(PS_ERR_BAD_ARG, "replicate_every must be >= 1");
   if (c->external_store != 0 && c->external_store != 1) return fail(PS_ERR_BAD_ARG, "external_store must be 0 or 1");
-  if (c->precision != PS_FP32) return fail(PS_ERR_BAD_ARG, "precision %d is not built", c->precision);
+  if (c->precision != PS_FP32 && c->precision != PS_TF32) return fail(PS_ERR_BAD_ARG, "precision %d is not built (PS_FP32 and PS_TF32 are)", c->precision);
   if (!(c->dropout_p >= 0.f) || !(c->dropout_p < 1.f)) return fail(PS_ERR_BAD_ARG, "dropout_p must be in [0,1)");
   if (c->queue_slots < 1) return fail(PS_ERR_BAD_ARG, "queue_slots must be >= 1");
   return PS_OK;
@@ -224,7 +224,7 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
   x->ckpt_version.assign(x->ckpt_buf.size(), 0);
   double t = std::floor((double)cfg->dropout_p * 4294967296.0);
   x->drop_thresh = t <= 0.0 ? 0u : (t >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)t);
-  if (psk::configure_grad_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
+  if (psk::configure_grad_kernels() != 0 || psk::configure_tc_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
   std::memcpy(x->io_stage, init_params_host, sizeof(float) * PS_PARAM_COUNT);
   std::memset(x->io_stage + PS_PARAM_COUNT, 0, sizeof(float) * (PS_PARAM_STRIDE - PS_PARAM_COUNT));
   cudaError_t e = cudaMemcpyAsync(x->ring[0], x->io_stage, VEC_BYTES, cudaMemcpyHostToDevice, x->st);
@@ -314,6 +314,7 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
   psk::GradStepArgs a;
   a.W = W; a.b = b; a.x = x_dev; a.y = y_dev; a.loss = loss_dev; a.argmax = argmax_dev;
   a.seed = seed; a.step = step; a.drop_p = x->cfg.dropout_p; a.drop_thresh = x->drop_thresh;
+  a.precision = x->cfg.precision;
   int n = psk::launch_grad_step_fp32(a, wt, gt, x->ws, x->st, &x->prof);
   if (n < 0) return cuda_fail(cudaGetLastError(), "grad step launch");
   x->launches += n;

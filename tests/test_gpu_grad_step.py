@@ -3,25 +3,27 @@ import numpy as np
 import pytest
 
 from paper_2406_05546_b200 import synth
-from tests.parity import TOL_FP32, assert_argmax_valid, assert_params_close
+from tests.parity import TOL_FP32, TOL_TENSOR, assert_argmax_valid, assert_params_close
 
 pytestmark = pytest.mark.gpu
 
 SEED = 0x5EED
 
 
-def _setup(W, b, n_versions=1, drop_p=0.25):
+def _setup(W, b, n_versions=1, drop_p=0.25, precision=0):
     import torch
     from paper_2406_05546_b200 import ps
     theta0 = synth.init_params(seed=1, bias_scale=0.05)
     srv = ps.ParameterServer(theta0, max_workers=W, max_batch=b, ring_depth=max(1, n_versions),
-                             queue_slots=max(W, n_versions), dropout_p=drop_p)
+                             queue_slots=max(W, n_versions), dropout_p=drop_p, precision=precision)
     return torch, ps, srv, theta0
 
 
-def _run_and_compare(W, b, lags=None, n_versions=1, step=3, drop_p=0.25, worker_ids=None, in_slots=False):
+def _run_and_compare(W, b, lags=None, n_versions=1, step=3, drop_p=0.25, worker_ids=None, in_slots=False,
+                     precision=0):
     from oracle import cnn
-    torch, ps, srv, theta0 = _setup(W, b, n_versions, drop_p)
+    tol = TOL_TENSOR if precision else TOL_FP32
+    torch, ps, srv, theta0 = _setup(W, b, n_versions, drop_p, precision)
     versions = {0: theta0}
     # produce older/newer versions with async applies of random "gradients" so that snapshots differ
     for v in range(1, n_versions):
@@ -48,12 +50,14 @@ def _run_and_compare(W, b, lags=None, n_versions=1, step=3, drop_p=0.25, worker_
         grads = gd.cpu().numpy()
     srv.ps_stats()
     thetas = [versions[s.version] for s in snaps]
-    og, ol, oa, oz = cnn.workers_grad_step(thetas, ids, x, y, SEED, step, drop_p)
+    og, ol, oa, oz = cnn.workers_grad_step(thetas, ids, x, y, SEED, step, drop_p, precision=precision)
     for w in range(W):
-        assert_params_close(grads[w, :ps.P], og[w], TOL_FP32, f"gradient of worker {w}")
+        errs = assert_params_close(grads[w, :ps.P], og[w], tol, f"gradient of worker {w}")
+        if precision and w == 0:
+            print("tensor-path relative errors:", {k: f"{v:.1e}" for k, v in errs.items()})
         assert (grads[w, ps.P:] == 0).all()
-    np.testing.assert_allclose(loss.cpu().numpy(), ol, rtol=1e-5, atol=1e-6)
-    assert_argmax_valid(am.cpu().numpy(), oz, TOL_FP32)
+    np.testing.assert_allclose(loss.cpu().numpy(), ol, rtol=3e-3 if precision else 1e-5, atol=1e-6)
+    assert_argmax_valid(am.cpu().numpy(), oz, tol)
     srv.close()
     return grads
 
@@ -73,6 +77,19 @@ def test_batch_spanning_several_tiles_with_tail():
 def test_stale_snapshots_grouped_over_three_versions():
     # five workers over three distinct weight versions, interleaved so that grouping must reorder
     _run_and_compare(5, 6, lags=[2, 0, 1, 2, 0], n_versions=3)
+
+
+@pytest.mark.parametrize("W,b,kw", [(2, 8, {}), (3, 5, {"worker_ids": [11, 4, 200]}), (2, 150, {}),
+                                     (5, 6, {"lags": [2, 0, 1, 2, 0], "n_versions": 3}), (1, 1, {}),
+                                     (2, 4, {"drop_p": 0.0})])
+def test_tf32_tensor_core_path(W, b, kw):
+    _run_and_compare(W, b, precision=1, **kw)
+
+
+def test_tf32_repeatable_bit_for_bit():
+    a = _run_and_compare(3, 9, precision=1)
+    b = _run_and_compare(3, 9, precision=1)
+    assert (a == b).all()
 
 
 def test_no_dropout():

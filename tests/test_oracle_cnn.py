@@ -148,3 +148,73 @@ def test_workers_entry_uses_philox_mask_and_fp32_inputs():
         keep = cnn.dropout_keep(0x5EED, ids[w], 12, b, 0.25)
         g, l, a, z = cnn.grad_step_f64(thetas[w].astype(np.float64), x[w].astype(np.float64), y[w], keep, 0.25)
         assert (g == grads[w]).all() and l == loss[w] and (a == am[w]).all() and (z == logits[w]).all()
+
+
+# ---- decisions taken in a tensor-core path's precision (precision=1: TF32 operands) -----------------
+
+def _tf32_numpy(a):
+    """Round fp32 values to TF32 (10 mantissa bits, nearest, ties away) with integer arithmetic."""
+    u = np.asarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = ((u + 0x1000) & 0xFFFFE000).astype(np.uint32)
+    return u.view(np.float32).astype(np.float64)
+
+
+def test_operand_rounding_is_tf32_nearest_ties_away():
+    assert cnn.round_operand(1.0, 1) == 1.0 and cnn.round_operand(0.3, 0) == 0.3
+    assert cnn.round_operand(1.0 + 2.0 ** -11, 1) == 1.0 + 2.0 ** -10            # tie goes away from zero
+    assert cnn.round_operand(-(1.0 + 2.0 ** -11), 1) == -(1.0 + 2.0 ** -10)
+    assert cnn.round_operand(1.0 + 2.0 ** -11 - 2.0 ** -23, 1) == 1.0            # just below the tie
+    assert cnn.round_operand(1.0 + 3 * 2.0 ** -12, 1) == 1.0 + 2.0 ** -10
+    vals = np.random.default_rng(0).standard_normal(2000).astype(np.float32) * np.float32(3.0)
+    ref = _tf32_numpy(vals)
+    got = np.array([cnn.round_operand(float(v), 1) for v in vals])
+    assert (got == ref).all()
+    assert np.abs(got - vals).max() <= 2.0 ** -11 * np.abs(vals).max()
+
+
+def test_precision_mode_changes_only_near_kink_decisions():
+    theta, x, y, keep = _case(1, 0)
+    theta = theta.astype(np.float32).astype(np.float64)
+    x = x.astype(np.float32).astype(np.float64)
+    g0 = cnn.grad_step_f64(theta, x, y, keep, 0.25, precision=0)
+    g1 = cnn.grad_step_f64(theta, x, y, keep, 0.25, precision=1)
+    # values are exact in both modes: a flipped decision sits at a pre-activation of ~1e-4, so the
+    # loss hardly moves and all but a few rows of the gradient are untouched
+    assert abs(g0[1] - g1[1]) < 1e-3
+    assert (g0[0] != g1[0]).mean() < 0.05
+
+
+def test_hidden_layer_signs_follow_the_tf32_product():
+    # Put every hidden pre-activation within 1e-6 of zero (exact arithmetic says "on" for all), so
+    # the sign of the TF32-operand product decides; recompute that product independently in numpy.
+    rng = np.random.default_rng(3)
+    theta = synth.init_params(seed=2, bias_scale=0.05).astype(np.float64)
+    x = rng.random((1, 28, 28), dtype=np.float32).astype(np.float64)
+    y = np.array([4], dtype=np.int32)
+    t = torch.tensor(theta)
+    seg = lambda name: t[cnn.TENSORS[name][0]:cnn.TENSORS[name][0] + int(np.prod(cnn.TENSORS[name][1]))].reshape(cnn.TENSORS[name][1])
+    xb = torch.tensor(x).reshape(1, 1, 28, 28)
+    a = F.max_pool2d(F.relu(F.conv2d(xb, seg("conv1.w"), seg("conv1.b"), padding=1)), 2)
+    # second convolution twice: exact, and with fp32-stored input and TF32 operands
+    a2 = F.conv2d(a, seg("conv2.w"), seg("conv2.b"), padding=1)
+    a_q = torch.tensor(_tf32_numpy(a.numpy().astype(np.float32))).reshape(a.shape)
+    w_q = torch.tensor(_tf32_numpy(seg("conv2.w").numpy().astype(np.float32))).reshape(seg("conv2.w").shape)
+    a2q = F.conv2d(a_q, w_q, seg("conv2.b"), padding=1)
+    p2 = F.max_pool2d(F.relu(a2), 2).flatten().numpy()
+    p2q, idx_q = F.max_pool2d(F.relu(a2q), 2, return_indices=True)
+    idx_e = F.max_pool2d(F.relu(a2), 2, return_indices=True)[1]
+    if not bool((idx_q == idx_e).all()) or not bool(((p2q > 0) == (torch.tensor(p2).reshape(p2q.shape) > 0)).all()):
+        pytest.skip("this seed has a conv2 decision inside TF32 rounding distance; the test needs equal pooling")
+    p2q = _tf32_numpy(p2q.flatten().numpy().astype(np.float32))
+    W1 = seg("fc1.w").numpy()
+    u_exact_nobias = W1 @ p2
+    off_b = cnn.TENSORS["fc1.b"][0]
+    theta[off_b:off_b + 512] = -u_exact_nobias + 1e-6          # exact u = +1e-6 for every unit
+    sq = _tf32_numpy(W1.astype(np.float32)) @ p2q + theta[off_b:off_b + 512]
+    assert 100 < (sq > 0).sum() < 412                            # the rounded products scatter both ways
+    g1 = cnn.grad_step_f64(theta, x, y, None, 0.25, precision=1)[0]
+    g0 = cnn.grad_step_f64(theta, x, y, None, 0.25, precision=0)[0]
+    on1 = g1[off_b:off_b + 512] != 0
+    on0 = g0[off_b:off_b + 512] != 0
+    assert on0.all()
+    assert (on1 == (sq > 0)).all()
