@@ -31,6 +31,7 @@ DROP_SEED = 0x5EED
 FLOP_PER_SAMPLE = 10_718_208            # 2 x (1,824,000 forward + 3,535,104 backward multiply-adds)
 GRAD_BYTES = 813258 * 4                 # algorithmic bytes per queued gradient
 N_BATCH_BUFFERS = 8
+REPLAY_TRAFFIC_PER_GRADIENT = 2.654663e9 / 816
 
 
 def measured_peaks():
@@ -159,6 +160,8 @@ def main():
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--precision", default="tf32", choices=["fp32", "tf32"],
+                    help="arithmetic of the dense contractions of the grad step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -197,7 +200,8 @@ def main():
     K_replay = DOWN_TICKS * W
     do_replay = True
     srv = ps.ParameterServer(synth.init_params(1), max_workers=W, max_batch=b, ring_depth=1,
-                             queue_slots=(K_replay if do_replay else 0) + W, external_store=True, dropout_p=0.25)
+                             queue_slots=(K_replay if do_replay else 0) + W, external_store=True, dropout_p=0.25,
+                             precision=ps.TF32 if args.precision == "tf32" else ps.FP32)
     # synthetic stand-in for the 60,000-image training pool, resident in HBM; every rank its own rows
     px, py = synth.image_pool(synth.POOL_IMAGES, seed=0)
     pool_x, pool_y = torch.from_numpy(px).cuda(), torch.from_numpy(py).cuda()
@@ -287,7 +291,10 @@ def main():
         gbs = bytes_alg / (ms * 1e-3) / 1e9
         replay = {"queue_gradients": K_replay, "bytes": bytes_alg, "ms": ms, "gb_per_s": gbs * world,
                   "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                               "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]},
+                               "frac": gbs / peaks["hbm_gbs"],
+                               # dram bytes per queued gradient from the ncu capture of a reduced case
+                               # (2.654663 GB over 816 gradients), scaled to this launch
+                               "traffic": K_replay * REPLAY_TRAFFIC_PER_GRADIENT, "peak_source": peaks["source"]},
                   "all_ms": reps}
     stats = srv.ps_stats()
 
@@ -298,11 +305,17 @@ def main():
         kernels = {k: {"ms_per_launch": ms / n, "launches": n, "share": ms / total_prof}
                    for k, (ms, n) in prof.items() if n}
         top = max(kernels, key=lambda k: kernels[k]["share"])
-        roof = kernel_roofline(top, kernels[top]["ms_per_launch"], W, b, peaks)
+        roof = kernel_roofline(top, kernels[top]["ms_per_launch"], W, b, peaks, args.precision)
+        grad_ms = sum(v["ms_per_launch"] for k, v in kernels.items()
+                      if not k.startswith("sum_") and k not in ("async_apply", "copy_rows"))
+        tensor_flop = 2 * (3 * 903_168 + 3 * 802_816) * W * b
+        grad_step = {"ms": grad_ms, "worker_samples_per_s": W * b / (grad_ms * 1e-3),
+                     "tflops": FLOP_PER_SAMPLE * W * b / (grad_ms * 1e-3) / 1e12,
+                     "tensor_flop_share": tensor_flop / (FLOP_PER_SAMPLE * W * b)}
         out = {
             "metric": "worker-samples/s", "value": value, "unit": "worker-samples/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": args.precision.replace("fp32", "f32"),
             "data": "synthetic",
             "config": {"workload": "config 5 (scale): W=128 workers x batch 128, stateless server, one tick = "
                                    "pull + grad step + enqueue + apply",
@@ -315,6 +328,7 @@ def main():
             "clocks": clocks,
             "roofline": roof,
             "kernels": kernels,
+            "grad_step": grad_step,
             "replay": replay,
             "cpu_baseline": cpu,
             "final_version": stats["version"],
@@ -325,23 +339,31 @@ def main():
         dist.destroy_process_group()
 
 
-def kernel_roofline(name, ms_per_launch, W, b, peaks):
+def kernel_roofline(name, ms_per_launch, W, b, peaks, precision):
     """Algorithmic work of one launch of the named kernel at (W, b) against the roofline that bounds it."""
     n = W * b
     sec = ms_per_launch * 1e-3
     sm_clock_ghz = peaks["sm_max_mhz"] / 1e3
     fp32_peak_tflops = 148 * 128 * 2 * sm_clock_ghz / 1e3        # 148 SMs x 128 FP32 lanes x FMA
+    # dense TF32 peak: the measured sustained bf16 GEMM rate x the nominal tf32/bf16 ratio (1.1 / 2.25 PFLOP/s)
+    tf32_peak_tflops = peaks["bf16_tflops_sustained"] * (1.1 / 2.25)
     flops = {
         "conv1_fwd": 2 * 112_896 * n, "conv2_fwd": 2 * 903_168 * n, "fc1_fwd": 2 * 802_816 * n,
-        "fc1_dw": 2 * 802_816 * n, "fc1_dx": 2 * 802_816 * n, "conv2_bwd": 2 * 2 * 903_168 * n,
+        "fc1_dw": 2 * 802_816 * n, "fc1_dx": 2 * 802_816 * n,
+        "conv2_bwd": 2 * (2 if precision == "fp32" else 1) * 903_168 * n, "conv2_dw": 2 * 903_168 * n,
         "conv1_bwd": 2 * 112_896 * n, "fc2_fwd_bwd": 2 * 3 * 5_120 * n,
     }
+    tensor_kernels = {"conv2_fwd", "fc1_fwd", "fc1_dw", "fc1_dx", "conv2_bwd", "conv2_dw"}
     if name in flops:
         ach = flops[name] / sec / 1e12
+        if precision == "tf32" and name in tensor_kernels:
+            return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": tf32_peak_tflops, "unit": "TFLOP/s",
+                    "frac": ach / tf32_peak_tflops, "traffic": None,
+                    "peak_source": f"{peaks['source']} sustained bf16 GEMM x nominal tf32/bf16 ratio 1.1/2.25"}
         return {"kernel": name, "bound": "alu", "achieved": ach, "peak": fp32_peak_tflops, "unit": "TFLOP/s",
                 "frac": ach / fp32_peak_tflops, "traffic": None,
                 "peak_source": "148 SMs x 128 FP32 lanes x 2 x max SM clock"}
-    bytes_ = {"sum_apply_direct": (W + 2) * GRAD_BYTES, "conv_grad_reduce": 0}.get(name, 0)
+    bytes_ = {"sum_apply_direct": (W + 2) * GRAD_BYTES, "sum_partial": (W + 2) * GRAD_BYTES}.get(name, 0)
     ach = bytes_ / sec / 1e9
     return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"]}

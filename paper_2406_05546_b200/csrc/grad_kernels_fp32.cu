@@ -481,12 +481,12 @@ __global__ void __launch_bounds__(256) conv1_bwd(GradStepArgs a, WorkerTable wt,
 }
 
 // ---- sums the per-block partial convolution gradients in block order and zeroes the padding.
-__global__ void __launch_bounds__(256) conv_grad_reduce(WorkerTable wt, Workspace ws, int n_chunks) {
+__global__ void __launch_bounds__(256) conv_grad_reduce(WorkerTable wt, Workspace ws, int n_chunks, int n_chunks2) {
   const int s = blockIdx.x, tid = threadIdx.x;
   float* grad = wt.grad[s];
   for (int o = tid; o < C2_GRAD; o += 256) {
     float t = 0.f;
-    for (int c = 0; c < n_chunks; ++c) t += ws.part2[((int64_t)s * n_chunks + c) * C2_GRAD + o];
+    for (int c = 0; c < n_chunks2; ++c) t += ws.part2[((int64_t)s * n_chunks2 + c) * C2_GRAD + o];
     grad[OFF_C2W + o] = t;
   }
   for (int o = tid; o < C1_GRAD; o += 256) {
@@ -530,8 +530,9 @@ int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const Gr
   const int n_chunks = (a.b + CONV_SPB - 1) / CONV_SPB;
   const int mt = group_tiles(gt, a.b, 64);
   TIMED(K_CONV1_FWD, (conv1_fwd<<<dim3(a.b, a.W), 256, 0, st>>>(a, wt, gt, ws)));
-  TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
   const bool tc = a.precision != 0;
+  if (tc) launch_conv2_fwd_tc(a, wt, gt, ws, st, prof);
+  else TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
   if (tc) launch_fc1_fwd_tc(a, wt, gt, ws, st, prof);
   else TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
   TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
@@ -542,10 +543,12 @@ int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const Gr
     TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
   }
-  TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
+  int n_chunks2 = n_chunks;
+  if (tc) n_chunks2 = launch_conv2_bwd_tc(a, wt, gt, ws, st, prof);
+  else TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
   TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
-  TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks)));
-  return cudaGetLastError() == cudaSuccess ? 9 : -1;
+  TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks, n_chunks2)));
+  return cudaGetLastError() == cudaSuccess ? (tc ? 10 : 9) : -1;
 }
 
 }  // namespace psk

@@ -239,6 +239,302 @@ __global__ void __launch_bounds__(256) fc1_dw_tc(GradStepArgs a, WorkerTable wt,
   store_tile(acc, wt.grad[s] + OFF_F1W, FLAT, m0, HID, n0, FLAT);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Second convolution (16 -> 32 channels, 3x3, pad 1) as implicit products on 14x14 maps.
+// Every block handles up to TC_SPB samples of one worker and keeps the (TF32-rounded) filter bank
+// in shared memory.  The reduction index is ordered tap-major: k = tap*C + channel, so that one
+// 8-wide k-step covers eight channels at one filter tap and a fragment element is one shared-memory
+// word of a zero-bordered image plane.
+// ------------------------------------------------------------------------------------------------
+constexpr int TC_SPB = 8;
+constexpr int FWD_PLANE = 264;   // 16 x 16 words + 8: plane stride = 8 (mod 32 banks)
+
+__device__ __forceinline__ float tf32f(float x) { return __uint_as_float(to_tf32(x)); }
+
+// Forward + ReLU + 2x2 max pool.  224 threads = 7 warps; warp w owns pooled positions 8w .. 8w+7
+// (49 used of 56).  The product's rows are ordered so that the four pre-pool positions of a pooled
+// element are rows g and g+8 of two 16-row tiles, i.e. they all land in one thread's accumulators and
+// the pooling decision needs no exchange.  Image planes are stored with even and odd columns apart
+// (offset = Y*16 + (X&1)*8 + X/2), which makes the eight positions a fragment load touches consecutive.
+__global__ void __launch_bounds__(224) conv2_fwd_tc(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+  __shared__ float Wk[144 * 40];          // [k = tap*16 + ic][oc], row stride 40
+  __shared__ float bias[32];
+  __shared__ float img[16 * FWD_PLANE];
+  const int s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const float* theta = group_theta(wt, gt, s);
+  for (int idx = tid; idx < 4608; idx += 224) {
+    int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
+    Wk[(tap * 16 + ic) * 40 + oc] = tf32f(theta[OFF_C2W + idx]);
+  }
+  if (tid < 32) bias[tid] = theta[OFF_C2B + tid];
+  for (int idx = tid; idx < 16 * FWD_PLANE; idx += 224) img[idx] = 0.f;
+  const int pp = warp * 8 + g;
+  const bool valid = pp < 49;
+  const int ppc = valid ? pp : 48;
+  const int py = ppc / 7, px = ppc - py * 7;
+  const int base = (2 * py) * 16 + px;
+  const int i0 = blockIdx.x * TC_SPB, i1 = min(i0 + TC_SPB, a.b);
+  for (int i = i0; i < i1; ++i) {
+    const int64_t row = (int64_t)s * a.b + i;
+    __syncthreads();
+    for (int idx = tid; idx < P1_ELEMS; idx += 224) {
+      int ic = idx / 196, p = idx - ic * 196, y = p / 14, x = p - y * 14;
+      int X = x + 1, Y = y + 1;
+      img[ic * FWD_PLANE + Y * 16 + (X & 1) * 8 + (X >> 1)] = tf32f(ws.p1[row * P1_ELEMS + idx]);
+    }
+    __syncthreads();
+    float acc[2][4][4];
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+      for (int n = 0; n < 4; ++n)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) acc[m][n][r] = 0.f;
+#pragma unroll
+    for (int tap = 0; tap < 9; ++tap) {
+      const int ky = tap / 3, kx = tap - ky * 3;
+      int off[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int jy = j >> 1, sx = (j & 1) + kx;
+        off[j] = base + (jy + ky) * 16 + (sx & 1) * 8 + (sx >> 1);
+      }
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const float* pa = img + (half * 8 + t) * FWD_PLANE;
+        const float* pb = pa + 4 * FWD_PLANE;
+        uint32_t fa[2][4], fb[4][2];
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+          fa[m][0] = __float_as_uint(pa[off[2 * m]]);
+          fa[m][1] = __float_as_uint(pa[off[2 * m + 1]]);
+          fa[m][2] = __float_as_uint(pb[off[2 * m]]);
+          fa[m][3] = __float_as_uint(pb[off[2 * m + 1]]);
+        }
+        const float* wk = Wk + (tap * 16 + half * 8 + t) * 40 + g;
+#pragma unroll
+        for (int n = 0; n < 4; ++n) {
+          fb[n][0] = __float_as_uint(wk[n * 8]);
+          fb[n][1] = __float_as_uint(wk[4 * 40 + n * 8]);
+        }
+#pragma unroll
+        for (int m = 0; m < 2; ++m)
+#pragma unroll
+          for (int n = 0; n < 4; ++n) mma_tf32(acc[m][n], fa[m], fb[n]);
+      }
+    }
+    if (valid) {
+#pragma unroll
+      for (int n = 0; n < 4; ++n)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int oc = n * 8 + 2 * t + e;
+          const float bv = bias[oc];
+          // window elements j = 0..3: (tile 0 row g), (tile 0 row g+8), (tile 1 row g), (tile 1 row g+8)
+          const float v[4] = {acc[0][n][e] + bv, acc[0][n][2 + e] + bv, acc[1][n][e] + bv, acc[1][n][2 + e] + bv};
+          float best = 0.f;
+          int bi = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            float r = fmaxf(v[j], 0.f);
+            if (j == 0 || r > best) { best = r; bi = j; }
+          }
+          ws.p2[row * FLAT + oc * 49 + pp] = best;
+          ws.code2[row * FLAT + oc * 49 + pp] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
+        }
+    }
+  }
+}
+
+// Gradient with respect to the convolution's input: dp1[ic][pos] = sum_{tap,oc} g2[oc][pos - tap] * w[oc][ic][tap],
+// rows = 196 positions (13 tiles of 16), 16 columns, k = tap*32 + oc (36 k-steps).  224 threads = 7 warps;
+// warp w owns row tiles w and w+7.  g2 is the gradient at the convolution's output, scattered from the
+// pooled gradient by the stored pooling decisions into zero-bordered 16x16 planes.
+constexpr int DX_PLANE = 264;
+constexpr int DX_SMEM_FLOATS = 288 * 24 + 32 * DX_PLANE;
+__global__ void __launch_bounds__(224) conv2_dx_tc(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+  extern __shared__ __align__(16) float smem[];
+  float* Wk = smem;                 // [k = tap*32 + oc][ic], row stride 24
+  float* g2 = smem + 288 * 24;      // [oc][Y][X]
+  const int s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const float* theta = group_theta(wt, gt, s);
+  for (int idx = tid; idx < 4608; idx += 224) {
+    int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
+    Wk[(tap * 32 + oc) * 24 + ic] = tf32f(theta[OFF_C2W + idx]);
+  }
+  // this warp's two row tiles; positions beyond 195 are computed on clamped addresses and not stored
+  int pos[2][2], offb[2][2];
+  bool ok[2][2];
+#pragma unroll
+  for (int m = 0; m < 2; ++m)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      int p = (warp + 7 * m) * 16 + g + 8 * h;
+      ok[m][h] = p < 196;
+      p = ok[m][h] ? p : 195;
+      pos[m][h] = p;
+      int y = p / 14, x = p - y * 14;
+      offb[m][h] = (y + 2) * 16 + (x + 2);
+    }
+  const bool second = warp + 7 < 13;
+  const int i0 = blockIdx.x * TC_SPB, i1 = min(i0 + TC_SPB, a.b);
+  for (int i = i0; i < i1; ++i) {
+    const int64_t row = (int64_t)s * a.b + i;
+    __syncthreads();
+    for (int idx = tid; idx < 32 * DX_PLANE / 4; idx += 224) reinterpret_cast<float4*>(g2)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncthreads();
+    for (int o = tid; o < FLAT; o += 224) {
+      int code = ws.code2[row * FLAT + o];
+      if (code < 4) {
+        int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
+        int y = 2 * py + (code >> 1), x = 2 * px + (code & 1);
+        g2[oc * DX_PLANE + (y + 1) * 16 + x + 1] = tf32f(ws.dp2[row * FLAT + o]);
+      }
+    }
+    __syncthreads();
+    float acc[2][2][4];
+#pragma unroll
+    for (int m = 0; m < 2; ++m)
+#pragma unroll
+      for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) acc[m][n][r] = 0.f;
+#pragma unroll
+    for (int tap = 0; tap < 9; ++tap) {
+      const int ky = tap / 3, kx = tap - ky * 3;
+      const int shift = ky * 16 + kx;        // g2 is read at (y - ky + 1, x - kx + 1) in bordered coordinates
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float* pa = g2 + (q * 8 + t) * DX_PLANE - shift;
+        const float* pb = pa + 4 * DX_PLANE;
+        uint32_t fa[2][4], fb[2][2];
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+          fa[m][0] = __float_as_uint(pa[offb[m][0]]);
+          fa[m][1] = __float_as_uint(pa[offb[m][1]]);
+          fa[m][2] = __float_as_uint(pb[offb[m][0]]);
+          fa[m][3] = __float_as_uint(pb[offb[m][1]]);
+        }
+        const float* wk = Wk + (tap * 32 + q * 8 + t) * 24 + g;
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+          fb[n][0] = __float_as_uint(wk[n * 8]);
+          fb[n][1] = __float_as_uint(wk[4 * 24 + n * 8]);
+        }
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+          mma_tf32(acc[0][n], fa[0], fb[n]);
+          if (second) mma_tf32(acc[1][n], fa[1], fb[n]);
+        }
+      }
+    }
+#pragma unroll
+    for (int m = 0; m < 2; ++m) {
+      if (m == 1 && !second) continue;
+#pragma unroll
+      for (int n = 0; n < 2; ++n) {
+        const int ic = n * 8 + 2 * t;
+        float* out = ws.dp1 + row * P1_ELEMS;
+        if (ok[m][0]) { out[ic * 196 + pos[m][0]] = acc[m][n][0]; out[(ic + 1) * 196 + pos[m][0]] = acc[m][n][1]; }
+        if (ok[m][1]) { out[ic * 196 + pos[m][1]] = acc[m][n][2]; out[(ic + 1) * 196 + pos[m][1]] = acc[m][n][3]; }
+      }
+    }
+  }
+}
+
+// Filter gradient: dW[oc][ic][tap] = sum_{samples,pos} g2[oc][pos] * p1[ic][pos + tap]: rows = 32 output
+// channels, columns = 16 input channels per tap, k = position (196 per sample, 25 k-steps, zero-padded).
+// 288 threads = 9 warps, warp = filter tap; accumulators persist over the block's samples and are
+// written once as the block's partial sum.  The bias gradient (sum of g2 over positions) is taken by
+// eight threads per channel straight from the pooled gradient, combined in a fixed order.
+constexpr int DW_G_STRIDE = 228;   // 196 positions + zeros; = 4 (mod 32 banks)
+constexpr int DW_PLANE = 260;      // 16 x 16 + 4;            = 4 (mod 32 banks)
+__global__ void __launch_bounds__(288) conv2_dw_tc(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
+  __shared__ __align__(16) float g2[32 * DW_G_STRIDE];   // [oc][pos]
+  __shared__ __align__(16) float img[16 * DW_PLANE];     // [ic][Y][X], zero border
+  const int s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  const int ky = warp / 3, kx = warp - ky * 3;
+  for (int idx = tid; idx < 16 * DW_PLANE; idx += 288) img[idx] = 0.f;
+  float acc[2][2][4];
+#pragma unroll
+  for (int m = 0; m < 2; ++m)
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) acc[m][n][r] = 0.f;
+  float gb = 0.f;
+  const int i0 = blockIdx.x * TC_SPB, i1 = min(i0 + TC_SPB, a.b);
+  for (int i = i0; i < i1; ++i) {
+    const int64_t row = (int64_t)s * a.b + i;
+    __syncthreads();
+    for (int idx = tid; idx < 32 * DW_G_STRIDE / 4; idx += 288) reinterpret_cast<float4*>(g2)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int idx = tid; idx < P1_ELEMS; idx += 288) {
+      int ic = idx / 196, p = idx - ic * 196, y = p / 14, x = p - y * 14;
+      img[ic * DW_PLANE + (y + 1) * 16 + x + 1] = tf32f(ws.p1[row * P1_ELEMS + idx]);
+    }
+    __syncthreads();
+    for (int o = tid; o < FLAT; o += 288) {
+      int code = ws.code2[row * FLAT + o];
+      if (code < 4) {
+        int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
+        int y = 2 * py + (code >> 1), x = 2 * px + (code & 1);
+        g2[oc * DW_G_STRIDE + y * 14 + x] = tf32f(ws.dp2[row * FLAT + o]);
+      }
+    }
+    if (tid < 256) {   // bias gradient: thread (oc, l) adds pooled entries l, l+8, ...; lanes combine in a fixed order
+      const int oc = tid >> 3, l = tid & 7;
+      float sum = 0.f;
+      for (int p = l; p < 49; p += 8) {
+        int o = oc * 49 + p;
+        if (ws.code2[row * FLAT + o] < 4) sum += ws.dp2[row * FLAT + o];
+      }
+      sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      gb += sum;
+    }
+    __syncthreads();
+#pragma unroll 5
+    for (int ks = 0; ks < 25; ++ks) {
+      const int p0 = ks * 8 + t, p1 = p0 + 4;
+      uint32_t fa[2][4], fb[2][2];
+#pragma unroll
+      for (int m = 0; m < 2; ++m) {
+        const float* ga = g2 + (m * 16 + g) * DW_G_STRIDE;
+        fa[m][0] = __float_as_uint(ga[p0]);
+        fa[m][1] = __float_as_uint(ga[8 * DW_G_STRIDE + p0]);
+        fa[m][2] = __float_as_uint(ga[p1]);
+        fa[m][3] = __float_as_uint(ga[8 * DW_G_STRIDE + p1]);
+      }
+      const int q0 = min(p0, 195), q1 = min(p1, 195);
+      const int y0 = q0 / 14, x0 = q0 - y0 * 14, y1 = q1 / 14, x1 = q1 - y1 * 14;
+      const int o0 = (y0 + ky) * 16 + x0 + kx, o1 = (y1 + ky) * 16 + x1 + kx;
+#pragma unroll
+      for (int n = 0; n < 2; ++n) {
+        const float* pi = img + (n * 8 + g) * DW_PLANE;
+        fb[n][0] = __float_as_uint(pi[o0]);
+        fb[n][1] = __float_as_uint(pi[o1]);
+      }
+#pragma unroll
+      for (int m = 0; m < 2; ++m)
+#pragma unroll
+        for (int n = 0; n < 2; ++n) mma_tf32(acc[m][n], fa[m], fb[n]);
+    }
+  }
+  float* part = ws.part2 + ((int64_t)s * n_chunks + blockIdx.x) * C2_GRAD;
+#pragma unroll
+  for (int m = 0; m < 2; ++m)
+#pragma unroll
+    for (int n = 0; n < 2; ++n) {
+      const int oc = m * 16 + g, ic = n * 8 + 2 * t;
+      part[(oc * 16 + ic) * 9 + warp] = acc[m][n][0];
+      part[(oc * 16 + ic + 1) * 9 + warp] = acc[m][n][1];
+      part[((oc + 8) * 16 + ic) * 9 + warp] = acc[m][n][2];
+      part[((oc + 8) * 16 + ic + 1) * 9 + warp] = acc[m][n][3];
+    }
+  if (tid < 256 && (tid & 7) == 0) part[4608 + (tid >> 3)] = gb;
+}
+
 }  // namespace
 
 #define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
@@ -247,6 +543,7 @@ int configure_tc_kernels() {
   cudaError_t e = cudaFuncSetAttribute(fc1_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fc1_dx_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fc1_dw_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(conv2_dx_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, DX_SMEM_FLOATS * 4);
   return e == cudaSuccess ? 0 : -1;
 }
 
@@ -265,6 +562,23 @@ void launch_fc1_dx_tc(const GradStepArgs& a, const GroupTable& gt, const Workspa
 void launch_fc1_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st,
                       Profiler* prof) {
   TIMED(K_FC1_DW, (fc1_dw_tc<<<dim3((FLAT + GN - 1) / GN, HID / GM, a.W), 256, GEMM_SMEM_BYTES, st>>>(a, wt, ws)));
+}
+
+int tc_conv_chunks(int b) { return (b + TC_SPB - 1) / TC_SPB; }
+
+void launch_conv2_fwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                         cudaStream_t st, Profiler* prof) {
+  TIMED(K_CONV2_FWD, (conv2_fwd_tc<<<dim3(tc_conv_chunks(a.b), a.W), 224, 0, st>>>(a, wt, gt, ws)));
+}
+
+// Launches the input-gradient and filter-gradient kernels; returns the number of per-worker partial
+// blocks the filter gradient was split into.
+int launch_conv2_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                        cudaStream_t st, Profiler* prof) {
+  const int chunks = tc_conv_chunks(a.b);
+  TIMED(K_CONV2_BWD, (conv2_dx_tc<<<dim3(chunks, a.W), 224, DX_SMEM_FLOATS * 4, st>>>(a, wt, gt, ws)));
+  TIMED(K_CONV2_DW, (conv2_dw_tc<<<dim3(chunks, a.W), 288, 0, st>>>(a, wt, ws, chunks)));
+  return chunks;
 }
 
 }  // namespace psk

@@ -32,7 +32,7 @@ constexpr uint32_t STATUS_BAD_LABEL = 1u;
 enum KernelId {
   K_CONV1_FWD = 0, K_CONV2_FWD, K_FC1_FWD, K_FC2_FWD_BWD, K_FC1_DW, K_FC1_DX, K_CONV2_BWD, K_CONV1_BWD,
   K_CONV_GRAD_REDUCE, K_SUM_APPLY_DIRECT, K_SUM_PARTIAL, K_SUM_FINISH, K_ASYNC_APPLY, K_COPY_ROWS,
-  K_DROPOUT_MASK, K_COUNT
+  K_DROPOUT_MASK, K_CONV2_DW, K_COUNT
 };
 const char* kernel_name(int id);
 
@@ -128,6 +128,10 @@ void launch_fc1_fwd_tc(const GradStepArgs& a, const WorkerTable& wt, const Group
                        cudaStream_t st, Profiler* prof);
 void launch_fc1_dx_tc(const GradStepArgs& a, const GroupTable& gt, const Workspace& ws, cudaStream_t st,
                       Profiler* prof);
+void launch_conv2_fwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                         cudaStream_t st, Profiler* prof);
+int launch_conv2_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                        cudaStream_t st, Profiler* prof);
 void launch_fc1_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st,
                       Profiler* prof);   // one-time function attributes (dynamic shared memory sizes)
 
