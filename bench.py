@@ -57,7 +57,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -157,7 +157,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--precision", default="tf32", choices=["fp32", "tf32"],
@@ -256,7 +256,7 @@ def main():
     hx = [torch.from_numpy(px[synth.batch_rows(t, W, b, px.shape[0])]).pin_memory() for t in range(2)]
     hy = [torch.from_numpy(py[synth.batch_rows(t, W, b, px.shape[0])]).pin_memory() for t in range(2)]
     loss_host = torch.empty(W, dtype=torch.float32).pin_memory()
-    e2e_steps = max(3, min(args.steps, 20))
+    e2e_steps = max(3, min(args.steps, 50))
     for t in range(3):
         srv.ps_tick_host(hx[t % 2], hy[t % 2], DROP_SEED, 10_000 + t, ps.REPLAY, LR, loss_host=loss_host)
     barrier()

@@ -12,7 +12,7 @@ def make_oracle(s, init_params):
                         external_store=s.external_store)
 
 
-def run(s, o, pool_x, pool_y, on_tick=None, first_tick=0, last_tick=None):
+def run(s, o, pool_x, pool_y, on_tick=None, first_tick=0, last_tick=None, precision=0):
     log = []
     last_tick = s.ticks if last_tick is None else last_tick
     ids = list(range(s.W))
@@ -34,7 +34,8 @@ def run(s, o, pool_x, pool_y, on_tick=None, first_tick=0, last_tick=None):
                 lags = np.minimum(synth.lags(t, s.W, s.max_lag), o.version - o.oldest_version())
             pulled = [o.pull_snapshot(w, int(lags[w])) for w in range(s.W)]
             x, y = synth.tick_batch(pool_x, pool_y, t, s.W, s.b)
-            g, l, am, z = cnn.workers_grad_step([th for _, th in pulled], ids, x, y, s.seed, t, s.dropout_p)
+            g, l, am, z = cnn.workers_grad_step([th for _, th in pulled], ids, x, y, s.seed, t, s.dropout_p,
+                                                 precision=precision)
             o.enqueue(g.astype(np.float32), ids, [v for v, _ in pulled], t)
             loss = (l, am, z)
             if p.apply:

@@ -5,14 +5,14 @@ import pytest
 
 from paper_2406_05546_b200 import schedules, synth
 from tests import oracle_driver
-from tests.parity import TOL_FP32, assert_argmax_valid, assert_params_close
+from tests.parity import TOL_FP32, TOL_TENSOR, assert_argmax_valid, assert_params_close
 
 pytestmark = pytest.mark.gpu
 
 LOCK_FROM = 20
 
 
-def _follow(n, pool=2048):
+def _follow(n, pool=2048, precision=0, lock_from=LOCK_FROM):
     """Runs reduced config n on the GPU and on the oracle, tick by tick.
 
     Integers (versions, queue lengths, events, apply counters) are compared exactly at every tick.
@@ -24,14 +24,15 @@ def _follow(n, pool=2048):
     s = schedules.reduced(n)
     px, py = synth.image_pool(pool, seed=0)
     theta = synth.init_params(1)
-    srv = harness.make_server(s, theta)
+    srv = harness.make_server(s, theta, precision=precision)
     o = oracle_driver.make_oracle(s, theta)
+    tol = TOL_TENSOR if precision else TOL_FP32
     glog, olog = [], []
     for t in range(s.ticks):
-        if t >= LOCK_FROM and o.ring and srv.ps_stats()["up"]:
+        if t >= lock_from and o.ring and srv.ps_stats()["up"]:
             srv.ps_import_params(o.head())
         g = harness.run(s, srv, px, py, first_tick=t, last_tick=t + 1)[0]
-        r = oracle_driver.run(s, o, px, py, first_tick=t, last_tick=t + 1)[0]
+        r = oracle_driver.run(s, o, px, py, first_tick=t, last_tick=t + 1, precision=precision)[0]
         glog.append(g); olog.append(r)
         assert g["version"] == r["version"], t
         assert g["queue_len"] == r["queue_len"], t
@@ -39,10 +40,11 @@ def _follow(n, pool=2048):
         assert g["apply"] == r["apply"], t
         assert (g["loss"] is None) == (r["loss"] is None)
         if g["loss"] is not None:
-            np.testing.assert_allclose(g["loss"][0], r["loss"][0], rtol=2e-4, atol=1e-5, err_msg=f"tick {t}")
-            assert_argmax_valid(g["loss"][1], r["loss"][2], 10 * TOL_FP32)
+            np.testing.assert_allclose(g["loss"][0], r["loss"][0], rtol=5e-3 if precision else 2e-4, atol=1e-5,
+                                       err_msg=f"tick {t}")
+            assert_argmax_valid(g["loss"][1], r["loss"][2], tol if precision else 10 * TOL_FP32)
         if o.ring and g["stats"]["up"]:
-            assert_params_close(srv.ps_export_params()[0], o.head(), TOL_FP32, f"config {n} tick {t}")
+            assert_params_close(srv.ps_export_params()[0], o.head(), tol, f"config {n} tick {t}")
     return s, srv, o, glog, olog
 
 
@@ -84,8 +86,18 @@ def test_config5_stateless_scale_reduced():
     srv.close()
 
 
-def test_full_size_config5_tick_on_sampled_workers():
+@pytest.mark.parametrize("n", [1, 3, 4])
+def test_reduced_configs_on_the_tf32_path(n):
+    # step-locked from the first tick: TF32 rounding separates the two trajectories within a few ticks
+    s, srv, o, glog, _ = _follow(n, precision=1, lock_from=1)
+    assert glog[-1]["version"] == o.version
+    srv.close()
+
+
+@pytest.mark.parametrize("precision", [0, 1])
+def test_full_size_config5_tick_on_sampled_workers(precision):
     """W=128 x b=128 in the launch configuration the benchmark times; the oracle recomputes three workers."""
+    tol = TOL_TENSOR if precision else TOL_FP32
     import torch
     from oracle import cnn
     from oracle import ps as ops
@@ -93,7 +105,7 @@ def test_full_size_config5_tick_on_sampled_workers():
     s = schedules.config(5)
     px, py = synth.image_pool(synth.POOL_IMAGES, seed=0)
     theta = synth.init_params(1)
-    srv = harness.make_server(s, theta, queue_slots=s.W)
+    srv = harness.make_server(s, theta, queue_slots=s.W, precision=precision)
     t = 3
     x, y = synth.tick_batch(px, py, t, s.W, s.b)
     snaps = [srv.ps_pull_snapshot(w) for w in range(s.W)]
@@ -102,13 +114,14 @@ def test_full_size_config5_tick_on_sampled_workers():
                                      s.seed, t, slot_ids=slots)
     loss, am = loss.cpu().numpy(), am.cpu().numpy()
     sample = [0, 77, 127]
-    og, ol, oa, oz = cnn.workers_grad_step([theta] * 3, sample, x[sample], y[sample], s.seed, t, 0.25)
+    og, ol, oa, oz = cnn.workers_grad_step([theta] * 3, sample, x[sample], y[sample], s.seed, t, 0.25,
+                                           precision=precision)
     for j, w in enumerate(sample):
         g = srv.slot_tensor(slots[w]).cpu().numpy()
-        assert_params_close(g[:ps.P], og[j], TOL_FP32, f"worker {w}")
+        assert_params_close(g[:ps.P], og[j], tol, f"worker {w}")
         assert (g[ps.P:] == 0).all()
-        assert abs(loss[w] - ol[j]) <= 1e-5 * abs(ol[j])
-        assert_argmax_valid(am[w], oz[j], TOL_FP32)
+        assert abs(loss[w] - ol[j]) <= (3e-3 if precision else 1e-5) * abs(ol[j])
+        assert_argmax_valid(am[w], oz[j], tol)
     for w in range(s.W):      # every worker wrote a finite, non-trivial gradient
         g = srv.slot_tensor(slots[w])
         assert bool(torch.isfinite(g).all()) and float(g.abs().max()) > 0
