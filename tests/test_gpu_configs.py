@@ -86,9 +86,12 @@ def test_config5_stateless_scale_reduced():
     srv.close()
 
 
-@pytest.mark.parametrize("n", [1, 3, 4])
+@pytest.mark.parametrize("n", [1, 3, 5])
 def test_reduced_configs_on_the_tf32_path(n):
-    # step-locked from the first tick: TF32 rounding separates the two trajectories within a few ticks
+    # step-locked from the first tick: TF32 rounding separates the two trajectories within a few ticks.
+    # (The async config is left to the FP32 run: only the head can be loaded with the oracle's weights,
+    # not the older ring versions its stale readers use; grouped stale snapshots under TF32 are covered
+    # by the grad-step tests, where both sides hold identical versions.)
     s, srv, o, glog, _ = _follow(n, precision=1, lock_from=1)
     assert glog[-1]["version"] == o.version
     srv.close()
