@@ -19,6 +19,13 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
   return c;
 }
 
+// Rounds to TF32 (10-bit mantissa, nearest, ties away from zero); the result is still an fp32 value.
+__device__ __forceinline__ float round_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return __uint_as_float(r);
+}
+
 __device__ __forceinline__ const float* group_theta(const WorkerTable& wt, const GroupTable& gt, int s) {
   return gt.theta[wt.group[s]];
 }

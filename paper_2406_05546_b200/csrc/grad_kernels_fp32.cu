@@ -274,7 +274,9 @@ __global__ void __launch_bounds__(256) fc2_fwd_bwd(GradStepArgs a, WorkerTable w
       float dd = 0.f;
 #pragma unroll
       for (int c = 0; c < NCLS; ++c) dd = fmaf(w2[c][j], dz[c], dd);
-      ws.da1[row * HID + j] = dv[t] > 0.f ? dd * scale : 0.f;
+      float dv1 = dv[t] > 0.f ? dd * scale : 0.f;
+      if (a.precision != 0) dv1 = round_tf32(dv1);   // it feeds tensor-core products only
+      ws.da1[row * HID + j] = dv1;
     }
   }
   if (lane == 0) warp_loss[warp] = loss_acc;
@@ -533,10 +535,16 @@ int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const Gr
   const bool tc = a.precision != 0;
   if (tc) launch_conv2_fwd_tc(a, wt, gt, ws, st, prof);
   else TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
-  if (tc) launch_fc1_fwd_tc(a, wt, gt, ws, st, prof);
+  int extra = 0;
+  const bool tc5 = tc && !a.fc1_legacy;
+  if (tc5) { int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1; }
+  else if (tc) launch_fc1_fwd_tc(a, wt, gt, ws, st, prof);
   else TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
   TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
-  if (tc) {
+  if (tc5) {
+    int n = launch_fc1_dw_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1;
+    n = launch_fc1_dx_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1;
+  } else if (tc) {
     launch_fc1_dw_tc(a, wt, ws, st, prof);
     launch_fc1_dx_tc(a, gt, ws, st, prof);
   } else {
@@ -548,7 +556,7 @@ int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const Gr
   else TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
   TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
   TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks, n_chunks2)));
-  return cudaGetLastError() == cudaSuccess ? (tc ? 10 : 9) : -1;
+  return cudaGetLastError() == cudaSuccess ? (tc ? 10 : 9) + extra : -1;
 }
 
 }  // namespace psk

@@ -339,7 +339,7 @@ __global__ void __launch_bounds__(224) conv2_fwd_tc(GradStepArgs a, WorkerTable 
             float r = fmaxf(v[j], 0.f);
             if (j == 0 || r > best) { best = r; bi = j; }
           }
-          ws.p2[row * FLAT + oc * 49 + pp] = best;
+          ws.p2[row * FLAT + oc * 49 + pp] = tf32f(best);   // its only readers are TF32 products
           ws.code2[row * FLAT + oc * 49 + pp] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
         }
     }

@@ -1,0 +1,361 @@
+// The three products of the 512-unit dense layer on the fifth-generation tensor cores:
+// tcgen05.mma (kind::tf32) issued by one thread, operands brought into 128-byte-swizzled shared
+// memory by TMA (cp.async.bulk.tensor, no multicast), accumulators in tensor memory, read back with
+// tcgen05.ld for the epilogue.
+//
+// All three are "both operands k-contiguous" products C[m][n] = sum_k A[m][k] * B[n][k]:
+//   forward          A = p2 [rows][1568]            B = W1 [512][1568]           (per weight group)
+//   input gradient   A = dA1 [rows][512]            B = W1^T [1568][512]         (per weight group)
+//   weight gradient  A = dA1^T of a worker [512][b] B = p2^T of that worker [1568][b]
+// The transposed copies are made by small kernels below; every operand is rounded to TF32 by its
+// producer, so the tensor core's own handling of the low mantissa bits cannot change a result.
+//
+// Every wait on an mbarrier is bounded: when a bound is exceeded the kernel raises a status flag,
+// stops issuing work, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "device_common.cuh"
+#include "kernels.h"
+
+namespace psk {
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 32;          // CTA tile; BK floats = one 128-byte swizzle row
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 4, B_BYTES = BN * BK * 4, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int TMEM_COLS = 256;
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000ll;   // about one second: no wait here lasts longer when all is well
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase with the given parity; false if the bound was exceeded.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t addr = smem_u32(bar);
+  const long long t0 = clock64();
+  for (;;) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+    if (done) return true;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) return false;
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+// Shared-memory matrix descriptor, k-contiguous operand, 128-byte swizzle: rows are 128 bytes apart,
+// groups of eight rows 1024 bytes apart (stride byte offset), descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)1 << 16;                // leading byte offset (unused for swizzled k-contiguous operands)
+  d |= (uint64_t)(1024 >> 4) << 32;      // stride byte offset
+  d |= (uint64_t)1 << 46;                // version
+  d |= (uint64_t)2 << 61;                // layout type: 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: fp32 accumulate, TF32 x TF32, both operands k-contiguous, tile M x N.
+__host__ __device__ constexpr uint32_t instr_desc_tf32(int m, int n) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Tensor maps of one launch, passed by value in the kernel's parameter space.
+struct GemmMaps {
+  CUtensorMap a;
+  CUtensorMap b[MAX_GROUPS];
+};
+
+enum { EPI_FC1_FWD = 0, EPI_STORE = 1 };
+
+struct GemmArgs {
+  int K;            // reduction length (columns beyond it are zero-filled by TMA)
+  int N;            // valid output columns
+  int ldc;
+  int per_worker;   // 1: blockIdx.z = sorted worker, rows 0..511 of its own output; 0: grouped rows
+  float* c;         // output base when !per_worker
+  int round_out;    // round stored values to TF32 (they feed another tensor-core product)
+};
+
+// 192 threads: warp 0 = TMA producer, warp 1 = tensor-memory owner and MMA issuer, warps 2..5 = epilogue
+// (each reads the 32 accumulator lanes of its quarter, quarter = warp index mod 4).
+template <int EPI>
+__global__ void __launch_bounds__(192) tc5_gemm(const __grid_constant__ GemmMaps maps, GemmArgs ga, GradStepArgs a,
+                                                WorkerTable wt, GroupTable gt, Workspace ws) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + STAGES * STAGE_BYTES);
+  uint64_t* full = bars;                 // [STAGES] TMA -> MMA
+  uint64_t* empty = bars + STAGES;       // [STAGES] MMA -> TMA
+  uint64_t* acc_full = bars + 2 * STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int grp = 0, m0, m_end, z = 0;
+  if (ga.per_worker) {
+    z = blockIdx.z; m0 = blockIdx.y * BM; m_end = HID;
+  } else if (!locate_group_tile<BM>(gt, a.b, blockIdx.y, grp, m0, m_end)) {
+    return;
+  }
+  const int n0 = blockIdx.x * BN;
+  const int n_k = (ga.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_acc = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const CUtensorMap* map_a = &maps.a;
+      const CUtensorMap* map_b = &maps.b[ga.per_worker ? 0 : grp];
+      for (int kb = 0; kb < n_k; ++kb) {
+        const int s = kb % STAGES;
+        if (kb >= STAGES && !mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1)) { *abort_flag = 1; break; }
+        if (*abort_flag) break;
+        mbar_expect_tx(&full[s], STAGE_BYTES);
+        tma_load_3d(tiles + s * STAGE_BYTES, map_a, &full[s], kb * BK, m0, z);
+        tma_load_3d(tiles + s * STAGE_BYTES + A_BYTES, map_b, &full[s], kb * BK, n0, z);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_tf32(BM, BN);
+      bool ok = true;
+      for (int kb = 0; kb < n_k && ok; ++kb) {
+        const int s = kb % STAGES;
+        if (!mbar_wait(&full[s], (kb / STAGES) & 1) || *abort_flag) { *abort_flag = 1; ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = base + s * STAGE_BYTES, b_addr = a_addr + A_BYTES;
+#pragma unroll
+        for (int k = 0; k < BK / 8; ++k) {
+          umma_tf32(tmem_acc, smem_desc_sw128(a_addr + k * 32), smem_desc_sw128(b_addr + k * 32), idesc,
+                    (kb > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(&empty[s]);      // the stage may be refilled once these MMAs have read it
+      }
+      if (ok) umma_commit(acc_full);
+    }
+  } else {
+    const int quarter = warp & 3;
+    const bool ready = mbar_wait(acc_full, 0) && !*abort_flag;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (!ready) {
+      if (lane == 0) { *abort_flag = 1; atomicOr(ws.status, STATUS_WAIT_TIMEOUT); }
+    } else {
+      const int m = m0 + quarter * 32 + lane;
+      const bool row_ok = m < m_end;
+      float* crow;
+      if (ga.per_worker) crow = wt.grad[z] + OFF_F1W + (int64_t)m * ga.ldc;
+      else crow = ga.c + (int64_t)m * ga.ldc;
+      int s_w = 0, smp = 0;
+      if (EPI == EPI_FC1_FWD && row_ok) { s_w = m / a.b; smp = m - s_w * a.b; }
+      const float scale = 1.0f / (1.0f - a.drop_p);
+      const uint2 key = make_uint2((uint32_t)a.seed, (uint32_t)(a.seed >> 32));
+      const float* bias = gt.theta[grp] + OFF_F1B;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        const int n = n0 + c * 32;
+        if (n >= ga.N) break;                    // warp-uniform
+        uint32_t r[32];
+        tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), r);
+        if (!row_ok) continue;
+        if (EPI == EPI_FC1_FWD) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int nq = n + q * 4;
+            uint4 rnd = philox4x32_10(make_uint4((uint32_t)((smp * HID + nq) >> 2), (uint32_t)wt.wid[s_w],
+                                                 (uint32_t)a.step, (uint32_t)(a.step >> 32)), key);
+            const float4 bv = *reinterpret_cast<const float4*>(bias + nq);
+            float4 o;
+            o.x = rnd.x >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 0]) + bv.x, 0.f) * scale : 0.f;
+            o.y = rnd.y >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 1]) + bv.y, 0.f) * scale : 0.f;
+            o.z = rnd.z >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 2]) + bv.z, 0.f) * scale : 0.f;
+            o.w = rnd.w >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 3]) + bv.w, 0.f) * scale : 0.f;
+            *reinterpret_cast<float4*>(crow + nq) = o;
+          }
+        } else {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            float4 o = make_float4(__uint_as_float(r[q * 4]), __uint_as_float(r[q * 4 + 1]),
+                                   __uint_as_float(r[q * 4 + 2]), __uint_as_float(r[q * 4 + 3]));
+            if (ga.round_out) {
+              o.x = round_tf32(o.x); o.y = round_tf32(o.y); o.z = round_tf32(o.z); o.w = round_tf32(o.w);
+            }
+            *reinterpret_cast<float4*>(crow + n + q * 4) = o;
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(TMEM_COLS) : "memory");
+  }
+  if (threadIdx.x == 0 && *abort_flag) {
+    atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
+    // give copies that were already issued time to land in this CTA's shared memory before it is released
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+  }
+}
+
+// ---- operand preparation ----------------------------------------------------------------------
+__device__ __forceinline__ float rna_tf32(float x) { return round_tf32(x); }
+
+// W1 of every weight group: a TF32-rounded copy [512][1568] and its transpose [1568][512].
+__global__ void __launch_bounds__(256) prep_w1(GroupTable gt, float* __restrict__ w1r, float* __restrict__ w1tr) {
+  __shared__ float tile[32][33];
+  const float* src = gt.theta[blockIdx.z] + OFF_F1W;
+  float* dr = w1r + (int64_t)blockIdx.z * HID * FLAT;
+  float* dt = w1tr + (int64_t)blockIdx.z * HID * FLAT;
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;      // c: 0..1567 (49 tiles), r: 0..511 (16 tiles)
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int i = ty; i < 32; i += 8) {
+    float v = rna_tf32(src[(int64_t)(r0 + i) * FLAT + c0 + tx]);
+    dr[(int64_t)(r0 + i) * FLAT + c0 + tx] = v;
+    tile[i][tx] = v;
+  }
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8) dt[(int64_t)(c0 + i) * HID + r0 + tx] = tile[tx][i];
+}
+
+// Per-worker transpose with TF32 rounding: src [W][b][F] -> dst [W][F][bp] (bp = b rounded up to 4).
+__global__ void __launch_bounds__(256) transpose_rows(const float* __restrict__ src, float* __restrict__ dst, int b, int bp, int F) {
+  __shared__ float tile[32][33];
+  const int s = blockIdx.z, f0 = blockIdx.x * 32, i0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const float* sp = src + (int64_t)s * b * F;
+  float* dp = dst + (int64_t)s * F * bp;
+  for (int i = ty; i < 32; i += 8)
+    tile[i][tx] = (i0 + i < b && f0 + tx < F) ? rna_tf32(sp[(int64_t)(i0 + i) * F + f0 + tx]) : 0.f;
+  __syncthreads();
+  for (int i = ty; i < 32; i += 8)
+    if (f0 + i < F && i0 + tx < bp) dp[(int64_t)(f0 + i) * bp + i0 + tx] = tile[tx][i];
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+// fp32 tensor [d2][d1][d0] (d0 contiguous, row pitch pitch1 floats, slab pitch pitch2 floats), box {32, rows, 1}.
+bool make_map(CUtensorMap* m, const float* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch1, uint64_t pitch2,
+              uint32_t box_rows) {
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {pitch1 * 4, pitch2 * 4};
+  cuuint32_t box[3] = {BK, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+#define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
+
+int configure_tc5_kernels() {
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return -1;
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  cudaError_t e = cudaFuncSetAttribute(tc5_gemm<EPI_FC1_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  return e == cudaSuccess ? 0 : -1;
+}
+
+// Rounded / transposed copies of W1 for every weight group of this call, then the forward product.
+int launch_fc1_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                       cudaStream_t st, Profiler* prof) {
+  TIMED(K_PREP_W1, (prep_w1<<<dim3(FLAT / 32, HID / 32, gt.n_groups), 256, 0, st>>>(gt, ws.w1r, ws.w1tr)));
+  GemmMaps maps;
+  const uint64_t rows = (uint64_t)a.W * a.b;
+  if (!make_map(&maps.a, ws.p2, FLAT, rows, 1, FLAT, rows * FLAT, BM)) return -1;
+  for (int g = 0; g < gt.n_groups; ++g)
+    if (!make_map(&maps.b[g], ws.w1r + (int64_t)g * HID * FLAT, FLAT, HID, 1, FLAT, (uint64_t)HID * FLAT, BN)) return -1;
+  GemmArgs ga{FLAT, HID, HID, 0, ws.d, 0};
+  const int mt = group_tiles(gt, a.b, BM);
+  TIMED(K_FC1_FWD, (tc5_gemm<EPI_FC1_FWD><<<dim3(HID / BN, mt, 1), 192, SMEM_BYTES, st>>>(maps, ga, a, wt, gt, ws)));
+  return 2;
+}
+
+int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                      cudaStream_t st, Profiler* prof) {
+  GemmMaps maps;
+  const uint64_t rows = (uint64_t)a.W * a.b;
+  if (!make_map(&maps.a, ws.da1, HID, rows, 1, HID, rows * HID, BM)) return -1;
+  for (int g = 0; g < gt.n_groups; ++g)
+    if (!make_map(&maps.b[g], ws.w1tr + (int64_t)g * HID * FLAT, HID, FLAT, 1, HID, (uint64_t)HID * FLAT, BN)) return -1;
+  GemmArgs ga{HID, FLAT, FLAT, 0, ws.dp2, 0};
+  const int mt = group_tiles(gt, a.b, BM);
+  TIMED(K_FC1_DX, (tc5_gemm<EPI_STORE><<<dim3((FLAT + BN - 1) / BN, mt, 1), 192, SMEM_BYTES, st>>>(maps, ga, a, wt, gt, ws)));
+  return 1;
+}
+
+int launch_fc1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                      cudaStream_t st, Profiler* prof) {
+  const int bp = (a.b + 3) & ~3;
+  TIMED(K_TRANSPOSE, (transpose_rows<<<dim3(HID / 32, (bp + 31) / 32, a.W), 256, 0, st>>>(ws.da1, ws.da1t, a.b, bp, HID)));
+  TIMED(K_TRANSPOSE, (transpose_rows<<<dim3(FLAT / 32, (bp + 31) / 32, a.W), 256, 0, st>>>(ws.p2, ws.p2t, a.b, bp, FLAT)));
+  GemmMaps maps;
+  if (!make_map(&maps.a, ws.da1t, a.b, HID, a.W, bp, (uint64_t)HID * bp, BM)) return -1;
+  if (!make_map(&maps.b[0], ws.p2t, a.b, FLAT, a.W, bp, (uint64_t)FLAT * bp, BN)) return -1;
+  GemmArgs ga{a.b, FLAT, FLAT, 1, nullptr, 0};
+  TIMED(K_FC1_DW, (tc5_gemm<EPI_STORE><<<dim3((FLAT + BN - 1) / BN, HID / BM, a.W), 192, SMEM_BYTES, st>>>(maps, ga, a, wt, gt, ws)));
+  return 3;
+}
+
+}  // namespace psk

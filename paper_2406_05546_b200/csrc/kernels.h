@@ -26,13 +26,14 @@ constexpr int CONV_SPB = 4;              // samples per block in the conv backwa
 constexpr int C2_GRAD = 4608 + 32, C1_GRAD = 144 + 16;
 
 constexpr uint32_t STATUS_BAD_LABEL = 1u;
+constexpr uint32_t STATUS_WAIT_TIMEOUT = 2u;   // a bounded barrier wait in a tensor-core kernel gave up
 
 // Optional per-kernel timing: when switched on, every launch is bracketed by two CUDA events on
 // the launching stream; totals per kernel are read back after a synchronisation.
 enum KernelId {
   K_CONV1_FWD = 0, K_CONV2_FWD, K_FC1_FWD, K_FC2_FWD_BWD, K_FC1_DW, K_FC1_DX, K_CONV2_BWD, K_CONV1_BWD,
   K_CONV_GRAD_REDUCE, K_SUM_APPLY_DIRECT, K_SUM_PARTIAL, K_SUM_FINISH, K_ASYNC_APPLY, K_COPY_ROWS,
-  K_DROPOUT_MASK, K_CONV2_DW, K_COUNT
+  K_DROPOUT_MASK, K_CONV2_DW, K_PREP_W1, K_TRANSPOSE, K_COUNT
 };
 const char* kernel_name(int id);
 
@@ -102,6 +103,10 @@ struct Workspace {
   float* dp1;      // [rows][3136]        gradient w.r.t. p1
   float* part2;    // [W][chunks][4640]   per-block partial conv2 weight/bias gradients
   float* part1;    // [W][chunks][160]    per-block partial conv1 weight/bias gradients
+  float* w1r;      // [groups][512][1568] TF32-rounded fc1 weights of each weight group of the call
+  float* w1tr;     // [groups][1568][512] and their transpose
+  float* da1t;     // [W][512][bp]        per-worker transpose of da1 (bp = batch rounded up to 4)
+  float* p2t;      // [W][1568][bp]       per-worker transpose of p2
   uint32_t* status;
 };
 
@@ -115,6 +120,7 @@ struct GradStepArgs {
   float drop_p;
   uint32_t drop_thresh;   // keep iff word >= thresh
   int precision;          // 0 = FP32 CUDA cores, 1 = TF32 tensor cores for the dense contractions
+  int fc1_legacy;         // 1 = dense-layer products on warp-level mma.sync instead of tcgen05
 };
 
 // Part A, FP32 CUDA-core path. Returns the number of kernels launched, or -1 on a launch error.
@@ -124,6 +130,13 @@ int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, ui
                         uint8_t* keep, cudaStream_t st, Profiler* prof);
 int configure_grad_kernels();
 int configure_tc_kernels();
+int configure_tc5_kernels();
+int launch_fc1_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                       cudaStream_t st, Profiler* prof);
+int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                      cudaStream_t st, Profiler* prof);
+int launch_fc1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                      cudaStream_t st, Profiler* prof);
 void launch_fc1_fwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                        cudaStream_t st, Profiler* prof);
 void launch_fc1_dx_tc(const GradStepArgs& a, const GroupTable& gt, const Workspace& ws, cudaStream_t st,

@@ -136,6 +136,15 @@ void layout(ps_ctx* x, const ps_config& c, void* arena, void* pinned, uint64_t* 
   ws.part2 = a.take<float>((uint64_t)c.max_workers * chunks * psk::C2_GRAD * 4);
   ws.part1 = a.take<float>((uint64_t)c.max_workers * chunks * psk::C1_GRAD * 4);
   ws.status = a.take<uint32_t>(ALIGN);
+  ws.w1r = ws.w1tr = ws.da1t = ws.p2t = nullptr;
+  if (c.precision != PS_FP32) {
+    const uint64_t groups = std::min<uint64_t>(psk::MAX_GROUPS, std::min<uint64_t>(c.max_workers, c.ring_depth));
+    const uint64_t bp = ((uint64_t)c.max_batch + 3) / 4 * 4;
+    ws.w1r = a.take<float>(groups * psk::HID * psk::FLAT * 4);
+    ws.w1tr = a.take<float>(groups * psk::HID * psk::FLAT * 4);
+    ws.da1t = a.take<float>((uint64_t)c.max_workers * psk::HID * bp * 4);
+    ws.p2t = a.take<float>((uint64_t)c.max_workers * psk::FLAT * bp * 4);
+  }
   float* x_stage = a.take<float>(rows * PS_IMAGE_PIXELS * 4);
   int32_t* y_stage = a.take<int32_t>(rows * 4);
   float* loss_stage = a.take<float>((uint64_t)c.max_workers * 4);
@@ -224,7 +233,7 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
   x->ckpt_version.assign(x->ckpt_buf.size(), 0);
   double t = std::floor((double)cfg->dropout_p * 4294967296.0);
   x->drop_thresh = t <= 0.0 ? 0u : (t >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)t);
-  if (psk::configure_grad_kernels() != 0 || psk::configure_tc_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
+  if (psk::configure_grad_kernels() != 0 || psk::configure_tc_kernels() != 0 || psk::configure_tc5_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
   std::memcpy(x->io_stage, init_params_host, sizeof(float) * PS_PARAM_COUNT);
   std::memset(x->io_stage + PS_PARAM_COUNT, 0, sizeof(float) * (PS_PARAM_STRIDE - PS_PARAM_COUNT));
   cudaError_t e = cudaMemcpyAsync(x->ring[0], x->io_stage, VEC_BYTES, cudaMemcpyHostToDevice, x->st);
@@ -315,6 +324,9 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
   a.W = W; a.b = b; a.x = x_dev; a.y = y_dev; a.loss = loss_dev; a.argmax = argmax_dev;
   a.seed = seed; a.step = step; a.drop_p = x->cfg.dropout_p; a.drop_thresh = x->drop_thresh;
   a.precision = x->cfg.precision;
+  a.fc1_legacy = 0;
+  if (a.precision != PS_FP32 && gt.n_groups > std::min(x->cfg.max_workers, x->cfg.ring_depth))
+    return fail(PS_ERR_BAD_ARG, "%d distinct snapshots but the tensor-core workspace holds ring_depth = %d", gt.n_groups, x->cfg.ring_depth);
   int n = psk::launch_grad_step_fp32(a, wt, gt, x->ws, x->st, &x->prof);
   if (n < 0) return cuda_fail(cudaGetLastError(), "grad step launch");
   x->launches += n;
@@ -573,7 +585,7 @@ int32_t ps_stats(ps_ctx* x, ps_stats_t* out) {
   out->replica_version = r ? r->version : 0;
   out->last_ckpt_version = x->ckpt_order.empty() ? 0 : x->ckpt_version[x->ckpt_order.back()];
   out->kernel_launches = x->launches;
-  if (out->device_status != 0) return fail(PS_ERR_DEVICE_STATUS, "device status 0x%x (bit 0: label outside 0..9)", out->device_status);
+  if (out->device_status != 0) return fail(PS_ERR_DEVICE_STATUS, "device status 0x%x (bit 0: label outside 0..9; bit 1: a bounded wait in a tensor-core kernel gave up)", out->device_status);
   return PS_OK;
 }
 
