@@ -1,0 +1,350 @@
+// Second convolution (16 -> 32 channels, 3x3, pad 1, 14x14 maps) on the fifth-generation tensor cores:
+// forward with fused ReLU + 2x2 max pooling, and the gradient with respect to the input.
+//
+// Both are implicit products with k = (filter tap, channel).  The trick that makes them fit
+// tcgen05.mma without an im2col copy: an un-swizzled k-contiguous shared-memory operand is a stack of
+// "core matrices" of 8 rows x 16 bytes, so if the image is stored as planes of FOUR channels
+// (one position = one 16-byte row), then for a fixed filter tap the operand "all positions x 4 channels"
+// is just that plane read from a shifted start address.  One MMA (K = 8) takes two such planes.
+//
+// Forward: rows are POOLED positions and the four pre-pool window elements go to four accumulators
+// (four column ranges of tensor memory), so that a thread of the epilogue holds the whole 2x2 window
+// and pools without exchanging data.  For that the planes keep even and odd columns apart
+// (position (Y, X) at row Y*16 + (X&1)*8 + X/2): consecutive pooled columns are then consecutive rows.
+//
+// Warp roles per CTA (288 threads): warp 0 issues the MMAs and owns tensor memory, warps 1-4 stage the
+// next tile's planes into shared memory, warps 5-8 run the epilogue of the previous tile; the three
+// stages overlap through mbarriers, and every wait is bounded.
+#include "device_common.cuh"
+#include "kernels.h"
+#include "tc5_common.cuh"
+
+namespace psk {
+
+namespace {
+
+constexpr int C5_SPB = 16;            // samples per CTA
+constexpr int THREADS = 288;
+constexpr int LOADERS = 128;
+
+__host__ __device__ constexpr uint32_t idesc_tf32(int m, int n) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// Barrier over the 128 staging threads that also tells every one of them whether any of them failed.
+__device__ __forceinline__ bool loaders_sync_any(bool failed) {
+  uint32_t any;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(any) : "r"((uint32_t)failed) : "memory");
+  return any != 0;
+}
+
+struct Pipe {
+  uint64_t a_full[2], a_empty[2], acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+  volatile uint32_t abort_flag;
+};
+
+__device__ __forceinline__ void pipe_init(Pipe* p) {
+  for (int i = 0; i < 2; ++i) {
+    mbar_init(&p->a_full[i], LOADERS);
+    mbar_init(&p->a_empty[i], 1);
+    mbar_init(&p->acc_full[i], 1);
+    mbar_init(&p->acc_empty[i], 4);
+  }
+  p->abort_flag = 0;
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// Forward.  Tile = two samples = 128 rows: row 8*g + i is pooled position (py = g mod 8, px = i) of
+// sample g / 8 (py = 7 and px = 7 are padding rows whose results are dropped).
+// ------------------------------------------------------------------------------------------------
+constexpr int F_PLANE_ROWS = 2 * 256 + 32;                 // two stacked 16x16 images + overrun of the padding rows
+constexpr int F_PLANE_BYTES = F_PLANE_ROWS * 16;           // 8704
+constexpr int F_BUF_BYTES = 4 * F_PLANE_BYTES;             // four channel quads
+constexpr int F_W_BYTES = 36 * 32 * 16;                    // [k quad = tap*4 + ic/4][oc][4]
+constexpr int F_SMEM = 2 * F_BUF_BYTES + F_W_BYTES + 32 * 4 + sizeof(Pipe) + 128;
+
+__global__ void __launch_bounds__(THREADS) conv2_fwd_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  float* bufs = reinterpret_cast<float*>(smem);
+  float* Wk = reinterpret_cast<float*>(smem + 2 * F_BUF_BYTES);
+  float* bias = reinterpret_cast<float*>(smem + 2 * F_BUF_BYTES + F_W_BYTES);
+  Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * F_BUF_BYTES + F_W_BYTES + 128);
+  const int s = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const float* theta = group_theta(wt, gt, s);
+  const int i_begin = blockIdx.x * C5_SPB, i_end = min(i_begin + C5_SPB, a.b);
+  const int n_tiles = (i_end - i_begin + 1) / 2;
+
+  for (int idx = tid; idx < 4608; idx += THREADS) {
+    int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
+    Wk[((tap * 4 + (ic >> 2)) * 32 + oc) * 4 + (ic & 3)] = round_tf32(theta[OFF_C2W + idx]);
+  }
+  if (tid < 32) bias[tid] = theta[OFF_C2B + tid];
+  for (int idx = tid; idx < 2 * F_BUF_BYTES / 16; idx += THREADS) reinterpret_cast<float4*>(bufs)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (tid == 0) pipe_init(pipe);
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(256) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_proxy_async_smem();      // the zeroed borders and the filter bank are read by the tensor core
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = pipe->tmem_base;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_tf32(128, 32);
+      const uint32_t w_addr = smem_u32(Wk);
+      for (int t = 0; t < n_tiles; ++t) {
+        const int buf = t & 1;
+        if (!mbar_wait(&pipe->a_full[buf], (t >> 1) & 1)) { pipe->abort_flag = 1; break; }
+        if (t >= 2 && !mbar_wait(&pipe->acc_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
+        if (pipe->abort_flag) break;
+        tc_fence_after();
+        const uint32_t a_base = smem_u32(bufs) + buf * F_BUF_BYTES;
+#pragma unroll 1
+        for (int j = 0; j < 4; ++j) {
+          const int jy = j >> 1, jx = j & 1;
+#pragma unroll 1
+          for (int tap = 0; tap < 9; ++tap) {
+            const int ky = tap / 3, kx = tap - ky * 3, sx = jx + kx;
+            const uint32_t row_off = (uint32_t)((jy + ky) * 16 + (sx & 1) * 8 + (sx >> 1)) * 16u;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const uint64_t da = smem_desc_plain(a_base + (2 * half) * F_PLANE_BYTES + row_off, F_PLANE_BYTES, 512);
+              const uint64_t db = smem_desc_plain(w_addr + (tap * 4 + half * 2) * 512, 512, 128);
+              umma_tf32(tmem + buf * 128 + j * 32, da, db, idesc, (tap | half) ? 1u : 0u);
+            }
+          }
+        }
+        umma_commit(&pipe->a_empty[buf]);
+        umma_commit(&pipe->acc_full[buf]);
+      }
+    }
+  } else if (warp <= 4) {
+    const int lt = tid - 32;                 // 0..127
+    for (int t = 0; t < n_tiles; ++t) {
+      const int buf = t & 1;
+      if (t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
+      if (pipe->abort_flag) break;
+      float* dst = bufs + buf * (F_BUF_BYTES / 4);
+#pragma unroll 1
+      for (int sp = 0; sp < 2; ++sp) {
+        const int i = i_begin + 2 * t + sp;
+        if (i >= i_end) break;
+        const float* src = ws.p1 + ((int64_t)s * a.b + i) * P1_ELEMS;
+        for (int e = lt; e < P1_ELEMS; e += LOADERS) {
+          int ic = e / 196, p = e - ic * 196, y = p / 14, x = p - y * 14;
+          int X = x + 1, Y = sp * 16 + y + 1;
+          dst[(ic >> 2) * (F_PLANE_BYTES / 4) + (Y * 16 + (X & 1) * 8 + (X >> 1)) * 4 + (ic & 3)] = round_tf32(src[e]);
+        }
+      }
+      fence_proxy_async_smem();
+      mbar_arrive(&pipe->a_full[buf]);
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane, g = r >> 3, px = r & 7, sp = g >> 3, py = g & 7;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int buf = t & 1;
+      if (!mbar_wait(&pipe->acc_full[buf], (t >> 1) & 1) || pipe->abort_flag) { pipe->abort_flag = 1; break; }
+      tc_fence_after();
+      const int i = i_begin + 2 * t + sp;
+      const bool valid = py < 7 && px < 7 && i < i_end;
+      const int64_t row = (int64_t)s * a.b + i;
+      const int pp = py * 7 + px;
+#pragma unroll 1
+      for (int ch = 0; ch < 2; ++ch) {
+        uint32_t v[4][16];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 128 + j * 32 + ch * 16), v[j]);
+        tmem_ld_wait();
+        if (valid) {
+#pragma unroll
+          for (int o = 0; o < 16; ++o) {
+            const int oc = ch * 16 + o;
+            const float bv = bias[oc];
+            float best = 0.f;
+            int bi = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              float rl = fmaxf(__uint_as_float(v[j][o]) + bv, 0.f);
+              if (j == 0 || rl > best) { best = rl; bi = j; }
+            }
+            ws.p2[row * FLAT + oc * 49 + pp] = round_tf32(best);   // its only readers are TF32 products
+            ws.code2[row * FLAT + oc * 49 + pp] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&pipe->acc_empty[buf]);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+  }
+  if (tid == 0 && pipe->abort_flag) atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Gradient with respect to the convolution's input.  Tile = one sample = two 128-row blocks of the
+// 16-wide position grid (row = y*16 + x; y, x >= 14 are padding rows).  g2, the gradient at the
+// convolution's output, is scattered from the pooled gradient by the stored pooling decisions into
+// zero-bordered planes of four output channels; tap (ky, kx) reads them shifted by (2-ky)*16 + (2-kx) rows.
+// ------------------------------------------------------------------------------------------------
+constexpr int X_PLANE_ROWS = 256 + 48;
+constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // 4864
+constexpr int X_BUF_BYTES = 8 * X_PLANE_BYTES;             // eight output-channel quads
+constexpr int X_W_BYTES = 72 * 16 * 16;                    // [k quad = tap*8 + oc/4][ic][4]
+constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + sizeof(Pipe) + 128;
+
+__global__ void __launch_bounds__(THREADS) conv2_dx_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  float* bufs = reinterpret_cast<float*>(smem);
+  float* Wk = reinterpret_cast<float*>(smem + 2 * X_BUF_BYTES);
+  Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * X_BUF_BYTES + X_W_BYTES);
+  const int s = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const float* theta = group_theta(wt, gt, s);
+  const int i_begin = blockIdx.x * C5_SPB, i_end = min(i_begin + C5_SPB, a.b);
+  const int n_tiles = i_end - i_begin;
+
+  for (int idx = tid; idx < 4608; idx += THREADS) {
+    int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
+    Wk[((tap * 8 + (oc >> 2)) * 16 + ic) * 4 + (oc & 3)] = round_tf32(theta[OFF_C2W + idx]);
+  }
+  for (int idx = tid; idx < 2 * X_BUF_BYTES / 16; idx += THREADS) reinterpret_cast<float4*>(bufs)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (tid == 0) pipe_init(pipe);
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(64) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_proxy_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = pipe->tmem_base;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_tf32(128, 16);
+      const uint32_t w_addr = smem_u32(Wk);
+      for (int t = 0; t < n_tiles; ++t) {
+        const int buf = t & 1;
+        if (!mbar_wait(&pipe->a_full[buf], (t >> 1) & 1)) { pipe->abort_flag = 1; break; }
+        if (t >= 2 && !mbar_wait(&pipe->acc_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
+        if (pipe->abort_flag) break;
+        tc_fence_after();
+        const uint32_t a_base = smem_u32(bufs) + buf * X_BUF_BYTES;
+#pragma unroll 1
+        for (int m = 0; m < 2; ++m) {
+#pragma unroll 1
+          for (int tap = 0; tap < 9; ++tap) {
+            const int ky = tap / 3, kx = tap - ky * 3;
+            const uint32_t row_off = (uint32_t)(m * 128 + (2 - ky) * 16 + (2 - kx)) * 16u;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint64_t da = smem_desc_plain(a_base + (2 * q) * X_PLANE_BYTES + row_off, X_PLANE_BYTES, 128);
+              const uint64_t db = smem_desc_plain(w_addr + (tap * 8 + q * 2) * 256, 256, 128);
+              umma_tf32(tmem + buf * 32 + m * 16, da, db, idesc, (tap | q) ? 1u : 0u);
+            }
+          }
+        }
+        umma_commit(&pipe->a_empty[buf]);
+        umma_commit(&pipe->acc_full[buf]);
+      }
+    }
+  } else if (warp <= 4) {
+    const int lt = tid - 32;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int buf = t & 1;
+      bool failed = false;
+      if (t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) failed = true;
+      // one uniform decision for all staging threads, so that none waits alone at the barrier below
+      if (loaders_sync_any(failed)) { pipe->abort_flag = 1; break; }
+      float* dst = bufs + buf * (X_BUF_BYTES / 4);
+      const int64_t row = (int64_t)s * a.b + i_begin + t;
+      if (t >= 2) {
+        // clear the interior (rows 16 .. 239 hold the 14x14 gradients of the sample staged two tiles ago)
+        for (int idx = lt; idx < 8 * 224; idx += LOADERS) {
+          int q = idx / 224, rr = idx - q * 224;
+          reinterpret_cast<float4*>(dst + q * (X_PLANE_BYTES / 4))[16 + rr] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+      loaders_sync_any(false);
+      for (int o = lt; o < FLAT; o += LOADERS) {
+        int code = ws.code2[row * FLAT + o];
+        if (code < 4) {
+          int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
+          int y = 2 * py + (code >> 1), x = 2 * px + (code & 1);
+          dst[(oc >> 2) * (X_PLANE_BYTES / 4) + ((y + 1) * 16 + x + 1) * 4 + (oc & 3)] = round_tf32(ws.dp2[row * FLAT + o]);
+        }
+      }
+      fence_proxy_async_smem();
+      mbar_arrive(&pipe->a_full[buf]);
+    }
+  } else {
+    const int quarter = warp & 3;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int buf = t & 1;
+      if (!mbar_wait(&pipe->acc_full[buf], (t >> 1) & 1) || pipe->abort_flag) { pipe->abort_flag = 1; break; }
+      tc_fence_after();
+      const int64_t row = (int64_t)s * a.b + i_begin + t;
+#pragma unroll
+      for (int m = 0; m < 2; ++m) {
+        uint32_t v[16];
+        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 32 + m * 16), v);
+        tmem_ld_wait();
+        const int r = m * 128 + quarter * 32 + lane, y = r >> 4, x = r & 15;
+        if (y < 14 && x < 14) {
+          float* out = ws.dp1 + row * P1_ELEMS + y * 14 + x;
+#pragma unroll
+          for (int ic = 0; ic < 16; ++ic) out[ic * 196] = __uint_as_float(v[ic]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&pipe->acc_empty[buf]);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64) : "memory");
+  }
+  if (tid == 0 && pipe->abort_flag) atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
+}
+
+}  // namespace
+
+#define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
+
+int configure_conv5_kernels() {
+  cudaError_t e = cudaFuncSetAttribute(conv2_fwd_tc5, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(conv2_dx_tc5, cudaFuncAttributeMaxDynamicSharedMemorySize, X_SMEM);
+  return e == cudaSuccess ? 0 : -1;
+}
+
+void launch_conv2_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                          cudaStream_t st, Profiler* prof) {
+  const int chunks = (a.b + C5_SPB - 1) / C5_SPB;
+  TIMED(K_CONV2_FWD, (conv2_fwd_tc5<<<dim3(chunks, a.W), THREADS, F_SMEM, st>>>(a, wt, gt, ws)));
+}
+
+void launch_conv2_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                         cudaStream_t st, Profiler* prof) {
+  const int chunks = (a.b + C5_SPB - 1) / C5_SPB;
+  TIMED(K_CONV2_BWD, (conv2_dx_tc5<<<dim3(chunks, a.W), THREADS, X_SMEM, st>>>(a, wt, gt, ws)));
+}
+
+}  // namespace psk

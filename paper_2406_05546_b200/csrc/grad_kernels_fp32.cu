@@ -533,7 +533,9 @@ int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const Gr
   const int mt = group_tiles(gt, a.b, 64);
   TIMED(K_CONV1_FWD, (conv1_fwd<<<dim3(a.b, a.W), 256, 0, st>>>(a, wt, gt, ws)));
   const bool tc = a.precision != 0;
-  if (tc) launch_conv2_fwd_tc(a, wt, gt, ws, st, prof);
+  const bool conv5 = tc && !a.fc1_legacy;
+  if (conv5) launch_conv2_fwd_tc5(a, wt, gt, ws, st, prof);
+  else if (tc) launch_conv2_fwd_tc(a, wt, gt, ws, st, prof);
   else TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
   int extra = 0;
   const bool tc5 = tc && !a.fc1_legacy;
@@ -552,7 +554,8 @@ int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const Gr
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
   }
   int n_chunks2 = n_chunks;
-  if (tc) n_chunks2 = launch_conv2_bwd_tc(a, wt, gt, ws, st, prof);
+  if (conv5) launch_conv2_dx_tc5(a, wt, gt, ws, st, prof);
+  if (tc) n_chunks2 = launch_conv2_bwd_tc(a, wt, gt, ws, st, prof, !conv5);
   else TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
   TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
   TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks, n_chunks2)));

@@ -574,9 +574,9 @@ void launch_conv2_fwd_tc(const GradStepArgs& a, const WorkerTable& wt, const Gro
 // Launches the input-gradient and filter-gradient kernels; returns the number of per-worker partial
 // blocks the filter gradient was split into.
 int launch_conv2_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
-                        cudaStream_t st, Profiler* prof) {
+                        cudaStream_t st, Profiler* prof, bool with_dx) {
   const int chunks = tc_conv_chunks(a.b);
-  TIMED(K_CONV2_BWD, (conv2_dx_tc<<<dim3(chunks, a.W), 224, DX_SMEM_FLOATS * 4, st>>>(a, wt, gt, ws)));
+  if (with_dx) TIMED(K_CONV2_BWD, (conv2_dx_tc<<<dim3(chunks, a.W), 224, DX_SMEM_FLOATS * 4, st>>>(a, wt, gt, ws)));
   TIMED(K_CONV2_DW, (conv2_dw_tc<<<dim3(chunks, a.W), 288, 0, st>>>(a, wt, ws, chunks)));
   return chunks;
 }

@@ -131,6 +131,11 @@ int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, ui
 int configure_grad_kernels();
 int configure_tc_kernels();
 int configure_tc5_kernels();
+int configure_conv5_kernels();
+void launch_conv2_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                          cudaStream_t st, Profiler* prof);
+void launch_conv2_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                         cudaStream_t st, Profiler* prof);
 int launch_fc1_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                        cudaStream_t st, Profiler* prof);
 int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
@@ -144,7 +149,7 @@ void launch_fc1_dx_tc(const GradStepArgs& a, const GroupTable& gt, const Workspa
 void launch_conv2_fwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                          cudaStream_t st, Profiler* prof);
 int launch_conv2_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
-                        cudaStream_t st, Profiler* prof);
+                        cudaStream_t st, Profiler* prof, bool with_dx);
 void launch_fc1_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st,
                       Profiler* prof);   // one-time function attributes (dynamic shared memory sizes)
 
