@@ -68,7 +68,7 @@ constexpr int F_BUF_BYTES = 4 * F_PLANE_BYTES;             // four channel quads
 constexpr int F_W_BYTES = 36 * 32 * 16;                    // [k quad = tap*4 + ic/4][oc][4]
 constexpr int F_SMEM = 2 * F_BUF_BYTES + F_W_BYTES + 32 * 4 + sizeof(Pipe) + 128;
 
-__global__ void __launch_bounds__(THREADS) conv2_fwd_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+__global__ void __launch_bounds__(THREADS, 2) conv2_fwd_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   extern __shared__ __align__(128) uint8_t smem[];
   float* bufs = reinterpret_cast<float*>(smem);
   float* Wk = reinterpret_cast<float*>(smem + 2 * F_BUF_BYTES);
@@ -128,20 +128,35 @@ __global__ void __launch_bounds__(THREADS) conv2_fwd_tc5(GradStepArgs a, WorkerT
     }
   } else if (warp <= 4) {
     const int lt = tid - 32;                 // 0..127
+    constexpr int PER = (P1_ELEMS + LOADERS - 1) / LOADERS;   // 25 elements per thread and sample
     for (int t = 0; t < n_tiles; ++t) {
       const int buf = t & 1;
+      // all global loads of the tile are issued before the wait for the buffer, so that their latency
+      // overlaps the MMAs still reading it
+      float v[2][PER];
+#pragma unroll
+      for (int sp = 0; sp < 2; ++sp) {
+        const int i = min(i_begin + 2 * t + sp, i_end - 1);
+        const float* src = ws.p1 + ((int64_t)s * a.b + i) * P1_ELEMS;
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+          const int e = lt + k * LOADERS;
+          v[sp][k] = e < P1_ELEMS ? __ldg(src + e) : 0.f;
+        }
+      }
       if (t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
       if (pipe->abort_flag) break;
       float* dst = bufs + buf * (F_BUF_BYTES / 4);
-#pragma unroll 1
+#pragma unroll
       for (int sp = 0; sp < 2; ++sp) {
-        const int i = i_begin + 2 * t + sp;
-        if (i >= i_end) break;
-        const float* src = ws.p1 + ((int64_t)s * a.b + i) * P1_ELEMS;
-        for (int e = lt; e < P1_ELEMS; e += LOADERS) {
-          int ic = e / 196, p = e - ic * 196, y = p / 14, x = p - y * 14;
-          int X = x + 1, Y = sp * 16 + y + 1;
-          dst[(ic >> 2) * (F_PLANE_BYTES / 4) + (Y * 16 + (X & 1) * 8 + (X >> 1)) * 4 + (ic & 3)] = round_tf32(src[e]);
+#pragma unroll
+        for (int k = 0; k < PER; ++k) {
+          const int e = lt + k * LOADERS;
+          if (e < P1_ELEMS) {
+            int ic = e / 196, p = e - ic * 196, y = p / 14, x = p - y * 14;
+            int X = x + 1, Y = sp * 16 + y + 1;
+            dst[(ic >> 2) * (F_PLANE_BYTES / 4) + (Y * 16 + (X & 1) * 8 + (X >> 1)) * 4 + (ic & 3)] = round_tf32(v[sp][k]);
+          }
         }
       }
       fence_proxy_async_smem();
@@ -208,7 +223,7 @@ constexpr int X_BUF_BYTES = 8 * X_PLANE_BYTES;             // eight output-chann
 constexpr int X_W_BYTES = 72 * 16 * 16;                    // [k quad = tap*8 + oc/4][ic][4]
 constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + sizeof(Pipe) + 128;
 
-__global__ void __launch_bounds__(THREADS) conv2_dx_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+__global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   extern __shared__ __align__(128) uint8_t smem[];
   float* bufs = reinterpret_cast<float*>(smem);
   float* Wk = reinterpret_cast<float*>(smem + 2 * X_BUF_BYTES);
@@ -265,14 +280,24 @@ __global__ void __launch_bounds__(THREADS) conv2_dx_tc5(GradStepArgs a, WorkerTa
     }
   } else if (warp <= 4) {
     const int lt = tid - 32;
+    constexpr int PER = (FLAT + LOADERS - 1) / LOADERS;      // 13 pooled entries per thread
     for (int t = 0; t < n_tiles; ++t) {
       const int buf = t & 1;
+      const int64_t row = (int64_t)s * a.b + i_begin + t;
+      // decisions and pooled gradients are fetched before the wait for the buffer
+      int code[PER];
+      float gv[PER];
+#pragma unroll
+      for (int k = 0; k < PER; ++k) {
+        const int o = lt + k * LOADERS;
+        code[k] = o < FLAT ? (int)ws.code2[row * FLAT + o] : 4;
+        gv[k] = o < FLAT ? __ldg(ws.dp2 + row * FLAT + o) : 0.f;
+      }
       bool failed = false;
       if (t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) failed = true;
       // one uniform decision for all staging threads, so that none waits alone at the barrier below
       if (loaders_sync_any(failed)) { pipe->abort_flag = 1; break; }
       float* dst = bufs + buf * (X_BUF_BYTES / 4);
-      const int64_t row = (int64_t)s * a.b + i_begin + t;
       if (t >= 2) {
         // clear the interior (rows 16 .. 239 hold the 14x14 gradients of the sample staged two tiles ago)
         for (int idx = lt; idx < 8 * 224; idx += LOADERS) {
@@ -281,12 +306,13 @@ __global__ void __launch_bounds__(THREADS) conv2_dx_tc5(GradStepArgs a, WorkerTa
         }
       }
       loaders_sync_any(false);
-      for (int o = lt; o < FLAT; o += LOADERS) {
-        int code = ws.code2[row * FLAT + o];
-        if (code < 4) {
+#pragma unroll
+      for (int k = 0; k < PER; ++k) {
+        if (code[k] < 4) {
+          const int o = lt + k * LOADERS;
           int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
-          int y = 2 * py + (code >> 1), x = 2 * px + (code & 1);
-          dst[(oc >> 2) * (X_PLANE_BYTES / 4) + ((y + 1) * 16 + x + 1) * 4 + (oc & 3)] = round_tf32(ws.dp2[row * FLAT + o]);
+          int y = 2 * py + (code[k] >> 1), x = 2 * px + (code[k] & 1);
+          dst[(oc >> 2) * (X_PLANE_BYTES / 4) + ((y + 1) * 16 + x + 1) * 4 + (oc & 3)] = round_tf32(gv[k]);
         }
       }
       fence_proxy_async_smem();
