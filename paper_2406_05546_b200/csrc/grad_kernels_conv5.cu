@@ -47,12 +47,12 @@ struct Pipe {
   volatile uint32_t abort_flag;
 };
 
-__device__ __forceinline__ void pipe_init(Pipe* p) {
+__device__ __forceinline__ void pipe_init(Pipe* p, int a_full_arrivals, int acc_empty_arrivals) {
   for (int i = 0; i < 2; ++i) {
-    mbar_init(&p->a_full[i], LOADERS);
+    mbar_init(&p->a_full[i], a_full_arrivals);
     mbar_init(&p->a_empty[i], 1);
     mbar_init(&p->acc_full[i], 1);
-    mbar_init(&p->acc_empty[i], 4);
+    mbar_init(&p->acc_empty[i], acc_empty_arrivals);
   }
   p->abort_flag = 0;
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -60,15 +60,20 @@ __device__ __forceinline__ void pipe_init(Pipe* p) {
 
 // ------------------------------------------------------------------------------------------------
 // Forward.  Tile = two samples = 128 rows: row 8*g + i is pooled position (py = g mod 8, px = i) of
-// sample g / 8 (py = 7 and px = 7 are padding rows whose results are dropped).
+// sample g / 8 (py = 7 and px = 7 are padding rows whose results are dropped).  The first convolution
+// already wrote its output in the plane layout, borders included, so staging a tile is eight plain
+// bulk copies of 4 KB issued by one thread.
+// Warps: 0 = MMA issuer and tensor-memory owner, 1 = copy producer, 2..9 = epilogue (warp w reads the
+// accumulator lanes of quarter w mod 4 and the output channels of half (w-2)/4).
 // ------------------------------------------------------------------------------------------------
+constexpr int F_THREADS = 320;
 constexpr int F_PLANE_ROWS = 2 * 256 + 32;                 // two stacked 16x16 images + overrun of the padding rows
 constexpr int F_PLANE_BYTES = F_PLANE_ROWS * 16;           // 8704
 constexpr int F_BUF_BYTES = 4 * F_PLANE_BYTES;             // four channel quads
 constexpr int F_W_BYTES = 36 * 32 * 16;                    // [k quad = tap*4 + ic/4][oc][4]
 constexpr int F_SMEM = 2 * F_BUF_BYTES + F_W_BYTES + 32 * 4 + sizeof(Pipe) + 128;
 
-__global__ void __launch_bounds__(THREADS, 2) conv2_fwd_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+__global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   extern __shared__ __align__(128) uint8_t smem[];
   float* bufs = reinterpret_cast<float*>(smem);
   float* Wk = reinterpret_cast<float*>(smem + 2 * F_BUF_BYTES);
@@ -79,18 +84,20 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Work
   const int i_begin = blockIdx.x * C5_SPB, i_end = min(i_begin + C5_SPB, a.b);
   const int n_tiles = (i_end - i_begin + 1) / 2;
 
-  for (int idx = tid; idx < 4608; idx += THREADS) {
+  for (int idx = tid; idx < 4608; idx += F_THREADS) {
     int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
     Wk[((tap * 4 + (ic >> 2)) * 32 + oc) * 4 + (ic & 3)] = round_tf32(theta[OFF_C2W + idx]);
   }
   if (tid < 32) bias[tid] = theta[OFF_C2B + tid];
-  for (int idx = tid; idx < 2 * F_BUF_BYTES / 16; idx += THREADS) reinterpret_cast<float4*>(bufs)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (tid == 0) pipe_init(pipe);
+  // rows never written by a copy (the overrun of the padding rows, a missing second sample) only feed
+  // results that are dropped; they are cleared once so that those results stay finite
+  for (int idx = tid; idx < 2 * F_BUF_BYTES / 16; idx += F_THREADS) reinterpret_cast<float4*>(bufs)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (tid == 0) pipe_init(pipe, 1, 8);
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(256) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  fence_proxy_async_smem();      // the zeroed borders and the filter bank are read by the tensor core
+  fence_proxy_async_smem();      // the filter bank and the cleared rows are read by the tensor core
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -126,44 +133,24 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Work
         umma_commit(&pipe->acc_full[buf]);
       }
     }
-  } else if (warp <= 4) {
-    const int lt = tid - 32;                 // 0..127
-    constexpr int PER = (P1_ELEMS + LOADERS - 1) / LOADERS;   // 25 elements per thread and sample
-    for (int t = 0; t < n_tiles; ++t) {
-      const int buf = t & 1;
-      // all global loads of the tile are issued before the wait for the buffer, so that their latency
-      // overlaps the MMAs still reading it
-      float v[2][PER];
+  } else if (warp == 1) {
+    if (lane == 0) {
+      for (int t = 0; t < n_tiles; ++t) {
+        const int buf = t & 1;
+        if (t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
+        if (pipe->abort_flag) break;
+        const int n_s = min(2, i_end - (i_begin + 2 * t));
+        mbar_expect_tx(&pipe->a_full[buf], (uint32_t)n_s * 4 * 4096u);
+        for (int sp = 0; sp < n_s; ++sp) {
+          const float* src = ws.p1 + ((int64_t)s * a.b + i_begin + 2 * t + sp) * P1_PLANE_ELEMS;
 #pragma unroll
-      for (int sp = 0; sp < 2; ++sp) {
-        const int i = min(i_begin + 2 * t + sp, i_end - 1);
-        const float* src = ws.p1 + ((int64_t)s * a.b + i) * P1_ELEMS;
-#pragma unroll
-        for (int k = 0; k < PER; ++k) {
-          const int e = lt + k * LOADERS;
-          v[sp][k] = e < P1_ELEMS ? __ldg(src + e) : 0.f;
+          for (int q = 0; q < 4; ++q)
+            bulk_load(smem + buf * F_BUF_BYTES + q * F_PLANE_BYTES + sp * 4096, src + q * 1024, 4096, &pipe->a_full[buf]);
         }
       }
-      if (t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
-      if (pipe->abort_flag) break;
-      float* dst = bufs + buf * (F_BUF_BYTES / 4);
-#pragma unroll
-      for (int sp = 0; sp < 2; ++sp) {
-#pragma unroll
-        for (int k = 0; k < PER; ++k) {
-          const int e = lt + k * LOADERS;
-          if (e < P1_ELEMS) {
-            int ic = e / 196, p = e - ic * 196, y = p / 14, x = p - y * 14;
-            int X = x + 1, Y = sp * 16 + y + 1;
-            dst[(ic >> 2) * (F_PLANE_BYTES / 4) + (Y * 16 + (X & 1) * 8 + (X >> 1)) * 4 + (ic & 3)] = round_tf32(v[sp][k]);
-          }
-        }
-      }
-      fence_proxy_async_smem();
-      mbar_arrive(&pipe->a_full[buf]);
     }
   } else {
-    const int quarter = warp & 3;
+    const int quarter = warp & 3, ch = (warp - 2) >> 2;
     const int r = quarter * 32 + lane, g = r >> 3, px = r & 7, sp = g >> 3, py = g & 7;
     for (int t = 0; t < n_tiles; ++t) {
       const int buf = t & 1;
@@ -173,33 +160,31 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Work
       const bool valid = py < 7 && px < 7 && i < i_end;
       const int64_t row = (int64_t)s * a.b + i;
       const int pp = py * 7 + px;
-#pragma unroll 1
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t v[4][16];
+      uint32_t v[4][16];
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-          tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 128 + j * 32 + ch * 16), v[j]);
-        tmem_ld_wait();
-        if (valid) {
-#pragma unroll
-          for (int o = 0; o < 16; ++o) {
-            const int oc = ch * 16 + o;
-            const float bv = bias[oc];
-            float best = 0.f;
-            int bi = 0;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              float rl = fmaxf(__uint_as_float(v[j][o]) + bv, 0.f);
-              if (j == 0 || rl > best) { best = rl; bi = j; }
-            }
-            ws.p2[row * FLAT + oc * 49 + pp] = round_tf32(best);   // its only readers are TF32 products
-            ws.code2[row * FLAT + oc * 49 + pp] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
-          }
-        }
-      }
+      for (int j = 0; j < 4; ++j)
+        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 128 + j * 32 + ch * 16), v[j]);
+      tmem_ld_wait();
+      // the accumulators are in registers: hand the buffer back before the pooling arithmetic
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&pipe->acc_empty[buf]);
+      if (valid) {
+#pragma unroll
+        for (int o = 0; o < 16; ++o) {
+          const int oc = ch * 16 + o;
+          const float bv = bias[oc];
+          float best = 0.f;
+          int bi = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            float rl = fmaxf(__uint_as_float(v[j][o]) + bv, 0.f);
+            if (j == 0 || rl > best) { best = rl; bi = j; }
+          }
+          ws.p2[row * FLAT + oc * 49 + pp] = round_tf32(best);   // its only readers are TF32 products
+          ws.code2[row * FLAT + oc * 49 + pp] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
+        }
+      }
     }
   }
   tc_fence_before();
@@ -208,7 +193,10 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Work
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
   }
-  if (tid == 0 && pipe->abort_flag) atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
+  if (tid == 0 && pipe->abort_flag) {
+    atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
+    for (int k = 0; k < 1000; ++k) __nanosleep(1000);   // let copies already issued land before the CTA ends
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -238,7 +226,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
     Wk[((tap * 8 + (oc >> 2)) * 16 + ic) * 4 + (oc & 3)] = round_tf32(theta[OFF_C2W + idx]);
   }
   for (int idx = tid; idx < 2 * X_BUF_BYTES / 16; idx += THREADS) reinterpret_cast<float4*>(bufs)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (tid == 0) pipe_init(pipe);
+  if (tid == 0) pipe_init(pipe, LOADERS, 4);
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(64) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -364,7 +352,7 @@ int configure_conv5_kernels() {
 void launch_conv2_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                           cudaStream_t st, Profiler* prof) {
   const int chunks = (a.b + C5_SPB - 1) / C5_SPB;
-  TIMED(K_CONV2_FWD, (conv2_fwd_tc5<<<dim3(chunks, a.W), THREADS, F_SMEM, st>>>(a, wt, gt, ws)));
+  TIMED(K_CONV2_FWD, (conv2_fwd_tc5<<<dim3(chunks, a.W), F_THREADS, F_SMEM, st>>>(a, wt, gt, ws)));
 }
 
 void launch_conv2_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,

@@ -14,42 +14,89 @@ namespace psk {
 
 namespace {
 
-// ---- conv1 (1->16, 3x3, pad 1) + ReLU + 2x2 max pool.  One sample per block.
-__global__ void __launch_bounds__(256) conv1_fwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
-  __shared__ float xs[30][31];
-  __shared__ float w[160];
-  const int s = blockIdx.y, i = blockIdx.x, tid = threadIdx.x;
-  const int64_t row = (int64_t)s * a.b + i;
+// ---- conv1 (1->16, 3x3, pad 1) + ReLU + 2x2 max pool.  A block handles up to CONV1_SPB samples of one
+// worker.  Thread = pooled position: it reads the 4x4 input patch under its 2x2 window once and
+// evaluates all 16 channels from registers (576 multiply-adds per 8 + 48 shared-memory loads).
+// PLANES selects the output layout: the compact [channel][14*14] rows of the FP32 path, or the layout
+// the tensor-core convolution copies straight into shared memory: per sample four planes of four
+// channels, one 16-byte row per position of a zero-bordered 16x16 grid with even and odd columns apart
+// (row = Y*16 + (X&1)*8 + X/2, Y = y+1, X = x+1), values rounded to TF32.
+constexpr int CONV1_SPB = 8;
+template <bool PLANES>
+__global__ void __launch_bounds__(224) conv1_fwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+  __shared__ __align__(16) float xs[2][30][32];
+  __shared__ __align__(16) float w[16][12];   // 9 taps + bias + padding
+  const int s = blockIdx.y, tid = threadIdx.x;
   const float* theta = group_theta(wt, gt, s);
-  const float* x = a.x + ((int64_t)wt.src[s] * a.b + i) * (IMG * IMG);
-  for (int t = tid; t < 30 * 30; t += 256) {
-    int yy = t / 30, xx = t % 30;
-    bool in = yy >= 1 && yy <= IMG && xx >= 1 && xx <= IMG;
-    xs[yy][xx] = in ? x[(yy - 1) * IMG + (xx - 1)] : 0.f;
+  if (tid < 160) {
+    if (tid < 144) w[tid / 9][tid % 9] = theta[OFF_C1W + tid];
+    else w[tid - 144][9] = theta[OFF_C1B + tid - 144];
   }
-  if (tid < 160) w[tid] = theta[OFF_C1W + tid];
+  for (int t = tid; t < 2 * 30 * 32; t += 224) (&xs[0][0][0])[t] = 0.f;
+  const int i0 = blockIdx.x * CONV1_SPB, i1 = min(i0 + CONV1_SPB, a.b);
+  const int py = tid / 14, px = tid - py * 14;
+  const bool active = tid < 196;
   __syncthreads();
-  for (int o = tid; o < P1_ELEMS; o += 256) {
-    int ch = o / 196, pp = o % 196, py = pp / 14, px = pp % 14;
-    float wv[9];
-#pragma unroll
-    for (int k = 0; k < 9; ++k) wv[k] = w[ch * 9 + k];
-    float bias = w[144 + ch];
-    float best = 0.f;
-    int bi = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      int yy = 2 * py + (j >> 1), xx = 2 * px + (j & 1);
-      float v = bias;
-#pragma unroll
-      for (int ky = 0; ky < 3; ++ky)
-#pragma unroll
-        for (int kx = 0; kx < 3; ++kx) v = fmaf(wv[ky * 3 + kx], xs[yy + ky][xx + kx], v);
-      float r = fmaxf(v, 0.f);
-      if (j == 0 || r > best) { best = r; bi = j; }
+  auto stage = [&](int i, int bufi) {
+    const float* x = a.x + ((int64_t)wt.src[s] * a.b + i) * (IMG * IMG);
+    for (int t = tid; t < IMG * IMG; t += 224) {
+      int yy = t / IMG, xx = t - yy * IMG;
+      xs[bufi][yy + 1][xx + 1] = x[t];
     }
-    ws.p1[row * P1_ELEMS + o] = best;
-    ws.code1[row * P1_ELEMS + o] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
+  };
+  stage(i0, 0);
+  for (int i = i0; i < i1; ++i) {
+    const int cur = (i - i0) & 1;
+    __syncthreads();                       // image `cur` is complete; image `cur^1` is no longer read
+    if (i + 1 < i1) stage(i + 1, cur ^ 1);
+    if (!active) continue;
+    const int64_t row = (int64_t)s * a.b + i;
+    float patch[4][4];
+#pragma unroll
+    for (int yy = 0; yy < 4; ++yy) {
+      float2 lo = *reinterpret_cast<const float2*>(&xs[cur][2 * py + yy][2 * px]);
+      float2 hi = *reinterpret_cast<const float2*>(&xs[cur][2 * py + yy][2 * px + 2]);
+      patch[yy][0] = lo.x; patch[yy][1] = lo.y; patch[yy][2] = hi.x; patch[yy][3] = hi.y;
+    }
+    float outv[16];
+    uint8_t outc[16];
+#pragma unroll
+    for (int ch = 0; ch < 16; ++ch) {
+      const float4 w0 = *reinterpret_cast<const float4*>(&w[ch][0]);
+      const float4 w1 = *reinterpret_cast<const float4*>(&w[ch][4]);
+      const float4 w2 = *reinterpret_cast<const float4*>(&w[ch][8]);
+      const float wv[9] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w, w2.x};
+      const float bias = w2.y;
+      float best = 0.f;
+      int bi = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int jy = j >> 1, jx = j & 1;
+        float v = bias;
+#pragma unroll
+        for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+          for (int kx = 0; kx < 3; ++kx) v = fmaf(wv[ky * 3 + kx], patch[jy + ky][jx + kx], v);
+        float r = fmaxf(v, 0.f);
+        if (j == 0 || r > best) { best = r; bi = j; }
+      }
+      outv[ch] = best;
+      outc[ch] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
+    }
+    const int pp = tid;
+#pragma unroll
+    for (int ch = 0; ch < 16; ++ch) ws.code1[row * P1_ELEMS + ch * 196 + pp] = outc[ch];
+    if (PLANES) {
+      const int X = px + 1, Y = py + 1;
+      float* dst = ws.p1 + row * P1_PLANE_ELEMS + (Y * 16 + (X & 1) * 8 + (X >> 1)) * 4;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<float4*>(dst + q * 1024) = make_float4(round_tf32(outv[4 * q]), round_tf32(outv[4 * q + 1]),
+                                                                  round_tf32(outv[4 * q + 2]), round_tf32(outv[4 * q + 3]));
+    } else {
+#pragma unroll
+      for (int ch = 0; ch < 16; ++ch) ws.p1[row * P1_ELEMS + ch * 196 + pp] = outv[ch];
+    }
   }
 }
 
@@ -531,31 +578,28 @@ int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const Gr
                           const Workspace& ws, cudaStream_t st, Profiler* prof) {
   const int n_chunks = (a.b + CONV_SPB - 1) / CONV_SPB;
   const int mt = group_tiles(gt, a.b, 64);
-  TIMED(K_CONV1_FWD, (conv1_fwd<<<dim3(a.b, a.W), 256, 0, st>>>(a, wt, gt, ws)));
   const bool tc = a.precision != 0;
-  const bool conv5 = tc && !a.fc1_legacy;
-  if (conv5) launch_conv2_fwd_tc5(a, wt, gt, ws, st, prof);
-  else if (tc) launch_conv2_fwd_tc(a, wt, gt, ws, st, prof);
+  const int n_chunks1 = (a.b + CONV1_SPB - 1) / CONV1_SPB;
+  if (tc) TIMED(K_CONV1_FWD, (conv1_fwd<true><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
+  else TIMED(K_CONV1_FWD, (conv1_fwd<false><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
+  if (tc) launch_conv2_fwd_tc5(a, wt, gt, ws, st, prof);
   else TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
   int extra = 0;
-  const bool tc5 = tc && !a.fc1_legacy;
-  if (tc5) { int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1; }
-  else if (tc) launch_fc1_fwd_tc(a, wt, gt, ws, st, prof);
+  if (tc) { int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1; }
   else TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
   TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
-  if (tc5) {
+  if (tc) {
     int n = launch_fc1_dw_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1;
     n = launch_fc1_dx_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1;
-  } else if (tc) {
-    launch_fc1_dw_tc(a, wt, ws, st, prof);
-    launch_fc1_dx_tc(a, gt, ws, st, prof);
   } else {
     TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
   }
   int n_chunks2 = n_chunks;
-  if (conv5) launch_conv2_dx_tc5(a, wt, gt, ws, st, prof);
-  if (tc) n_chunks2 = launch_conv2_bwd_tc(a, wt, gt, ws, st, prof, !conv5);
+  if (tc) {
+    launch_conv2_dx_tc5(a, wt, gt, ws, st, prof);
+    n_chunks2 = launch_conv2_dw_tc(a, wt, ws, st, prof);
+  }
   else TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
   TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
   TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks, n_chunks2)));

@@ -19,6 +19,7 @@ constexpr int OFF_F1W = 4800, OFF_F1B = 807616, OFF_F2W = 808128, OFF_F2B = 8132
 
 constexpr int IMG = 28, C1 = 16, H1 = 14, C2 = 32, H2 = 7;
 constexpr int P1_ELEMS = C1 * H1 * H1;   // 3136
+constexpr int P1_PLANE_ELEMS = 4 * 256 * 4;   // 4096: p1 of one sample in the tensor-core plane layout
 constexpr int FLAT = C2 * H2 * H2;       // 1568
 constexpr int HID = 512, NCLS = 10;
 constexpr int DZ_STRIDE = 16;            // logits gradient row, padded
@@ -92,7 +93,7 @@ struct GroupTable {
 
 // Activation workspace carved from the arena (rows = sorted worker * b + sample).
 struct Workspace {
-  float* p1;       // [rows][16][14][14]  conv1 -> ReLU -> pool
+  float* p1;       // conv1 -> ReLU -> pool: [rows][16][14][14] (FP32 path) or [rows][4 planes][256][4] (tensor-core path)
   uint8_t* code1;  // [rows][3136]        pool-1 argmax 0..3, 4 = no gradient (max <= 0)
   float* p2;       // [rows][1568]        conv2 -> ReLU -> pool, channel-major flatten
   uint8_t* code2;  // [rows][1568]
@@ -120,7 +121,6 @@ struct GradStepArgs {
   float drop_p;
   uint32_t drop_thresh;   // keep iff word >= thresh
   int precision;          // 0 = FP32 CUDA cores, 1 = TF32 tensor cores for the dense contractions
-  int fc1_legacy;         // 1 = dense-layer products on warp-level mma.sync instead of tcgen05
 };
 
 // Part A, FP32 CUDA-core path. Returns the number of kernels launched, or -1 on a launch error.
@@ -130,6 +130,7 @@ int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, ui
                         uint8_t* keep, cudaStream_t st, Profiler* prof);
 int configure_grad_kernels();
 int configure_tc_kernels();
+int launch_conv2_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof);
 int configure_tc5_kernels();
 int configure_conv5_kernels();
 void launch_conv2_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,

@@ -124,7 +124,8 @@ void layout(ps_ctx* x, const ps_config& c, void* arena, void* pinned, uint64_t* 
   float* partial = a.take<float>(VEC_BYTES * MAX_SPLIT);
   float* queue = a.take<float>(VEC_BYTES * (uint64_t)c.queue_slots);
   psk::Workspace ws;
-  ws.p1 = a.take<float>(rows * psk::P1_ELEMS * 4);
+  const uint64_t p1_elems = c.precision != PS_FP32 ? psk::P1_PLANE_ELEMS : psk::P1_ELEMS;
+  ws.p1 = a.take<float>(rows * p1_elems * 4);
   ws.code1 = a.take<uint8_t>(rows * psk::P1_ELEMS);
   ws.p2 = a.take<float>(rows * psk::FLAT * 4);
   ws.code2 = a.take<uint8_t>(rows * psk::FLAT);
@@ -240,6 +241,9 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
   for (auto& r : x->replicas)
     if (e == cudaSuccess) e = cudaMemcpyAsync(r.buf, x->io_stage, VEC_BYTES, cudaMemcpyHostToDevice, x->st);
   if (e == cudaSuccess) e = cudaMemsetAsync(x->status_dev, 0, ALIGN, x->st);
+  // tensor-core path: the zero borders of the plane-layout activations are written once, here
+  if (e == cudaSuccess && cfg->precision != PS_FP32)
+    e = cudaMemsetAsync(x->ws.p1, 0, (uint64_t)cfg->max_workers * cfg->max_batch * psk::P1_PLANE_ELEMS * 4, x->st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(x->st);
   if (e != cudaSuccess) { delete x; return cuda_fail(e, "ps_create upload"); }
   *out = x;
@@ -324,7 +328,6 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
   a.W = W; a.b = b; a.x = x_dev; a.y = y_dev; a.loss = loss_dev; a.argmax = argmax_dev;
   a.seed = seed; a.step = step; a.drop_p = x->cfg.dropout_p; a.drop_thresh = x->drop_thresh;
   a.precision = x->cfg.precision;
-  a.fc1_legacy = 0;
   if (a.precision != PS_FP32 && gt.n_groups > std::min(x->cfg.max_workers, x->cfg.ring_depth))
     return fail(PS_ERR_BAD_ARG, "%d distinct snapshots but the tensor-core workspace holds ring_depth = %d", gt.n_groups, x->cfg.ring_depth);
   int n = psk::launch_grad_step_fp32(a, wt, gt, x->ws, x->st, &x->prof);
