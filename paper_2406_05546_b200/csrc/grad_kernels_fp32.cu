@@ -482,30 +482,54 @@ __global__ void __launch_bounds__(256) conv2_bwd(GradStepArgs a, WorkerTable wt,
 }
 
 // ---- backward through pool1, ReLU and conv1 (filter / bias gradients only: the input needs none).
+// Thread (channel, lane of 16) owns 13 pooled positions of its channel.  The image, the pooling decisions
+// and the pooled gradients of the NEXT sample are fetched into registers while the current one is
+// accumulated, so that no global-memory latency sits between the multiply-adds.
 __global__ void __launch_bounds__(256) conv1_bwd(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
   __shared__ float xs[30][31];
+  constexpr int PER = 13;                   // ceil(196 / 16)
   const int s = blockIdx.y, tid = threadIdx.x;
   const int oc = tid >> 4, l = tid & 15;
   float gw[9], gb = 0.f;
 #pragma unroll
   for (int k = 0; k < 9; ++k) gw[k] = 0.f;
+  for (int t = tid; t < 30 * 31; t += 256) (&xs[0][0])[t] = 0.f;
   const int i0 = blockIdx.x * CONV_SPB;
   const int i1 = min(i0 + CONV_SPB, a.b);
-  for (int i = i0; i < i1; ++i) {
+  float xr[4], gr[PER];
+  int cr[PER];
+  auto prefetch = [&](int i) {
     const int64_t row = (int64_t)s * a.b + i;
     const float* x = a.x + ((int64_t)wt.src[s] * a.b + i) * (IMG * IMG);
-    __syncthreads();
-    for (int t = tid; t < 30 * 30; t += 256) {
-      int yy = t / 30, xx = t % 30;
-      bool in = yy >= 1 && yy <= IMG && xx >= 1 && xx <= IMG;
-      xs[yy][xx] = in ? x[(yy - 1) * IMG + (xx - 1)] : 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) xr[k] = tid + 256 * k < IMG * IMG ? x[tid + 256 * k] : 0.f;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      const int pp = l + 16 * k;
+      cr[k] = pp < 196 ? (int)ws.code1[row * P1_ELEMS + oc * 196 + pp] : 4;
+      gr[k] = pp < 196 ? ws.dp1[row * P1_ELEMS + oc * 196 + pp] : 0.f;
     }
+  };
+  prefetch(i0);
+  for (int i = i0; i < i1; ++i) {
+    __syncthreads();                        // the previous sample's image is no longer read
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int t = tid + 256 * k;
+      if (t < IMG * IMG) xs[t / IMG + 1][t % IMG + 1] = xr[k];
+    }
+    float g_cur[PER];
+    int c_cur[PER];
+#pragma unroll
+    for (int k = 0; k < PER; ++k) { g_cur[k] = gr[k]; c_cur[k] = cr[k]; }
     __syncthreads();
-    for (int pp = l; pp < 196; pp += 16) {
-      int code = ws.code1[row * P1_ELEMS + oc * 196 + pp];
-      if (code < 4) {
-        float g = ws.dp1[row * P1_ELEMS + oc * 196 + pp];
-        int y = 2 * (pp / 14) + (code >> 1), xq = 2 * (pp % 14) + (code & 1);
+    if (i + 1 < i1) prefetch(i + 1);
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      if (c_cur[k] < 4) {
+        const int pp = l + 16 * k;
+        const float g = g_cur[k];
+        const int y = 2 * (pp / 14) + (c_cur[k] >> 1), xq = 2 * (pp % 14) + (c_cur[k] & 1);
         gb += g;
 #pragma unroll
         for (int ky = 0; ky < 3; ++ky)

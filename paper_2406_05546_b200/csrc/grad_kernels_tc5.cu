@@ -22,11 +22,14 @@ namespace psk {
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 32;          // CTA tile; BK floats = one 128-byte swizzle row
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BM * BK * 4, B_BYTES = BN * BK * 4, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int BM = 128, BK = 32;                    // CTA tile rows; BK floats = one 128-byte swizzle row
+constexpr int A_BYTES = BM * BK * 4;
 constexpr int TMEM_COLS = 256;
+constexpr int MAX_STAGES = 4;
+__host__ __device__ constexpr int stage_bytes(int bn) { return A_BYTES + bn * BK * 4; }
+__host__ __device__ constexpr int gemm_smem_bytes(int bn, int stages) {
+  return stages * stage_bytes(bn) + 1024 /* alignment slack */ + 256 /* barriers */;
+}
 
 // Shared-memory matrix descriptor, k-contiguous operand, 128-byte swizzle: rows are 128 bytes apart,
 // groups of eight rows 1024 bytes apart (stride byte offset), descriptor version 1.
@@ -64,9 +67,13 @@ struct GemmArgs {
 
 // 192 threads: warp 0 = TMA producer, warp 1 = tensor-memory owner and MMA issuer, warps 2..5 = epilogue
 // (each reads the 32 accumulator lanes of its quarter, quarter = warp index mod 4).
-template <int EPI>
+// BN = tile columns (256 for the 512-wide forward product, 224 = 1568/7 for the other two), STAGES = depth
+// of the operand pipeline (2 for the weight gradient, whose reduction is only b long: two CTAs then share an SM).
+template <int EPI, int BN, int STAGES>
 __global__ void __launch_bounds__(192) tc5_gemm(const __grid_constant__ GemmMaps maps, GemmArgs ga, GradStepArgs a,
                                                 WorkerTable wt, GroupTable gt, Workspace ws) {
+  constexpr int B_BYTES = BN * BK * 4, STAGE_BYTES = A_BYTES + B_BYTES;
+  static_assert(STAGE_BYTES % 1024 == 0 && STAGES <= MAX_STAGES && BN % 32 == 0 && BN <= TMEM_COLS, "tile shape");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
@@ -261,8 +268,9 @@ int configure_tc5_kernels() {
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return -1;
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
-  cudaError_t e = cudaFuncSetAttribute(tc5_gemm<EPI_FC1_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(tc5_gemm<EPI_FC1_FWD, 256, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(256, 4));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, 4));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, 2));
   return e == cudaSuccess ? 0 : -1;
 }
 
@@ -274,10 +282,10 @@ int launch_fc1_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const Group
   const uint64_t rows = (uint64_t)a.W * a.b;
   if (!make_map(&maps.a, ws.p2, FLAT, rows, 1, FLAT, rows * FLAT, BM)) return -1;
   for (int g = 0; g < gt.n_groups; ++g)
-    if (!make_map(&maps.b[g], ws.w1r + (int64_t)g * HID * FLAT, FLAT, HID, 1, FLAT, (uint64_t)HID * FLAT, BN)) return -1;
+    if (!make_map(&maps.b[g], ws.w1r + (int64_t)g * HID * FLAT, FLAT, HID, 1, FLAT, (uint64_t)HID * FLAT, 256)) return -1;
   GemmArgs ga{FLAT, HID, HID, 0, ws.d, 0};
   const int mt = group_tiles(gt, a.b, BM);
-  TIMED(K_FC1_FWD, (tc5_gemm<EPI_FC1_FWD><<<dim3(HID / BN, mt, 1), 192, SMEM_BYTES, st>>>(maps, ga, a, wt, gt, ws)));
+  TIMED(K_FC1_FWD, (tc5_gemm<EPI_FC1_FWD, 256, 4><<<dim3(HID / 256, mt, 1), 192, gemm_smem_bytes(256, 4), st>>>(maps, ga, a, wt, gt, ws)));
   return 2;
 }
 
@@ -287,10 +295,10 @@ int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupT
   const uint64_t rows = (uint64_t)a.W * a.b;
   if (!make_map(&maps.a, ws.da1, HID, rows, 1, HID, rows * HID, BM)) return -1;
   for (int g = 0; g < gt.n_groups; ++g)
-    if (!make_map(&maps.b[g], ws.w1tr + (int64_t)g * HID * FLAT, HID, FLAT, 1, HID, (uint64_t)HID * FLAT, BN)) return -1;
+    if (!make_map(&maps.b[g], ws.w1tr + (int64_t)g * HID * FLAT, HID, FLAT, 1, HID, (uint64_t)HID * FLAT, 224)) return -1;
   GemmArgs ga{HID, FLAT, FLAT, 0, ws.dp2, 0};
   const int mt = group_tiles(gt, a.b, BM);
-  TIMED(K_FC1_DX, (tc5_gemm<EPI_STORE><<<dim3((FLAT + BN - 1) / BN, mt, 1), 192, SMEM_BYTES, st>>>(maps, ga, a, wt, gt, ws)));
+  TIMED(K_FC1_DX, (tc5_gemm<EPI_STORE, 224, 4><<<dim3(FLAT / 224, mt, 1), 192, gemm_smem_bytes(224, 4), st>>>(maps, ga, a, wt, gt, ws)));
   return 1;
 }
 
@@ -301,9 +309,9 @@ int launch_fc1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupT
   TIMED(K_TRANSPOSE, (transpose_rows<<<dim3(FLAT / 32, (bp + 31) / 32, a.W), 256, 0, st>>>(ws.p2, ws.p2t, a.b, bp, FLAT)));
   GemmMaps maps;
   if (!make_map(&maps.a, ws.da1t, a.b, HID, a.W, bp, (uint64_t)HID * bp, BM)) return -1;
-  if (!make_map(&maps.b[0], ws.p2t, a.b, FLAT, a.W, bp, (uint64_t)FLAT * bp, BN)) return -1;
+  if (!make_map(&maps.b[0], ws.p2t, a.b, FLAT, a.W, bp, (uint64_t)FLAT * bp, 224)) return -1;
   GemmArgs ga{a.b, FLAT, FLAT, 1, nullptr, 0};
-  TIMED(K_FC1_DW, (tc5_gemm<EPI_STORE><<<dim3((FLAT + BN - 1) / BN, HID / BM, a.W), 192, SMEM_BYTES, st>>>(maps, ga, a, wt, gt, ws)));
+  TIMED(K_FC1_DW, (tc5_gemm<EPI_STORE, 224, 2><<<dim3(FLAT / 224, HID / BM, a.W), 192, gemm_smem_bytes(224, 2), st>>>(maps, ga, a, wt, gt, ws)));
   return 3;
 }
 
