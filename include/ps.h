@@ -230,7 +230,9 @@ int32_t ps_tick_host(ps_ctx* ctx, int32_t W, int32_t b, const int32_t* lags, con
 
 /* Per-kernel timing for measurement (no counterpart in the paper's method; it serves the roofline
  * report).  ps_profile(ctx, 1) clears the totals and from then on brackets every kernel launch with
- * two CUDA events on the context's stream; ps_profile(ctx, 0) stops.  ps_profile_read() synchronises
+ * two CUDA events on the context's stream (and runs the branches of the backward pass one after the
+ * other instead of side by side, so that each kernel is timed alone); ps_profile(ctx, 0) stops.
+ * ps_profile_read() synchronises
  * the stream and returns, for kernel index 0..n-1, its name (static string), summed device time in
  * milliseconds and launch count; an index past the last kernel returns PS_ERR_BAD_ARG. */
 int32_t ps_profile(ps_ctx* ctx, int32_t enable);

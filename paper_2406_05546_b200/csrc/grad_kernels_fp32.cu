@@ -598,36 +598,57 @@ int configure_grad_kernels() {
   return e == cudaSuccess ? 0 : -1;
 }
 
-int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt,
-                          const Workspace& ws, cudaStream_t st, Profiler* prof) {
+// Launch order of one grad step.  On the tensor-core path the backward pass forks: once the output
+// layer's backward has produced da1, the dense layer's per-worker weight gradient (bound by its 3.2 MB
+// per worker of writes) runs on a side stream next to the input-gradient chain, and once dp2 exists the
+// second convolution's filter gradient runs on another side stream next to its input gradient and the
+// first convolution's backward.  Everything joins before the final reduction.
+int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                     cudaStream_t st, const SideStreams& side, Profiler* prof) {
   const int n_chunks = (a.b + CONV_SPB - 1) / CONV_SPB;
   const int mt = group_tiles(gt, a.b, 64);
   const bool tc = a.precision != 0;
   const int n_chunks1 = (a.b + CONV1_SPB - 1) / CONV1_SPB;
-  if (tc) TIMED(K_CONV1_FWD, (conv1_fwd<true><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
-  else TIMED(K_CONV1_FWD, (conv1_fwd<false><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
-  if (tc) launch_conv2_fwd_tc5(a, wt, gt, ws, st, prof);
-  else TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
-  int extra = 0;
-  if (tc) { int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1; }
-  else TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
-  TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
+  int launches = 0, n_chunks2 = n_chunks;
   if (tc) {
-    int n = launch_fc1_dw_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1;
-    n = launch_fc1_dx_tc5(a, wt, gt, ws, st, prof); if (n < 0) return -1; extra += n - 1;
+    TIMED(K_CONV1_FWD, (conv1_fwd<true><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
+    launch_conv2_fwd_tc5(a, wt, gt, ws, st, prof);
+    int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof);
+    if (n < 0) return -1;
+    launches += 2 + n;
+    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
+    launches += 1;
+    cudaStream_t s1 = side.s1 ? side.s1 : st, s2 = side.s2 ? side.s2 : st;
+    if (side.s1) { cudaEventRecord(side.fork1, st); cudaStreamWaitEvent(s1, side.fork1, 0); }
+    n = launch_fc1_dw_tc5(a, wt, gt, ws, s1, prof);
+    if (n < 0) return -1;
+    launches += n;
+    if (side.s1) cudaEventRecord(side.join1, s1);
+    n = launch_fc1_dx_tc5(a, wt, gt, ws, st, prof);
+    if (n < 0) return -1;
+    launches += n;
+    if (side.s2) { cudaEventRecord(side.fork2, st); cudaStreamWaitEvent(s2, side.fork2, 0); }
+    n_chunks2 = launch_conv2_dw_tc(a, wt, ws, s2, prof);
+    if (side.s2) cudaEventRecord(side.join2, s2);
+    launch_conv2_dx_tc5(a, wt, gt, ws, st, prof);
+    TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
+    if (side.s1) cudaStreamWaitEvent(st, side.join1, 0);
+    if (side.s2) cudaStreamWaitEvent(st, side.join2, 0);
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks, n_chunks2)));
+    launches += 4;
   } else {
+    TIMED(K_CONV1_FWD, (conv1_fwd<false><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
+    TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
+    TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks, n_chunks2)));
+    launches = 9;
   }
-  int n_chunks2 = n_chunks;
-  if (tc) {
-    launch_conv2_dx_tc5(a, wt, gt, ws, st, prof);
-    n_chunks2 = launch_conv2_dw_tc(a, wt, ws, st, prof);
-  }
-  else TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
-  TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
-  TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks, n_chunks2)));
-  return cudaGetLastError() == cudaSuccess ? (tc ? 10 : 9) + extra : -1;
+  return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 }  // namespace psk

@@ -123,9 +123,16 @@ struct GradStepArgs {
   int precision;          // 0 = FP32 CUDA cores, 1 = TF32 tensor cores for the dense contractions
 };
 
-// Part A, FP32 CUDA-core path. Returns the number of kernels launched, or -1 on a launch error.
-int launch_grad_step_fp32(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt,
-                          const Workspace& ws, cudaStream_t st, Profiler* prof);
+// Side streams (and the events that fork from / join into the caller's stream) for the independent
+// branches of the backward pass; null streams mean "run everything on the caller's stream".
+struct SideStreams {
+  cudaStream_t s1 = nullptr, s2 = nullptr;
+  cudaEvent_t fork1 = nullptr, join1 = nullptr, fork2 = nullptr, join2 = nullptr;
+};
+
+// Part A. Returns the number of kernels launched, or -1 on a launch error.
+int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                     cudaStream_t st, const SideStreams& side, Profiler* prof);
 int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, uint32_t thresh,
                         uint8_t* keep, cudaStream_t st, Profiler* prof);
 int configure_grad_kernels();

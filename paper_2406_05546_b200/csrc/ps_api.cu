@@ -73,6 +73,7 @@ struct ps_ctx {
   std::vector<QueueMeta> meta;
   uint32_t drop_thresh = 0;
   psk::Profiler prof;
+  psk::SideStreams side;
   double prof_ms[psk::K_COUNT] = {0};
   int64_t prof_n[psk::K_COUNT] = {0};
 };
@@ -235,6 +236,14 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
   double t = std::floor((double)cfg->dropout_p * 4294967296.0);
   x->drop_thresh = t <= 0.0 ? 0u : (t >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)t);
   if (psk::configure_grad_kernels() != 0 || psk::configure_tc_kernels() != 0 || psk::configure_tc5_kernels() != 0 || psk::configure_conv5_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
+  if (cfg->precision != PS_FP32) {
+    // two side streams let independent branches of the backward pass overlap (they allocate no device memory)
+    bool ok = cudaStreamCreateWithFlags(&x->side.s1, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&x->side.s2, cudaStreamNonBlocking) == cudaSuccess;
+    cudaEvent_t* evs[4] = {&x->side.fork1, &x->side.join1, &x->side.fork2, &x->side.join2};
+    for (auto ev : evs) ok = ok && cudaEventCreateWithFlags(ev, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { delete x; return fail(PS_ERR_CUDA, "side stream set-up failed: %s", cudaGetErrorString(cudaGetLastError())); }
+  }
   std::memcpy(x->io_stage, init_params_host, sizeof(float) * PS_PARAM_COUNT);
   std::memset(x->io_stage + PS_PARAM_COUNT, 0, sizeof(float) * (PS_PARAM_STRIDE - PS_PARAM_COUNT));
   cudaError_t e = cudaMemcpyAsync(x->ring[0], x->io_stage, VEC_BYTES, cudaMemcpyHostToDevice, x->st);
@@ -253,6 +262,9 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
 int32_t ps_destroy(ps_ctx* x) {
   if (!x) return fail(PS_ERR_BAD_ARG, "ctx is NULL");
   cudaError_t e = cudaStreamSynchronize(x->st);
+  if (x->side.s1) { cudaStreamSynchronize(x->side.s1); cudaStreamDestroy(x->side.s1); }
+  if (x->side.s2) { cudaStreamSynchronize(x->side.s2); cudaStreamDestroy(x->side.s2); }
+  for (cudaEvent_t ev : {x->side.fork1, x->side.join1, x->side.fork2, x->side.join2}) if (ev) cudaEventDestroy(ev);
   delete x;
   if (e != cudaSuccess) return cuda_fail(e, "ps_destroy");
   return PS_OK;
@@ -330,7 +342,7 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
   a.precision = x->cfg.precision;
   if (a.precision != PS_FP32 && gt.n_groups > std::min(x->cfg.max_workers, x->cfg.ring_depth))
     return fail(PS_ERR_BAD_ARG, "%d distinct snapshots but the tensor-core workspace holds ring_depth = %d", gt.n_groups, x->cfg.ring_depth);
-  int n = psk::launch_grad_step_fp32(a, wt, gt, x->ws, x->st, &x->prof);
+  int n = psk::launch_grad_step(a, wt, gt, x->ws, x->st, x->prof.on ? psk::SideStreams() : x->side, &x->prof);
   if (n < 0) return cuda_fail(cudaGetLastError(), "grad step launch");
   x->launches += n;
   return PS_OK;
