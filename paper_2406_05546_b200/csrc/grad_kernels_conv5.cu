@@ -106,27 +106,27 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
   if (warp == 0) {
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_tf32(128, 32);
-      const uint32_t w_addr = smem_u32(Wk);
+      const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), 512);
       for (int t = 0; t < n_tiles; ++t) {
         const int buf = t & 1;
         if (!mbar_wait(&pipe->a_full[buf], (t >> 1) & 1)) { pipe->abort_flag = 1; break; }
         if (t >= 2 && !mbar_wait(&pipe->acc_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
         if (pipe->abort_flag) break;
         tc_fence_after();
-        const uint32_t a_base = smem_u32(bufs) + buf * F_BUF_BYTES;
-#pragma unroll 1
+        // 72 MMAs, fully unrolled: every descriptor is a per-tile base plus a compile-time constant
+        const uint32_t a_lo = plain_desc_lo(smem_u32(bufs) + buf * F_BUF_BYTES, F_PLANE_BYTES);
+        const uint32_t d_tmem = tmem + buf * 128;
+#pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int jy = j >> 1, jx = j & 1;
-#pragma unroll 1
+#pragma unroll
           for (int tap = 0; tap < 9; ++tap) {
             const int ky = tap / 3, kx = tap - ky * 3, sx = jx + kx;
-            const uint32_t row_off = (uint32_t)((jy + ky) * 16 + (sx & 1) * 8 + (sx >> 1)) * 16u;
+            const int row_off = (jy + ky) * 16 + (sx & 1) * 8 + (sx >> 1);     // in 16-byte rows
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              const uint64_t da = smem_desc_plain(a_base + (2 * half) * F_PLANE_BYTES + row_off, F_PLANE_BYTES, 512);
-              const uint64_t db = smem_desc_plain(w_addr + (tap * 4 + half * 2) * 512, 512, 128);
-              umma_tf32(tmem + buf * 128 + j * 32, da, db, idesc, (tap | half) ? 1u : 0u);
-            }
+            for (int half = 0; half < 2; ++half)
+              umma_tf32_split(d_tmem + j * 32, a_lo + (2 * half) * (F_PLANE_BYTES / 16) + row_off, plain_desc_hi(512),
+                              w_lo + (tap * 4 + half * 2) * (512 / 16), plain_desc_hi(128), idesc, (tap | half) ? 1u : 0u);
           }
         }
         umma_commit(&pipe->a_empty[buf]);
@@ -240,26 +240,25 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
   if (warp == 0) {
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_tf32(128, 16);
-      const uint32_t w_addr = smem_u32(Wk);
+      const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), 256);
       for (int t = 0; t < n_tiles; ++t) {
         const int buf = t & 1;
         if (!mbar_wait(&pipe->a_full[buf], (t >> 1) & 1)) { pipe->abort_flag = 1; break; }
         if (t >= 2 && !mbar_wait(&pipe->acc_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
         if (pipe->abort_flag) break;
         tc_fence_after();
-        const uint32_t a_base = smem_u32(bufs) + buf * X_BUF_BYTES;
-#pragma unroll 1
+        const uint32_t a_lo = plain_desc_lo(smem_u32(bufs) + buf * X_BUF_BYTES, X_PLANE_BYTES);
+        const uint32_t d_tmem = tmem + buf * 32;
+#pragma unroll
         for (int m = 0; m < 2; ++m) {
-#pragma unroll 1
+#pragma unroll
           for (int tap = 0; tap < 9; ++tap) {
             const int ky = tap / 3, kx = tap - ky * 3;
-            const uint32_t row_off = (uint32_t)(m * 128 + (2 - ky) * 16 + (2 - kx)) * 16u;
+            const int row_off = m * 128 + (2 - ky) * 16 + (2 - kx);           // in 16-byte rows
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const uint64_t da = smem_desc_plain(a_base + (2 * q) * X_PLANE_BYTES + row_off, X_PLANE_BYTES, 128);
-              const uint64_t db = smem_desc_plain(w_addr + (tap * 8 + q * 2) * 256, 256, 128);
-              umma_tf32(tmem + buf * 32 + m * 16, da, db, idesc, (tap | q) ? 1u : 0u);
-            }
+            for (int q = 0; q < 4; ++q)
+              umma_tf32_split(d_tmem + m * 16, a_lo + (2 * q) * (X_PLANE_BYTES / 16) + row_off, plain_desc_hi(128),
+                              w_lo + (tap * 8 + q * 2) * (256 / 16), plain_desc_hi(128), idesc, (tap | q) ? 1u : 0u);
           }
         }
         umma_commit(&pipe->a_empty[buf]);
