@@ -24,11 +24,12 @@ namespace {
 
 constexpr int BM = 128, BK = 32;                    // CTA tile rows; BK floats = one 128-byte swizzle row
 constexpr int A_BYTES = BM * BK * 4;
-constexpr int TMEM_COLS = 256;
 constexpr int MAX_STAGES = 4;
+constexpr int EPI_ROW_FLOATS = 36;                       // 32 columns + 4 of padding: conflict-free both ways
+constexpr int EPI_WARP_BYTES = 32 * EPI_ROW_FLOATS * 4;  // per epilogue warp: a 32 x 32 block being transposed
 __host__ __device__ constexpr int stage_bytes(int bn) { return A_BYTES + bn * BK * 4; }
 __host__ __device__ constexpr int gemm_smem_bytes(int bn, int stages) {
-  return stages * stage_bytes(bn) + 1024 /* alignment slack */ + 256 /* barriers */;
+  return stages * stage_bytes(bn) + 1024 /* alignment slack */ + 256 /* barriers */ + 4 * EPI_WARP_BYTES;
 }
 
 // Shared-memory matrix descriptor, k-contiguous operand, 128-byte swizzle: rows are 128 bytes apart,
@@ -60,143 +61,186 @@ struct GemmArgs {
   int K;            // reduction length (columns beyond it are zero-filled by TMA)
   int N;            // valid output columns
   int ldc;
-  int per_worker;   // 1: blockIdx.z = sorted worker, rows 0..511 of its own output; 0: grouped rows
+  int per_worker;   // 1: one 512-row output per sorted worker (tensor-map slab z); 0: grouped rows
   float* c;         // output base when !per_worker
-  int round_out;    // round stored values to TF32 (they feed another tensor-core product)
+  int n_tiles_n;    // tiles along the columns
+  int n_tiles;      // all tiles of the launch
 };
 
-// 192 threads: warp 0 = TMA producer, warp 1 = tensor-memory owner and MMA issuer, warps 2..5 = epilogue
-// (each reads the 32 accumulator lanes of its quarter, quarter = warp index mod 4).
-// BN = tile columns (256 for the 512-wide forward product, 224 = 1568/7 for the other two), STAGES = depth
-// of the operand pipeline (2 for the weight gradient, whose reduction is only b long: two CTAs then share an SM).
-template <int EPI, int BN, int STAGES>
-__global__ void __launch_bounds__(192) tc5_gemm(const __grid_constant__ GemmMaps maps, GemmArgs ga, GradStepArgs a,
-                                                WorkerTable wt, GroupTable gt, Workspace ws) {
+// Persistent kernel: one CTA per SM walks over output tiles (columns fastest, so that neighbouring CTAs
+// share their A rows in L2).  192 threads: warp 0 = TMA producer, warp 1 = tensor-memory owner and MMA
+// issuer, warps 2..5 = epilogue (each reads the 32 accumulator lanes of its quarter, quarter = warp index
+// mod 4).  The accumulator is double-buffered in tensor memory (2 x BN columns), so the epilogue of one
+// tile (tensor memory -> registers -> global) overlaps the loads and MMAs of the next.
+// BN = tile columns: 256 for the 512-wide forward product, 224 = 1568/7 for the other two.
+struct TileCoord { int grp, m0, m_end, n0, z; };
+
+template <int BN>
+__device__ __forceinline__ bool decode_tile(int t, const GemmArgs& ga, const GroupTable& gt, int b, TileCoord& c) {
+  const int nt = t % ga.n_tiles_n;
+  const int rest = t / ga.n_tiles_n;
+  c.n0 = nt * BN;
+  c.grp = 0;
+  if (ga.per_worker) {
+    c.z = rest / (HID / BM);
+    c.m0 = (rest % (HID / BM)) * BM;
+    c.m_end = HID;
+    return true;
+  }
+  c.z = 0;
+  return locate_group_tile<BM>(gt, b, rest, c.grp, c.m0, c.m_end);
+}
+
+template <int EPI, int BN>
+__global__ void __launch_bounds__(192, 1) tc5_gemm(const __grid_constant__ GemmMaps maps, GemmArgs ga, GradStepArgs a,
+                                                   WorkerTable wt, GroupTable gt, Workspace ws) {
+  constexpr int STAGES = MAX_STAGES;
   constexpr int B_BYTES = BN * BK * 4, STAGE_BYTES = A_BYTES + B_BYTES;
-  static_assert(STAGE_BYTES % 1024 == 0 && STAGES <= MAX_STAGES && BN % 32 == 0 && BN <= TMEM_COLS, "tile shape");
+  static_assert(STAGE_BYTES % 1024 == 0 && BN % 32 == 0 && 2 * BN <= 512, "tile shape");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* tiles = smem_raw + (base - smem_u32(smem_raw));
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + STAGES * STAGE_BYTES);
-  uint64_t* full = bars;                 // [STAGES] TMA -> MMA
-  uint64_t* empty = bars + STAGES;       // [STAGES] MMA -> TMA
-  uint64_t* acc_full = bars + 2 * STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
+  uint64_t* full = bars;                     // [STAGES] TMA -> MMA
+  uint64_t* empty = bars + STAGES;           // [STAGES] MMA -> TMA
+  uint64_t* acc_full = bars + 2 * STAGES;    // [2] MMA -> epilogue
+  uint64_t* acc_empty = bars + 2 * STAGES + 2;   // [2] epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* epi_stage = reinterpret_cast<float*>(tiles + STAGES * STAGE_BYTES + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int grp = 0, m0, m_end, z = 0;
-  if (ga.per_worker) {
-    z = blockIdx.z; m0 = blockIdx.y * BM; m_end = HID;
-  } else if (!locate_group_tile<BM>(gt, a.b, blockIdx.y, grp, m0, m_end)) {
-    return;
-  }
-  const int n0 = blockIdx.x * BN;
   const int n_k = (ga.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(acc_full, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  tc_fence_before();
   __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  tc_fence_after();
   const uint32_t tmem_acc = *tmem_slot;
 
   if (warp == 0) {
     if (lane == 0) {
-      const CUtensorMap* map_a = &maps.a;
-      const CUtensorMap* map_b = &maps.b[ga.per_worker ? 0 : grp];
-      for (int kb = 0; kb < n_k; ++kb) {
-        const int s = kb % STAGES;
-        if (kb >= STAGES && !mbar_wait(&empty[s], ((kb / STAGES) - 1) & 1)) { *abort_flag = 1; break; }
-        if (*abort_flag) break;
-        mbar_expect_tx(&full[s], STAGE_BYTES);
-        tma_load_3d(tiles + s * STAGE_BYTES, map_a, &full[s], kb * BK, m0, z);
-        tma_load_3d(tiles + s * STAGE_BYTES + A_BYTES, map_b, &full[s], kb * BK, n0, z);
+      int it = 0;                            // k-blocks issued so far, over all tiles
+      bool ok = true;
+      for (int t = blockIdx.x; t < ga.n_tiles && ok; t += gridDim.x) {
+        TileCoord c;
+        if (!decode_tile<BN>(t, ga, gt, a.b, c)) continue;
+        const CUtensorMap* map_a = &maps.a;
+        const CUtensorMap* map_b = &maps.b[c.grp];
+        for (int kb = 0; kb < n_k; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (it >= STAGES && !mbar_wait(&empty[s], ((it / STAGES) - 1) & 1)) { *abort_flag = 1; ok = false; break; }
+          if (*abort_flag) { ok = false; break; }
+          mbar_expect_tx(&full[s], STAGE_BYTES);
+          tma_load_3d(tiles + s * STAGE_BYTES, map_a, &full[s], kb * BK, c.m0, c.z);
+          tma_load_3d(tiles + s * STAGE_BYTES + A_BYTES, map_b, &full[s], kb * BK, c.n0, c.z);
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc_tf32(BM, BN);
+      const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0) >> 32);
+      int it = 0, tile_i = 0;
       bool ok = true;
-      for (int kb = 0; kb < n_k && ok; ++kb) {
-        const int s = kb % STAGES;
-        if (!mbar_wait(&full[s], (kb / STAGES) & 1) || *abort_flag) { *abort_flag = 1; ok = false; break; }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_addr = base + s * STAGE_BYTES, b_addr = a_addr + A_BYTES;
+      for (int t = blockIdx.x; t < ga.n_tiles && ok; t += gridDim.x) {
+        TileCoord c;
+        if (!decode_tile<BN>(t, ga, gt, a.b, c)) continue;
+        const int ab = tile_i & 1;
+        if (tile_i >= 2 && !mbar_wait(&acc_empty[ab], ((tile_i >> 1) - 1) & 1)) { *abort_flag = 1; break; }
+        tc_fence_after();
+        for (int kb = 0; kb < n_k; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&full[s], (it / STAGES) & 1) || *abort_flag) { *abort_flag = 1; ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_lo = (uint32_t)smem_desc_sw128(base + s * STAGE_BYTES);
+          const uint32_t b_lo = (uint32_t)smem_desc_sw128(base + s * STAGE_BYTES + A_BYTES);
 #pragma unroll
-        for (int k = 0; k < BK / 8; ++k) {
-          umma_tf32(tmem_acc, smem_desc_sw128(a_addr + k * 32), smem_desc_sw128(b_addr + k * 32), idesc,
-                    (kb > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < BK / 8; ++k)
+            umma_tf32_split(tmem_acc + ab * BN, a_lo + k * 2, desc_hi, b_lo + k * 2, desc_hi, idesc, (kb | k) ? 1u : 0u);
+          umma_commit(&empty[s]);            // the stage may be refilled once these MMAs have read it
         }
-        umma_commit(&empty[s]);      // the stage may be refilled once these MMAs have read it
+        if (ok) umma_commit(&acc_full[ab]);
+        ++tile_i;
       }
-      if (ok) umma_commit(acc_full);
     }
   } else {
     const int quarter = warp & 3;
-    const bool ready = mbar_wait(acc_full, 0) && !*abort_flag;
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (!ready) {
-      if (lane == 0) { *abort_flag = 1; atomicOr(ws.status, STATUS_WAIT_TIMEOUT); }
-    } else {
-      const int m = m0 + quarter * 32 + lane;
-      const bool row_ok = m < m_end;
-      float* crow;
-      if (ga.per_worker) crow = wt.grad[z] + OFF_F1W + (int64_t)m * ga.ldc;
-      else crow = ga.c + (int64_t)m * ga.ldc;
+    int tile_i = 0;
+    const float scale = 1.0f / (1.0f - a.drop_p);
+    const uint2 key = make_uint2((uint32_t)a.seed, (uint32_t)(a.seed >> 32));
+    for (int t = blockIdx.x; t < ga.n_tiles; t += gridDim.x) {
+      TileCoord c;
+      if (!decode_tile<BN>(t, ga, gt, a.b, c)) continue;
+      const int ab = tile_i & 1;
+      if (!mbar_wait(&acc_full[ab], (tile_i >> 1) & 1) || *abort_flag) {
+        if (lane == 0) { *abort_flag = 1; atomicOr(ws.status, STATUS_WAIT_TIMEOUT); }
+        break;
+      }
+      tc_fence_after();
+      // Each lane reads one accumulator row (32 columns at a time); the 32 x 32 block then goes through a
+      // padded shared-memory buffer so that one store instruction writes four full 128-byte row segments
+      // instead of 32 scattered 16-byte pieces.
+      const int m_lane = c.m0 + quarter * 32 + lane;
+      const bool row_ok = m_lane < c.m_end;
+      float* stage = epi_stage + (warp - 2) * (EPI_WARP_BYTES / 4);
+      float* cbase = ga.per_worker ? wt.grad[c.z] + OFF_F1W : ga.c;
       int s_w = 0, smp = 0;
-      if (EPI == EPI_FC1_FWD && row_ok) { s_w = m / a.b; smp = m - s_w * a.b; }
-      const float scale = 1.0f / (1.0f - a.drop_p);
-      const uint2 key = make_uint2((uint32_t)a.seed, (uint32_t)(a.seed >> 32));
-      const float* bias = gt.theta[grp] + OFF_F1B;
+      if (EPI == EPI_FC1_FWD && row_ok) { s_w = m_lane / a.b; smp = m_lane - s_w * a.b; }
+      const float* bias = gt.theta[c.grp] + OFF_F1B;
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int n = n0 + c * 32;
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        const int n = c.n0 + ch * 32;
         if (n >= ga.N) break;                    // warp-uniform
         uint32_t r[32];
-        tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), r);
-        if (!row_ok) continue;
-        if (EPI == EPI_FC1_FWD) {
+        tmem_ld32(tmem_acc + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + ch * 32), r);
+        if (EPI == EPI_FC1_FWD && row_ok) {
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             const int nq = n + q * 4;
             uint4 rnd = philox4x32_10(make_uint4((uint32_t)((smp * HID + nq) >> 2), (uint32_t)wt.wid[s_w],
                                                  (uint32_t)a.step, (uint32_t)(a.step >> 32)), key);
             const float4 bv = *reinterpret_cast<const float4*>(bias + nq);
-            float4 o;
-            o.x = rnd.x >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 0]) + bv.x, 0.f) * scale : 0.f;
-            o.y = rnd.y >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 1]) + bv.y, 0.f) * scale : 0.f;
-            o.z = rnd.z >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 2]) + bv.z, 0.f) * scale : 0.f;
-            o.w = rnd.w >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 3]) + bv.w, 0.f) * scale : 0.f;
-            *reinterpret_cast<float4*>(crow + nq) = o;
-          }
-        } else {
-#pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            float4 o = make_float4(__uint_as_float(r[q * 4]), __uint_as_float(r[q * 4 + 1]),
-                                   __uint_as_float(r[q * 4 + 2]), __uint_as_float(r[q * 4 + 3]));
-            if (ga.round_out) {
-              o.x = round_tf32(o.x); o.y = round_tf32(o.y); o.z = round_tf32(o.z); o.w = round_tf32(o.w);
-            }
-            *reinterpret_cast<float4*>(crow + n + q * 4) = o;
+            r[q * 4 + 0] = __float_as_uint(rnd.x >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 0]) + bv.x, 0.f) * scale : 0.f);
+            r[q * 4 + 1] = __float_as_uint(rnd.y >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 1]) + bv.y, 0.f) * scale : 0.f);
+            r[q * 4 + 2] = __float_as_uint(rnd.z >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 2]) + bv.z, 0.f) * scale : 0.f);
+            r[q * 4 + 3] = __float_as_uint(rnd.w >= a.drop_thresh ? fmaxf(__uint_as_float(r[q * 4 + 3]) + bv.w, 0.f) * scale : 0.f);
           }
         }
+        __syncwarp();                            // the previous block has been read out of the buffer
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<uint4*>(stage + lane * EPI_ROW_FLOATS + q * 4) = make_uint4(r[q * 4], r[q * 4 + 1], r[q * 4 + 2], r[q * 4 + 3]);
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int rr = i * 4 + (lane >> 3), cc = (lane & 7) * 4;
+          const int m = c.m0 + quarter * 32 + rr;
+          const uint4 v = *reinterpret_cast<const uint4*>(stage + rr * EPI_ROW_FLOATS + cc);
+          if (m < c.m_end) *reinterpret_cast<uint4*>(cbase + (int64_t)m * ga.ldc + n + cc) = v;
+        }
       }
+      // all of this warp's tensor-memory reads of the buffer are complete (tmem_ld32 waits): hand it back
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[ab]);
+      ++tile_i;
     }
   }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  tc_fence_before();
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(TMEM_COLS) : "memory");
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(512) : "memory");
   }
   if (threadIdx.x == 0 && *abort_flag) {
     atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
@@ -261,6 +305,8 @@ bool make_map(CUtensorMap* m, const float* base, uint64_t d0, uint64_t d1, uint6
 
 #define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
 
+int g_sm_count = 0;
+
 int configure_tc5_kernels() {
   if (!g_encode) {
     void* fn = nullptr;
@@ -268,9 +314,11 @@ int configure_tc5_kernels() {
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return -1;
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
-  cudaError_t e = cudaFuncSetAttribute(tc5_gemm<EPI_FC1_FWD, 256, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(256, 4));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, 4));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, 2));
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_sm_count <= 0) return -1;
+  cudaError_t e = cudaFuncSetAttribute(tc5_gemm<EPI_FC1_FWD, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(256, MAX_STAGES));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES));
   return e == cudaSuccess ? 0 : -1;
 }
 
@@ -283,9 +331,10 @@ int launch_fc1_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const Group
   if (!make_map(&maps.a, ws.p2, FLAT, rows, 1, FLAT, rows * FLAT, BM)) return -1;
   for (int g = 0; g < gt.n_groups; ++g)
     if (!make_map(&maps.b[g], ws.w1r + (int64_t)g * HID * FLAT, FLAT, HID, 1, FLAT, (uint64_t)HID * FLAT, 256)) return -1;
-  GemmArgs ga{FLAT, HID, HID, 0, ws.d, 0};
   const int mt = group_tiles(gt, a.b, BM);
-  TIMED(K_FC1_FWD, (tc5_gemm<EPI_FC1_FWD, 256, 4><<<dim3(HID / 256, mt, 1), 192, gemm_smem_bytes(256, 4), st>>>(maps, ga, a, wt, gt, ws)));
+  GemmArgs ga{FLAT, HID, HID, 0, ws.d, HID / 256, (HID / 256) * mt};
+  const int grid = ga.n_tiles < g_sm_count ? ga.n_tiles : g_sm_count;
+  TIMED(K_FC1_FWD, (tc5_gemm<EPI_FC1_FWD, 256><<<grid, 192, gemm_smem_bytes(256, MAX_STAGES), st>>>(maps, ga, a, wt, gt, ws)));
   return 2;
 }
 
@@ -296,9 +345,10 @@ int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupT
   if (!make_map(&maps.a, ws.da1, HID, rows, 1, HID, rows * HID, BM)) return -1;
   for (int g = 0; g < gt.n_groups; ++g)
     if (!make_map(&maps.b[g], ws.w1tr + (int64_t)g * HID * FLAT, HID, FLAT, 1, HID, (uint64_t)HID * FLAT, 224)) return -1;
-  GemmArgs ga{HID, FLAT, FLAT, 0, ws.dp2, 0};
   const int mt = group_tiles(gt, a.b, BM);
-  TIMED(K_FC1_DX, (tc5_gemm<EPI_STORE, 224, 4><<<dim3(FLAT / 224, mt, 1), 192, gemm_smem_bytes(224, 4), st>>>(maps, ga, a, wt, gt, ws)));
+  GemmArgs ga{HID, FLAT, FLAT, 0, ws.dp2, FLAT / 224, (FLAT / 224) * mt};
+  const int grid = ga.n_tiles < g_sm_count ? ga.n_tiles : g_sm_count;
+  TIMED(K_FC1_DX, (tc5_gemm<EPI_STORE, 224><<<grid, 192, gemm_smem_bytes(224, MAX_STAGES), st>>>(maps, ga, a, wt, gt, ws)));
   return 1;
 }
 
@@ -310,8 +360,9 @@ int launch_fc1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupT
   GemmMaps maps;
   if (!make_map(&maps.a, ws.da1t, a.b, HID, a.W, bp, (uint64_t)HID * bp, BM)) return -1;
   if (!make_map(&maps.b[0], ws.p2t, a.b, FLAT, a.W, bp, (uint64_t)FLAT * bp, 224)) return -1;
-  GemmArgs ga{a.b, FLAT, FLAT, 1, nullptr, 0};
-  TIMED(K_FC1_DW, (tc5_gemm<EPI_STORE, 224, 2><<<dim3(FLAT / 224, HID / BM, a.W), 192, gemm_smem_bytes(224, 2), st>>>(maps, ga, a, wt, gt, ws)));
+  GemmArgs ga{a.b, FLAT, FLAT, 1, nullptr, FLAT / 224, (FLAT / 224) * (HID / BM) * a.W};
+  const int grid = ga.n_tiles < g_sm_count ? ga.n_tiles : g_sm_count;
+  TIMED(K_FC1_DW, (tc5_gemm<EPI_STORE, 224><<<grid, 192, gemm_smem_bytes(224, MAX_STAGES), st>>>(maps, ga, a, wt, gt, ws)));
   return 3;
 }
 
