@@ -1,4 +1,4 @@
-// Filter gradient of the second convolution on the tensor cores (TF32, warp-level mma.sync): the one
+// Filter gradient of the second convolution on the tensor cores (BF16 operands, warp-level mma.sync): the one
 // contraction of the step whose output (32 x 144 per worker) is too small for a 128-row tcgen05 tile,
 // while its reduction (all positions of all samples of a worker) is long.
 //
@@ -10,40 +10,51 @@ namespace psk {
 
 namespace {
 
-// D += A(16x8, row) * B(8x8, col), TF32 inputs, fp32 accumulate.  Lane = 4*g + t:
-//   a0 (g, t)  a1 (g+8, t)  a2 (g, t+4)  a3 (g+8, t+4);  b0 (k=t, n=g)  b1 (k=t+4, n=g);
-//   c0 (g, 2t) c1 (g, 2t+1) c2 (g+8, 2t) c3 (g+8, 2t+1).
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
-}
-
 constexpr int TC_SPB = 8;
-__device__ __forceinline__ float tf32f(float x) { return round_tf32(x); }
 
 // Filter gradient: dW[oc][ic][tap] = sum_{samples,pos} g2[oc][pos] * p1[ic][pos + tap]: rows = 32 output
-// channels, columns = 16 input channels per tap, k = position (196 per sample, 25 k-steps, zero-padded).
+// channels, columns = 16 input channels per tap, k = position (196 per sample, 13 k-steps of 16, zero-padded).
+// Both operands are rounded to BF16 here (fp32 accumulation): this product only yields gradient values, no
+// ReLU or pooling decision depends on it, and at 16 positions per instruction it needs half the
+// instructions and shared-memory loads of the TF32 form.
 // 288 threads = 9 warps, warp = filter tap; accumulators persist over the block's samples and are
 // written once as the block's partial sum.  The bias gradient (sum of g2 over positions) rides along as
 // a product with a column of ones, each warp taking every ninth k-step; the nine partial sums are
 // combined in a fixed order at the end.
-// The next sample's inputs are fetched into registers while the current one is being multiplied, so
-// that global-memory latency stays off the critical path.
-constexpr int DW_G_STRIDE = 228;   // 196 positions + zeros; = 4 (mod 32 banks)
-constexpr int DW_PLANE = 260;      // 16 x 16 + 4;            = 4 (mod 32 banks)
+// A BF16 fragment register holds two consecutive k = two horizontally adjacent positions (x even, x+1).
+// For the taps that shift by an odd number of columns such a pair is not word-aligned in the image plane,
+// so the planes are kept twice, the second copy shifted by one element.
+// The next sample's inputs are fetched into registers while the current one is being multiplied.
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+__device__ __forceinline__ uint16_t bf16_bits(float x) {
+  uint16_t r;
+  asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {   // lo in the low half (lower k index)
+  return (uint32_t)bf16_bits(lo) | ((uint32_t)bf16_bits(hi) << 16);
+}
+
+constexpr int DW_G_WORDS = 108;    // 216 bf16 per output channel: 196 positions + zeros; 108 = 12 (mod 32 banks)
+constexpr int DW_P_WORDS = 132;    // 16 x 16 bf16 per input channel + 8; 132 = 4 (mod 32 banks)
 constexpr int DW_THREADS = 288;
+constexpr int DW_KSTEPS = 13;      // 208 positions / 16
 constexpr int DW_QUADS = (4 * 196 + DW_THREADS - 1) / DW_THREADS;   // 3 four-channel positions per thread
 constexpr int DW_ENTRIES = (FLAT + DW_THREADS - 1) / DW_THREADS;    // 6 pooled gradient entries per thread
 __global__ void __launch_bounds__(DW_THREADS) conv2_dw_tc(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
-  __shared__ __align__(16) float g2[32 * DW_G_STRIDE];   // [oc][pos]
-  __shared__ __align__(16) float img[16 * DW_PLANE];     // [ic][Y][X], zero border
+  __shared__ __align__(16) uint32_t g2w[32 * DW_G_WORDS];        // [oc][position pair]
+  __shared__ __align__(16) uint32_t imgw[2][16 * DW_P_WORDS];    // [copy][ic][(Y*16 + X - copy) / 2], zero border
   __shared__ float bias_part[9][32];
+  uint16_t* img_h[2] = {reinterpret_cast<uint16_t*>(imgw[0]), reinterpret_cast<uint16_t*>(imgw[1])};
   const int s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   const int ky = warp / 3, kx = warp - ky * 3;
-  for (int idx = tid; idx < 16 * DW_PLANE; idx += DW_THREADS) img[idx] = 0.f;
-  for (int idx = tid; idx < 32 * DW_G_STRIDE; idx += DW_THREADS) g2[idx] = 0.f;
+  for (int idx = tid; idx < 2 * 16 * DW_P_WORDS; idx += DW_THREADS) (&imgw[0][0])[idx] = 0u;
+  for (int idx = tid; idx < 32 * DW_G_WORDS; idx += DW_THREADS) g2w[idx] = 0u;
   float acc[2][2][4], accb[2][4];
 #pragma unroll
   for (int m = 0; m < 2; ++m) {
@@ -55,7 +66,11 @@ __global__ void __launch_bounds__(DW_THREADS) conv2_dw_tc(GradStepArgs a, Worker
     for (int r = 0; r < 4; ++r) accb[m][r] = 0.f;
   }
   // the column of ones: B(k, n) = 1 for n == 0; this lane supplies column n = g
-  const uint32_t one_frag[2] = {g == 0 ? __float_as_uint(1.0f) : 0u, g == 0 ? __float_as_uint(1.0f) : 0u};
+  const uint32_t one_frag[2] = {g == 0 ? 0x3F803F80u : 0u, g == 0 ? 0x3F803F80u : 0u};
+  // this warp's B fragments: pair index j = ks*8 + t (+4): position 2j = (y, x even); element (y+ky)*16 + x + kx
+  // in the bordered plane, taken from the copy that makes it even
+  const int copy = kx & 1;
+  const uint32_t* plane = imgw[copy];
   const int i0 = blockIdx.x * TC_SPB, i1 = min(i0 + TC_SPB, a.b);
 
   float4 pq[DW_QUADS];
@@ -86,8 +101,14 @@ __global__ void __launch_bounds__(DW_THREADS) conv2_dw_tc(GradStepArgs a, Worker
       const int e = tid + k * DW_THREADS;
       if (e < 4 * 196) {
         const int q = e / 196, p = e - q * 196, y = p / 14, x = p - y * 14;
-        float* d = img + (4 * q) * DW_PLANE + (y + 1) * 16 + x + 1;
-        d[0] = pq[k].x; d[DW_PLANE] = pq[k].y; d[2 * DW_PLANE] = pq[k].z; d[3 * DW_PLANE] = pq[k].w;
+        const int el = (y + 1) * 16 + x + 1;
+        const float v[4] = {pq[k].x, pq[k].y, pq[k].z, pq[k].w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const uint16_t h = bf16_bits(v[c]);
+          img_h[0][(4 * q + c) * (2 * DW_P_WORDS) + el] = h;
+          img_h[1][(4 * q + c) * (2 * DW_P_WORDS) + el - 1] = h;
+        }
       }
     }
 #pragma unroll
@@ -97,42 +118,42 @@ __global__ void __launch_bounds__(DW_THREADS) conv2_dw_tc(GradStepArgs a, Worker
         // every pooled entry owns the four positions of its window: the gradient goes to the chosen one,
         // the others are cleared, so no separate clearing pass is needed
         const int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
-        float* d = g2 + oc * DW_G_STRIDE + (2 * py) * 14 + 2 * px;
-        const float v = tf32f(pg[k]);
-        d[0] = pc[k] == 0 ? v : 0.f; d[1] = pc[k] == 1 ? v : 0.f;
-        d[14] = pc[k] == 2 ? v : 0.f; d[15] = pc[k] == 3 ? v : 0.f;
+        uint32_t* d = g2w + oc * DW_G_WORDS + (2 * py) * 7 + px;     // word of positions (2py, 2px), (2py, 2px+1)
+        const float v = pg[k];
+        d[0] = bf16_pair(pc[k] == 0 ? v : 0.f, pc[k] == 1 ? v : 0.f);
+        d[7] = bf16_pair(pc[k] == 2 ? v : 0.f, pc[k] == 3 ? v : 0.f);
       }
     }
     __syncthreads();
     if (i + 1 < i1) prefetch(i + 1);
-#pragma unroll 5
-    for (int ks = 0; ks < 25; ++ks) {
-      const int p0 = ks * 8 + t, p1 = p0 + 4;
+#pragma unroll
+    for (int ks = 0; ks < DW_KSTEPS; ++ks) {
+      const int j0 = ks * 8 + t, j1 = j0 + 4;                  // position pairs of this lane's k columns
       uint32_t fa[2][4], fb[2][2];
 #pragma unroll
       for (int m = 0; m < 2; ++m) {
-        const float* ga = g2 + (m * 16 + g) * DW_G_STRIDE;
-        fa[m][0] = __float_as_uint(ga[p0]);
-        fa[m][1] = __float_as_uint(ga[8 * DW_G_STRIDE + p0]);
-        fa[m][2] = __float_as_uint(ga[p1]);
-        fa[m][3] = __float_as_uint(ga[8 * DW_G_STRIDE + p1]);
+        const uint32_t* ga = g2w + (m * 16 + g) * DW_G_WORDS;
+        fa[m][0] = ga[j0];
+        fa[m][1] = ga[8 * DW_G_WORDS + j0];
+        fa[m][2] = ga[j1];
+        fa[m][3] = ga[8 * DW_G_WORDS + j1];
       }
-      const int q0 = min(p0, 195), q1 = min(p1, 195);
-      const int y0 = q0 / 14, x0 = q0 - y0 * 14, y1 = q1 / 14, x1 = q1 - y1 * 14;
-      const int o0 = (y0 + ky) * 16 + x0 + kx, o1 = (y1 + ky) * 16 + x1 + kx;
+      const int q0 = min(j0, 97), q1 = min(j1, 97);            // pairs beyond 97 meet zeros in g2
+      const int y0 = q0 / 7, x0 = 2 * (q0 - y0 * 7), y1 = q1 / 7, x1 = 2 * (q1 - y1 * 7);
+      const int w0 = ((y0 + ky) * 16 + x0 + kx - copy) >> 1, w1 = ((y1 + ky) * 16 + x1 + kx - copy) >> 1;
 #pragma unroll
       for (int n = 0; n < 2; ++n) {
-        const float* pi = img + (n * 8 + g) * DW_PLANE;
-        fb[n][0] = __float_as_uint(pi[o0]);
-        fb[n][1] = __float_as_uint(pi[o1]);
+        const uint32_t* pi = plane + (n * 8 + g) * DW_P_WORDS;
+        fb[n][0] = pi[w0];
+        fb[n][1] = pi[w1];
       }
 #pragma unroll
       for (int m = 0; m < 2; ++m)
 #pragma unroll
-        for (int n = 0; n < 2; ++n) mma_tf32(acc[m][n], fa[m], fb[n]);
+        for (int n = 0; n < 2; ++n) mma_bf16(acc[m][n], fa[m], fb[n]);
       if (ks % 9 == warp) {            // warp-uniform
-        mma_tf32(accb[0], fa[0], one_frag);
-        mma_tf32(accb[1], fa[1], one_frag);
+        mma_bf16(accb[0], fa[0], one_frag);
+        mma_bf16(accb[1], fa[1], one_frag);
       }
     }
   }
