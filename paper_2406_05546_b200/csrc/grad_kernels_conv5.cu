@@ -42,7 +42,7 @@ __device__ __forceinline__ bool loaders_sync_any(bool failed) {
 }
 
 struct Pipe {
-  uint64_t a_full[2], a_empty[2], acc_full[2], acc_empty[2];
+  uint64_t a_full[2], a_empty[2], acc_full[2], acc_empty[2], raw_full[2];
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -53,6 +53,7 @@ __device__ __forceinline__ void pipe_init(Pipe* p, int a_full_arrivals, int acc_
     mbar_init(&p->a_empty[i], 1);
     mbar_init(&p->acc_full[i], 1);
     mbar_init(&p->acc_empty[i], acc_empty_arrivals);
+    mbar_init(&p->raw_full[i], 1);
   }
   p->abort_flag = 0;
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -209,13 +210,15 @@ constexpr int X_PLANE_ROWS = 256 + 48;
 constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // 4864
 constexpr int X_BUF_BYTES = 8 * X_PLANE_BYTES;             // eight output-channel quads
 constexpr int X_W_BYTES = 72 * 16 * 16;                    // [k quad = tap*8 + oc/4][ic][4]
-constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + sizeof(Pipe) + 128;
+constexpr int X_RAW_BYTES = FLAT * 4 + FLAT;                // one sample's pooled gradients (fp32) and pooling decisions (bytes)
+constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + 2 * X_RAW_BYTES + sizeof(Pipe) + 128;
 
 __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   extern __shared__ __align__(128) uint8_t smem[];
   float* bufs = reinterpret_cast<float*>(smem);
   float* Wk = reinterpret_cast<float*>(smem + 2 * X_BUF_BYTES);
-  Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * X_BUF_BYTES + X_W_BYTES);
+  uint8_t* raw = smem + 2 * X_BUF_BYTES + X_W_BYTES;        // two raw staging slots filled by bulk copies
+  Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * X_BUF_BYTES + X_W_BYTES + 2 * X_RAW_BYTES);
   const int s = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const float* theta = group_theta(wt, gt, s);
   const int i_begin = blockIdx.x * C5_SPB, i_end = min(i_begin + C5_SPB, a.b);
@@ -268,42 +271,44 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
   } else if (warp <= 4) {
     const int lt = tid - 32;
     constexpr int PER = (FLAT + LOADERS - 1) / LOADERS;      // 13 pooled entries per thread
+    // The pooled gradients and decisions of a sample arrive in a raw slot by two bulk copies issued two
+    // tiles ahead, so no global-memory latency sits in this loop.
+    auto fetch_raw = [&](int t) {
+      const int64_t row = (int64_t)s * a.b + i_begin + t;
+      uint8_t* slot = raw + (t & 1) * X_RAW_BYTES;
+      mbar_expect_tx(&pipe->raw_full[t & 1], X_RAW_BYTES);
+      bulk_load(slot, ws.dp2 + row * FLAT, FLAT * 4, &pipe->raw_full[t & 1]);
+      bulk_load(slot + FLAT * 4, ws.code2 + row * FLAT, FLAT, &pipe->raw_full[t & 1]);
+    };
+    if (lt == 0) { fetch_raw(0); if (n_tiles > 1) fetch_raw(1); }
     for (int t = 0; t < n_tiles; ++t) {
       const int buf = t & 1;
-      const int64_t row = (int64_t)s * a.b + i_begin + t;
-      // decisions and pooled gradients are fetched before the wait for the buffer
-      int code[PER];
-      float gv[PER];
+      bool failed = !mbar_wait(&pipe->raw_full[buf], (t >> 1) & 1);
+      if (!failed && t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) failed = true;
+      // one uniform decision for all staging threads, so that none waits alone at a later barrier
+      if (loaders_sync_any(failed)) { pipe->abort_flag = 1; break; }
+      float* dst = bufs + buf * (X_BUF_BYTES / 4);
+      const float* rg = reinterpret_cast<const float*>(raw + buf * X_RAW_BYTES);
+      const uint8_t* rc = raw + buf * X_RAW_BYTES + FLAT * 4;
 #pragma unroll
       for (int k = 0; k < PER; ++k) {
         const int o = lt + k * LOADERS;
-        code[k] = o < FLAT ? (int)ws.code2[row * FLAT + o] : 4;
-        gv[k] = o < FLAT ? __ldg(ws.dp2 + row * FLAT + o) : 0.f;
-      }
-      bool failed = false;
-      if (t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) failed = true;
-      // one uniform decision for all staging threads, so that none waits alone at the barrier below
-      if (loaders_sync_any(failed)) { pipe->abort_flag = 1; break; }
-      float* dst = bufs + buf * (X_BUF_BYTES / 4);
-      if (t >= 2) {
-        // clear the interior (rows 16 .. 239 hold the 14x14 gradients of the sample staged two tiles ago)
-        for (int idx = lt; idx < 8 * 224; idx += LOADERS) {
-          int q = idx / 224, rr = idx - q * 224;
-          reinterpret_cast<float4*>(dst + q * (X_PLANE_BYTES / 4))[16 + rr] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-      }
-      loaders_sync_any(false);
-#pragma unroll
-      for (int k = 0; k < PER; ++k) {
-        if (code[k] < 4) {
-          const int o = lt + k * LOADERS;
-          int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
-          int y = 2 * py + (code[k] >> 1), x = 2 * px + (code[k] & 1);
-          dst[(oc >> 2) * (X_PLANE_BYTES / 4) + ((y + 1) * 16 + x + 1) * 4 + (oc & 3)] = round_tf32(gv[k]);
+        if (o < FLAT) {
+          // every pooled entry owns the four positions of its window: the gradient goes to the chosen one
+          // and the other three are cleared, so the planes need no separate clearing pass
+          const int code = rc[o];
+          const float v = round_tf32(rg[o]);
+          const int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
+          float* d = dst + (oc >> 2) * (X_PLANE_BYTES / 4) + ((2 * py + 1) * 16 + 2 * px + 1) * 4 + (oc & 3);
+          d[0] = code == 0 ? v : 0.f; d[4] = code == 1 ? v : 0.f;
+          d[64] = code == 2 ? v : 0.f; d[68] = code == 3 ? v : 0.f;
         }
       }
       fence_proxy_async_smem();
       mbar_arrive(&pipe->a_full[buf]);
+      // the raw slot may be refilled once every staging thread has read it
+      loaders_sync_any(false);
+      if (lt == 0 && t + 2 < n_tiles) fetch_raw(t + 2);
     }
   } else {
     const int quarter = warp & 3;
@@ -335,7 +340,10 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64) : "memory");
   }
-  if (tid == 0 && pipe->abort_flag) atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
+  if (tid == 0 && pipe->abort_flag) {
+    atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
+    for (int k = 0; k < 1000; ++k) __nanosleep(1000);   // let copies already issued land before the CTA ends
+  }
 }
 
 }  // namespace

@@ -46,7 +46,7 @@ constexpr int DW_THREADS = 288;
 constexpr int DW_KSTEPS = 13;      // 208 positions / 16
 constexpr int DW_QUADS = (4 * 196 + DW_THREADS - 1) / DW_THREADS;   // 3 four-channel positions per thread
 constexpr int DW_ENTRIES = (FLAT + DW_THREADS - 1) / DW_THREADS;    // 6 pooled gradient entries per thread
-__global__ void __launch_bounds__(DW_THREADS) conv2_dw_tc(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
+__global__ void __launch_bounds__(DW_THREADS, 2) conv2_dw_tc(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
   __shared__ __align__(16) uint32_t g2w[32 * DW_G_WORDS];        // [oc][position pair]
   __shared__ __align__(16) uint32_t imgw[2][16 * DW_P_WORDS];    // [copy][ic][(Y*16 + X - copy) / 2], zero border
   __shared__ float bias_part[9][32];
