@@ -485,6 +485,7 @@ __global__ void __launch_bounds__(256) conv2_bwd(GradStepArgs a, WorkerTable wt,
 // Thread (channel, lane of 16) owns 13 pooled positions of its channel.  The image, the pooling decisions
 // and the pooled gradients of the NEXT sample are fetched into registers while the current one is
 // accumulated, so that no global-memory latency sits between the multiply-adds.
+constexpr int CONV1B_SPB = 16;
 __global__ void __launch_bounds__(256) conv1_bwd(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
   __shared__ float xs[30][31];
   constexpr int PER = 13;                   // ceil(196 / 16)
@@ -494,8 +495,8 @@ __global__ void __launch_bounds__(256) conv1_bwd(GradStepArgs a, WorkerTable wt,
 #pragma unroll
   for (int k = 0; k < 9; ++k) gw[k] = 0.f;
   for (int t = tid; t < 30 * 31; t += 256) (&xs[0][0])[t] = 0.f;
-  const int i0 = blockIdx.x * CONV_SPB;
-  const int i1 = min(i0 + CONV_SPB, a.b);
+  const int i0 = blockIdx.x * CONV1B_SPB;
+  const int i1 = min(i0 + CONV1B_SPB, a.b);
   float xr[4], gr[PER];
   int cr[PER];
   auto prefetch = [&](int i) {
@@ -609,6 +610,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
   const int mt = group_tiles(gt, a.b, 64);
   const bool tc = a.precision != 0;
   const int n_chunks1 = (a.b + CONV1_SPB - 1) / CONV1_SPB;
+  const int n_chunks1b = (a.b + CONV1B_SPB - 1) / CONV1B_SPB;
   int launches = 0, n_chunks2 = n_chunks;
   if (tc) {
     TIMED(K_CONV1_FWD, (conv1_fwd<true><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
@@ -631,10 +633,10 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     n_chunks2 = launch_conv2_dw_tc(a, wt, ws, s2, prof);
     if (side.s2) cudaEventRecord(side.join2, s2);
     launch_conv2_dx_tc5(a, wt, gt, ws, st, prof);
-    TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
+    const int n_chunks1t = launch_conv1_bwd_tc(a, wt, ws, st, prof);
     if (side.s1) cudaStreamWaitEvent(st, side.join1, 0);
     if (side.s2) cudaStreamWaitEvent(st, side.join2, 0);
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks, n_chunks2)));
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks1t, n_chunks2)));
     launches += 4;
   } else {
     TIMED(K_CONV1_FWD, (conv1_fwd<false><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
@@ -644,8 +646,8 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
     TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
-    TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, ws, n_chunks)));
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks, n_chunks2)));
+    TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks1b, a.W), 256, 0, st>>>(a, wt, ws, n_chunks1b)));
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks1b, n_chunks2)));
     launches = 9;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;

@@ -185,6 +185,115 @@ __global__ void __launch_bounds__(DW_THREADS, 2) conv2_dw_tc(GradStepArgs a, Wor
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Filter gradient of the first convolution: dW[oc][tap] = sum_{samples,pos} da1[oc][pos] * x[pos + tap],
+// rows = 16 channels, columns = 9 taps (+ one column of ones for the bias gradient), k = the 784 positions
+// of a sample (49 k-steps of 16).  BF16 operands, fp32 accumulation; values only.  da1, the gradient at
+// the convolution's output, is written densely from the pooled gradient and the pooling decisions (each
+// pooled entry owns its 2x2 window).  The eight warps split the k-steps; their accumulators persist over
+// the block's samples and are combined in a fixed order at the end.
+// ------------------------------------------------------------------------------------------------
+constexpr int C1B_SPB = 16;
+constexpr int C1B_A_WORDS = 396;       // 392 position pairs per channel + 4: 396 = 12 (mod 32 banks)
+constexpr int C1B_X_WORDS = 15 * 32;   // bordered 30 x 32 image as bf16 pairs
+constexpr int C1B_ENTRIES = (P1_ELEMS + 255) / 256;   // 13 pooled entries per thread
+__global__ void __launch_bounds__(256) conv1_bwd_tc(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
+  __shared__ __align__(16) uint32_t da1w[16 * C1B_A_WORDS];
+  __shared__ __align__(16) uint32_t xw[2][C1B_X_WORDS + 16];   // copy 1 is shifted by one element
+  __shared__ float red[8][16][17];
+  uint16_t* xh[2] = {reinterpret_cast<uint16_t*>(xw[0]), reinterpret_cast<uint16_t*>(xw[1])};
+  const int s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+  for (int idx = tid; idx < 2 * (C1B_X_WORDS + 16); idx += 256) (&xw[0][0])[idx] = 0u;
+  for (int idx = tid; idx < 16 * C1B_A_WORDS; idx += 256) da1w[idx] = 0u;
+  // this lane's B columns: tile 0 column g = tap g; tile 1 column 0 = tap 8, column 1 = ones
+  const int ky0 = g / 3, kx0 = g - ky0 * 3;                  // tap g (g < 8)
+  const int copy0 = kx0 & 1;
+  const int off0 = ky0 * 32 + kx0 - copy0;                   // element offset of tap g in its copy (even)
+  const int off8 = 2 * 32 + 2;                               // tap 8 = (2, 2) in copy 0
+  float acc[2][4];
+#pragma unroll
+  for (int n = 0; n < 2; ++n)
+#pragma unroll
+    for (int r = 0; r < 4; ++r) acc[n][r] = 0.f;
+  const int i0 = blockIdx.x * C1B_SPB, i1 = min(i0 + C1B_SPB, a.b);
+
+  float xr[4], gr[C1B_ENTRIES];
+  int cr[C1B_ENTRIES];
+  auto prefetch = [&](int i) {
+    const int64_t row = (int64_t)s * a.b + i;
+    const float* x = a.x + ((int64_t)wt.src[s] * a.b + i) * (IMG * IMG);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) xr[k] = tid + 256 * k < IMG * IMG ? x[tid + 256 * k] : 0.f;
+#pragma unroll
+    for (int k = 0; k < C1B_ENTRIES; ++k) {
+      const int o = tid + 256 * k;
+      cr[k] = o < P1_ELEMS ? (int)ws.code1[row * P1_ELEMS + o] : 4;
+      gr[k] = o < P1_ELEMS ? ws.dp1[row * P1_ELEMS + o] : 0.f;
+    }
+  };
+  prefetch(i0);
+  for (int i = i0; i < i1; ++i) {
+    __syncthreads();                        // the previous sample's products are done with shared memory
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int e = tid + 256 * k;
+      if (e < IMG * IMG) {
+        const int yy = e / IMG, xx = e - yy * IMG, el = (yy + 1) * 32 + xx + 1;
+        const uint16_t h = bf16_bits(xr[k]);
+        xh[0][el] = h;
+        xh[1][el - 1] = h;
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < C1B_ENTRIES; ++k) {
+      const int o = tid + 256 * k;
+      if (o < P1_ELEMS) {
+        const int oc = o / 196, p = o - oc * 196, py = p / 14, px = p - py * 14;
+        uint32_t* d = da1w + oc * C1B_A_WORDS + py * 28 + px;     // pair of positions (2py, 2px), (2py, 2px+1)
+        const float v = gr[k];
+        d[0] = bf16_pair(cr[k] == 0 ? v : 0.f, cr[k] == 1 ? v : 0.f);
+        d[14] = bf16_pair(cr[k] == 2 ? v : 0.f, cr[k] == 3 ? v : 0.f);
+      }
+    }
+    __syncthreads();
+    if (i + 1 < i1) prefetch(i + 1);
+    for (int ks = warp; ks < 49; ks += 8) {
+      const int j0 = ks * 8 + t, j1 = j0 + 4;               // position pairs of this lane's k columns
+      uint32_t fa[4], fb[2][2];
+      fa[0] = da1w[g * C1B_A_WORDS + j0];
+      fa[1] = da1w[(g + 8) * C1B_A_WORDS + j0];
+      fa[2] = da1w[g * C1B_A_WORDS + j1];
+      fa[3] = da1w[(g + 8) * C1B_A_WORDS + j1];
+      const int y0 = j0 / 14, x0 = 2 * (j0 - y0 * 14), y1 = j1 / 14, x1 = 2 * (j1 - y1 * 14);
+      const int e0 = y0 * 32 + x0, e1 = y1 * 32 + x1;       // bordered element (y, x) of tap (0, 0)
+      fb[0][0] = xw[copy0][(e0 + off0) >> 1];
+      fb[0][1] = xw[copy0][(e1 + off0) >> 1];
+      const uint32_t t8a = xw[0][(e0 + off8) >> 1], t8b = xw[0][(e1 + off8) >> 1];
+      fb[1][0] = g == 0 ? t8a : (g == 1 ? 0x3F803F80u : 0u);
+      fb[1][1] = g == 0 ? t8b : (g == 1 ? 0x3F803F80u : 0u);
+      mma_bf16(acc[0], fa, fb[0]);
+      mma_bf16(acc[1], fa, fb[1]);
+    }
+  }
+  // c0 (row g, col 2t), c1 (g, 2t+1), c2 (g+8, 2t), c3 (g+8, 2t+1); columns 0..7 = taps, 8 = tap 8, 9 = bias
+#pragma unroll
+  for (int n = 0; n < 2; ++n) {
+    red[warp][g][n * 8 + 2 * t] = acc[n][0];
+    red[warp][g][n * 8 + 2 * t + 1] = acc[n][1];
+    red[warp][g + 8][n * 8 + 2 * t] = acc[n][2];
+    red[warp][g + 8][n * 8 + 2 * t + 1] = acc[n][3];
+  }
+  __syncthreads();
+  if (tid < 160) {
+    const int oc = tid / 10, col = tid - oc * 10;
+    float sum = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) sum += red[w][oc][col];
+    float* part = ws.part1 + ((int64_t)s * n_chunks + blockIdx.x) * C1_GRAD;
+    part[col < 9 ? oc * 9 + col : 144 + oc] = sum;
+  }
+}
+
 }  // namespace
 
 #define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
@@ -195,6 +304,12 @@ int configure_tc_kernels() { return 0; }
 int launch_conv2_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof) {
   const int chunks = (a.b + TC_SPB - 1) / TC_SPB;
   TIMED(K_CONV2_DW, (conv2_dw_tc<<<dim3(chunks, a.W), DW_THREADS, 0, st>>>(a, wt, ws, chunks)));
+  return chunks;
+}
+
+int launch_conv1_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof) {
+  const int chunks = (a.b + C1B_SPB - 1) / C1B_SPB;
+  TIMED(K_CONV1_BWD, (conv1_bwd_tc<<<dim3(chunks, a.W), 256, 0, st>>>(a, wt, ws, chunks)));
   return chunks;
 }
 

@@ -137,6 +137,7 @@ int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, ui
                         uint8_t* keep, cudaStream_t st, Profiler* prof);
 int configure_grad_kernels();
 int configure_tc_kernels();
+int launch_conv1_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof);
 int launch_conv2_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof);
 int configure_tc5_kernels();
 int configure_conv5_kernels();
