@@ -30,6 +30,14 @@ constexpr int LOADERS = 128;
 __host__ __device__ constexpr uint32_t idesc_tf32(int m, int n) {
   return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
+__host__ __device__ constexpr uint32_t idesc_bf16(int m, int n) {     // fp32 accumulate, BF16 x BF16, k-contiguous
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ uint16_t bf16_bits(float x) {
+  uint16_t r;
+  asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(x));
+  return r;
+}
 
 // Barrier over the 128 staging threads that also tells every one of them whether any of them failed.
 __device__ __forceinline__ bool loaders_sync_any(bool failed) {
@@ -203,20 +211,22 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
 // ------------------------------------------------------------------------------------------------
 // Gradient with respect to the convolution's input.  Tile = one sample = two 128-row blocks of the
 // 16-wide position grid (row = y*16 + x; y, x >= 14 are padding rows).  g2, the gradient at the
-// convolution's output, is scattered from the pooled gradient by the stored pooling decisions into
-// zero-bordered planes of four output channels; tap (ky, kx) reads them shifted by (2-ky)*16 + (2-kx) rows.
+// convolution's output, is written from the pooled gradient and the stored pooling decisions into
+// zero-bordered planes of EIGHT output channels in BF16 (one position = one 16-byte row); tap (ky, kx)
+// reads them shifted by (2-ky)*16 + (2-kx) rows.  BF16 operands, fp32 accumulation: this product only
+// yields gradient values, and at K = 16 per instruction it needs half the MMAs and half the operand bytes.
 // ------------------------------------------------------------------------------------------------
 constexpr int X_PLANE_ROWS = 256 + 48;
 constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // 4864
-constexpr int X_BUF_BYTES = 8 * X_PLANE_BYTES;             // eight output-channel quads
-constexpr int X_W_BYTES = 72 * 16 * 16;                    // [k quad = tap*8 + oc/4][ic][4]
+constexpr int X_BUF_BYTES = 4 * X_PLANE_BYTES;             // four planes of eight output channels
+constexpr int X_W_BYTES = 36 * 16 * 16;                    // [k chunk = tap*4 + oc/8][ic][8 bf16]
 constexpr int X_RAW_BYTES = FLAT * 4 + FLAT;                // one sample's pooled gradients (fp32) and pooling decisions (bytes)
 constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + 2 * X_RAW_BYTES + sizeof(Pipe) + 128;
 
 __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   extern __shared__ __align__(128) uint8_t smem[];
-  float* bufs = reinterpret_cast<float*>(smem);
-  float* Wk = reinterpret_cast<float*>(smem + 2 * X_BUF_BYTES);
+  uint16_t* bufs = reinterpret_cast<uint16_t*>(smem);
+  uint16_t* Wk = reinterpret_cast<uint16_t*>(smem + 2 * X_BUF_BYTES);
   uint8_t* raw = smem + 2 * X_BUF_BYTES + X_W_BYTES;        // two raw staging slots filled by bulk copies
   Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * X_BUF_BYTES + X_W_BYTES + 2 * X_RAW_BYTES);
   const int s = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -226,9 +236,9 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
 
   for (int idx = tid; idx < 4608; idx += THREADS) {
     int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
-    Wk[((tap * 8 + (oc >> 2)) * 16 + ic) * 4 + (oc & 3)] = round_tf32(theta[OFF_C2W + idx]);
+    Wk[((tap * 4 + (oc >> 3)) * 16 + ic) * 8 + (oc & 7)] = bf16_bits(theta[OFF_C2W + idx]);
   }
-  for (int idx = tid; idx < 2 * X_BUF_BYTES / 16; idx += THREADS) reinterpret_cast<float4*>(bufs)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int idx = tid; idx < 2 * X_BUF_BYTES / 16; idx += THREADS) reinterpret_cast<float4*>(smem)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
   if (tid == 0) pipe_init(pipe, LOADERS, 4);
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(64) : "memory");
@@ -242,7 +252,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
 
   if (warp == 0) {
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_tf32(128, 16);
+      constexpr uint32_t idesc = idesc_bf16(128, 16);
       const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), 256);
       for (int t = 0; t < n_tiles; ++t) {
         const int buf = t & 1;
@@ -250,7 +260,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
         if (t >= 2 && !mbar_wait(&pipe->acc_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
         if (pipe->abort_flag) break;
         tc_fence_after();
-        const uint32_t a_lo = plain_desc_lo(smem_u32(bufs) + buf * X_BUF_BYTES, X_PLANE_BYTES);
+        const uint32_t a_lo = plain_desc_lo(smem_u32(smem) + buf * X_BUF_BYTES, X_PLANE_BYTES);
         const uint32_t d_tmem = tmem + buf * 32;
 #pragma unroll
         for (int m = 0; m < 2; ++m) {
@@ -259,9 +269,9 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
             const int ky = tap / 3, kx = tap - ky * 3;
             const int row_off = m * 128 + (2 - ky) * 16 + (2 - kx);           // in 16-byte rows
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-              umma_tf32_split(d_tmem + m * 16, a_lo + (2 * q) * (X_PLANE_BYTES / 16) + row_off, plain_desc_hi(128),
-                              w_lo + (tap * 8 + q * 2) * (256 / 16), plain_desc_hi(128), idesc, (tap | q) ? 1u : 0u);
+            for (int q = 0; q < 2; ++q)                                        // 16 output channels per MMA
+              umma_f16_split(d_tmem + m * 16, a_lo + (2 * q) * (X_PLANE_BYTES / 16) + row_off, plain_desc_hi(128),
+                             w_lo + (tap * 4 + q * 2) * (256 / 16), plain_desc_hi(128), idesc, (tap | q) ? 1u : 0u);
           }
         }
         umma_commit(&pipe->a_empty[buf]);
@@ -287,7 +297,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
       if (!failed && t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) failed = true;
       // one uniform decision for all staging threads, so that none waits alone at a later barrier
       if (loaders_sync_any(failed)) { pipe->abort_flag = 1; break; }
-      float* dst = bufs + buf * (X_BUF_BYTES / 4);
+      uint16_t* dst = bufs + buf * (X_BUF_BYTES / 2);
       const float* rg = reinterpret_cast<const float*>(raw + buf * X_RAW_BYTES);
       const uint8_t* rc = raw + buf * X_RAW_BYTES + FLAT * 4;
 #pragma unroll
@@ -297,11 +307,11 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
           // every pooled entry owns the four positions of its window: the gradient goes to the chosen one
           // and the other three are cleared, so the planes need no separate clearing pass
           const int code = rc[o];
-          const float v = round_tf32(rg[o]);
+          const uint16_t v = bf16_bits(rg[o]);
           const int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
-          float* d = dst + (oc >> 2) * (X_PLANE_BYTES / 4) + ((2 * py + 1) * 16 + 2 * px + 1) * 4 + (oc & 3);
-          d[0] = code == 0 ? v : 0.f; d[4] = code == 1 ? v : 0.f;
-          d[64] = code == 2 ? v : 0.f; d[68] = code == 3 ? v : 0.f;
+          uint16_t* d = dst + (oc >> 3) * (X_PLANE_BYTES / 2) + ((2 * py + 1) * 16 + 2 * px + 1) * 8 + (oc & 7);
+          d[0] = code == 0 ? v : (uint16_t)0; d[8] = code == 1 ? v : (uint16_t)0;
+          d[128] = code == 2 ? v : (uint16_t)0; d[136] = code == 3 ? v : (uint16_t)0;
         }
       }
       fence_proxy_async_smem();
