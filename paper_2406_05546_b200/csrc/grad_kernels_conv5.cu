@@ -216,8 +216,8 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
 // reads them shifted by (2-ky)*16 + (2-kx) rows.  BF16 operands, fp32 accumulation: this product only
 // yields gradient values, and at K = 16 per instruction it needs half the MMAs and half the operand bytes.
 // ------------------------------------------------------------------------------------------------
-constexpr int X_PLANE_ROWS = 256 + 48;
-constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // 4864
+constexpr int X_PLANE_ROWS = 256 + 50;                     // 34 rows of tap overrun; 306 rows = 32 bytes (mod 128): the
+constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // four planes then start in different shared-memory banks
 constexpr int X_BUF_BYTES = 4 * X_PLANE_BYTES;             // four planes of eight output channels
 constexpr int X_W_BYTES = 36 * 16 * 16;                    // [k chunk = tap*4 + oc/8][ic][8 bf16]
 constexpr int X_RAW_BYTES = FLAT * 4 + FLAT;                // one sample's pooled gradients (fp32) and pooling decisions (bytes)
@@ -300,15 +300,19 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
       uint16_t* dst = bufs + buf * (X_BUF_BYTES / 2);
       const float* rg = reinterpret_cast<const float*>(raw + buf * X_RAW_BYTES);
       const uint8_t* rc = raw + buf * X_RAW_BYTES + FLAT * 4;
+      // Entry e = lt + 128 k is (pooled position e / 32, output channel e % 32): the 32 lanes of a warp write
+      // the 32 channels of one position (64 contiguous bytes spread over the four planes, no bank conflict)
+      // and read the raw slot at a stride of 49 words (odd, no conflict either).
 #pragma unroll
       for (int k = 0; k < PER; ++k) {
-        const int o = lt + k * LOADERS;
-        if (o < FLAT) {
+        const int e = lt + k * LOADERS;
+        if (e < FLAT) {
           // every pooled entry owns the four positions of its window: the gradient goes to the chosen one
           // and the other three are cleared, so the planes need no separate clearing pass
+          const int p = e >> 5, oc = e & 31, o = oc * 49 + p;
           const int code = rc[o];
           const uint16_t v = bf16_bits(rg[o]);
-          const int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
+          const int py = p / 7, px = p - py * 7;
           uint16_t* d = dst + (oc >> 3) * (X_PLANE_BYTES / 2) + ((2 * py + 1) * 16 + 2 * px + 1) * 8 + (oc & 7);
           d[0] = code == 0 ? v : (uint16_t)0; d[8] = code == 1 ? v : (uint16_t)0;
           d[128] = code == 2 ? v : (uint16_t)0; d[136] = code == 3 ? v : (uint16_t)0;
