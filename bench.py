@@ -172,6 +172,7 @@ def main():
 
     import torch
     from paper_2406_05546_b200 import ps, synth
+    from paper_2406_05546_b200.ranks import Ranks
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -182,22 +183,8 @@ def main():
     if rank == 0 and world == 1:
         cpu = cpu_baseline()
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(v):
-        if dist is None:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    ranks = Ranks("nccl")
+    barrier, max_over_ranks = ranks.barrier, ranks.max_over_ranks
 
     W, b = W_WORKERS, BATCH
     K_replay = DOWN_TICKS * W
@@ -210,7 +197,7 @@ def main():
     pool_x, pool_y = torch.from_numpy(px).cuda(), torch.from_numpy(py).cuda()
     bufs = []
     for t in range(N_BATCH_BUFFERS):
-        rows = torch.from_numpy(synth.batch_rows(t + rank * 1000, W, b, px.shape[0])).cuda()
+        rows = torch.from_numpy(synth.batch_rows(ranks.batch_seed(t), W, b, px.shape[0])).cuda()
         bufs.append((pool_x[rows].contiguous(), pool_y[rows].contiguous()))
     loss_dev = torch.empty(W, dtype=torch.float32, device="cuda")
     am_dev = torch.empty((W, b), dtype=torch.int32, device="cuda")
@@ -302,8 +289,7 @@ def main():
     stats = srv.ps_stats()
 
     if rank == 0:
-        samples = W * b * args.steps * world
-        value = samples / (ms_total * 1e-3)
+        value = ranks.whole_job_rate(W * b * args.steps, ms_total)
         total_prof = sum(ms for ms, _ in prof.values()) or 1.0
         kernels = {k: {"ms_per_launch": ms / n, "launches": n, "share": ms / total_prof}
                    for k, (ms, n) in prof.items() if n}
@@ -342,8 +328,7 @@ def main():
         }
         print(json.dumps(out))
     srv.close()
-    if dist is not None:
-        dist.destroy_process_group()
+    ranks.close()
 
 
 def kernel_roofline(name, ms_per_launch, W, b, peaks, precision):

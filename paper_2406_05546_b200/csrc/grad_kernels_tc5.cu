@@ -1,6 +1,6 @@
 // The three products of the 512-unit dense layer on the fifth-generation tensor cores:
 // tcgen05.mma (kind::tf32) issued by one thread, operands brought into 128-byte-swizzled shared
-// memory by TMA (cp.async.bulk.tensor, no multicast), accumulators in tensor memory, read back with
+// memory by TMA (cp.async.bulk.tensor, each CTA loading its own tiles), accumulators in tensor memory, read back with
 // tcgen05.ld for the epilogue.
 //
 // All three are "both operands k-contiguous" products C[m][n] = sum_k A[m][k] * B[n][k]:

@@ -1,5 +1,5 @@
 // PTX wrappers for the fifth-generation tensor-core path: mbarriers with bounded waits, TMA tile
-// loads (no multicast), tcgen05 MMA / commit / tensor-memory loads.
+// loads (each CTA loads its own tiles), tcgen05 MMA / commit / tensor-memory loads.
 #pragma once
 #include <cuda.h>
 #include <stdint.h>
