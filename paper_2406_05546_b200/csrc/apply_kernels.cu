@@ -133,7 +133,7 @@ const char* kernel_name(int id) {
   static const char* names[K_COUNT] = {
       "conv1_fwd", "conv2_fwd", "fc1_fwd", "fc2_fwd_bwd", "fc1_dw", "fc1_dx", "conv2_bwd", "conv1_bwd",
       "conv_grad_reduce", "sum_apply_direct", "sum_partial", "sum_finish", "async_apply", "copy_rows",
-      "dropout_mask", "conv2_dw", "prep_w1", "transpose_rows"};
+      "dropout_mask", "conv2_dw", "prep_w1"};
   return id >= 0 && id < K_COUNT ? names[id] : "?";
 }
 

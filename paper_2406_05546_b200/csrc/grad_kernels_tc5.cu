@@ -3,12 +3,14 @@
 // memory by TMA (cp.async.bulk.tensor, each CTA loading its own tiles), accumulators in tensor memory, read back with
 // tcgen05.ld for the epilogue.
 //
-// All three are "both operands k-contiguous" products C[m][n] = sum_k A[m][k] * B[n][k]:
+// Two are "both operands k-contiguous" products C[m][n] = sum_k A[m][k] * B[n][k]:
 //   forward          A = p2 [rows][1568]            B = W1 [512][1568]           (per weight group)
 //   input gradient   A = dA1 [rows][512]            B = W1^T [1568][512]         (per weight group)
-//   weight gradient  A = dA1^T of a worker [512][b] B = p2^T of that worker [1568][b]
-// The transposed copies are made by small kernels below; every operand is rounded to TF32 by its
-// producer, so the tensor core's own handling of the low mantissa bits cannot change a result.
+// The weight gradient of a worker, C[m][n] = sum_k dA1[k][m] * p2[k][n] over the worker's samples k, reads
+// both operands as they lie in memory (m and n contiguous, one row per sample): the tensor core takes them
+// "MN-major", so no transposed copy is made.
+// Every operand is rounded to TF32 by its producer, so the tensor core's own handling of the low mantissa
+// bits cannot change a result.
 //
 // Every wait on an mbarrier is bounded: when a bound is exceeded the kernel raises a status flag,
 // stops issuing work, frees its tensor memory and returns.
@@ -44,9 +46,27 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
   return d;
 }
 
-// Instruction descriptor: fp32 accumulate, TF32 x TF32, both operands k-contiguous, tile M x N.
-__host__ __device__ constexpr uint32_t instr_desc_tf32(int m, int n) {
-  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+// Shared-memory matrix descriptor of a 32-bit operand whose m (or n) index is contiguous.  The only layout the
+// tensor core takes for it is the 128-byte swizzle with 32-byte atoms (layout type 1): the tile is a row of
+// blocks of 32 columns; inside a block the k-th row (one sample) is 128 bytes, and the four 32-byte pieces of
+// a row are permuted by the row index modulo 4.  Blocks are `block_bytes` apart (leading byte offset),
+// groups of four rows 512 bytes apart (stride byte offset).  TMA writes the same pattern with
+// CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t block_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)(block_bytes >> 4) << 16;
+  d |= (uint64_t)(512 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)1 << 61;
+  return d;
+}
+
+// Instruction descriptor: fp32 accumulate, TF32 x TF32, tile M x N; bits 15 / 16 say that A / B are stored
+// with their m / n index contiguous instead of k.
+__host__ __device__ constexpr uint32_t instr_desc_tf32(int m, int n, bool mn_major = false) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | (mn_major ? (3u << 15) : 0u) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(m >> 4) << 24);
 }
 
 // Tensor maps of one launch, passed by value in the kernel's parameter space.
@@ -91,7 +111,7 @@ __device__ __forceinline__ bool decode_tile(int t, const GemmArgs& ga, const Gro
   return locate_group_tile<BM>(gt, b, rest, c.grp, c.m0, c.m_end);
 }
 
-template <int EPI, int BN>
+template <int EPI, int BN, bool MN = false>
 __global__ void __launch_bounds__(192, 1) tc5_gemm(const __grid_constant__ GemmMaps maps, GemmArgs ga, GradStepArgs a,
                                                    WorkerTable wt, GroupTable gt, Workspace ws) {
   constexpr int STAGES = MAX_STAGES;
@@ -141,15 +161,20 @@ __global__ void __launch_bounds__(192, 1) tc5_gemm(const __grid_constant__ GemmM
           if (it >= STAGES && !mbar_wait(&empty[s], ((it / STAGES) - 1) & 1)) { *abort_flag = 1; ok = false; break; }
           if (*abort_flag) { ok = false; break; }
           mbar_expect_tx(&full[s], STAGE_BYTES);
-          tma_load_3d(tiles + s * STAGE_BYTES, map_a, &full[s], kb * BK, c.m0, c.z);
-          tma_load_3d(tiles + s * STAGE_BYTES + A_BYTES, map_b, &full[s], kb * BK, c.n0, c.z);
+          if (MN) {      // boxes of {32 columns, BK samples, BM/32 or BN/32 column blocks} of worker z
+            tma_load_4d(tiles + s * STAGE_BYTES, map_a, &full[s], 0, kb * BK, c.m0 / 32, c.z);
+            tma_load_4d(tiles + s * STAGE_BYTES + A_BYTES, map_b, &full[s], 0, kb * BK, c.n0 / 32, c.z);
+          } else {
+            tma_load_3d(tiles + s * STAGE_BYTES, map_a, &full[s], kb * BK, c.m0, c.z);
+            tma_load_3d(tiles + s * STAGE_BYTES + A_BYTES, map_b, &full[s], kb * BK, c.n0, c.z);
+          }
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc_tf32(BM, BN);
-      const uint32_t desc_hi = (uint32_t)(smem_desc_sw128(0) >> 32);
+      constexpr uint32_t idesc = instr_desc_tf32(BM, BN, MN);
+      const uint32_t desc_hi = (uint32_t)((MN ? smem_desc_mn_sw128(0, 0) : smem_desc_sw128(0)) >> 32);
       int it = 0, tile_i = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < ga.n_tiles && ok; t += gridDim.x) {
@@ -162,11 +187,16 @@ __global__ void __launch_bounds__(192, 1) tc5_gemm(const __grid_constant__ GemmM
           const int s = it % STAGES;
           if (!mbar_wait(&full[s], (it / STAGES) & 1) || *abort_flag) { *abort_flag = 1; ok = false; break; }
           tc_fence_after();
-          const uint32_t a_lo = (uint32_t)smem_desc_sw128(base + s * STAGE_BYTES);
-          const uint32_t b_lo = (uint32_t)smem_desc_sw128(base + s * STAGE_BYTES + A_BYTES);
+          // k-contiguous operands: eight k = 32 bytes along the swizzled row; m/n-contiguous operands: eight k
+          // = eight 128-byte rows.  (Descriptor addresses count 16-byte units.)
+          const uint32_t a_lo = MN ? (uint32_t)smem_desc_mn_sw128(base + s * STAGE_BYTES, BK * 128)
+                                   : (uint32_t)smem_desc_sw128(base + s * STAGE_BYTES);
+          const uint32_t b_lo = MN ? (uint32_t)smem_desc_mn_sw128(base + s * STAGE_BYTES + A_BYTES, BK * 128)
+                                   : (uint32_t)smem_desc_sw128(base + s * STAGE_BYTES + A_BYTES);
+          constexpr uint32_t K_STEP = MN ? 1024 / 16 : 32 / 16;
 #pragma unroll
           for (int k = 0; k < BK / 8; ++k)
-            umma_tf32_split(tmem_acc + ab * BN, a_lo + k * 2, desc_hi, b_lo + k * 2, desc_hi, idesc, (kb | k) ? 1u : 0u);
+            umma_tf32_split(tmem_acc + ab * BN, a_lo + k * K_STEP, desc_hi, b_lo + k * K_STEP, desc_hi, idesc, (kb | k) ? 1u : 0u);
           umma_commit(&empty[s]);            // the stage may be refilled once these MMAs have read it
         }
         if (ok) umma_commit(&acc_full[ab]);
@@ -269,20 +299,6 @@ __global__ void __launch_bounds__(256) prep_w1(GroupTable gt, float* __restrict_
   for (int i = ty; i < 32; i += 8) dt[(int64_t)(c0 + i) * HID + r0 + tx] = tile[tx][i];
 }
 
-// Per-worker transpose with TF32 rounding: src [W][b][F] -> dst [W][F][bp] (bp = b rounded up to 4).
-__global__ void __launch_bounds__(256) transpose_rows(const float* __restrict__ src, float* __restrict__ dst, int b, int bp, int F) {
-  __shared__ float tile[32][33];
-  const int s = blockIdx.z, f0 = blockIdx.x * 32, i0 = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  const float* sp = src + (int64_t)s * b * F;
-  float* dp = dst + (int64_t)s * F * bp;
-  for (int i = ty; i < 32; i += 8)
-    tile[i][tx] = (i0 + i < b && f0 + tx < F) ? rna_tf32(sp[(int64_t)(i0 + i) * F + f0 + tx]) : 0.f;
-  __syncthreads();
-  for (int i = ty; i < 32; i += 8)
-    if (f0 + i < F && i0 + tx < bp) dp[(int64_t)(f0 + i) * bp + i0 + tx] = tile[tx][i];
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -298,6 +314,19 @@ bool make_map(CUtensorMap* m, const float* base, uint64_t d0, uint64_t d1, uint6
   CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// One worker's [b][F] rows as {32 columns, b samples, F/32 column blocks, W workers}; box {32, BK, blocks, 1}.
+// Samples beyond b are out of bounds in their own dimension and arrive as zeros.
+bool make_map_mn(CUtensorMap* m, const float* base, uint64_t F, uint64_t b, uint64_t W, uint32_t box_blocks) {
+  cuuint64_t dims[4] = {32, b, F / 32, W};
+  cuuint64_t strides[3] = {F * 4, 128, b * F * 4};
+  cuuint32_t box[4] = {32, BK, box_blocks, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
@@ -319,6 +348,7 @@ int configure_tc5_kernels() {
       cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_sm_count <= 0) return -1;
   cudaError_t e = cudaFuncSetAttribute(tc5_gemm<EPI_FC1_FWD, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(256, MAX_STAGES));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES));
   return e == cudaSuccess ? 0 : -1;
 }
 
@@ -354,16 +384,13 @@ int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupT
 
 int launch_fc1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                       cudaStream_t st, Profiler* prof) {
-  const int bp = (a.b + 3) & ~3;
-  TIMED(K_TRANSPOSE, (transpose_rows<<<dim3(HID / 32, (bp + 31) / 32, a.W), 256, 0, st>>>(ws.da1, ws.da1t, a.b, bp, HID)));
-  TIMED(K_TRANSPOSE, (transpose_rows<<<dim3(FLAT / 32, (bp + 31) / 32, a.W), 256, 0, st>>>(ws.p2, ws.p2t, a.b, bp, FLAT)));
   GemmMaps maps;
-  if (!make_map(&maps.a, ws.da1t, a.b, HID, a.W, bp, (uint64_t)HID * bp, BM)) return -1;
-  if (!make_map(&maps.b[0], ws.p2t, a.b, FLAT, a.W, bp, (uint64_t)FLAT * bp, 224)) return -1;
+  if (!make_map_mn(&maps.a, ws.da1, HID, a.b, a.W, BM / 32)) return -1;
+  if (!make_map_mn(&maps.b[0], ws.p2, FLAT, a.b, a.W, 224 / 32)) return -1;
   GemmArgs ga{a.b, FLAT, FLAT, 1, nullptr, FLAT / 224, (FLAT / 224) * (HID / BM) * a.W};
   const int grid = ga.n_tiles < g_sm_count ? ga.n_tiles : g_sm_count;
-  TIMED(K_FC1_DW, (tc5_gemm<EPI_STORE, 224><<<grid, 192, gemm_smem_bytes(224, MAX_STAGES), st>>>(maps, ga, a, wt, gt, ws)));
-  return 3;
+  TIMED(K_FC1_DW, (tc5_gemm<EPI_STORE, 224, true><<<grid, 192, gemm_smem_bytes(224, MAX_STAGES), st>>>(maps, ga, a, wt, gt, ws)));
+  return 1;
 }
 
 }  // namespace psk

@@ -34,7 +34,7 @@ constexpr uint32_t STATUS_WAIT_TIMEOUT = 2u;   // a bounded barrier wait in a te
 enum KernelId {
   K_CONV1_FWD = 0, K_CONV2_FWD, K_FC1_FWD, K_FC2_FWD_BWD, K_FC1_DW, K_FC1_DX, K_CONV2_BWD, K_CONV1_BWD,
   K_CONV_GRAD_REDUCE, K_SUM_APPLY_DIRECT, K_SUM_PARTIAL, K_SUM_FINISH, K_ASYNC_APPLY, K_COPY_ROWS,
-  K_DROPOUT_MASK, K_CONV2_DW, K_PREP_W1, K_TRANSPOSE, K_COUNT
+  K_DROPOUT_MASK, K_CONV2_DW, K_PREP_W1, K_COUNT
 };
 const char* kernel_name(int id);
 
@@ -106,8 +106,6 @@ struct Workspace {
   float* part1;    // [W][chunks][160]    per-block partial conv1 weight/bias gradients
   float* w1r;      // [groups][512][1568] TF32-rounded fc1 weights of each weight group of the call
   float* w1tr;     // [groups][1568][512] and their transpose
-  float* da1t;     // [W][512][bp]        per-worker transpose of da1 (bp = batch rounded up to 4)
-  float* p2t;      // [W][1568][bp]       per-worker transpose of p2
   uint32_t* status;
 };
 

@@ -138,14 +138,11 @@ void layout(ps_ctx* x, const ps_config& c, void* arena, void* pinned, uint64_t* 
   ws.part2 = a.take<float>((uint64_t)c.max_workers * chunks * psk::C2_GRAD * 4);
   ws.part1 = a.take<float>((uint64_t)c.max_workers * chunks * psk::C1_GRAD * 4);
   ws.status = a.take<uint32_t>(ALIGN);
-  ws.w1r = ws.w1tr = ws.da1t = ws.p2t = nullptr;
+  ws.w1r = ws.w1tr = nullptr;
   if (c.precision != PS_FP32) {
     const uint64_t groups = std::min<uint64_t>(psk::MAX_GROUPS, std::min<uint64_t>(c.max_workers, c.ring_depth));
-    const uint64_t bp = ((uint64_t)c.max_batch + 3) / 4 * 4;
     ws.w1r = a.take<float>(groups * psk::HID * psk::FLAT * 4);
     ws.w1tr = a.take<float>(groups * psk::HID * psk::FLAT * 4);
-    ws.da1t = a.take<float>((uint64_t)c.max_workers * psk::HID * bp * 4);
-    ws.p2t = a.take<float>((uint64_t)c.max_workers * psk::FLAT * bp * 4);
   }
   float* x_stage = a.take<float>(rows * PS_IMAGE_PIXELS * 4);
   int32_t* y_stage = a.take<int32_t>(rows * 4);
