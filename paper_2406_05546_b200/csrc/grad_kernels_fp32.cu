@@ -259,108 +259,148 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // ---- fc2 forward, softmax cross-entropy, argmax, and the backward pass down to the gradient with
 // respect to fc1's pre-activation; then the worker's fc2 weight/bias and fc1 bias gradients.
-// One block per worker, one warp per sample at a time.
-__global__ void __launch_bounds__(256) fc2_fwd_bwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+// One block of 16 warps per worker: first one warp per sample at a time; then thread = hidden unit sums its
+// outputs over the worker's samples in sample order, several loads in flight.
+constexpr int FC2_THREADS = 512;
+__global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   __shared__ float w2[NCLS][HID];
   __shared__ float b2[NCLS];
-  __shared__ float warp_loss[8];
+  __shared__ float warp_loss[FC2_THREADS / 32];
   const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* theta = group_theta(wt, gt, s);
   const int src = wt.src[s];
-  for (int t = tid; t < NCLS * HID; t += 256) (&w2[0][0])[t] = theta[OFF_F2W + t];
+  for (int t = tid; t < NCLS * HID; t += FC2_THREADS) (&w2[0][0])[t] = theta[OFF_F2W + t];
   if (tid < NCLS) b2[tid] = theta[OFF_F2B + tid];
   __syncthreads();
   const float scale = 1.0f / (1.0f - a.drop_p);
   const float inv_b = 1.0f / (float)a.b;
   float loss_acc = 0.f;
-  for (int i = warp; i < a.b; i += 8) {
-    const int64_t row = (int64_t)s * a.b + i;
-    float dv[16];
-#pragma unroll
-    for (int t = 0; t < 16; ++t) dv[t] = ws.d[row * HID + lane + 32 * t];
-    float z[NCLS];
-#pragma unroll
-    for (int c = 0; c < NCLS; ++c) {
-      float p = 0.f;
-#pragma unroll
-      for (int t = 0; t < 16; ++t) p = fmaf(w2[c][lane + 32 * t], dv[t], p);
-      z[c] = warp_sum(p) + b2[c];
-    }
-    float zmax = z[0];
-    int am = 0;
-#pragma unroll
-    for (int c = 1; c < NCLS; ++c)
-      if (z[c] > zmax) { zmax = z[c]; am = c; }
-    float se = 0.f;
-#pragma unroll
-    for (int c = 0; c < NCLS; ++c) se += expf(z[c] - zmax);
-    const float lse = zmax + logf(se);
-    int label = a.y[(int64_t)src * a.b + i];
-    if (label < 0 || label >= NCLS) {
-      if (lane == 0) atomicOr(ws.status, STATUS_BAD_LABEL);
-      label = 0;
-    }
-    float zy = 0.f, dz[NCLS];
-#pragma unroll
-    for (int c = 0; c < NCLS; ++c) {
-      if (c == label) zy = z[c];
-      dz[c] = (expf(z[c] - lse) - (c == label ? 1.f : 0.f)) * inv_b;
-    }
-    loss_acc += lse - zy;
-    if (lane == 0) a.argmax[(int64_t)src * a.b + i] = am;
-    if (lane < DZ_STRIDE) {
-      float v = 0.f;
-#pragma unroll
-      for (int c = 0; c < NCLS; ++c)
-        if (lane == c) v = dz[c];
-      ws.dz[row * DZ_STRIDE + lane] = v;
-    }
+  // two samples per warp and pass, so that every weight read from shared memory is used twice
+  for (int i0 = 2 * warp; i0 < a.b; i0 += 2 * (FC2_THREADS / 32)) {
+    const bool two = i0 + 1 < a.b;                       // warp-uniform
+    // the weights are re-read from shared memory on every pass: 160 of them per lane would not fit in the
+    // registers of a 512-thread block, so their address is made to look pass-dependent
+    uint32_t opaque_zero;
+    asm volatile("mov.u32 %0, 0;" : "=r"(opaque_zero));
+    const float (*w2p)[HID] = reinterpret_cast<const float (*)[HID]>(&w2[0][0] + opaque_zero);
+    const int64_t row0 = (int64_t)s * a.b + i0, row1 = two ? row0 + 1 : row0;
+    float dv[2][16];
 #pragma unroll
     for (int t = 0; t < 16; ++t) {
-      int j = lane + 32 * t;
-      float dd = 0.f;
+      dv[0][t] = ws.d[row0 * HID + lane + 32 * t];
+      dv[1][t] = ws.d[row1 * HID + lane + 32 * t];
+    }
+    float z[2][NCLS];
 #pragma unroll
-      for (int c = 0; c < NCLS; ++c) dd = fmaf(w2[c][j], dz[c], dd);
-      float dv1 = dv[t] > 0.f ? dd * scale : 0.f;
-      if (a.precision != 0) dv1 = round_tf32(dv1);   // it feeds tensor-core products only
-      ws.da1[row * HID + j] = dv1;
+    for (int c = 0; c < NCLS; ++c) z[0][c] = z[1][c] = 0.f;
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+#pragma unroll
+      for (int c = 0; c < NCLS; ++c) {
+        const float wv = w2p[c][lane + 32 * t];
+        z[0][c] = fmaf(wv, dv[0][t], z[0][c]);
+        z[1][c] = fmaf(wv, dv[1][t], z[1][c]);
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < NCLS; ++c) {
+      z[0][c] = warp_sum(z[0][c]) + b2[c];
+      z[1][c] = warp_sum(z[1][c]) + b2[c];
+    }
+    float dz[2][NCLS];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      if (u == 1 && !two) continue;
+      const int i = i0 + u;
+      float zmax = z[u][0];
+      int am = 0;
+#pragma unroll
+      for (int c = 1; c < NCLS; ++c)
+        if (z[u][c] > zmax) { zmax = z[u][c]; am = c; }
+      float se = 0.f;
+#pragma unroll
+      for (int c = 0; c < NCLS; ++c) se += expf(z[u][c] - zmax);
+      const float lse = zmax + logf(se);
+      int label = a.y[(int64_t)src * a.b + i];
+      if (label < 0 || label >= NCLS) {
+        if (lane == 0) atomicOr(ws.status, STATUS_BAD_LABEL);
+        label = 0;
+      }
+      float zy = 0.f;
+#pragma unroll
+      for (int c = 0; c < NCLS; ++c) {
+        if (c == label) zy = z[u][c];
+        dz[u][c] = (expf(z[u][c] - lse) - (c == label ? 1.f : 0.f)) * inv_b;
+      }
+      loss_acc += lse - zy;
+      if (lane == 0) a.argmax[(int64_t)src * a.b + i] = am;
+      if (lane < DZ_STRIDE) {
+        float v = 0.f;
+#pragma unroll
+        for (int c = 0; c < NCLS; ++c)
+          if (lane == c) v = dz[u][c];
+        ws.dz[(row0 + u) * DZ_STRIDE + lane] = v;
+      }
+    }
+    if (!two) {
+#pragma unroll
+      for (int c = 0; c < NCLS; ++c) dz[1][c] = 0.f;
+    }
+    asm volatile("mov.u32 %0, 0;" : "=r"(opaque_zero));    // second read of the weights, as above
+    w2p = reinterpret_cast<const float (*)[HID]>(&w2[0][0] + opaque_zero);
+    uint32_t live0 = 0u, live1 = 0u;                         // which of the lane's 16 units passed ReLU and dropout
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      live0 |= (dv[0][t] > 0.f ? 1u : 0u) << t;
+      live1 |= (dv[1][t] > 0.f ? 1u : 0u) << t;
+    }
+#pragma unroll 2
+    for (int t = 0; t < 16; ++t) {
+      const int j = lane + 32 * t;
+      float dd0 = 0.f, dd1 = 0.f;
+#pragma unroll
+      for (int c = 0; c < NCLS; ++c) {
+        const float wv = w2p[c][j];
+        dd0 = fmaf(wv, dz[0][c], dd0);
+        dd1 = fmaf(wv, dz[1][c], dd1);
+      }
+      float v0 = (live0 >> t) & 1u ? dd0 * scale : 0.f, v1 = (live1 >> t) & 1u ? dd1 * scale : 0.f;
+      if (a.precision != 0) { v0 = round_tf32(v0); v1 = round_tf32(v1); }   // they feed tensor-core products only
+      ws.da1[row0 * HID + j] = v0;
+      if (two) ws.da1[row1 * HID + j] = v1;
     }
   }
   if (lane == 0) warp_loss[warp] = loss_acc;
   __syncthreads();   // also makes this block's dz / da1 stores visible to all of its threads
   if (tid == 0) {
     float t = 0.f;
-    for (int w = 0; w < 8; ++w) t += warp_loss[w];
+    for (int w = 0; w < FC2_THREADS / 32; ++w) t += warp_loss[w];
     a.loss[src] = t * inv_b;
   }
   float* grad = wt.grad[s];
-  float gw[2][NCLS], gb1[2] = {0.f, 0.f};
+  const int j = tid;                                  // hidden unit (FC2_THREADS == HID)
+  float gw[NCLS], gb1 = 0.f, gb2 = 0.f;
 #pragma unroll
-  for (int h = 0; h < 2; ++h)
-#pragma unroll
-    for (int c = 0; c < NCLS; ++c) gw[h][c] = 0.f;
-  float gb2 = 0.f;
+  for (int c = 0; c < NCLS; ++c) gw[c] = 0.f;
+  const float* dzp = ws.dz + (int64_t)s * a.b * DZ_STRIDE;
+  const float* dp = ws.d + (int64_t)s * a.b * HID + j;
+  const float* da1p = ws.da1 + (int64_t)s * a.b * HID + j;
+#pragma unroll 4
   for (int i = 0; i < a.b; ++i) {
-    const int64_t row = (int64_t)s * a.b + i;
-    float dzv[NCLS];
+    const float dval = dp[(int64_t)i * HID];
+    const float4 z0 = *reinterpret_cast<const float4*>(dzp + i * DZ_STRIDE);
+    const float4 z1 = *reinterpret_cast<const float4*>(dzp + i * DZ_STRIDE + 4);
+    const float2 z2 = *reinterpret_cast<const float2*>(dzp + i * DZ_STRIDE + 8);
+    const float dzv[NCLS] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w, z2.x, z2.y};
 #pragma unroll
-    for (int c = 0; c < NCLS; ++c) dzv[c] = ws.dz[row * DZ_STRIDE + c];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      float dval = ws.d[row * HID + tid + 256 * h];
-#pragma unroll
-      for (int c = 0; c < NCLS; ++c) gw[h][c] = fmaf(dzv[c], dval, gw[h][c]);
-      gb1[h] += ws.da1[row * HID + tid + 256 * h];
-    }
-    if (tid < NCLS) gb2 += ws.dz[row * DZ_STRIDE + tid];
+    for (int c = 0; c < NCLS; ++c) gw[c] = fmaf(dzv[c], dval, gw[c]);
+    gb1 += da1p[(int64_t)i * HID];
+    if (j < NCLS) gb2 += dzp[i * DZ_STRIDE + j];
   }
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
-#pragma unroll
-    for (int c = 0; c < NCLS; ++c) grad[OFF_F2W + c * HID + tid + 256 * h] = gw[h][c];
-    grad[OFF_F1B + tid + 256 * h] = gb1[h];
-  }
-  if (tid < NCLS) grad[OFF_F2B + tid] = gb2;
+  for (int c = 0; c < NCLS; ++c) grad[OFF_F2W + c * HID + j] = gw[c];
+  grad[OFF_F1B + j] = gb1;
+  if (j < NCLS) grad[OFF_F2B + j] = gb2;
 }
 
 // ---- fc1 weight gradient of one worker: dW1 [512][1568] = da1^T [512 x b] * p2 [b x 1568].
@@ -618,7 +658,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof);
     if (n < 0) return -1;
     launches += 2 + n;
-    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
     launches += 1;
     cudaStream_t s1 = side.s1 ? side.s1 : st, s2 = side.s2 ? side.s2 : st;
     if (side.s1) { cudaEventRecord(side.fork1, st); cudaStreamWaitEvent(s1, side.fork1, 0); }
@@ -642,7 +682,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     TIMED(K_CONV1_FWD, (conv1_fwd<false><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
-    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, 256, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
     TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
