@@ -595,12 +595,16 @@ __global__ void __launch_bounds__(256) conv1_bwd(GradStepArgs a, WorkerTable wt,
 }
 
 // ---- sums the per-block partial convolution gradients in block order and zeroes the padding.
-__global__ void __launch_bounds__(256) conv_grad_reduce(WorkerTable wt, Workspace ws, int n_chunks, int n_chunks2) {
+// part2 holds n_chunks2 slots per worker; all of them are summed when seg_len == 0, otherwise four for every
+// range of seg_len rows that meets the worker's b rows (the tensor-core filter-gradient kernel's layout).
+__global__ void __launch_bounds__(256) conv_grad_reduce(WorkerTable wt, Workspace ws, int n_chunks, int n_chunks2,
+                                                        int seg_len, int b) {
   const int s = blockIdx.x, tid = threadIdx.x;
   float* grad = wt.grad[s];
+  const int used2 = seg_len > 0 ? 4 * ((s * b + b - 1) / seg_len - (s * b) / seg_len + 1) : n_chunks2;
   for (int o = tid; o < C2_GRAD; o += 256) {
     float t = 0.f;
-    for (int c = 0; c < n_chunks2; ++c) t += ws.part2[((int64_t)s * n_chunks2 + c) * C2_GRAD + o];
+    for (int c = 0; c < used2; ++c) t += ws.part2[((int64_t)s * n_chunks2 + c) * C2_GRAD + o];
     grad[OFF_C2W + o] = t;
   }
   for (int o = tid; o < C1_GRAD; o += 256) {
@@ -651,7 +655,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
   const bool tc = a.precision != 0;
   const int n_chunks1 = (a.b + CONV1_SPB - 1) / CONV1_SPB;
   const int n_chunks1b = (a.b + CONV1B_SPB - 1) / CONV1B_SPB;
-  int launches = 0, n_chunks2 = n_chunks;
+  int launches = 0, n_chunks2 = n_chunks, seg_len = 0;
   if (tc) {
     TIMED(K_CONV1_FWD, (conv1_fwd<true><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
     launch_conv2_fwd_tc5(a, wt, gt, ws, st, prof);
@@ -670,13 +674,13 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     if (n < 0) return -1;
     launches += n;
     if (side.s2) { cudaEventRecord(side.fork2, st); cudaStreamWaitEvent(s2, side.fork2, 0); }
-    n_chunks2 = launch_conv2_dw_tc(a, wt, ws, s2, prof);
+    n_chunks2 = launch_conv2_dw_tc(a, wt, ws, s2, prof, &seg_len);
     if (side.s2) cudaEventRecord(side.join2, s2);
     launch_conv2_dx_tc5(a, wt, gt, ws, st, prof);
     const int n_chunks1t = launch_conv1_bwd_tc(a, wt, ws, st, prof);
     if (side.s1) cudaStreamWaitEvent(st, side.join1, 0);
     if (side.s2) cudaStreamWaitEvent(st, side.join2, 0);
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks1t, n_chunks2)));
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks1t, n_chunks2, seg_len, a.b)));
     launches += 4;
   } else {
     TIMED(K_CONV1_FWD, (conv1_fwd<false><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
@@ -687,7 +691,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
     TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
     TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks1b, a.W), 256, 0, st>>>(a, wt, ws, n_chunks1b)));
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks1b, n_chunks2)));
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks1b, n_chunks2, 0, a.b)));
     launches = 9;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;

@@ -5,6 +5,7 @@
 // Reductions keep a fixed order, so results are reproducible bit for bit.
 #include "device_common.cuh"
 #include "kernels.h"
+#include "tc5_common.cuh"
 
 namespace psk {
 
@@ -17,14 +18,21 @@ constexpr int TC_SPB = 8;
 // Both operands are rounded to BF16 here (fp32 accumulation): this product only yields gradient values, no
 // ReLU or pooling decision depends on it, and at 16 positions per instruction it needs half the
 // instructions and shared-memory loads of the TF32 form.
-// 288 threads = 9 warps, warp = filter tap; accumulators persist over the block's samples and are
-// written once as the block's partial sum.  The bias gradient (sum of g2 over positions) rides along as
-// a product with a column of ones, each warp taking every ninth k-step; the nine partial sums are
-// combined in a fixed order at the end.
-// A BF16 fragment register holds two consecutive k = two horizontally adjacent positions (x even, x+1).
-// For the taps that shift by an odd number of columns such a pair is not word-aligned in the image plane,
-// so the planes are kept twice, the second copy shifted by one element.
-// The next sample's inputs are fetched into registers while the current one is being multiplied.
+// 512 threads: twelve MMA warps and four loader warps, one CTA per SM walking over a contiguous range of samples.
+// The loaders fetch a sample's pooled gradient, pooling decisions and input planes one sample ahead, write
+// them as BF16 operands into one of two shared-memory buffers and signal an mbarrier; the MMA warps never
+// wait for staging.  MMA warp = (share of the 13 k-steps, filter row): it multiplies one set of g2 fragments
+// (ldmatrix) with the image fragments of the three taps of its filter row, twelve independent MMAs per
+// k-step; accumulators persist over the range and are written as partial sums at its end (and where the
+// range passes from one worker to the next); a later kernel adds the partial sums in a fixed order.  The bias
+// gradient (sum of g2 over positions) rides along as a product with a column of ones in the warps of
+// filter row 0.
+// A BF16 fragment register holds two consecutive k = two horizontally adjacent positions (x even, x+1) of
+// the flattened 14-wide image, so a tap is a constant word offset (7 words per filter row).  The image
+// is kept three times, once per filter column: the copy of the left (right) taps is shifted by one element
+// so that its pairs are word-aligned, and leaves out column 13 (0), whose shifted slot is the neighbouring
+// row's out-of-image column and must read zero.
+// Every mbarrier wait is bounded; on a timeout the kernel raises a status flag and all warps leave.
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -37,152 +45,231 @@ __device__ __forceinline__ uint16_t bf16_bits(float x) {
   return r;
 }
 __device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {   // lo in the low half (lower k index)
-  return (uint32_t)bf16_bits(lo) | ((uint32_t)bf16_bits(hi) << 16);
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
 }
 
 constexpr int DW_G_WORDS = 108;    // 216 bf16 per output channel: 196 positions + zeros; 108 = 12 (mod 32 banks)
-constexpr int DW_P_WORDS = 132;    // 16 x 16 bf16 per input channel + 8; 132 = 4 (mod 32 banks)
-constexpr int DW_THREADS = 288;
-constexpr int DW_KSTEPS = 13;      // 208 positions / 16
-constexpr int DW_QUADS = (4 * 196 + DW_THREADS - 1) / DW_THREADS;   // 3 four-channel positions per thread
-constexpr int DW_ENTRIES = (FLAT + DW_THREADS - 1) / DW_THREADS;    // 6 pooled gradient entries per thread
-__global__ void __launch_bounds__(DW_THREADS, 2) conv2_dw_tc(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
-  __shared__ __align__(16) uint32_t g2w[32 * DW_G_WORDS];        // [oc][position pair]
-  __shared__ __align__(16) uint32_t imgw[2][16 * DW_P_WORDS];    // [copy][ic][(Y*16 + X - copy) / 2], zero border
-  __shared__ float bias_part[9][32];
-  uint16_t* img_h[2] = {reinterpret_cast<uint16_t*>(imgw[0]), reinterpret_cast<uint16_t*>(imgw[1])};
-  const int s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-  const int ky = warp / 3, kx = warp - ky * 3;
-  for (int idx = tid; idx < 2 * 16 * DW_P_WORDS; idx += DW_THREADS) (&imgw[0][0])[idx] = 0u;
-  for (int idx = tid; idx < 32 * DW_G_WORDS; idx += DW_THREADS) g2w[idx] = 0u;
-  float acc[2][2][4], accb[2][4];
-#pragma unroll
-  for (int m = 0; m < 2; ++m) {
-#pragma unroll
-    for (int n = 0; n < 2; ++n)
-#pragma unroll
-      for (int r = 0; r < 4; ++r) acc[m][n][r] = 0.f;
-#pragma unroll
-    for (int r = 0; r < 4; ++r) accb[m][r] = 0.f;
-  }
-  // the column of ones: B(k, n) = 1 for n == 0; this lane supplies column n = g
-  const uint32_t one_frag[2] = {g == 0 ? 0x3F803F80u : 0u, g == 0 ? 0x3F803F80u : 0u};
-  // this warp's B fragments: pair index j = ks*8 + t (+4): position 2j = (y, x even); element (y+ky)*16 + x + kx
-  // in the bordered plane, taken from the copy that makes it even
-  const int copy = kx & 1;
-  const uint32_t* plane = imgw[copy];
-  const int i0 = blockIdx.x * TC_SPB, i1 = min(i0 + TC_SPB, a.b);
+constexpr int DW_P_WORDS = 132;    // plane of one input channel: 16 rows x 14 bf16 (rows 0 and 15 stay zero) = 112
+                                   // words, + the words the zero-padded k tail reaches; 132 = 4 (mod 32 banks)
+constexpr int DW_MMA_WARPS = 12, DW_LOAD_WARPS = 8;
+constexpr int DW_THREADS = 32 * (DW_MMA_WARPS + DW_LOAD_WARPS);
+constexpr int DW_LOADERS = 32 * DW_LOAD_WARPS;
+constexpr int DW_BUF_WORDS = 32 * DW_G_WORDS + 3 * 16 * DW_P_WORDS;   // one sample: g2 and three image copies
+constexpr int DW_RAW_P1 = P1_PLANE_ELEMS * 4, DW_RAW_DP2 = FLAT * 4, DW_RAW_CODE = FLAT;   // bytes of one sample's inputs
+constexpr int DW_RAW_BYTES = DW_RAW_P1 + DW_RAW_DP2 + DW_RAW_CODE;
+constexpr int DW_RAW_WORDS = (DW_RAW_BYTES + 127) / 128 * 32;          // raw buffer, padded to 128 bytes
+constexpr int DW_NRAW = 3;         // raw input buffers: copies run three samples ahead of the MMAs
+constexpr int DW_SMEM_BYTES = (2 * DW_BUF_WORDS + DW_NRAW * DW_RAW_WORDS) * 4 + 128;
+static_assert(DW_RAW_P1 % 16 == 0 && DW_RAW_DP2 % 16 == 0 && DW_RAW_CODE % 16 == 0, "bulk copies move multiples of 16 bytes");
+constexpr int DW_MIN_SEG = 16;     // a CTA's range is at least this long (bounds the partial sums per worker)
+constexpr int DW_PAIRS = (4 * 98 + DW_LOADERS - 1) / DW_LOADERS;      // 2 (plane, position pair) items per loader thread
+constexpr int DW_ENTRIES = (FLAT + DW_LOADERS - 1) / DW_LOADERS;      // 7 pooled gradient entries per loader thread
 
-  float4 pq[DW_QUADS];
-  float pg[DW_ENTRIES];
-  int pc[DW_ENTRIES];
-  auto prefetch = [&](int i) {
-    const int64_t row = (int64_t)s * a.b + i;
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+
+// The k-steps K0..K1-1 of one sample for one warp: two ldmatrix for g2, twelve word loads for the three taps of the
+// warp's filter row, twelve MMAs (+ two for the bias in the warps of filter row 0).
+template <int K0, int K1>
+__device__ __forceinline__ void dw_ksteps(uint32_t a_addr, const uint32_t* b_base, float (&acc)[3][2][2][4],
+                                          float (&accb)[2][4], bool with_bias, const uint32_t (&one_frag)[2]) {
 #pragma unroll
-    for (int k = 0; k < DW_QUADS; ++k) {
-      const int e = tid + k * DW_THREADS;                      // (plane q, position p)
-      if (e < 4 * 196) {
-        const int q = e / 196, p = e - q * 196, y = p / 14, x = p - y * 14, X = x + 1, Y = y + 1;
-        pq[k] = *reinterpret_cast<const float4*>(ws.p1 + row * P1_PLANE_ELEMS + q * 1024 + (Y * 16 + (X & 1) * 8 + (X >> 1)) * 4);
-      }
-    }
+  for (int ks = K0; ks < K1; ++ks) {
+    uint32_t fa[2][4], fb[3][2][2];
+    ldmatrix_x4(fa[0], a_addr + ks * 32);
+    ldmatrix_x4(fa[1], a_addr + 16 * DW_G_WORDS * 4 + ks * 32);
 #pragma unroll
-    for (int k = 0; k < DW_ENTRIES; ++k) {
-      const int o = tid + k * DW_THREADS;
-      pc[k] = o < FLAT ? (int)ws.code2[row * FLAT + o] : 4;
-      pg[k] = o < FLAT ? ws.dp2[row * FLAT + o] : 0.f;
-    }
-  };
-  prefetch(i0);
-  for (int i = i0; i < i1; ++i) {
-    __syncthreads();                 // the previous sample's products are done with shared memory
-#pragma unroll
-    for (int k = 0; k < DW_QUADS; ++k) {
-      const int e = tid + k * DW_THREADS;
-      if (e < 4 * 196) {
-        const int q = e / 196, p = e - q * 196, y = p / 14, x = p - y * 14;
-        const int el = (y + 1) * 16 + x + 1;
-        const float v[4] = {pq[k].x, pq[k].y, pq[k].z, pq[k].w};
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint16_t h = bf16_bits(v[c]);
-          img_h[0][(4 * q + c) * (2 * DW_P_WORDS) + el] = h;
-          img_h[1][(4 * q + c) * (2 * DW_P_WORDS) + el - 1] = h;
-        }
-      }
-    }
-#pragma unroll
-    for (int k = 0; k < DW_ENTRIES; ++k) {
-      const int o = tid + k * DW_THREADS;
-      if (o < FLAT) {
-        // every pooled entry owns the four positions of its window: the gradient goes to the chosen one,
-        // the others are cleared, so no separate clearing pass is needed
-        const int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
-        uint32_t* d = g2w + oc * DW_G_WORDS + (2 * py) * 7 + px;     // word of positions (2py, 2px), (2py, 2px+1)
-        const float v = pg[k];
-        d[0] = bf16_pair(pc[k] == 0 ? v : 0.f, pc[k] == 1 ? v : 0.f);
-        d[7] = bf16_pair(pc[k] == 2 ? v : 0.f, pc[k] == 3 ? v : 0.f);
-      }
-    }
-    __syncthreads();
-    if (i + 1 < i1) prefetch(i + 1);
-#pragma unroll
-    for (int ks = 0; ks < DW_KSTEPS; ++ks) {
-      const int j0 = ks * 8 + t, j1 = j0 + 4;                  // position pairs of this lane's k columns
-      uint32_t fa[2][4], fb[2][2];
-#pragma unroll
-      for (int m = 0; m < 2; ++m) {
-        const uint32_t* ga = g2w + (m * 16 + g) * DW_G_WORDS;
-        fa[m][0] = ga[j0];
-        fa[m][1] = ga[8 * DW_G_WORDS + j0];
-        fa[m][2] = ga[j1];
-        fa[m][3] = ga[8 * DW_G_WORDS + j1];
-      }
-      const int q0 = min(j0, 97), q1 = min(j1, 97);            // pairs beyond 97 meet zeros in g2
-      const int y0 = q0 / 7, x0 = 2 * (q0 - y0 * 7), y1 = q1 / 7, x1 = 2 * (q1 - y1 * 7);
-      const int w0 = ((y0 + ky) * 16 + x0 + kx - copy) >> 1, w1 = ((y1 + ky) * 16 + x1 + kx - copy) >> 1;
+    for (int kx = 0; kx < 3; ++kx)
 #pragma unroll
       for (int n = 0; n < 2; ++n) {
-        const uint32_t* pi = plane + (n * 8 + g) * DW_P_WORDS;
-        fb[n][0] = pi[w0];
-        fb[n][1] = pi[w1];
+        fb[kx][n][0] = b_base[(kx * 16 + n * 8) * DW_P_WORDS + ks * 8];
+        fb[kx][n][1] = b_base[(kx * 16 + n * 8) * DW_P_WORDS + ks * 8 + 4];
       }
+#pragma unroll
+    for (int kx = 0; kx < 3; ++kx)
 #pragma unroll
       for (int m = 0; m < 2; ++m)
 #pragma unroll
-        for (int n = 0; n < 2; ++n) mma_bf16(acc[m][n], fa[m], fb[n]);
-      if (ks % 9 == warp) {            // warp-uniform
-        mma_bf16(accb[0], fa[0], one_frag);
-        mma_bf16(accb[1], fa[1], one_frag);
+        for (int n = 0; n < 2; ++n) mma_bf16(acc[kx][m][n], fa[m], fb[kx][n]);
+    if (with_bias) {                   // warp-uniform
+      mma_bf16(accb[0], fa[0], one_frag);
+      mma_bf16(accb[1], fa[1], one_frag);
+    }
+  }
+}
+
+// Rows (sorted worker, sample) are split into gridDim.x contiguous ranges of seg_len; a range may cross from one
+// worker into the next, where the accumulators are written out and cleared.  Partial sums of worker s go to
+// part2[s][4 * (range index - first range of s) + k-share].
+__global__ void __launch_bounds__(DW_THREADS, 1) conv2_dw_tc(GradStepArgs a, WorkerTable wt, Workspace ws, int seg_len, int slots) {
+  extern __shared__ __align__(128) uint32_t dw_smem[];
+  uint32_t* raw = dw_smem + 2 * DW_BUF_WORDS;                                   // [DW_NRAW][DW_RAW_WORDS]
+  uint64_t* full = reinterpret_cast<uint64_t*>(raw + DW_NRAW * DW_RAW_WORDS);   // [2] loaders -> MMA warps
+  uint64_t* empty = full + 2;                                                    // [2] MMA warps -> loaders
+  uint64_t* raw_full = full + 4;                                                 // [DW_NRAW] bulk copies -> loaders
+  uint64_t* raw_empty = raw_full + DW_NRAW;                                      // [DW_NRAW] loaders -> copy issuer
+  volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(raw_empty + DW_NRAW);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int total = a.W * a.b;
+  const int r0 = blockIdx.x * seg_len, r1 = min(r0 + seg_len, total);
+  for (int idx = tid; idx < 2 * DW_BUF_WORDS; idx += DW_THREADS) dw_smem[idx] = 0u;
+  if (tid == 0) {
+    mbar_init(&full[0], DW_LOADERS); mbar_init(&full[1], DW_LOADERS);
+    mbar_init(&empty[0], 32 * DW_MMA_WARPS); mbar_init(&empty[1], 32 * DW_MMA_WARPS);
+    for (int i = 0; i < DW_NRAW; ++i) { mbar_init(&raw_full[i], 1); mbar_init(&raw_empty[i], DW_LOADERS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp >= DW_MMA_WARPS) {
+    // ---------------- loaders: bulk copies global -> raw buffers (three samples ahead), then BF16 operands
+    const int lt = tid - 32 * DW_MMA_WARPS;
+    auto issue = [&](int n) {            // one thread: the three input rows of sample r0 + n
+      const int64_t row = r0 + n;
+      uint8_t* dst = reinterpret_cast<uint8_t*>(raw + (n % DW_NRAW) * DW_RAW_WORDS);
+      uint64_t* bar = &raw_full[n % DW_NRAW];
+      mbar_expect_tx(bar, DW_RAW_BYTES);
+      bulk_load(dst, ws.p1 + row * P1_PLANE_ELEMS, DW_RAW_P1, bar);
+      bulk_load(dst + DW_RAW_P1, ws.dp2 + row * FLAT, DW_RAW_DP2, bar);
+      bulk_load(dst + DW_RAW_P1 + DW_RAW_DP2, ws.code2 + row * FLAT, DW_RAW_CODE, bar);
+    };
+    if (lt == 0)
+      for (int n = 0; n < DW_NRAW && r0 + n < r1; ++n) issue(n);
+    for (int row = r0, n = 0; row < r1; ++row, ++n) {
+      const int buf = n & 1, rb = n % DW_NRAW;
+      bool ok = mbar_wait(&raw_full[rb], (n / DW_NRAW) & 1);
+      if (ok && n >= 2) ok = mbar_wait(&empty[buf], ((n >> 1) - 1) & 1);
+      if (!ok) { *abort_flag = 1; atomicOr(ws.status, STATUS_WAIT_TIMEOUT); }
+      if (*abort_flag) break;
+      const float* rp1 = reinterpret_cast<const float*>(raw + rb * DW_RAW_WORDS);
+      const float* rdp2 = rp1 + P1_PLANE_ELEMS;
+      const uint8_t* rcode = reinterpret_cast<const uint8_t*>(rdp2 + FLAT);
+      uint32_t* g2w = dw_smem + buf * DW_BUF_WORDS;
+      // Item = (plane q of four channels, pair w of horizontally adjacent positions 2w, 2w+1 of the flattened
+      // 14-wide image).  Word w + 7 of a channel's plane holds positions (x, x+1) in the middle copy,
+      // (x-1, x) in the copy of the left taps and (x+1, x+2) in the copy of the right taps; x-1 = -1 and
+      // x+2 = 14 read the zero border of the source plane.
+#pragma unroll
+      for (int k = 0; k < DW_PAIRS; ++k) {
+        const int e = lt + k * DW_LOADERS;
+        if (e < 4 * 98) {
+          const int q = e / 98, w = e - q * 98, y = w / 7, x = 2 * (w - y * 7);
+          const float* src = rp1 + q * 1024 + (y + 1) * 64;        // row Y = y + 1: even X in floats 0..31, odd X in 32..63
+          // X = x + 1 + j for j = -1..2: X = x (even), x + 1 (odd), x + 2 (even), x + 3 (odd)
+          const float4 v0 = *reinterpret_cast<const float4*>(src + (x >> 1) * 4);
+          const float4 v1 = *reinterpret_cast<const float4*>(src + 32 + (x >> 1) * 4);
+          const float4 v2 = *reinterpret_cast<const float4*>(src + ((x >> 1) + 1) * 4);
+          const float4 v3 = *reinterpret_cast<const float4*>(src + 32 + ((x >> 1) + 1) * 4);
+          const float a0[4] = {v0.x, v0.y, v0.z, v0.w}, a1[4] = {v1.x, v1.y, v1.z, v1.w};
+          const float a2[4] = {v2.x, v2.y, v2.z, v2.w}, a3[4] = {v3.x, v3.y, v3.z, v3.w};
+          uint32_t* d = g2w + 32 * DW_G_WORDS + (4 * q) * DW_P_WORDS + w + 7;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            d[c * DW_P_WORDS] = bf16_pair(a0[c], a1[c]);
+            d[(16 + c) * DW_P_WORDS] = bf16_pair(a1[c], a2[c]);
+            d[(32 + c) * DW_P_WORDS] = bf16_pair(a2[c], a3[c]);
+          }
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < DW_ENTRIES; ++k) {
+        const int o = lt + k * DW_LOADERS;
+        if (o < FLAT) {
+          // every pooled entry owns the four positions of its window: the gradient goes to the chosen one,
+          // the others are cleared, so no separate clearing pass is needed
+          const int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
+          uint32_t* d = g2w + oc * DW_G_WORDS + (2 * py) * 7 + px;     // word of positions (2py, 2px), (2py, 2px+1)
+          const float v = rdp2[o];
+          const int code = rcode[o];
+          d[0] = bf16_pair(code == 0 ? v : 0.f, code == 1 ? v : 0.f);
+          d[7] = bf16_pair(code == 2 ? v : 0.f, code == 3 ? v : 0.f);
+        }
+      }
+      mbar_arrive(&full[buf]);
+      mbar_arrive(&raw_empty[rb]);
+      if (lt == 0 && row + DW_NRAW < r1) {
+        // every loader has read this raw buffer: refill it with the sample three ahead
+        if (!mbar_wait(&raw_empty[rb], (n / DW_NRAW) & 1)) { *abort_flag = 1; atomicOr(ws.status, STATUS_WAIT_TIMEOUT); break; }
+        issue(n + DW_NRAW);
+      }
+    }
+  } else {
+    // ---------------- MMA warps: warp = (k-share, filter row); the k-shares are 4, 3, 3, 3 of the 13 k-steps
+    const int g = lane >> 2, t = lane & 3;
+    const int kpart = warp / 3, ky = warp - kpart * 3;
+    float acc[3][2][2][4], accb[2][4];
+    auto clear = [&]() {
+#pragma unroll
+      for (int m = 0; m < 2; ++m) {
+#pragma unroll
+        for (int kx = 0; kx < 3; ++kx)
+#pragma unroll
+          for (int n = 0; n < 2; ++n)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) acc[kx][m][n][r] = 0.f;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) accb[m][r] = 0.f;
+      }
+    };
+    clear();
+    // the column of ones: B(k, n) = 1 for n == 0; this lane supplies column n = g
+    const uint32_t one_frag[2] = {g == 0 ? 0x3F803F80u : 0u, g == 0 ? 0x3F803F80u : 0u};
+    // A fragments by ldmatrix: lane l addresses row (l & 7) + 8 * ((l >> 3) & 1) of the 16-row tile, k half l >> 4
+    const uint32_t a_off = (uint32_t)(((lane & 7) + ((lane >> 3) & 1) * 8) * DW_G_WORDS * 4 + (lane >> 4) * 16);
+    // B fragments: column n = input channel g (+8), k pair ks*8 + t (+4) -> word ks*8 + t + 7*ky of the tap's copy
+    const int b_off = 32 * DW_G_WORDS + g * DW_P_WORDS + t + 7 * ky;
+    for (int row = r0, n = 0; row < r1; ++row, ++n) {
+      const int buf = n & 1;
+      // the products below are warp-wide instructions: the decision to go on must be the same in all lanes
+      const bool ready = mbar_wait(&full[buf], (n >> 1) & 1) && *abort_flag == 0;
+      if (!__all_sync(0xffffffffu, ready)) {
+        if (lane == 0) { *abort_flag = 1; atomicOr(ws.status, STATUS_WAIT_TIMEOUT); }
+        break;
+      }
+      const uint32_t a_addr = smem_u32(dw_smem + buf * DW_BUF_WORDS) + a_off;
+      const uint32_t* b_base = dw_smem + buf * DW_BUF_WORDS + b_off;
+      if (kpart == 0) dw_ksteps<0, 4>(a_addr, b_base, acc, accb, ky == 0, one_frag);
+      else if (kpart == 1) dw_ksteps<4, 7>(a_addr, b_base, acc, accb, ky == 0, one_frag);
+      else if (kpart == 2) dw_ksteps<7, 10>(a_addr, b_base, acc, accb, ky == 0, one_frag);
+      else dw_ksteps<10, 13>(a_addr, b_base, acc, accb, ky == 0, one_frag);
+      mbar_arrive(&empty[buf]);
+      const int s = row / a.b;
+      if (row + 1 == r1 || (row + 1) % a.b == 0) {
+        // last row of the range or of worker s: write this warp's partial sums and start over
+        const int sub = 4 * (blockIdx.x - (s * a.b) / seg_len) + kpart;
+        float* part = ws.part2 + ((int64_t)s * slots + sub) * C2_GRAD;
+#pragma unroll
+        for (int kx = 0; kx < 3; ++kx)
+#pragma unroll
+          for (int m = 0; m < 2; ++m)
+#pragma unroll
+            for (int nn = 0; nn < 2; ++nn) {
+              const int oc = m * 16 + g, ic = nn * 8 + 2 * t, tap = ky * 3 + kx;
+              part[(oc * 16 + ic) * 9 + tap] = acc[kx][m][nn][0];
+              part[(oc * 16 + ic + 1) * 9 + tap] = acc[kx][m][nn][1];
+              part[((oc + 8) * 16 + ic) * 9 + tap] = acc[kx][m][nn][2];
+              part[((oc + 8) * 16 + ic + 1) * 9 + tap] = acc[kx][m][nn][3];
+            }
+        // column 0 of the ones-product lives in the lanes with t == 0: rows g and g+8 of each 16-row tile
+        if (ky == 0 && t == 0) {
+#pragma unroll
+          for (int m = 0; m < 2; ++m) {
+            part[4608 + m * 16 + g] = accb[m][0];
+            part[4608 + m * 16 + g + 8] = accb[m][2];
+          }
+        }
+        clear();
       }
     }
   }
-  float* part = ws.part2 + ((int64_t)s * n_chunks + blockIdx.x) * C2_GRAD;
-#pragma unroll
-  for (int m = 0; m < 2; ++m)
-#pragma unroll
-    for (int n = 0; n < 2; ++n) {
-      const int oc = m * 16 + g, ic = n * 8 + 2 * t;
-      part[(oc * 16 + ic) * 9 + warp] = acc[m][n][0];
-      part[(oc * 16 + ic + 1) * 9 + warp] = acc[m][n][1];
-      part[((oc + 8) * 16 + ic) * 9 + warp] = acc[m][n][2];
-      part[((oc + 8) * 16 + ic + 1) * 9 + warp] = acc[m][n][3];
-    }
-  // column 0 of the ones-product lives in the lanes with t == 0: rows g and g+8 of each 16-row tile
-  if (t == 0) {
-#pragma unroll
-    for (int m = 0; m < 2; ++m) {
-      bias_part[warp][m * 16 + g] = accb[m][0];
-      bias_part[warp][m * 16 + g + 8] = accb[m][2];
-    }
-  }
-  __syncthreads();
-  if (tid < 32) {
-    float sum = 0.f;
-#pragma unroll
-    for (int w = 0; w < 9; ++w) sum += bias_part[w][tid];
-    part[4608 + tid] = sum;
-  }
+  // after a timeout, give bulk copies that are still in flight time to land before the CTA's shared memory is released
+  if (tid == 32 * DW_MMA_WARPS && *abort_flag)
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -298,13 +385,24 @@ __global__ void __launch_bounds__(256) conv1_bwd_tc(GradStepArgs a, WorkerTable 
 
 #define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
 
-int configure_tc_kernels() { return 0; }
+int configure_tc_kernels() {
+  return cudaFuncSetAttribute(conv2_dw_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, DW_SMEM_BYTES) == cudaSuccess ? 0 : -1;
+}
 
-// Returns the number of per-worker partial blocks the filter gradient was split into.
-int launch_conv2_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof) {
-  const int chunks = (a.b + TC_SPB - 1) / TC_SPB;
-  TIMED(K_CONV2_DW, (conv2_dw_tc<<<dim3(chunks, a.W), DW_THREADS, 0, st>>>(a, wt, ws, chunks)));
-  return chunks;
+// Returns the number of partial-sum slots reserved per worker (the stride of part2) and, in *seg_len, the length
+// of a CTA's range of rows: worker s owns 4 x (ranges that meet its rows) partial sums.
+int launch_conv2_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof,
+                       int* seg_len) {
+  const int total = a.W * a.b;
+  int grid = total / DW_MIN_SEG;
+  if (grid > g_sm_count) grid = g_sm_count;
+  if (grid < 1) grid = 1;
+  const int len = (total + grid - 1) / grid;
+  grid = (total + len - 1) / len;
+  const int slots = 4 * ((a.b - 1) / len + 2);
+  TIMED(K_CONV2_DW, (conv2_dw_tc<<<grid, DW_THREADS, DW_SMEM_BYTES, st>>>(a, wt, ws, len, slots)));
+  *seg_len = len;
+  return slots;
 }
 
 int launch_conv1_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof) {

@@ -118,7 +118,9 @@ int32_t check_cfg(const ps_config* c) {
 // Lays the context's device and pinned buffers out over the two caller-owned blocks.
 void layout(ps_ctx* x, const ps_config& c, void* arena, void* pinned, uint64_t* arena_bytes, uint64_t* pinned_bytes) {
   const uint64_t rows = (uint64_t)c.max_workers * c.max_batch;
-  const uint64_t chunks = ((uint64_t)c.max_batch + psk::CONV_SPB - 1) / psk::CONV_SPB;
+  // partial-sum slots per worker: one per block of CONV_SPB samples, or four per range of the tensor-core
+  // filter-gradient kernel (at most (b - 1) / 16 + 2 ranges meet a worker)
+  const uint64_t chunks = ((uint64_t)c.max_batch + psk::CONV_SPB - 1) / psk::CONV_SPB + 8;
   Carver a(arena);
   for (int i = 0; i < c.ring_depth; ++i) { float* p = a.take<float>(VEC_BYTES); if (x) x->ring[i] = p; }
   for (int i = 0; i + 1 < c.chain_len; ++i) { float* p = a.take<float>(VEC_BYTES); if (x) x->replicas.push_back({p, 0, true}); }
