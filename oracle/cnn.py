@@ -69,7 +69,8 @@ def dropout_keep(seed, worker, step, b, p):
 
 def grad_step_f64(theta, x, y, keep=None, drop_p=0.25, precision=0):
     """One worker, everything double.  Returns (grad[P], loss, argmax[b], logits[b,10]).
-    precision 1: ReLU/pooling decisions are taken on a TF32-operand forward pass (values stay exact)."""
+    precision 1: ReLU/pooling decisions are taken on a TF32-operand forward pass (values stay exact);
+    precision 2: the same with BF16 operands in the second convolution (the 512-unit layer stays TF32)."""
     theta = np.ascontiguousarray(theta, dtype=np.float64)
     x = np.ascontiguousarray(x, dtype=np.float64)
     y = np.ascontiguousarray(y, dtype=np.int32)

@@ -168,21 +168,30 @@ static void pool_bwd(const double* dpooled, const int* code, int c, int hw, doub
  * A tensor-core path rounds the operands of its dense contractions (second convolution, 512-unit
  * layer) to a short mantissa and accumulates exactly enough that the products dominate the error.
  * ReLU signs and pooling winners are integer decisions taken on those rounded results, so the
- * oracle must be able to take them in the same precision: precision 1 rounds an fp32 value to
- * TF32 (10 explicit mantissa bits, round to nearest, ties away from zero). */
-static double round_operand(double v, int precision) {
-    if (precision == 0) return v;
+ * oracle must be able to take them in the same precision.  Rounding modes of an fp32 value:
+ *   0  none
+ *   1  TF32: 10 explicit mantissa bits, round to nearest, ties away from zero
+ *   2  BF16:  7 explicit mantissa bits, round to nearest, ties to even */
+static double round_operand(double v, int mode) {
+    if (mode == 0) return v;
     float f = (float)v;
     uint32_t u;
     memcpy(&u, &f, 4);
-    u = (u + 0x1000u) & 0xFFFFE000u;
+    if (mode == 1) u = (u + 0x1000u) & 0xFFFFE000u;
+    else u = (u + 0x7FFFu + ((u >> 16) & 1u)) & 0xFFFF0000u;
     memcpy(&f, &u, 4);
     return (double)f;
 }
 
-double oracle_round_operand(double v, int32_t precision) { return round_operand(v, precision); }
+double oracle_round_operand(double v, int32_t mode) { return round_operand(v, mode); }
 
-/* conv3x3 with both operands rounded (precision 0 = plain conv3x3). */
+/* Which rounding the two reduced-precision contractions use under a given `precision` of the
+ * gradient step: 1 = TF32 everywhere; 2 = BF16 operands in the second convolution, TF32 in the
+ * 512-unit layer. */
+static int conv_rounding(int precision) { return precision == 2 ? 2 : (precision == 1 ? 1 : 0); }
+static int dense_rounding(int precision) { return precision != 0 ? 1 : 0; }
+
+/* conv3x3 with both operands rounded in the given mode (0 = plain conv3x3). */
 static void conv3x3_rounded(const double* in, int cin, int hw, const double* w, const double* bias,
                             int cout, int precision, double* out) {
     size_t nin = (size_t)cin * hw * hw, nw = (size_t)cout * cin * 9;
@@ -247,6 +256,8 @@ static void conv3x3_bwd_x(const double* dout, int cout, int hw, const double* w,
  *                       tensor-core path takes them, on a second forward pass whose second
  *                       convolution and 512-unit layer use TF32-rounded operands (and fp32-stored
  *                       activations); all VALUES are still the exact double-precision ones.
+ *                       2: the same, with BF16-rounded operands in the second convolution (the
+ *                       512-unit layer stays TF32).
  * Outputs (any may be NULL except grad):
  *   grad   [P]          d(mean loss)/d(theta)
  *   loss                mean over the batch of logsumexp(z) - z[y]
@@ -292,10 +303,10 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
         } else {
             /* decision pass in the kernel's precision: activations are stored as fp32 there */
             for (size_t k = 0; k < np1; ++k) p1q[k] = (double)(float)p1[k];
-            conv3x3_rounded(p1q, C1, H1, c2w, c2b, C2, precision, a2q);
+            conv3x3_rounded(p1q, C1, H1, c2w, c2b, C2, conv_rounding(precision), a2q);
             pool_decide(a2q, C2, H1, i2);
             pool_apply(a2q, i2, C2, H1, p2q);
-            for (size_t k = 0; k < np2; ++k) p2q[k] = round_operand((double)(float)p2q[k], precision);
+            for (size_t k = 0; k < np2; ++k) p2q[k] = round_operand((double)(float)p2q[k], dense_rounding(precision));
         }
         pool_apply(a2, i2, C2, H1, p2); /* p2 is already the channel-major flatten */
         for (int j = 0; j < HID; ++j) {
@@ -306,7 +317,7 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
                 on[j] = s > 0.0;
             } else {
                 double sq = f1b[j];
-                for (int k = 0; k < FLAT; ++k) sq += round_operand(f1w[(size_t)j * FLAT + k], precision) * p2q[k];
+                for (int k = 0; k < FLAT; ++k) sq += round_operand(f1w[(size_t)j * FLAT + k], dense_rounding(precision)) * p2q[k];
                 on[j] = sq > 0.0;
             }
             double h = on[j] ? s : 0.0;

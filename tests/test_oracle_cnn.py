@@ -150,7 +150,7 @@ def test_workers_entry_uses_philox_mask_and_fp32_inputs():
         assert (g == grads[w]).all() and l == loss[w] and (a == am[w]).all() and (z == logits[w]).all()
 
 
-# ---- decisions taken in a tensor-core path's precision (precision=1: TF32 operands) -----------------
+# ---- decisions taken in a tensor-core path's precision (precision=1: TF32 operands; 2: BF16 in conv2) ----
 
 def _tf32_numpy(a):
     """Round fp32 values to TF32 (10 mantissa bits, nearest, ties away) with integer arithmetic."""
@@ -218,3 +218,64 @@ def test_hidden_layer_signs_follow_the_tf32_product():
     on0 = g0[off_b:off_b + 512] != 0
     assert on0.all()
     assert (on1 == (sq > 0)).all()
+
+
+# ---- precision=2: BF16 operands in the second convolution, TF32 in the 512-unit layer -----------------
+
+def _bf16_numpy(a):
+    """Round fp32 values to BF16 (7 mantissa bits, nearest, ties to even) with integer arithmetic."""
+    u = np.asarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = ((u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000).astype(np.uint32)
+    return u.view(np.float32).astype(np.float64)
+
+
+def test_operand_rounding_mode_2_is_bf16_nearest_even():
+    assert cnn.round_operand(1.0, 2) == 1.0
+    assert cnn.round_operand(1.0 + 2.0 ** -8, 2) == 1.0                          # tie, even mantissa below
+    assert cnn.round_operand(1.0 + 3 * 2.0 ** -8, 2) == 1.0 + 2.0 ** -6          # tie, even mantissa above
+    assert cnn.round_operand(1.0 + 2.0 ** -8 + 2.0 ** -20, 2) == 1.0 + 2.0 ** -7
+    assert cnn.round_operand(-(1.0 + 3 * 2.0 ** -8), 2) == -(1.0 + 2.0 ** -6)
+    vals = np.random.default_rng(1).standard_normal(2000).astype(np.float32) * np.float32(3.0)
+    got = np.array([cnn.round_operand(float(v), 2) for v in vals])
+    assert (got == _bf16_numpy(vals)).all()
+    # the library's own fp32 -> bfloat16 conversion agrees
+    assert (got == torch.tensor(vals).to(torch.bfloat16).to(torch.float64).numpy()).all()
+
+
+@pytest.mark.parametrize("precision", [1, 2])
+def test_reduced_precision_decisions_against_a_torch_restatement(precision):
+    """The decisions (pooling winners and ReLU signs of the second convolution, signs of the 512-unit
+    layer) are recomputed with torch's conv2d / max_pool2d / matmul on operands rounded by torch's own
+    casts or integer arithmetic; the exact gradient under those decisions comes from autograd through
+    a graph that gathers the exact pre-activations at the decided positions."""
+    conv_round = _tf32_numpy if precision == 1 else _bf16_numpy
+    b = 3
+    theta, x, y, keep = _case(b, 5)
+    theta = theta.astype(np.float32).astype(np.float64)
+    x = x.astype(np.float32).astype(np.float64)
+    t = torch.tensor(theta, requires_grad=True)
+    seg = lambda name: t[cnn.TENSORS[name][0]:cnn.TENSORS[name][0] + int(np.prod(cnn.TENSORS[name][1]))].reshape(cnn.TENSORS[name][1])
+    rq = lambda v, f: torch.tensor(f(v.detach().numpy().astype(np.float32))).reshape(v.shape)
+    xb = torch.tensor(x).reshape(b, 1, 28, 28)
+    p1 = F.max_pool2d(F.relu(F.conv2d(xb, seg("conv1.w"), seg("conv1.b"), padding=1)), 2)
+    # decision pass on rounded operands
+    a2q = F.conv2d(rq(p1, conv_round), rq(seg("conv2.w"), conv_round), seg("conv2.b").detach(), padding=1)
+    p2q, idx = F.max_pool2d(F.relu(a2q), 2, return_indices=True)
+    live2 = (p2q > 0).double()
+    uq = rq(p2q, _tf32_numpy).flatten(1) @ rq(seg("fc1.w"), _tf32_numpy).T + seg("fc1.b").detach()
+    on = (uq > 0).double()
+    # exact values under those decisions
+    a2 = F.conv2d(p1, seg("conv2.w"), seg("conv2.b"), padding=1)
+    p2 = (a2.flatten(2).gather(2, idx.flatten(2)).reshape(p2q.shape) * live2).flatten(1)
+    h = F.linear(p2, seg("fc1.w"), seg("fc1.b")) * on
+    d = h * torch.tensor(keep, dtype=torch.float64) / 0.75
+    z = F.linear(d, seg("fc2.w"), seg("fc2.b"))
+    loss = F.cross_entropy(z, torch.tensor(y, dtype=torch.long), reduction="mean")
+    loss.backward()
+    g, l, am, logits = cnn.grad_step_f64(theta, x, y, keep, 0.25, precision=precision)
+    assert abs(l - float(loss.detach())) < 1e-12
+    ref = t.grad.numpy()
+    assert np.abs(g - ref).max() <= 1e-11 * max(1.0, np.abs(ref).max())
+    # the case is a discriminating one: these decisions differ from the exact ones and from the other mode's
+    for other in {0, 1, 2} - {precision}:
+        assert (cnn.grad_step_f64(theta, x, y, keep, 0.25, precision=other)[0] != g).sum() > 1000
