@@ -1,20 +1,20 @@
 // Second convolution (16 -> 32 channels, 3x3, pad 1, 14x14 maps) on the fifth-generation tensor cores:
-// forward with fused ReLU + 2x2 max pooling, and the gradient with respect to the input.
+// forward with fused ReLU + 2x2 max pooling, and the gradient with respect to the input.  BF16 operands,
+// fp32 accumulation in tensor memory.
 //
 // Both are implicit products with k = (filter tap, channel).  The trick that makes them fit
 // tcgen05.mma without an im2col copy: an un-swizzled k-contiguous shared-memory operand is a stack of
-// "core matrices" of 8 rows x 16 bytes, so if the image is stored as planes of FOUR channels
-// (one position = one 16-byte row), then for a fixed filter tap the operand "all positions x 4 channels"
-// is just that plane read from a shifted start address.  One MMA (K = 8) takes two such planes.
+// "core matrices" of 8 rows x 16 bytes, so if the image is stored as planes of EIGHT BF16 channels
+// (one position = one 16-byte row), then for a fixed filter tap the operand "all positions x 8 channels"
+// is just that plane read from a shifted start address.  One MMA (K = 16) takes two such planes.
 //
 // Forward: rows are POOLED positions and the four pre-pool window elements go to four accumulators
 // (four column ranges of tensor memory), so that a thread of the epilogue holds the whole 2x2 window
 // and pools without exchanging data.  For that the planes keep even and odd columns apart
 // (position (Y, X) at row Y*16 + (X&1)*8 + X/2): consecutive pooled columns are then consecutive rows.
 //
-// Warp roles per CTA (288 threads): warp 0 issues the MMAs and owns tensor memory, warps 1-4 stage the
-// next tile's planes into shared memory, warps 5-8 run the epilogue of the previous tile; the three
-// stages overlap through mbarriers, and every wait is bounded.
+// The stages of each kernel (staging, MMA issue, epilogue) run in different warps and overlap through
+// mbarriers; every wait is bounded.
 #include "device_common.cuh"
 #include "kernels.h"
 #include "tc5_common.cuh"
@@ -27,16 +27,8 @@ constexpr int C5_SPB = 16;            // samples per CTA
 constexpr int THREADS = 288;
 constexpr int LOADERS = 128;
 
-__host__ __device__ constexpr uint32_t idesc_tf32(int m, int n) {
-  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
 __host__ __device__ constexpr uint32_t idesc_bf16(int m, int n) {     // fp32 accumulate, BF16 x BF16, k-contiguous
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
-__device__ __forceinline__ uint16_t bf16_bits(float x) {
-  uint16_t r;
-  asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(x));
-  return r;
 }
 
 // Barrier over the 128 staging threads that also tells every one of them whether any of them failed.
@@ -70,7 +62,7 @@ __device__ __forceinline__ void pipe_init(Pipe* p, int a_full_arrivals, int acc_
 // ------------------------------------------------------------------------------------------------
 // Forward.  Tile = two samples = 128 rows: row 8*g + i is pooled position (py = g mod 8, px = i) of
 // sample g / 8 (py = 7 and px = 7 are padding rows whose results are dropped).  The first convolution
-// already wrote its output in the plane layout, borders included, so staging a tile is eight plain
+// already wrote its output in the plane layout, borders included, so staging a tile is four plain
 // bulk copies of 4 KB issued by one thread.
 // Warps: 0 = MMA issuer and tensor-memory owner, 1 = copy producer, 2..9 = epilogue (warp w reads the
 // accumulator lanes of quarter w mod 4 and the output channels of half (w-2)/4).
@@ -78,14 +70,14 @@ __device__ __forceinline__ void pipe_init(Pipe* p, int a_full_arrivals, int acc_
 constexpr int F_THREADS = 320;
 constexpr int F_PLANE_ROWS = 2 * 256 + 32;                 // two stacked 16x16 images + overrun of the padding rows
 constexpr int F_PLANE_BYTES = F_PLANE_ROWS * 16;           // 8704
-constexpr int F_BUF_BYTES = 4 * F_PLANE_BYTES;             // four channel quads
-constexpr int F_W_BYTES = 36 * 32 * 16;                    // [k quad = tap*4 + ic/4][oc][4]
+constexpr int F_BUF_BYTES = 2 * F_PLANE_BYTES;             // two planes of eight channels
+constexpr int F_W_BYTES = 18 * 32 * 16;                    // [k chunk = tap*2 + ic/8][oc][8 bf16]
 constexpr int F_SMEM = 2 * F_BUF_BYTES + F_W_BYTES + 32 * 4 + sizeof(Pipe) + 128;
 
 __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   extern __shared__ __align__(128) uint8_t smem[];
-  float* bufs = reinterpret_cast<float*>(smem);
-  float* Wk = reinterpret_cast<float*>(smem + 2 * F_BUF_BYTES);
+  uint8_t* bufs = smem;
+  uint16_t* Wk = reinterpret_cast<uint16_t*>(smem + 2 * F_BUF_BYTES);
   float* bias = reinterpret_cast<float*>(smem + 2 * F_BUF_BYTES + F_W_BYTES);
   Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * F_BUF_BYTES + F_W_BYTES + 128);
   const int s = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -95,12 +87,12 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
 
   for (int idx = tid; idx < 4608; idx += F_THREADS) {
     int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
-    Wk[((tap * 4 + (ic >> 2)) * 32 + oc) * 4 + (ic & 3)] = round_tf32(theta[OFF_C2W + idx]);
+    Wk[((tap * 2 + (ic >> 3)) * 32 + oc) * 8 + (ic & 7)] = bf16_bits(theta[OFF_C2W + idx]);
   }
   if (tid < 32) bias[tid] = theta[OFF_C2B + tid];
   // rows never written by a copy (the overrun of the padding rows, a missing second sample) only feed
   // results that are dropped; they are cleared once so that those results stay finite
-  for (int idx = tid; idx < 2 * F_BUF_BYTES / 16; idx += F_THREADS) reinterpret_cast<float4*>(bufs)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int idx = tid; idx < 2 * F_BUF_BYTES / 16; idx += F_THREADS) reinterpret_cast<float4*>(smem)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
   if (tid == 0) pipe_init(pipe, 1, 8);
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(256) : "memory");
@@ -114,7 +106,7 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
 
   if (warp == 0) {
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_tf32(128, 32);
+      constexpr uint32_t idesc = idesc_bf16(128, 32);
       const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), 512);
       for (int t = 0; t < n_tiles; ++t) {
         const int buf = t & 1;
@@ -122,8 +114,9 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
         if (t >= 2 && !mbar_wait(&pipe->acc_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
         if (pipe->abort_flag) break;
         tc_fence_after();
-        // 72 MMAs, fully unrolled: every descriptor is a per-tile base plus a compile-time constant
-        const uint32_t a_lo = plain_desc_lo(smem_u32(bufs) + buf * F_BUF_BYTES, F_PLANE_BYTES);
+        // 36 MMAs (one per window element and tap: K = 16 channels), fully unrolled: every descriptor is a
+        // per-tile base plus a compile-time constant
+        const uint32_t a_lo = plain_desc_lo(smem_u32(smem) + buf * F_BUF_BYTES, F_PLANE_BYTES);
         const uint32_t d_tmem = tmem + buf * 128;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -132,10 +125,8 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
           for (int tap = 0; tap < 9; ++tap) {
             const int ky = tap / 3, kx = tap - ky * 3, sx = jx + kx;
             const int row_off = (jy + ky) * 16 + (sx & 1) * 8 + (sx >> 1);     // in 16-byte rows
-#pragma unroll
-            for (int half = 0; half < 2; ++half)
-              umma_tf32_split(d_tmem + j * 32, a_lo + (2 * half) * (F_PLANE_BYTES / 16) + row_off, plain_desc_hi(512),
-                              w_lo + (tap * 4 + half * 2) * (512 / 16), plain_desc_hi(128), idesc, (tap | half) ? 1u : 0u);
+            umma_f16_split(d_tmem + j * 32, a_lo + row_off, plain_desc_hi(512), w_lo + (tap * 2) * (512 / 16),
+                           plain_desc_hi(128), idesc, tap ? 1u : 0u);
           }
         }
         umma_commit(&pipe->a_empty[buf]);
@@ -149,11 +140,11 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
         if (t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
         if (pipe->abort_flag) break;
         const int n_s = min(2, i_end - (i_begin + 2 * t));
-        mbar_expect_tx(&pipe->a_full[buf], (uint32_t)n_s * 4 * 4096u);
+        mbar_expect_tx(&pipe->a_full[buf], (uint32_t)n_s * 2 * 4096u);
         for (int sp = 0; sp < n_s; ++sp) {
           const float* src = ws.p1 + ((int64_t)s * a.b + i_begin + 2 * t + sp) * P1_PLANE_ELEMS;
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
+          for (int q = 0; q < 2; ++q)
             bulk_load(smem + buf * F_BUF_BYTES + q * F_PLANE_BYTES + sp * 4096, src + q * 1024, 4096, &pipe->a_full[buf]);
         }
       }

@@ -18,9 +18,9 @@ namespace {
 // worker.  Thread = pooled position: it reads the 4x4 input patch under its 2x2 window once and
 // evaluates all 16 channels from registers (576 multiply-adds per 8 + 48 shared-memory loads).
 // PLANES selects the output layout: the compact [channel][14*14] rows of the FP32 path, or the layout
-// the tensor-core convolution copies straight into shared memory: per sample four planes of four
-// channels, one 16-byte row per position of a zero-bordered 16x16 grid with even and odd columns apart
-// (row = Y*16 + (X&1)*8 + X/2, Y = y+1, X = x+1), values rounded to TF32.
+// the tensor-core convolution copies straight into shared memory: per sample two planes of eight
+// channels in BF16, one 16-byte row per position of a zero-bordered 16x16 grid with even and odd columns
+// apart (row = Y*16 + (X&1)*8 + X/2, Y = y+1, X = x+1).
 constexpr int CONV1_SPB = 8;
 template <bool PLANES>
 __global__ void __launch_bounds__(224) conv1_fwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
@@ -88,11 +88,11 @@ __global__ void __launch_bounds__(224) conv1_fwd(GradStepArgs a, WorkerTable wt,
     for (int ch = 0; ch < 16; ++ch) ws.code1[row * P1_ELEMS + ch * 196 + pp] = outc[ch];
     if (PLANES) {
       const int X = px + 1, Y = py + 1;
-      float* dst = ws.p1 + row * P1_PLANE_ELEMS + (Y * 16 + (X & 1) * 8 + (X >> 1)) * 4;
+      uint4* dst = reinterpret_cast<uint4*>(ws.p1 + row * P1_PLANE_ELEMS) + (Y * 16 + (X & 1) * 8 + (X >> 1));
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
-        *reinterpret_cast<float4*>(dst + q * 1024) = make_float4(round_tf32(outv[4 * q]), round_tf32(outv[4 * q + 1]),
-                                                                  round_tf32(outv[4 * q + 2]), round_tf32(outv[4 * q + 3]));
+      for (int q = 0; q < 2; ++q)
+        dst[q * 256] = make_uint4(bf16_pair(outv[8 * q], outv[8 * q + 1]), bf16_pair(outv[8 * q + 2], outv[8 * q + 3]),
+                                  bf16_pair(outv[8 * q + 4], outv[8 * q + 5]), bf16_pair(outv[8 * q + 6], outv[8 * q + 7]));
     } else {
 #pragma unroll
       for (int ch = 0; ch < 16; ++ch) ws.p1[row * P1_ELEMS + ch * 196 + pp] = outv[ch];

@@ -11,8 +11,6 @@ namespace psk {
 
 namespace {
 
-constexpr int TC_SPB = 8;
-
 // Filter gradient: dW[oc][ic][tap] = sum_{samples,pos} g2[oc][pos] * p1[ic][pos + tap]: rows = 32 output
 // channels, columns = 16 input channels per tap, k = position (196 per sample, 13 k-steps of 16, zero-padded).
 // Both operands are rounded to BF16 here (fp32 accumulation): this product only yields gradient values, no
@@ -39,16 +37,6 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
-__device__ __forceinline__ uint16_t bf16_bits(float x) {
-  uint16_t r;
-  asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(x));
-  return r;
-}
-__device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {   // lo in the low half (lower k index)
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
 
 constexpr int DW_G_WORDS = 108;    // 216 bf16 per output channel: 196 positions + zeros; 108 = 12 (mod 32 banks)
 constexpr int DW_P_WORDS = 132;    // plane of one input channel: 16 rows x 14 bf16 (rows 0 and 15 stay zero) = 112
@@ -64,7 +52,7 @@ constexpr int DW_NRAW = 3;         // raw input buffers: copies run three sample
 constexpr int DW_SMEM_BYTES = (2 * DW_BUF_WORDS + DW_NRAW * DW_RAW_WORDS) * 4 + 128;
 static_assert(DW_RAW_P1 % 16 == 0 && DW_RAW_DP2 % 16 == 0 && DW_RAW_CODE % 16 == 0, "bulk copies move multiples of 16 bytes");
 constexpr int DW_MIN_SEG = 16;     // a CTA's range is at least this long (bounds the partial sums per worker)
-constexpr int DW_PAIRS = (4 * 98 + DW_LOADERS - 1) / DW_LOADERS;      // 2 (plane, position pair) items per loader thread
+constexpr int DW_PAIRS = (2 * 98 + DW_LOADERS - 1) / DW_LOADERS;      // (plane, position pair) items per loader thread
 constexpr int DW_ENTRIES = (FLAT + DW_LOADERS - 1) / DW_LOADERS;      // 7 pooled gradient entries per loader thread
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
@@ -150,29 +138,30 @@ __global__ void __launch_bounds__(DW_THREADS, 1) conv2_dw_tc(GradStepArgs a, Wor
       const float* rdp2 = rp1 + P1_PLANE_ELEMS;
       const uint8_t* rcode = reinterpret_cast<const uint8_t*>(rdp2 + FLAT);
       uint32_t* g2w = dw_smem + buf * DW_BUF_WORDS;
-      // Item = (plane q of four channels, pair w of horizontally adjacent positions 2w, 2w+1 of the flattened
+      // Item = (plane q of eight channels, pair w of horizontally adjacent positions 2w, 2w+1 of the flattened
       // 14-wide image).  Word w + 7 of a channel's plane holds positions (x, x+1) in the middle copy,
       // (x-1, x) in the copy of the left taps and (x+1, x+2) in the copy of the right taps; x-1 = -1 and
-      // x+2 = 14 read the zero border of the source plane.
+      // x+2 = 14 read the zero border of the source plane.  The source is already BF16 (one position =
+      // eight channels = 16 bytes), so a pair is two half-words picked out of two rows.
 #pragma unroll
       for (int k = 0; k < DW_PAIRS; ++k) {
         const int e = lt + k * DW_LOADERS;
-        if (e < 4 * 98) {
+        if (e < 2 * 98) {
           const int q = e / 98, w = e - q * 98, y = w / 7, x = 2 * (w - y * 7);
-          const float* src = rp1 + q * 1024 + (y + 1) * 64;        // row Y = y + 1: even X in floats 0..31, odd X in 32..63
+          const uint4* src = reinterpret_cast<const uint4*>(rp1) + q * 256 + (y + 1) * 16;   // row Y = y + 1: even X in rows 0..7, odd X in 8..15
           // X = x + 1 + j for j = -1..2: X = x (even), x + 1 (odd), x + 2 (even), x + 3 (odd)
-          const float4 v0 = *reinterpret_cast<const float4*>(src + (x >> 1) * 4);
-          const float4 v1 = *reinterpret_cast<const float4*>(src + 32 + (x >> 1) * 4);
-          const float4 v2 = *reinterpret_cast<const float4*>(src + ((x >> 1) + 1) * 4);
-          const float4 v3 = *reinterpret_cast<const float4*>(src + 32 + ((x >> 1) + 1) * 4);
-          const float a0[4] = {v0.x, v0.y, v0.z, v0.w}, a1[4] = {v1.x, v1.y, v1.z, v1.w};
-          const float a2[4] = {v2.x, v2.y, v2.z, v2.w}, a3[4] = {v3.x, v3.y, v3.z, v3.w};
-          uint32_t* d = g2w + 32 * DW_G_WORDS + (4 * q) * DW_P_WORDS + w + 7;
+          const uint4 v0 = src[x >> 1], v1 = src[8 + (x >> 1)], v2 = src[(x >> 1) + 1], v3 = src[8 + (x >> 1) + 1];
+          const uint32_t a0[4] = {v0.x, v0.y, v0.z, v0.w}, a1[4] = {v1.x, v1.y, v1.z, v1.w};
+          const uint32_t a2[4] = {v2.x, v2.y, v2.z, v2.w}, a3[4] = {v3.x, v3.y, v3.z, v3.w};
+          uint32_t* d = g2w + 32 * DW_G_WORDS + (8 * q) * DW_P_WORDS + w + 7;
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            d[c * DW_P_WORDS] = bf16_pair(a0[c], a1[c]);
-            d[(16 + c) * DW_P_WORDS] = bf16_pair(a1[c], a2[c]);
-            d[(32 + c) * DW_P_WORDS] = bf16_pair(a2[c], a3[c]);
+          for (int j = 0; j < 4; ++j) {      // word j of a row holds channels 2j (low half) and 2j + 1 (high half)
+            d[(2 * j) * DW_P_WORDS] = __byte_perm(a0[j], a1[j], 0x5410);
+            d[(2 * j + 1) * DW_P_WORDS] = __byte_perm(a0[j], a1[j], 0x7632);
+            d[(16 + 2 * j) * DW_P_WORDS] = __byte_perm(a1[j], a2[j], 0x5410);
+            d[(16 + 2 * j + 1) * DW_P_WORDS] = __byte_perm(a1[j], a2[j], 0x7632);
+            d[(32 + 2 * j) * DW_P_WORDS] = __byte_perm(a2[j], a3[j], 0x5410);
+            d[(32 + 2 * j + 1) * DW_P_WORDS] = __byte_perm(a2[j], a3[j], 0x7632);
           }
         }
       }

@@ -19,7 +19,7 @@ constexpr int OFF_F1W = 4800, OFF_F1B = 807616, OFF_F2W = 808128, OFF_F2B = 8132
 
 constexpr int IMG = 28, C1 = 16, H1 = 14, C2 = 32, H2 = 7;
 constexpr int P1_ELEMS = C1 * H1 * H1;   // 3136
-constexpr int P1_PLANE_ELEMS = 4 * 256 * 4;   // 4096: p1 of one sample in the tensor-core plane layout
+constexpr int P1_PLANE_ELEMS = 2 * 256 * 4;   // 32-bit words of one sample's p1 in the tensor-core plane layout (8 KB of BF16)
 constexpr int FLAT = C2 * H2 * H2;       // 1568
 constexpr int HID = 512, NCLS = 10;
 constexpr int DZ_STRIDE = 16;            // logits gradient row, padded
@@ -93,7 +93,7 @@ struct GroupTable {
 
 // Activation workspace carved from the arena (rows = sorted worker * b + sample).
 struct Workspace {
-  float* p1;       // conv1 -> ReLU -> pool: [rows][16][14][14] (FP32 path) or [rows][4 planes][256][4] (tensor-core path)
+  float* p1;       // conv1 -> ReLU -> pool: [rows][16][14][14] fp32 (FP32 path) or [rows][2 planes][256][8] BF16 (tensor-core path)
   uint8_t* code1;  // [rows][3136]        pool-1 argmax 0..3, 4 = no gradient (max <= 0)
   float* p2;       // [rows][1568]        conv2 -> ReLU -> pool, channel-major flatten
   uint8_t* code2;  // [rows][1568]
@@ -118,7 +118,7 @@ struct GradStepArgs {
   uint64_t seed, step;
   float drop_p;
   uint32_t drop_thresh;   // keep iff word >= thresh
-  int precision;          // 0 = FP32 CUDA cores, 1 = TF32 tensor cores for the dense contractions
+  int precision;          // 0 = FP32 CUDA cores; otherwise tensor cores (BF16 convolution products, TF32 dense layer)
 };
 
 // Side streams (and the events that fork from / join into the caller's stream) for the independent

@@ -109,7 +109,7 @@ int32_t check_cfg(const ps_config* c) {
   if (c->chain_len < 1 || c->chain_len > 8) return fail(PS_ERR_BAD_ARG, "chain_len must be 1..8");
   if (c->replicate_every < 1) return fail(PS_ERR_BAD_ARG, "replicate_every must be >= 1");
   if (c->external_store != 0 && c->external_store != 1) return fail(PS_ERR_BAD_ARG, "external_store must be 0 or 1");
-  if (c->precision != PS_FP32 && c->precision != PS_TF32) return fail(PS_ERR_BAD_ARG, "precision %d is not built (PS_FP32 and PS_TF32 are)", c->precision);
+  if (c->precision != PS_FP32 && c->precision != PS_BF16) return fail(PS_ERR_BAD_ARG, "precision %d is not built (PS_FP32 and PS_BF16 are)", c->precision);
   if (!(c->dropout_p >= 0.f) || !(c->dropout_p < 1.f)) return fail(PS_ERR_BAD_ARG, "dropout_p must be in [0,1)");
   if (c->queue_slots < 1) return fail(PS_ERR_BAD_ARG, "queue_slots must be >= 1");
   return PS_OK;

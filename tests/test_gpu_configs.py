@@ -92,12 +92,12 @@ def test_reduced_configs_on_the_tf32_path(n):
     # (The async config is left to the FP32 run: only the head can be loaded with the oracle's weights,
     # not the older ring versions its stale readers use; grouped stale snapshots under TF32 are covered
     # by the grad-step tests, where both sides hold identical versions.)
-    s, srv, o, glog, _ = _follow(n, precision=1, lock_from=1)
+    s, srv, o, glog, _ = _follow(n, precision=2, lock_from=1)
     assert glog[-1]["version"] == o.version
     srv.close()
 
 
-@pytest.mark.parametrize("precision", [0, 1])
+@pytest.mark.parametrize("precision", [0, 2])
 def test_full_size_config5_tick_on_sampled_workers(precision):
     """W=128 x b=128 in the launch configuration the benchmark times; the oracle recomputes three workers."""
     tol = TOL_TENSOR if precision else TOL_FP32

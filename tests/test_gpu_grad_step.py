@@ -83,12 +83,12 @@ def test_stale_snapshots_grouped_over_three_versions():
                                      (5, 6, {"lags": [2, 0, 1, 2, 0], "n_versions": 3}), (1, 1, {}),
                                      (2, 4, {"drop_p": 0.0})])
 def test_tf32_tensor_core_path(W, b, kw):
-    _run_and_compare(W, b, precision=1, **kw)
+    _run_and_compare(W, b, precision=2, **kw)
 
 
 def test_tf32_repeatable_bit_for_bit():
-    a = _run_and_compare(3, 9, precision=1)
-    b = _run_and_compare(3, 9, precision=1)
+    a = _run_and_compare(3, 9, precision=2)
+    b = _run_and_compare(3, 9, precision=2)
     assert (a == b).all()
 
 
