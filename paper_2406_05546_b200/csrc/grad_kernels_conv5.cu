@@ -76,7 +76,6 @@ constexpr int F_SMEM = 2 * F_BUF_BYTES + F_W_BYTES + 32 * 4 + sizeof(Pipe) + 128
 
 __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   extern __shared__ __align__(128) uint8_t smem[];
-  uint8_t* bufs = smem;
   uint16_t* Wk = reinterpret_cast<uint16_t*>(smem + 2 * F_BUF_BYTES);
   float* bias = reinterpret_cast<float*>(smem + 2 * F_BUF_BYTES + F_W_BYTES);
   Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * F_BUF_BYTES + F_W_BYTES + 128);

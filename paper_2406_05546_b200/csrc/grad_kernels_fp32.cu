@@ -259,8 +259,9 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 // ---- fc2 forward, softmax cross-entropy, argmax, and the backward pass down to the gradient with
 // respect to fc1's pre-activation; then the worker's fc2 weight/bias and fc1 bias gradients.
-// One block of 16 warps per worker: first one warp per sample at a time; then thread = hidden unit sums its
-// outputs over the worker's samples in sample order, several loads in flight.
+// FC2_SPLIT blocks of 16 warps per worker, each with its share of the worker's samples: first two samples per
+// warp at a time; then thread = hidden unit sums its outputs over the block's samples in sample order, several
+// loads in flight.  The block's sums (and its share of the loss) are partial results added later in block order.
 constexpr int FC2_THREADS = 512;
 __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   __shared__ float w2[NCLS][HID];
@@ -269,6 +270,8 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
   const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* theta = group_theta(wt, gt, s);
   const int src = wt.src[s];
+  const int per = ((a.b + FC2_SPLIT - 1) / FC2_SPLIT + 1) & ~1;          // samples per block, even
+  const int i_lo = min(a.b, (int)blockIdx.y * per), i_hi = min(a.b, i_lo + per);
   for (int t = tid; t < NCLS * HID; t += FC2_THREADS) (&w2[0][0])[t] = theta[OFF_F2W + t];
   if (tid < NCLS) b2[tid] = theta[OFF_F2B + tid];
   __syncthreads();
@@ -276,8 +279,8 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
   const float inv_b = 1.0f / (float)a.b;
   float loss_acc = 0.f;
   // two samples per warp and pass, so that every weight read from shared memory is used twice
-  for (int i0 = 2 * warp; i0 < a.b; i0 += 2 * (FC2_THREADS / 32)) {
-    const bool two = i0 + 1 < a.b;                       // warp-uniform
+  for (int i0 = i_lo + 2 * warp; i0 < i_hi; i0 += 2 * (FC2_THREADS / 32)) {
+    const bool two = i0 + 1 < i_hi;                      // warp-uniform
     // the weights are re-read from shared memory on every pass: 160 of them per lane would not fit in the
     // registers of a 512-thread block, so their address is made to look pass-dependent
     uint32_t opaque_zero;
@@ -372,12 +375,12 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
   }
   if (lane == 0) warp_loss[warp] = loss_acc;
   __syncthreads();   // also makes this block's dz / da1 stores visible to all of its threads
+  float* part = ws.partf + ((int64_t)s * FC2_SPLIT + blockIdx.y) * FC_PART;
   if (tid == 0) {
     float t = 0.f;
     for (int w = 0; w < FC2_THREADS / 32; ++w) t += warp_loss[w];
-    a.loss[src] = t * inv_b;
+    part[NCLS * HID + HID + NCLS] = t;
   }
-  float* grad = wt.grad[s];
   const int j = tid;                                  // hidden unit (FC2_THREADS == HID)
   float gw[NCLS], gb1 = 0.f, gb2 = 0.f;
 #pragma unroll
@@ -386,7 +389,7 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
   const float* dp = ws.d + (int64_t)s * a.b * HID + j;
   const float* da1p = ws.da1 + (int64_t)s * a.b * HID + j;
 #pragma unroll 4
-  for (int i = 0; i < a.b; ++i) {
+  for (int i = i_lo; i < i_hi; ++i) {
     const float dval = dp[(int64_t)i * HID];
     const float4 z0 = *reinterpret_cast<const float4*>(dzp + i * DZ_STRIDE);
     const float4 z1 = *reinterpret_cast<const float4*>(dzp + i * DZ_STRIDE + 4);
@@ -398,9 +401,9 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
     if (j < NCLS) gb2 += dzp[i * DZ_STRIDE + j];
   }
 #pragma unroll
-  for (int c = 0; c < NCLS; ++c) grad[OFF_F2W + c * HID + j] = gw[c];
-  grad[OFF_F1B + j] = gb1;
-  if (j < NCLS) grad[OFF_F2B + j] = gb2;
+  for (int c = 0; c < NCLS; ++c) part[c * HID + j] = gw[c];
+  part[NCLS * HID + j] = gb1;
+  if (j < NCLS) part[NCLS * HID + HID + j] = gb2;
 }
 
 // ---- fc1 weight gradient of one worker: dW1 [512][1568] = da1^T [512 x b] * p2 [b x 1568].
@@ -594,25 +597,48 @@ __global__ void __launch_bounds__(256) conv1_bwd(GradStepArgs a, WorkerTable wt,
   }
 }
 
-// ---- sums the per-block partial convolution gradients in block order and zeroes the padding.
+// ---- sums the per-block partial gradients in block order, finishes the loss and zeroes the padding.
 // part2 holds n_chunks2 slots per worker; all of them are summed when seg_len == 0, otherwise four for every
 // range of seg_len rows that meets the worker's b rows (the tensor-core filter-gradient kernel's layout).
-__global__ void __launch_bounds__(256) conv_grad_reduce(WorkerTable wt, Workspace ws, int n_chunks, int n_chunks2,
-                                                        int seg_len, int b) {
-  const int s = blockIdx.x, tid = threadIdx.x;
+// A worker's outputs are numbered conv2 (4640), conv1 (160), output layer (5642), loss, padding; a block takes
+// RED_PER_BLOCK of them.
+constexpr int RED_PER_BLOCK = 1024;
+constexpr int RED_OUTPUTS = C2_GRAD + C1_GRAD + (NCLS * HID + HID + NCLS) + 1 + (P_PAD - P);
+constexpr int RED_BLOCKS = (RED_OUTPUTS + RED_PER_BLOCK - 1) / RED_PER_BLOCK;
+__global__ void __launch_bounds__(256) conv_grad_reduce(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks, int n_chunks2,
+                                                        int seg_len) {
+  const int s = blockIdx.x, b = a.b;
   float* grad = wt.grad[s];
   const int used2 = seg_len > 0 ? 4 * ((s * b + b - 1) / seg_len - (s * b) / seg_len + 1) : n_chunks2;
-  for (int o = tid; o < C2_GRAD; o += 256) {
-    float t = 0.f;
-    for (int c = 0; c < used2; ++c) t += ws.part2[((int64_t)s * n_chunks2 + c) * C2_GRAD + o];
-    grad[OFF_C2W + o] = t;
+  for (int v = blockIdx.y * RED_PER_BLOCK + threadIdx.x; v < min(RED_OUTPUTS, ((int)blockIdx.y + 1) * RED_PER_BLOCK); v += 256) {
+    int o = v;
+    if (o < C2_GRAD) {
+      float t = 0.f;
+      for (int c = 0; c < used2; ++c) t += ws.part2[((int64_t)s * n_chunks2 + c) * C2_GRAD + o];
+      grad[OFF_C2W + o] = t;
+      continue;
+    }
+    o -= C2_GRAD;
+    if (o < C1_GRAD) {
+      float t = 0.f;
+      for (int c = 0; c < n_chunks; ++c) t += ws.part1[((int64_t)s * n_chunks + c) * C1_GRAD + o];
+      grad[OFF_C1W + o] = t;
+      continue;
+    }
+    o -= C1_GRAD;
+    if (o <= NCLS * HID + HID + NCLS) {
+      float t = 0.f;
+#pragma unroll
+      for (int c = 0; c < FC2_SPLIT; ++c) t += ws.partf[((int64_t)s * FC2_SPLIT + c) * FC_PART + o];
+      if (o < NCLS * HID) grad[OFF_F2W + o] = t;
+      else if (o < NCLS * HID + HID) grad[OFF_F1B + o - NCLS * HID] = t;
+      else if (o < NCLS * HID + HID + NCLS) grad[OFF_F2B + o - NCLS * HID - HID] = t;
+      else a.loss[wt.src[s]] = t * (1.0f / (float)b);
+      continue;
+    }
+    o -= NCLS * HID + HID + NCLS + 1;
+    grad[P + o] = 0.f;
   }
-  for (int o = tid; o < C1_GRAD; o += 256) {
-    float t = 0.f;
-    for (int c = 0; c < n_chunks; ++c) t += ws.part1[((int64_t)s * n_chunks + c) * C1_GRAD + o];
-    grad[OFF_C1W + o] = t;
-  }
-  for (int o = P + tid; o < P_PAD; o += 256) grad[o] = 0.f;
 }
 
 // ---- the keep mask on its own: thread e/4 draws the four words of elements 4*(e/4) .. +3.
@@ -662,7 +688,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof);
     if (n < 0) return -1;
     launches += 2 + n;
-    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<dim3(a.W, FC2_SPLIT), FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
     launches += 1;
     cudaStream_t s1 = side.s1 ? side.s1 : st, s2 = side.s2 ? side.s2 : st;
     if (side.s1) { cudaEventRecord(side.fork1, st); cudaStreamWaitEvent(s1, side.fork1, 0); }
@@ -680,18 +706,18 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     const int n_chunks1t = launch_conv1_bwd_tc(a, wt, ws, st, prof);
     if (side.s1) cudaStreamWaitEvent(st, side.join1, 0);
     if (side.s2) cudaStreamWaitEvent(st, side.join2, 0);
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks1t, n_chunks2, seg_len, a.b)));
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1t, n_chunks2, seg_len)));
     launches += 4;
   } else {
     TIMED(K_CONV1_FWD, (conv1_fwd<false><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
-    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<a.W, FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<dim3(a.W, FC2_SPLIT), FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
     TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
     TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks1b, a.W), 256, 0, st>>>(a, wt, ws, n_chunks1b)));
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<a.W, 256, 0, st>>>(wt, ws, n_chunks1b, n_chunks2, 0, a.b)));
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1b, n_chunks2, 0)));
     launches = 9;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;

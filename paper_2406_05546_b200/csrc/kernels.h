@@ -25,6 +25,8 @@ constexpr int HID = 512, NCLS = 10;
 constexpr int DZ_STRIDE = 16;            // logits gradient row, padded
 constexpr int CONV_SPB = 4;              // samples per block in the conv backward kernels
 constexpr int C2_GRAD = 4608 + 32, C1_GRAD = 144 + 16;
+constexpr int FC2_SPLIT = 1;             // blocks per worker in the output-layer kernel, each with its own partial sums (at 128 registers x 512 threads one block fills an SM, so more blocks only queue)
+constexpr int FC_PART = NCLS * HID + HID + NCLS + 2;   // fc2.w, fc1.b, fc2.b gradients, loss sum, padding
 
 constexpr uint32_t STATUS_BAD_LABEL = 1u;
 constexpr uint32_t STATUS_WAIT_TIMEOUT = 2u;   // a bounded barrier wait in a tensor-core kernel gave up
@@ -104,6 +106,7 @@ struct Workspace {
   float* dp1;      // [rows][3136]        gradient w.r.t. p1
   float* part2;    // [W][chunks][4640]   per-block partial conv2 weight/bias gradients
   float* part1;    // [W][chunks][160]    per-block partial conv1 weight/bias gradients
+  float* partf;    // [W][FC2_SPLIT][FC_PART] per-block partial output-layer gradients and loss sums
   float* w1r;      // [groups][512][1568] TF32-rounded fc1 weights of each weight group of the call
   float* w1tr;     // [groups][1568][512] and their transpose
   uint32_t* status;
