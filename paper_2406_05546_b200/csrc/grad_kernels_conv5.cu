@@ -327,10 +327,10 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
         tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 32 + m * 16), v);
         tmem_ld_wait();
         const int r = m * 128 + quarter * 32 + lane, y = r >> 4, x = r & 15;
-        if (y < 14 && x < 14) {
-          float* out = ws.dp1 + row * P1_ELEMS + y * 14 + x;
+        if (y < 14 && x < 14) {      // dp1 of a sample is [channel quad][position][4 channels]: a warp writes 448 contiguous bytes
+          uint4* out = reinterpret_cast<uint4*>(ws.dp1 + row * P1_ELEMS) + (y * 14 + x);
 #pragma unroll
-          for (int ic = 0; ic < 16; ++ic) out[ic * 196] = __uint_as_float(v[ic]);
+          for (int q = 0; q < 4; ++q) out[q * 196] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
         }
       }
       tc_fence_before();

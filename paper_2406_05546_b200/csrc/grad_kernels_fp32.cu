@@ -17,12 +17,8 @@ namespace {
 // ---- conv1 (1->16, 3x3, pad 1) + ReLU + 2x2 max pool.  A block handles up to CONV1_SPB samples of one
 // worker.  Thread = pooled position: it reads the 4x4 input patch under its 2x2 window once and
 // evaluates all 16 channels from registers (576 multiply-adds per 8 + 48 shared-memory loads).
-// PLANES selects the output layout: the compact [channel][14*14] rows of the FP32 path, or the layout
-// the tensor-core convolution copies straight into shared memory: per sample two planes of eight
-// channels in BF16, one 16-byte row per position of a zero-bordered 16x16 grid with even and odd columns
-// apart (row = Y*16 + (X&1)*8 + X/2, Y = y+1, X = x+1).
+// (FP32 path; the tensor-core path has its own kernel, which writes the layout its convolutions copy from.)
 constexpr int CONV1_SPB = 8;
-template <bool PLANES>
 __global__ void __launch_bounds__(224) conv1_fwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
   __shared__ __align__(16) float xs[2][30][32];
   __shared__ __align__(16) float w[16][12];   // 9 taps + bias + padding
@@ -86,17 +82,8 @@ __global__ void __launch_bounds__(224) conv1_fwd(GradStepArgs a, WorkerTable wt,
     const int pp = tid;
 #pragma unroll
     for (int ch = 0; ch < 16; ++ch) ws.code1[row * P1_ELEMS + ch * 196 + pp] = outc[ch];
-    if (PLANES) {
-      const int X = px + 1, Y = py + 1;
-      uint4* dst = reinterpret_cast<uint4*>(ws.p1 + row * P1_PLANE_ELEMS) + (Y * 16 + (X & 1) * 8 + (X >> 1));
 #pragma unroll
-      for (int q = 0; q < 2; ++q)
-        dst[q * 256] = make_uint4(bf16_pair(outv[8 * q], outv[8 * q + 1]), bf16_pair(outv[8 * q + 2], outv[8 * q + 3]),
-                                  bf16_pair(outv[8 * q + 4], outv[8 * q + 5]), bf16_pair(outv[8 * q + 6], outv[8 * q + 7]));
-    } else {
-#pragma unroll
-      for (int ch = 0; ch < 16; ++ch) ws.p1[row * P1_ELEMS + ch * 196 + pp] = outv[ch];
-    }
+    for (int ch = 0; ch < 16; ++ch) ws.p1[row * P1_ELEMS + ch * 196 + pp] = outv[ch];
   }
 }
 
@@ -683,7 +670,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
   const int n_chunks1b = (a.b + CONV1B_SPB - 1) / CONV1B_SPB;
   int launches = 0, n_chunks2 = n_chunks, seg_len = 0;
   if (tc) {
-    TIMED(K_CONV1_FWD, (conv1_fwd<true><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
+    if (launch_conv1_fwd_planes(a, wt, gt, ws, st, prof) < 0) return -1;
     launch_conv2_fwd_tc5(a, wt, gt, ws, st, prof);
     int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof);
     if (n < 0) return -1;
@@ -709,7 +696,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1t, n_chunks2, seg_len)));
     launches += 4;
   } else {
-    TIMED(K_CONV1_FWD, (conv1_fwd<false><<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_CONV1_FWD, (conv1_fwd<<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<dim3(a.W, FC2_SPLIT), FC2_THREADS, 0, st>>>(a, wt, gt, ws)));

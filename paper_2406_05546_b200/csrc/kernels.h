@@ -96,14 +96,14 @@ struct GroupTable {
 // Activation workspace carved from the arena (rows = sorted worker * b + sample).
 struct Workspace {
   float* p1;       // conv1 -> ReLU -> pool: [rows][16][14][14] fp32 (FP32 path) or [rows][2 planes][256][8] BF16 (tensor-core path)
-  uint8_t* code1;  // [rows][3136]        pool-1 argmax 0..3, 4 = no gradient (max <= 0)
+  uint8_t* code1;  // [rows][3136]        pool-1 argmax 0..3, 4 = no gradient (max <= 0); [16][196] (FP32 path) or [4 channel quads][196][4] (tensor-core path)
   float* p2;       // [rows][1568]        conv2 -> ReLU -> pool, channel-major flatten
   uint8_t* code2;  // [rows][1568]
   float* d;        // [rows][512]         fc1 -> ReLU -> dropout (scaled)
   float* da1;      // [rows][512]         gradient w.r.t. fc1 pre-activation
   float* dz;       // [rows][16]          gradient w.r.t. logits (10 used)
   float* dp2;      // [rows][1568]        gradient w.r.t. p2
-  float* dp1;      // [rows][3136]        gradient w.r.t. p1
+  float* dp1;      // [rows][3136]        gradient w.r.t. p1; [16][196] (FP32 path) or [4 channel quads][196][4] (tensor-core path)
   float* part2;    // [W][chunks][4640]   per-block partial conv2 weight/bias gradients
   float* part1;    // [W][chunks][160]    per-block partial conv1 weight/bias gradients
   float* partf;    // [W][FC2_SPLIT][FC_PART] per-block partial output-layer gradients and loss sums
@@ -144,6 +144,9 @@ int launch_conv2_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Works
 extern int g_sm_count;   // SMs of the current device, set by configure_tc5_kernels
 int configure_tc5_kernels();
 int configure_conv5_kernels();
+int configure_conv1_kernels();
+int launch_conv1_fwd_planes(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
+                            cudaStream_t st, Profiler* prof);
 void launch_conv2_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                           cudaStream_t st, Profiler* prof);
 void launch_conv2_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,

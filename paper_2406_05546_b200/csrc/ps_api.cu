@@ -235,7 +235,7 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
   x->ckpt_version.assign(x->ckpt_buf.size(), 0);
   double t = std::floor((double)cfg->dropout_p * 4294967296.0);
   x->drop_thresh = t <= 0.0 ? 0u : (t >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)t);
-  if (psk::configure_grad_kernels() != 0 || psk::configure_tc_kernels() != 0 || psk::configure_tc5_kernels() != 0 || psk::configure_conv5_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
+  if (psk::configure_grad_kernels() != 0 || psk::configure_tc_kernels() != 0 || psk::configure_tc5_kernels() != 0 || psk::configure_conv5_kernels() != 0 || psk::configure_conv1_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
   if (cfg->precision != PS_FP32) {
     // two side streams let independent branches of the backward pass overlap (they allocate no device memory)
     bool ok = cudaStreamCreateWithFlags(&x->side.s1, cudaStreamNonBlocking) == cudaSuccess &&
@@ -340,6 +340,7 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
   a.W = W; a.b = b; a.x = x_dev; a.y = y_dev; a.loss = loss_dev; a.argmax = argmax_dev;
   a.seed = seed; a.step = step; a.drop_p = x->cfg.dropout_p; a.drop_thresh = x->drop_thresh;
   a.precision = x->cfg.precision;
+  if (a.precision != PS_FP32 && ((uintptr_t)x_dev & 15) != 0) return fail(PS_ERR_BAD_ARG, "x_dev must be 16-byte aligned on the tensor-core path");
   if (a.precision != PS_FP32 && gt.n_groups > std::min(x->cfg.max_workers, x->cfg.ring_depth))
     return fail(PS_ERR_BAD_ARG, "%d distinct snapshots but the tensor-core workspace holds ring_depth = %d", gt.n_groups, x->cfg.ring_depth);
   int n = psk::launch_grad_step(a, wt, gt, x->ws, x->st, x->prof.on ? psk::SideStreams() : x->side, &x->prof);

@@ -96,6 +96,15 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
                ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// Plain bulk copy shared -> global (both 16-byte aligned, size a multiple of 16), tracked by the thread's bulk groups.
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// All of this thread's committed bulk copies have finished reading shared memory / have completed.
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -130,5 +139,10 @@ __host__ __device__ constexpr uint32_t plain_desc_hi(uint32_t sbo) { return ((sb
 __device__ __forceinline__ uint32_t plain_desc_lo(uint32_t addr, uint32_t lbo) {
   return ((addr & 0x3FFFF) >> 4) | (((lbo >> 4) & 0x3FFF) << 16);
 }
+
+// Host: tensor map of an fp32 tensor of `rank` dimensions (dims[0] contiguous; strides_bytes[i] = pitch of
+// dimension i + 1), box as given, no swizzle, out-of-range elements read as zero.  False on failure.
+bool encode_tensor_map_f32(CUtensorMap* m, const float* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                           const uint32_t* box);
 
 }  // namespace psk
