@@ -38,6 +38,14 @@ __device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {   // lo in t
   return r;
 }
 
+// Where element (channel oc, pooled position p) of a sample's pooled gradient dp2 and of its pooling decisions
+// sits on the tensor-core path: [channel quad][position][4 channels], so that a thread of the backward
+// kernels takes four channels of a position with one vector load.  `canonical` = oc * 49 + p.
+__host__ __device__ __forceinline__ int dp2_column(int canonical) {
+  const int oc = canonical / 49, p = canonical - oc * 49;
+  return (oc >> 2) * 196 + p * 4 + (oc & 3);
+}
+
 __device__ __forceinline__ const float* group_theta(const WorkerTable& wt, const GroupTable& gt, int s) {
   return gt.theta[wt.group[s]];
 }

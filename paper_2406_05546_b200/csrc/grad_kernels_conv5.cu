@@ -169,20 +169,23 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
       __syncwarp();
       if (lane == 0) mbar_arrive(&pipe->acc_empty[buf]);
       if (valid) {
+        // the bias is the same for the four window elements, so the winner is taken on the raw sums:
+        // ReLU then max = max then ReLU, first element that reaches the maximum wins
+        uint32_t codes[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
         for (int o = 0; o < 16; ++o) {
           const int oc = ch * 16 + o;
-          const float bv = bias[oc];
-          float best = 0.f;
-          int bi = 0;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            float rl = fmaxf(__uint_as_float(v[j][o]) + bv, 0.f);
-            if (j == 0 || rl > best) { best = rl; bi = j; }
-          }
+          const float v0 = __uint_as_float(v[0][o]), v1 = __uint_as_float(v[1][o]), v2 = __uint_as_float(v[2][o]), v3 = __uint_as_float(v[3][o]);
+          const float m = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
+          const uint32_t bi = v0 == m ? 0u : (v1 == m ? 1u : (v2 == m ? 2u : 3u));
+          const float best = fmaxf(m + bias[oc], 0.f);
           ws.p2[row * FLAT + oc * 49 + pp] = round_tf32(best);   // its only readers are TF32 products
-          ws.code2[row * FLAT + oc * 49 + pp] = best > 0.f ? (uint8_t)bi : (uint8_t)4;
+          codes[o >> 2] |= (best > 0.f ? bi : 4u) << (8 * (o & 3));
         }
+        // decisions as [channel quad][position][4 channels] bytes
+        uint32_t* c2 = reinterpret_cast<uint32_t*>(ws.code2 + row * FLAT);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) c2[(ch * 4 + q) * 49 + pp] = codes[q];
       }
     }
   }
@@ -206,8 +209,8 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
 // reads them shifted by (2-ky)*16 + (2-kx) rows.  BF16 operands, fp32 accumulation: this product only
 // yields gradient values, and at K = 16 per instruction it needs half the MMAs and half the operand bytes.
 // ------------------------------------------------------------------------------------------------
-constexpr int X_PLANE_ROWS = 256 + 50;                     // 34 rows of tap overrun; 306 rows = 32 bytes (mod 128): the
-constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // four planes then start in different shared-memory banks
+constexpr int X_PLANE_ROWS = 256 + 51;                     // 34 rows of tap overrun (+ 17: a plane pitch of 3 rows mod 8 spreads the
+constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // staging stores of the four planes over all shared-memory banks)
 constexpr int X_BUF_BYTES = 4 * X_PLANE_BYTES;             // four planes of eight output channels
 constexpr int X_W_BYTES = 36 * 16 * 16;                    // [k chunk = tap*4 + oc/8][ic][8 bf16]
 constexpr int X_RAW_BYTES = FLAT * 4 + FLAT;                // one sample's pooled gradients (fp32) and pooling decisions (bytes)
@@ -270,7 +273,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
     }
   } else if (warp <= 4) {
     const int lt = tid - 32;
-    constexpr int PER = (FLAT + LOADERS - 1) / LOADERS;      // 13 pooled entries per thread
+    constexpr int X_ITEMS = (4 * 49 + LOADERS - 1) / LOADERS;      // (channel octet, position) items per thread
     // The pooled gradients and decisions of a sample arrive in a raw slot by two bulk copies issued two
     // tiles ahead, so no global-memory latency sits in this loop.
     auto fetch_raw = [&](int t) {
@@ -290,22 +293,26 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
       uint16_t* dst = bufs + buf * (X_BUF_BYTES / 2);
       const float* rg = reinterpret_cast<const float*>(raw + buf * X_RAW_BYTES);
       const uint8_t* rc = raw + buf * X_RAW_BYTES + FLAT * 4;
-      // Entry e = lt + 128 k is (pooled position e / 32, output channel e % 32): the 32 lanes of a warp write
-      // the 32 channels of one position (64 contiguous bytes spread over the four planes, no bank conflict)
-      // and read the raw slot at a stride of 49 words (odd, no conflict either).
+      // Item e = lt + 128 k is (octet of output channels e / 49, pooled position e % 49).  The raw slot holds
+      // the gradients and the decisions as [channel quad][position][4 channels], so an item is two 16-byte and
+      // two 4-byte loads.  Its eight gradients become four BF16 pairs once; for each of the four positions of
+      // the window the pairs are masked by "this position won" (a per-byte comparison of the four decisions,
+      // spread to half-words) and stored as the position's 16-byte row, which also clears the losers.
 #pragma unroll
-      for (int k = 0; k < PER; ++k) {
+      for (int k = 0; k < X_ITEMS; ++k) {
         const int e = lt + k * LOADERS;
-        if (e < FLAT) {
-          // every pooled entry owns the four positions of its window: the gradient goes to the chosen one
-          // and the other three are cleared, so the planes need no separate clearing pass
-          const int p = e >> 5, oc = e & 31, o = oc * 49 + p;
-          const int code = rc[o];
-          const uint16_t v = bf16_bits(rg[o]);
-          const int py = p / 7, px = p - py * 7;
-          uint16_t* d = dst + (oc >> 3) * (X_PLANE_BYTES / 2) + ((2 * py + 1) * 16 + 2 * px + 1) * 8 + (oc & 7);
-          d[0] = code == 0 ? v : (uint16_t)0; d[8] = code == 1 ? v : (uint16_t)0;
-          d[128] = code == 2 ? v : (uint16_t)0; d[136] = code == 3 ? v : (uint16_t)0;
+        if (e < 4 * 49) {
+          const int o8 = e / 49, p = e - o8 * 49, py = p / 7, px = p - py * 7;
+          const float4 va = reinterpret_cast<const float4*>(rg)[(2 * o8) * 49 + p], vb = reinterpret_cast<const float4*>(rg)[(2 * o8 + 1) * 49 + p];
+          const uint32_t ca = reinterpret_cast<const uint32_t*>(rc)[(2 * o8) * 49 + p], cb = reinterpret_cast<const uint32_t*>(rc)[(2 * o8 + 1) * 49 + p];
+          const uint32_t h0 = bf16_pair(va.x, va.y), h1 = bf16_pair(va.z, va.w), h2 = bf16_pair(vb.x, vb.y), h3 = bf16_pair(vb.z, vb.w);
+          uint4* d = reinterpret_cast<uint4*>(dst) + o8 * (X_PLANE_BYTES / 16) + (2 * py + 1) * 16 + 2 * px + 1;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t ma = __vcmpeq4(ca, 0x01010101u * j), mb = __vcmpeq4(cb, 0x01010101u * j);   // 0xFF where the code is j
+            d[(j >> 1) * 16 + (j & 1)] = make_uint4(h0 & __byte_perm(ma, 0u, 0x1100), h1 & __byte_perm(ma, 0u, 0x3322),
+                                                    h2 & __byte_perm(mb, 0u, 0x1100), h3 & __byte_perm(mb, 0u, 0x3322));
+          }
         }
       }
       fence_proxy_async_smem();

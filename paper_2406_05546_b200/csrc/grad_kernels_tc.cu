@@ -53,7 +53,7 @@ constexpr int DW_SMEM_BYTES = (2 * DW_BUF_WORDS + DW_NRAW * DW_RAW_WORDS) * 4 + 
 static_assert(DW_RAW_P1 % 16 == 0 && DW_RAW_DP2 % 16 == 0 && DW_RAW_CODE % 16 == 0, "bulk copies move multiples of 16 bytes");
 constexpr int DW_MIN_SEG = 16;     // a CTA's range is at least this long (bounds the partial sums per worker)
 constexpr int DW_PAIRS = (2 * 98 + DW_LOADERS - 1) / DW_LOADERS;      // (plane, position pair) items per loader thread
-constexpr int DW_ENTRIES = (FLAT + DW_LOADERS - 1) / DW_LOADERS;      // 7 pooled gradient entries per loader thread
+constexpr int DW_ENTRIES = (8 * 49 + DW_LOADERS - 1) / DW_LOADERS;    // (channel quad, position) items per loader thread
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -165,18 +165,25 @@ __global__ void __launch_bounds__(DW_THREADS, 1) conv2_dw_tc(GradStepArgs a, Wor
           }
         }
       }
+      // Item = (quad of output channels, pooled position): the raw buffer holds gradients and decisions as
+      // [channel quad][position][4 channels].  Every pooled entry owns the four positions of its window: its
+      // gradient goes to the chosen one, the others are cleared, so no separate clearing pass is needed.
 #pragma unroll
       for (int k = 0; k < DW_ENTRIES; ++k) {
-        const int o = lt + k * DW_LOADERS;
-        if (o < FLAT) {
-          // every pooled entry owns the four positions of its window: the gradient goes to the chosen one,
-          // the others are cleared, so no separate clearing pass is needed
-          const int oc = o / 49, p = o - oc * 49, py = p / 7, px = p - py * 7;
-          uint32_t* d = g2w + oc * DW_G_WORDS + (2 * py) * 7 + px;     // word of positions (2py, 2px), (2py, 2px+1)
-          const float v = rdp2[o];
-          const int code = rcode[o];
-          d[0] = bf16_pair(code == 0 ? v : 0.f, code == 1 ? v : 0.f);
-          d[7] = bf16_pair(code == 2 ? v : 0.f, code == 3 ? v : 0.f);
+        const int e = lt + k * DW_LOADERS;
+        if (e < 8 * 49) {
+          const int q = e / 49, p = e - q * 49, py = p / 7, px = p - py * 7;
+          const float4 v4 = reinterpret_cast<const float4*>(rdp2)[e];
+          const uint32_t c4 = reinterpret_cast<const uint32_t*>(rcode)[e];
+          const float v[4] = {v4.x, v4.y, v4.z, v4.w};
+          uint32_t* d = g2w + (4 * q) * DW_G_WORDS + (2 * py) * 7 + px;    // word of positions (2py, 2px), (2py, 2px+1)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint32_t code = (c4 >> (8 * c)) & 0xFFu;
+            const uint32_t h = (uint32_t)bf16_bits(v[c]) << ((code & 1u) * 16u);    // low half: even column, high half: odd column
+            d[c * DW_G_WORDS] = (code >> 1) == 0u ? h : 0u;
+            d[c * DW_G_WORDS + 7] = (code >> 1) == 1u ? h : 0u;
+          }
         }
       }
       mbar_arrive(&full[buf]);

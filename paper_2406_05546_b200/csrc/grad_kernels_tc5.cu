@@ -282,7 +282,7 @@ __global__ void __launch_bounds__(192, 1) tc5_gemm(const __grid_constant__ GemmM
 // ---- operand preparation ----------------------------------------------------------------------
 __device__ __forceinline__ float rna_tf32(float x) { return round_tf32(x); }
 
-// W1 of every weight group: a TF32-rounded copy [512][1568] and its transpose [1568][512].
+// W1 of every weight group: a TF32-rounded copy [512][1568] and its transpose [1568][512] (rows permuted, below).
 __global__ void __launch_bounds__(256) prep_w1(GroupTable gt, float* __restrict__ w1r, float* __restrict__ w1tr) {
   __shared__ float tile[32][33];
   const float* src = gt.theta[blockIdx.z] + OFF_F1W;
@@ -296,7 +296,9 @@ __global__ void __launch_bounds__(256) prep_w1(GroupTable gt, float* __restrict_
     tile[i][tx] = v;
   }
   __syncthreads();
-  for (int i = ty; i < 32; i += 8) dt[(int64_t)(c0 + i) * HID + r0 + tx] = tile[tx][i];
+  // row of the transpose = column of W1 in the order the convolution's backward kernels read dp2:
+  // [channel quad][position][4 channels] instead of channel * 49 + position
+  for (int i = ty; i < 32; i += 8) dt[(int64_t)dp2_column(c0 + i) * HID + r0 + tx] = tile[tx][i];
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
