@@ -68,6 +68,35 @@ __device__ __forceinline__ bool locate_group_tile(const GroupTable& gt, int b, i
   return false;
 }
 
+// Same with a run-time range length: range `index` covers rows [r0, r1) of weight group g (ranges never cross
+// from one weight group into the next).  False past the last range.
+__device__ __forceinline__ bool locate_row_range(const GroupTable& gt, int b, int len, int index, int& g, int& r0, int& r1) {
+  for (g = 0; g < gt.n_groups; ++g) {
+    const int first = gt.first[g] * b, end = gt.first[g + 1] * b;
+    const int n = (end - first + len - 1) / len;
+    if (index < n) {
+      r0 = first + index * len;
+      r1 = min(r0 + len, end);
+      return true;
+    }
+    index -= n;
+  }
+  return false;
+}
+
+// Host: a range length (a multiple of `unit` rows) that gives about `slots` ranges over all rows, and the number
+// of ranges it makes when no range crosses a weight-group boundary.
+inline int plan_row_ranges(const GroupTable& gt, int b, int slots, int unit, int* len_out) {
+  const int total = gt.first[gt.n_groups] * b;
+  int len = (total + slots - 1) / slots;
+  len = (len + unit - 1) / unit * unit;
+  if (len < unit) len = unit;
+  int n = 0;
+  for (int g = 0; g < gt.n_groups; ++g) n += ((gt.first[g + 1] - gt.first[g]) * b + len - 1) / len;
+  *len_out = len;
+  return n;
+}
+
 inline int group_tiles(const GroupTable& gt, int b, int tm) {
   int t = 0;
   for (int g = 0; g < gt.n_groups; ++g) t += ((gt.first[g + 1] - gt.first[g]) * b + tm - 1) / tm;

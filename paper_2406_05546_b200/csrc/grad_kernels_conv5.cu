@@ -23,7 +23,6 @@ namespace psk {
 
 namespace {
 
-constexpr int C5_SPB = 16;            // samples per CTA
 constexpr int THREADS = 288;
 constexpr int LOADERS = 128;
 
@@ -41,16 +40,19 @@ __device__ __forceinline__ bool loaders_sync_any(bool failed) {
   return any != 0;
 }
 
+constexpr int F_NBUF = 4;             // shared-memory tile buffers of the forward kernel (copies run four tiles ahead)
 struct Pipe {
-  uint64_t a_full[2], a_empty[2], acc_full[2], acc_empty[2], raw_full[2];
+  uint64_t a_full[F_NBUF], a_empty[F_NBUF], acc_full[2], acc_empty[2], raw_full[2];
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
 
 __device__ __forceinline__ void pipe_init(Pipe* p, int a_full_arrivals, int acc_empty_arrivals) {
-  for (int i = 0; i < 2; ++i) {
+  for (int i = 0; i < F_NBUF; ++i) {
     mbar_init(&p->a_full[i], a_full_arrivals);
     mbar_init(&p->a_empty[i], 1);
+  }
+  for (int i = 0; i < 2; ++i) {
     mbar_init(&p->acc_full[i], 1);
     mbar_init(&p->acc_empty[i], acc_empty_arrivals);
     mbar_init(&p->raw_full[i], 1);
@@ -72,17 +74,19 @@ constexpr int F_PLANE_ROWS = 2 * 256 + 32;                 // two stacked 16x16 
 constexpr int F_PLANE_BYTES = F_PLANE_ROWS * 16;           // 8704
 constexpr int F_BUF_BYTES = 2 * F_PLANE_BYTES;             // two planes of eight channels
 constexpr int F_W_BYTES = 18 * 32 * 16;                    // [k chunk = tap*2 + ic/8][oc][8 bf16]
-constexpr int F_SMEM = 2 * F_BUF_BYTES + F_W_BYTES + 32 * 4 + sizeof(Pipe) + 128;
+constexpr int F_SMEM = F_NBUF * F_BUF_BYTES + F_W_BYTES + 32 * 4 + sizeof(Pipe) + 128;
 
-__global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+__global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, GroupTable gt, Workspace ws, int range_len) {
   extern __shared__ __align__(128) uint8_t smem[];
-  uint16_t* Wk = reinterpret_cast<uint16_t*>(smem + 2 * F_BUF_BYTES);
-  float* bias = reinterpret_cast<float*>(smem + 2 * F_BUF_BYTES + F_W_BYTES);
-  Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * F_BUF_BYTES + F_W_BYTES + 128);
-  const int s = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const float* theta = group_theta(wt, gt, s);
-  const int i_begin = blockIdx.x * C5_SPB, i_end = min(i_begin + C5_SPB, a.b);
-  const int n_tiles = (i_end - i_begin + 1) / 2;
+  uint16_t* Wk = reinterpret_cast<uint16_t*>(smem + F_NBUF * F_BUF_BYTES);
+  float* bias = reinterpret_cast<float*>(smem + F_NBUF * F_BUF_BYTES + F_W_BYTES);
+  Pipe* pipe = reinterpret_cast<Pipe*>(smem + F_NBUF * F_BUF_BYTES + F_W_BYTES + 128);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // a CTA walks over a contiguous range of rows (worker-major samples) that share one weight snapshot
+  int grp, r_begin, r_end;
+  if (!locate_row_range(gt, a.b, range_len, blockIdx.x, grp, r_begin, r_end)) return;
+  const float* theta = gt.theta[grp];
+  const int n_tiles = (r_end - r_begin + 1) / 2;
 
   for (int idx = tid; idx < 4608; idx += F_THREADS) {
     int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
@@ -91,7 +95,7 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
   if (tid < 32) bias[tid] = theta[OFF_C2B + tid];
   // rows never written by a copy (the overrun of the padding rows, a missing second sample) only feed
   // results that are dropped; they are cleared once so that those results stay finite
-  for (int idx = tid; idx < 2 * F_BUF_BYTES / 16; idx += F_THREADS) reinterpret_cast<float4*>(smem)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int idx = tid; idx < F_NBUF * F_BUF_BYTES / 16; idx += F_THREADS) reinterpret_cast<float4*>(smem)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
   if (tid == 0) pipe_init(pipe, 1, 8);
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(256) : "memory");
@@ -108,40 +112,41 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
       constexpr uint32_t idesc = idesc_bf16(128, 32);
       const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), 512);
       for (int t = 0; t < n_tiles; ++t) {
-        const int buf = t & 1;
-        if (!mbar_wait(&pipe->a_full[buf], (t >> 1) & 1)) { pipe->abort_flag = 1; break; }
-        if (t >= 2 && !mbar_wait(&pipe->acc_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
+        const int buf = t % F_NBUF, ab = t & 1;
+        if (!mbar_wait(&pipe->a_full[buf], (t / F_NBUF) & 1)) { pipe->abort_flag = 1; break; }
+        if (t >= 2 && !mbar_wait(&pipe->acc_empty[ab], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
         if (pipe->abort_flag) break;
         tc_fence_after();
         // 36 MMAs (one per window element and tap: K = 16 channels), fully unrolled: every descriptor is a
         // per-tile base plus a compile-time constant
         const uint32_t a_lo = plain_desc_lo(smem_u32(smem) + buf * F_BUF_BYTES, F_PLANE_BYTES);
-        const uint32_t d_tmem = tmem + buf * 128;
+        const uint32_t d_tmem = tmem + ab * 128;
+        // (taps outermost: consecutive MMAs go to the four different accumulators)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int jy = j >> 1, jx = j & 1;
+        for (int tap = 0; tap < 9; ++tap) {
+          const int ky = tap / 3, kx = tap - ky * 3;
 #pragma unroll
-          for (int tap = 0; tap < 9; ++tap) {
-            const int ky = tap / 3, kx = tap - ky * 3, sx = jx + kx;
+          for (int j = 0; j < 4; ++j) {
+            const int jy = j >> 1, jx = j & 1, sx = jx + kx;
             const int row_off = (jy + ky) * 16 + (sx & 1) * 8 + (sx >> 1);     // in 16-byte rows
             umma_f16_split(d_tmem + j * 32, a_lo + row_off, plain_desc_hi(512), w_lo + (tap * 2) * (512 / 16),
                            plain_desc_hi(128), idesc, tap ? 1u : 0u);
           }
         }
         umma_commit(&pipe->a_empty[buf]);
-        umma_commit(&pipe->acc_full[buf]);
+        umma_commit(&pipe->acc_full[ab]);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       for (int t = 0; t < n_tiles; ++t) {
-        const int buf = t & 1;
-        if (t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
+        const int buf = t % F_NBUF;
+        if (t >= F_NBUF && !mbar_wait(&pipe->a_empty[buf], ((t / F_NBUF) - 1) & 1)) { pipe->abort_flag = 1; break; }
         if (pipe->abort_flag) break;
-        const int n_s = min(2, i_end - (i_begin + 2 * t));
+        const int n_s = min(2, r_end - (r_begin + 2 * t));
         mbar_expect_tx(&pipe->a_full[buf], (uint32_t)n_s * 2 * 4096u);
         for (int sp = 0; sp < n_s; ++sp) {
-          const float* src = ws.p1 + ((int64_t)s * a.b + i_begin + 2 * t + sp) * P1_PLANE_ELEMS;
+          const float* src = ws.p1 + (int64_t)(r_begin + 2 * t + sp) * P1_PLANE_ELEMS;
 #pragma unroll
           for (int q = 0; q < 2; ++q)
             bulk_load(smem + buf * F_BUF_BYTES + q * F_PLANE_BYTES + sp * 4096, src + q * 1024, 4096, &pipe->a_full[buf]);
@@ -155,9 +160,8 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
       const int buf = t & 1;
       if (!mbar_wait(&pipe->acc_full[buf], (t >> 1) & 1) || pipe->abort_flag) { pipe->abort_flag = 1; break; }
       tc_fence_after();
-      const int i = i_begin + 2 * t + sp;
-      const bool valid = py < 7 && px < 7 && i < i_end;
-      const int64_t row = (int64_t)s * a.b + i;
+      const int64_t row = r_begin + 2 * t + sp;
+      const bool valid = py < 7 && px < 7 && row < r_end;
       const int pp = py * 7 + px;
       uint32_t v[4][16];
 #pragma unroll
@@ -212,29 +216,30 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Wo
 constexpr int X_PLANE_ROWS = 256 + 51;                     // 34 rows of tap overrun (+ 17: a plane pitch of 3 rows mod 8 spreads the
 constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // staging stores of the four planes over all shared-memory banks)
 constexpr int X_BUF_BYTES = 4 * X_PLANE_BYTES;             // four planes of eight output channels
-constexpr int X_W_BYTES = 36 * 16 * 16;                    // [k chunk = tap*4 + oc/8][ic][8 bf16]
+constexpr int X_W_BYTES = 12 * 48 * 16;                    // [filter row ky][k chunk oc/8][column = kx*16 + ic][8 bf16]
 constexpr int X_RAW_BYTES = FLAT * 4 + FLAT;                // one sample's pooled gradients (fp32) and pooling decisions (bytes)
 constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + 2 * X_RAW_BYTES + sizeof(Pipe) + 128;
 
-__global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
+__global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, GroupTable gt, Workspace ws, int range_len) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint16_t* bufs = reinterpret_cast<uint16_t*>(smem);
   uint16_t* Wk = reinterpret_cast<uint16_t*>(smem + 2 * X_BUF_BYTES);
   uint8_t* raw = smem + 2 * X_BUF_BYTES + X_W_BYTES;        // two raw staging slots filled by bulk copies
   Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * X_BUF_BYTES + X_W_BYTES + 2 * X_RAW_BYTES);
-  const int s = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const float* theta = group_theta(wt, gt, s);
-  const int i_begin = blockIdx.x * C5_SPB, i_end = min(i_begin + C5_SPB, a.b);
-  const int n_tiles = i_end - i_begin;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int grp, r_begin, r_end;
+  if (!locate_row_range(gt, a.b, range_len, blockIdx.x, grp, r_begin, r_end)) return;
+  const float* theta = gt.theta[grp];
+  const int n_tiles = r_end - r_begin;
 
   for (int idx = tid; idx < 4608; idx += THREADS) {
     int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
-    Wk[((tap * 4 + (oc >> 3)) * 16 + ic) * 8 + (oc & 7)] = bf16_bits(theta[OFF_C2W + idx]);
+    Wk[(((tap / 3) * 4 + (oc >> 3)) * 48 + (tap % 3) * 16 + ic) * 8 + (oc & 7)] = bf16_bits(theta[OFF_C2W + idx]);
   }
   for (int idx = tid; idx < 2 * X_BUF_BYTES / 16; idx += THREADS) reinterpret_cast<float4*>(smem)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
   if (tid == 0) pipe_init(pipe, LOADERS, 4);
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(64) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(256) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   fence_proxy_async_smem();
@@ -245,8 +250,8 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
 
   if (warp == 0) {
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(128, 16);
-      const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), 256);
+      constexpr uint32_t idesc = idesc_bf16(128, 48);
+      const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), 48 * 16);
       for (int t = 0; t < n_tiles; ++t) {
         const int buf = t & 1;
         if (!mbar_wait(&pipe->a_full[buf], (t >> 1) & 1)) { pipe->abort_flag = 1; break; }
@@ -254,19 +259,17 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
         if (pipe->abort_flag) break;
         tc_fence_after();
         const uint32_t a_lo = plain_desc_lo(smem_u32(smem) + buf * X_BUF_BYTES, X_PLANE_BYTES);
-        const uint32_t d_tmem = tmem + buf * 32;
+        const uint32_t d_tmem = tmem + buf * 128;
+        // 12 MMAs: per block of 128 positions and filter row ky, the products with the three taps of that row sit
+        // side by side in the 48 accumulator columns (kx, ic); the rows read are shifted by the filter row only
 #pragma unroll
-        for (int m = 0; m < 2; ++m) {
+        for (int ky = 0; ky < 3; ++ky)
 #pragma unroll
-          for (int tap = 0; tap < 9; ++tap) {
-            const int ky = tap / 3, kx = tap - ky * 3;
-            const int row_off = m * 128 + (2 - ky) * 16 + (2 - kx);           // in 16-byte rows
+          for (int q = 0; q < 2; ++q)                                        // 16 output channels per MMA
 #pragma unroll
-            for (int q = 0; q < 2; ++q)                                        // 16 output channels per MMA
-              umma_f16_split(d_tmem + m * 16, a_lo + (2 * q) * (X_PLANE_BYTES / 16) + row_off, plain_desc_hi(128),
-                             w_lo + (tap * 4 + q * 2) * (256 / 16), plain_desc_hi(128), idesc, (tap | q) ? 1u : 0u);
-          }
-        }
+            for (int m = 0; m < 2; ++m)
+              umma_f16_split(d_tmem + m * 48, a_lo + (2 * q) * (X_PLANE_BYTES / 16) + m * 128 + (2 - ky) * 16 + 1, plain_desc_hi(128),
+                             w_lo + ((ky * 4 + 2 * q) * 48), plain_desc_hi(128), idesc, (ky | q) ? 1u : 0u);
         umma_commit(&pipe->a_empty[buf]);
         umma_commit(&pipe->acc_full[buf]);
       }
@@ -277,7 +280,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
     // The pooled gradients and decisions of a sample arrive in a raw slot by two bulk copies issued two
     // tiles ahead, so no global-memory latency sits in this loop.
     auto fetch_raw = [&](int t) {
-      const int64_t row = (int64_t)s * a.b + i_begin + t;
+      const int64_t row = r_begin + t;
       uint8_t* slot = raw + (t & 1) * X_RAW_BYTES;
       mbar_expect_tx(&pipe->raw_full[t & 1], X_RAW_BYTES);
       bulk_load(slot, ws.dp2 + row * FLAT, FLAT * 4, &pipe->raw_full[t & 1]);
@@ -327,17 +330,30 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
       const int buf = t & 1;
       if (!mbar_wait(&pipe->acc_full[buf], (t >> 1) & 1) || pipe->abort_flag) { pipe->abort_flag = 1; break; }
       tc_fence_after();
-      const int64_t row = (int64_t)s * a.b + i_begin + t;
+      const int64_t row = r_begin + t;
 #pragma unroll
       for (int m = 0; m < 2; ++m) {
-        uint32_t v[16];
-        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 32 + m * 16), v);
+        // the thread's position holds, per filter column kx, the sum over filter rows of what the gradient AT this
+        // position sends through tap (ky, kx); the input gradient here collects kx = 0 from the position to the
+        // right, kx = 1 from itself and kx = 2 from the position to the left (zero borders make the rows' ends right)
+        uint32_t e0[16], e1[16], e2[16];
+        const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 128 + m * 48);
+        tmem_ld16(taddr, e0);
+        tmem_ld16(taddr + 16, e1);
+        tmem_ld16(taddr + 32, e2);
         tmem_ld_wait();
         const int r = m * 128 + quarter * 32 + lane, y = r >> 4, x = r & 15;
-        if (y < 14 && x < 14) {      // dp1 of a sample is [channel quad][position][4 channels]: a warp writes 448 contiguous bytes
-          uint4* out = reinterpret_cast<uint4*>(ws.dp1 + row * P1_ELEMS) + (y * 14 + x);
+        float v[16];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) out[q * 196] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        for (int ic = 0; ic < 16; ++ic) {
+          const float right = __shfl_down_sync(0xffffffffu, __uint_as_float(e0[ic]), 1);
+          const float left = __shfl_up_sync(0xffffffffu, __uint_as_float(e2[ic]), 1);
+          v[ic] = (__uint_as_float(e1[ic]) + right) + (x == 0 ? 0.f : left);
+        }
+        if (y < 14 && x < 14) {      // dp1 of a sample is [channel quad][position][4 channels]: a warp writes 448 contiguous bytes
+          float4* out = reinterpret_cast<float4*>(ws.dp1 + row * P1_ELEMS) + (y * 14 + x);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) out[q * 196] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
         }
       }
       tc_fence_before();
@@ -349,7 +365,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Worke
   __syncthreads();
   if (warp == 0) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
   }
   if (tid == 0 && pipe->abort_flag) {
     atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
@@ -369,14 +385,16 @@ int configure_conv5_kernels() {
 
 void launch_conv2_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                           cudaStream_t st, Profiler* prof) {
-  const int chunks = (a.b + C5_SPB - 1) / C5_SPB;
-  TIMED(K_CONV2_FWD, (conv2_fwd_tc5<<<dim3(chunks, a.W), F_THREADS, F_SMEM, st>>>(a, wt, gt, ws)));
+  int len;
+  const int n = plan_row_ranges(gt, a.b, 2 * g_sm_count, 2, &len);      // two CTAs per SM, tiles of two samples
+  TIMED(K_CONV2_FWD, (conv2_fwd_tc5<<<n, F_THREADS, F_SMEM, st>>>(a, gt, ws, len)));
 }
 
 void launch_conv2_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                          cudaStream_t st, Profiler* prof) {
-  const int chunks = (a.b + C5_SPB - 1) / C5_SPB;
-  TIMED(K_CONV2_BWD, (conv2_dx_tc5<<<dim3(chunks, a.W), THREADS, X_SMEM, st>>>(a, wt, gt, ws)));
+  int len;
+  const int n = plan_row_ranges(gt, a.b, 2 * g_sm_count, 1, &len);
+  TIMED(K_CONV2_BWD, (conv2_dx_tc5<<<n, THREADS, X_SMEM, st>>>(a, gt, ws, len)));
 }
 
 }  // namespace psk
