@@ -23,26 +23,16 @@ namespace psk {
 
 namespace {
 
-constexpr int THREADS = 288;
-constexpr int LOADERS = 128;
+constexpr int THREADS = 416;           // input-gradient kernel: 1 MMA warp, 8 staging warps, 4 epilogue warps
+constexpr int LOADERS = 256;
 
 __host__ __device__ constexpr uint32_t idesc_bf16(int m, int n) {     // fp32 accumulate, BF16 x BF16, k-contiguous
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-// Barrier over the 128 staging threads that also tells every one of them whether any of them failed.
-__device__ __forceinline__ bool loaders_sync_any(bool failed) {
-  uint32_t any;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(any) : "r"((uint32_t)failed) : "memory");
-  return any != 0;
-}
-
 constexpr int F_NBUF = 4;             // shared-memory tile buffers of the forward kernel (copies run four tiles ahead)
 struct Pipe {
-  uint64_t a_full[F_NBUF], a_empty[F_NBUF], acc_full[2], acc_empty[2], raw_full[2];
+  uint64_t a_full[F_NBUF], a_empty[F_NBUF], acc_full[2], acc_empty[2], raw_full[2], raw_empty[2];
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -56,6 +46,7 @@ __device__ __forceinline__ void pipe_init(Pipe* p, int a_full_arrivals, int acc_
     mbar_init(&p->acc_full[i], 1);
     mbar_init(&p->acc_empty[i], acc_empty_arrivals);
     mbar_init(&p->raw_full[i], 1);
+    mbar_init(&p->raw_empty[i], LOADERS / 32);
   }
   p->abort_flag = 0;
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -237,7 +228,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
     Wk[(((tap / 3) * 4 + (oc >> 3)) * 48 + (tap % 3) * 16 + ic) * 8 + (oc & 7)] = bf16_bits(theta[OFF_C2W + idx]);
   }
   for (int idx = tid; idx < 2 * X_BUF_BYTES / 16; idx += THREADS) reinterpret_cast<float4*>(smem)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (tid == 0) pipe_init(pipe, LOADERS, 4);
+  if (tid == 0) pipe_init(pipe, LOADERS / 32, 4);
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(256) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -274,7 +265,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
         umma_commit(&pipe->acc_full[buf]);
       }
     }
-  } else if (warp <= 4) {
+  } else if (warp <= LOADERS / 32) {
     const int lt = tid - 32;
     constexpr int X_ITEMS = (4 * 49 + LOADERS - 1) / LOADERS;      // (channel octet, position) items per thread
     // The pooled gradients and decisions of a sample arrive in a raw slot by two bulk copies issued two
@@ -289,14 +280,14 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
     if (lt == 0) { fetch_raw(0); if (n_tiles > 1) fetch_raw(1); }
     for (int t = 0; t < n_tiles; ++t) {
       const int buf = t & 1;
-      bool failed = !mbar_wait(&pipe->raw_full[buf], (t >> 1) & 1);
-      if (!failed && t >= 2 && !mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1)) failed = true;
-      // one uniform decision for all staging threads, so that none waits alone at a later barrier
-      if (loaders_sync_any(failed)) { pipe->abort_flag = 1; break; }
+      // every staging warp waits and reports on its own (no block-level barrier among them)
+      bool ok = mbar_wait(&pipe->raw_full[buf], (t >> 1) & 1);
+      if (ok && t >= 2) ok = mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1);
+      if (!__all_sync(0xffffffffu, ok) || pipe->abort_flag) { pipe->abort_flag = 1; break; }
       uint16_t* dst = bufs + buf * (X_BUF_BYTES / 2);
       const float* rg = reinterpret_cast<const float*>(raw + buf * X_RAW_BYTES);
       const uint8_t* rc = raw + buf * X_RAW_BYTES + FLAT * 4;
-      // Item e = lt + 128 k is (octet of output channels e / 49, pooled position e % 49).  The raw slot holds
+      // Item e = lt + 256 k is (octet of output channels e / 49, pooled position e % 49).  The raw slot holds
       // the gradients and the decisions as [channel quad][position][4 channels], so an item is two 16-byte and
       // two 4-byte loads.  Its eight gradients become four BF16 pairs once; for each of the four positions of
       // the window the pairs are masked by "this position won" (a per-byte comparison of the four decisions,
@@ -319,10 +310,13 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
         }
       }
       fence_proxy_async_smem();
-      mbar_arrive(&pipe->a_full[buf]);
-      // the raw slot may be refilled once every staging thread has read it
-      loaders_sync_any(false);
-      if (lt == 0 && t + 2 < n_tiles) fetch_raw(t + 2);
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&pipe->a_full[buf]); mbar_arrive(&pipe->raw_empty[buf]); }
+      // the raw slot is refilled once every staging warp has read it
+      if (lt == 0 && t + 2 < n_tiles) {
+        if (!mbar_wait(&pipe->raw_empty[buf], (t >> 1) & 1)) { pipe->abort_flag = 1; break; }
+        fetch_raw(t + 2);
+      }
     }
   } else {
     const int quarter = warp & 3;
