@@ -122,6 +122,7 @@ struct GradStepArgs {
   float drop_p;
   uint32_t drop_thresh;   // keep iff word >= thresh
   int precision;          // 0 = FP32 CUDA cores; otherwise tensor cores (BF16 convolution products, TF32 dense layer)
+  int skip_prep_w1;       // the rounded copies of the dense-layer weights of these very snapshots are still valid
 };
 
 // Side streams (and the events that fork from / join into the caller's stream) for the independent

@@ -74,6 +74,13 @@ struct ps_ctx {
   uint32_t drop_thresh = 0;
   psk::Profiler prof;
   psk::SideStreams side;
+  // rounded copies of the dense-layer weights: which snapshots they were made from, and in which state of the weights
+  uint64_t weights_epoch = 1, prep_epoch = 0;
+  const float* prep_theta[psk::MAX_GROUPS] = {nullptr};
+  int prep_n = 0;
+  // ps_tick_host copies its inputs in on a stream of its own, chunk by chunk, while earlier chunks compute
+  cudaStream_t copy_st = nullptr;
+  cudaEvent_t copy_ev[8] = {nullptr};
   double prof_ms[psk::K_COUNT] = {0};
   int64_t prof_n[psk::K_COUNT] = {0};
 };
@@ -244,6 +251,11 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
     for (auto ev : evs) ok = ok && cudaEventCreateWithFlags(ev, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { delete x; return fail(PS_ERR_CUDA, "side stream set-up failed: %s", cudaGetErrorString(cudaGetLastError())); }
   }
+  {
+    bool ok = cudaStreamCreateWithFlags(&x->copy_st, cudaStreamNonBlocking) == cudaSuccess;
+    for (auto& ev : x->copy_ev) ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { delete x; return fail(PS_ERR_CUDA, "copy stream set-up failed: %s", cudaGetErrorString(cudaGetLastError())); }
+  }
   std::memcpy(x->io_stage, init_params_host, sizeof(float) * PS_PARAM_COUNT);
   std::memset(x->io_stage + PS_PARAM_COUNT, 0, sizeof(float) * (PS_PARAM_STRIDE - PS_PARAM_COUNT));
   cudaError_t e = cudaMemcpyAsync(x->ring[0], x->io_stage, VEC_BYTES, cudaMemcpyHostToDevice, x->st);
@@ -265,6 +277,8 @@ int32_t ps_destroy(ps_ctx* x) {
   if (x->side.s1) { cudaStreamSynchronize(x->side.s1); cudaStreamDestroy(x->side.s1); }
   if (x->side.s2) { cudaStreamSynchronize(x->side.s2); cudaStreamDestroy(x->side.s2); }
   for (cudaEvent_t ev : {x->side.fork1, x->side.join1, x->side.fork2, x->side.join2}) if (ev) cudaEventDestroy(ev);
+  if (x->copy_st) { cudaStreamSynchronize(x->copy_st); cudaStreamDestroy(x->copy_st); }
+  for (cudaEvent_t ev : x->copy_ev) if (ev) cudaEventDestroy(ev);
   delete x;
   if (e != cudaSuccess) return cuda_fail(e, "ps_destroy");
   return PS_OK;
@@ -343,7 +357,14 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
   if (a.precision != PS_FP32 && ((uintptr_t)x_dev & 15) != 0) return fail(PS_ERR_BAD_ARG, "x_dev must be 16-byte aligned on the tensor-core path");
   if (a.precision != PS_FP32 && gt.n_groups > std::min(x->cfg.max_workers, x->cfg.ring_depth))
     return fail(PS_ERR_BAD_ARG, "%d distinct snapshots but the tensor-core workspace holds ring_depth = %d", gt.n_groups, x->cfg.ring_depth);
+  // the rounded / transposed copies of the dense-layer weights are reused while the same snapshots hold the same weights
+  a.skip_prep_w1 = x->prep_epoch == x->weights_epoch && x->prep_n == gt.n_groups;
+  for (int g = 0; g < gt.n_groups && a.skip_prep_w1; ++g) a.skip_prep_w1 = x->prep_theta[g] == gt.theta[g];
   int n = psk::launch_grad_step(a, wt, gt, x->ws, x->st, x->prof.on ? psk::SideStreams() : x->side, &x->prof);
+  if (n >= 0 && a.precision != PS_FP32) {
+    x->prep_epoch = x->weights_epoch; x->prep_n = gt.n_groups;
+    for (int g = 0; g < gt.n_groups; ++g) x->prep_theta[g] = gt.theta[g];
+  }
   if (n < 0) return cuda_fail(cudaGetLastError(), "grad step launch");
   x->launches += n;
   return PS_OK;
@@ -431,6 +452,7 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
     if (n < 0) return cuda_fail(cudaGetLastError(), "apply launch");
     x->launches += n;
     x->version += 1;
+    x->weights_epoch++;
     advance_oldest(x);
     if (mirror) { int32_t rc = propagate_chain(x, x->version); if (rc != PS_OK) return rc; res.replicated = 1; }
     if (x->cfg.ckpt_every > 0 && x->version % (uint64_t)x->cfg.ckpt_every == 0) {
@@ -469,6 +491,7 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
       if (n < 0) return cuda_fail(cudaGetLastError(), "async apply launch");
       x->launches += n;
       x->version += (uint64_t)seg;
+      x->weights_epoch++;
       advance_oldest(x);
       if (mirrored) { int32_t rc = propagate_chain(x, mirrored); if (rc != PS_OK) return rc; }
       if (x->cfg.ckpt_every > 0 && x->version % (uint64_t)x->cfg.ckpt_every == 0) {
@@ -518,6 +541,7 @@ int32_t ps_restore(ps_ctx* x, uint64_t* version_out) {
   uint64_t v = x->ckpt_version[slot];
   CUDA_TRY(cudaMemcpyAsync(x->ring[v % (uint64_t)x->cfg.ring_depth], x->ckpt_buf[slot], VEC_BYTES, cudaMemcpyHostToDevice, x->st));
   x->version = v; x->oldest = v;
+  x->weights_epoch++;
   x->queue_len = 0; x->reserved = 0; x->meta.clear();
   x->up = true; x->weights_lost = false;
   if (version_out) *version_out = v;
@@ -535,6 +559,7 @@ int32_t ps_failover(ps_ctx* x, uint64_t* version_out) {
   x->ring[slot] = r.buf;   // the dead frontend's buffer in that slot is retired
   x->replicas.erase(x->replicas.begin(), x->replicas.begin() + (long)i + 1);
   x->version = r.version; x->oldest = r.version;
+  x->weights_epoch++;
   x->queue_len = 0; x->reserved = 0; x->meta.clear();
   x->up = true; x->weights_lost = false;
   if (version_out) *version_out = r.version;
@@ -542,6 +567,7 @@ int32_t ps_failover(ps_ctx* x, uint64_t* version_out) {
 }
 
 int32_t ps_import_params(ps_ctx* x, const float* host_in) {
+  if (x) x->weights_epoch++;
   if (!x || !host_in) return fail(PS_ERR_BAD_ARG, "NULL argument");
   if (x->weights_lost) return fail(PS_ERR_DOWN, "server is down");
   CUDA_TRY(cudaStreamSynchronize(x->st));
@@ -643,10 +669,27 @@ int32_t ps_tick_host(ps_ctx* x, int32_t W, int32_t b, const int32_t* lags, const
   int32_t rc = ps_queue_reserve(x, W, slots);
   if (rc != PS_OK) return rc;
   const size_t rows = (size_t)W * b;
-  CUDA_TRY(cudaMemcpyAsync(x->x_stage, x_host, rows * PS_IMAGE_PIXELS * sizeof(float), cudaMemcpyHostToDevice, x->st));
-  CUDA_TRY(cudaMemcpyAsync(x->y_stage, y_host, rows * sizeof(int32_t), cudaMemcpyHostToDevice, x->st));
-  rc = workers_grad_step(x, W, b, snaps, ids, x->x_stage, x->y_stage, seed, step, slots, nullptr, x->loss_stage, x->argmax_stage);
-  if (rc != PS_OK) return rc;
+  // The inputs go in on the copy stream in up to four chunks of workers; the grad step of a chunk starts as soon as
+  // its chunk has landed, so most of the host-to-device copy hides behind the computation of earlier chunks.
+  // (The staging buffers are free: the previous call synchronised the context's stream before it returned.)
+  const int n_chunks = W >= 8 ? 4 : 1, per = (W + n_chunks - 1) / n_chunks;
+  for (int c = 0; c < n_chunks; ++c) {
+    const int w0 = c * per, w1 = std::min(W, w0 + per);
+    if (w0 >= w1) break;
+    const size_t r0 = (size_t)w0 * b, nr = (size_t)(w1 - w0) * b;
+    CUDA_TRY(cudaMemcpyAsync(x->x_stage + r0 * PS_IMAGE_PIXELS, x_host + r0 * PS_IMAGE_PIXELS, nr * PS_IMAGE_PIXELS * sizeof(float), cudaMemcpyHostToDevice, x->copy_st));
+    CUDA_TRY(cudaMemcpyAsync(x->y_stage + r0, y_host + r0, nr * sizeof(int32_t), cudaMemcpyHostToDevice, x->copy_st));
+    CUDA_TRY(cudaEventRecord(x->copy_ev[c], x->copy_st));
+  }
+  for (int c = 0; c < n_chunks; ++c) {
+    const int w0 = c * per, w1 = std::min(W, w0 + per);
+    if (w0 >= w1) break;
+    const size_t r0 = (size_t)w0 * b;
+    CUDA_TRY(cudaStreamWaitEvent(x->st, x->copy_ev[c], 0));
+    rc = workers_grad_step(x, w1 - w0, b, snaps + w0, ids + w0, x->x_stage + r0 * PS_IMAGE_PIXELS, x->y_stage + r0, seed, step,
+                           slots + w0, nullptr, x->loss_stage + w0, x->argmax_stage + r0);
+    if (rc != PS_OK) { cudaStreamSynchronize(x->copy_st); return rc; }
+  }
   rc = ps_enqueue(x, W, slots, nullptr, ids, bases, step);
   if (rc != PS_OK) return rc;
   ps_apply_result res = {0, x->version, 0, 0};
