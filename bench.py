@@ -32,6 +32,9 @@ FLOP_PER_SAMPLE = 10_718_208            # 2 x (1,824,000 forward + 3,535,104 bac
 GRAD_BYTES = 813258 * 4                 # algorithmic bytes per queued gradient
 N_BATCH_BUFFERS = 8
 REPLAY_TRAFFIC_PER_GRADIENT = 2.654663e9 / 816
+# dram bytes (read + written) per sample of the grad-step kernels, from one ncu capture of a reduced case
+# (W=128, b=64: 8,192 samples; traffic grows in proportion to the samples); None = not captured since the kernel changed
+KERNEL_TRAFFIC_PER_SAMPLE = {}
 
 
 def measured_peaks():
@@ -297,6 +300,9 @@ def main():
         top = max(kernels, key=lambda k: kernels[k]["share"])
         roof = kernel_roofline(top, kernels[top]["ms_per_launch"], W, b, peaks, args.precision)
         roof.pop("flops", None)
+        per_sample = KERNEL_TRAFFIC_PER_SAMPLE.get(top) if args.precision != "fp32" else None
+        if per_sample is not None:
+            roof["traffic"] = per_sample * W * b
         grad_ms = sum(v["ms_per_launch"] for k, v in kernels.items()
                       if not k.startswith("sum_") and k not in ("async_apply", "copy_rows"))
         tensor_flop = 2 * (3 * 903_168 + 3 * 802_816) * W * b

@@ -65,7 +65,11 @@ enum {
   PS_ERR_DEVICE_STATUS = -9     /* a kernel's own input check tripped (e.g. a label outside 0..9) */
 };
 
-enum { PS_FP32 = 0, PS_TF32 = 1, PS_BF16 = 2 };   /* arithmetic of the dense contractions of part A */
+/* Arithmetic of the dense contractions of part A.  PS_FP32: everything on the FP32 pipes.  PS_BF16: the
+ * tensor-core path: BF16 operands (fp32 accumulation) in the products of the second convolution and in the
+ * first convolution's filter gradient, TF32 operands in the 512-unit layer; the first convolution's forward
+ * pass and the output layer stay FP32.  PS_TF32 is reserved and not built (ps_create refuses it). */
+enum { PS_FP32 = 0, PS_TF32 = 1, PS_BF16 = 2 };
 typedef enum { PS_SYNC = 0, PS_ASYNC = 1, PS_REPLAY = 2 } ps_mode;
 
 typedef struct ps_ctx ps_ctx;   /* opaque; owned by the library */
@@ -129,7 +133,8 @@ int32_t ps_slot_ptr(ps_ctx* ctx, int64_t slot_id, float** dev_ptr_out);
  *   slot_ids[w] if slot_ids != NULL, else to grads_dev + w*PS_PARAM_STRIDE      (dev, written)
  *   loss_dev [W] mean cross-entropy per worker; argmax_dev [W][b] lowest index of the largest
  *   logit                                                                       (dev, written)
- * Errors: PS_ERR_BAD_ARG (W, b out of range; NULL pointers; slot not reserved). A label outside
+ * On the tensor-core path x_dev must be 16-byte aligned (the images are read by TMA tile copies).
+ * Errors: PS_ERR_BAD_ARG (W, b out of range; NULL pointers; slot not reserved; misaligned x_dev). A label outside
  * 0..9 is reported as PS_ERR_DEVICE_STATUS by ps_stats(). */
 int32_t workers_grad_step(ps_ctx* ctx, int32_t W, int32_t b, const ps_snapshot* snaps,
                           const int32_t* worker_ids, const float* x_dev, const int32_t* y_dev,

@@ -38,6 +38,20 @@ __device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {   // lo in t
   return r;
 }
 
+// prmt.b32 in its default mode: selector nibble n picks byte (n & 7) of {b, a}; with bit 3 of the nibble set, the
+// picked byte's top bit is replicated over the whole output byte instead.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t selector) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(selector));
+  return r;
+}
+// x << n for a 64-bit x, with n >= 64 giving 0 (PTX clamps the shift amount; C++ leaves it undefined).
+__device__ __forceinline__ unsigned long long shl64_clamped(unsigned long long x, uint32_t n) {
+  unsigned long long r;
+  asm("shl.b64 %0, %1, %2;" : "=l"(r) : "l"(x), "r"(n));
+  return r;
+}
+
 // Where element (channel oc, pooled position p) of a sample's pooled gradient dp2 and of its pooling decisions
 // sits on the tensor-core path: [channel quad][position][4 channels], so that a thread of the backward
 // kernels takes four channels of a position with one vector load.  `canonical` = oc * 49 + p.

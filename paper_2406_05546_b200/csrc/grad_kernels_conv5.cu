@@ -290,8 +290,8 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
       // Item e = lt + 256 k is (octet of output channels e / 49, pooled position e % 49).  The raw slot holds
       // the gradients and the decisions as [channel quad][position][4 channels], so an item is two 16-byte and
       // two 4-byte loads.  Its eight gradients become four BF16 pairs once; for each of the four positions of
-      // the window the pairs are masked by "this position won" (a per-byte comparison of the four decisions,
-      // spread to half-words) and stored as the position's 16-byte row, which also clears the losers.
+      // the window the pairs are masked by "this position won" and stored as the position's 16-byte row, which
+      // also clears the losers.
 #pragma unroll
       for (int k = 0; k < X_ITEMS; ++k) {
         const int e = lt + k * LOADERS;
@@ -303,9 +303,12 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
           uint4* d = reinterpret_cast<uint4*>(dst) + o8 * (X_PLANE_BYTES / 16) + (2 * py + 1) * 16 + 2 * px + 1;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const uint32_t ma = __vcmpeq4(ca, 0x01010101u * j), mb = __vcmpeq4(cb, 0x01010101u * j);   // 0xFF where the code is j
-            d[(j >> 1) * 16 + (j & 1)] = make_uint4(h0 & __byte_perm(ma, 0u, 0x1100), h1 & __byte_perm(ma, 0u, 0x3322),
-                                                    h2 & __byte_perm(mb, 0u, 0x1100), h3 & __byte_perm(mb, 0u, 0x3322));
+            // a decision byte is 0..4, so (byte xor j) + 0x7F has its top bit set exactly when the byte differs from j;
+            // byte permutes that replicate the top bit turn the four flags into two pairs of half-word masks
+            const uint32_t ea = ~((ca ^ (0x01010101u * j)) + 0x7F7F7F7Fu) & 0x80808080u;
+            const uint32_t eb = ~((cb ^ (0x01010101u * j)) + 0x7F7F7F7Fu) & 0x80808080u;
+            d[(j >> 1) * 16 + (j & 1)] = make_uint4(h0 & prmt(ea, 0u, 0x9988u), h1 & prmt(ea, 0u, 0xBBAAu),
+                                                    h2 & prmt(eb, 0u, 0x9988u), h3 & prmt(eb, 0u, 0xBBAAu));
           }
         }
       }

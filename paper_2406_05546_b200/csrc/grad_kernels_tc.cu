@@ -179,10 +179,12 @@ __global__ void __launch_bounds__(DW_THREADS, 1) conv2_dw_tc(GradStepArgs a, Wor
           uint32_t* d = g2w + (4 * q) * DW_G_WORDS + (2 * py) * 7 + px;    // word of positions (2py, 2px), (2py, 2px+1)
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
+            // shifted left by 16 bits per decision, the BF16 value lands in the half-word of the winning window position
+            // (low word: row 2py, high word: row 2py + 1); decision 4 shifts it out entirely
             const uint32_t code = (c4 >> (8 * c)) & 0xFFu;
-            const uint32_t h = (uint32_t)bf16_bits(v[c]) << ((code & 1u) * 16u);    // low half: even column, high half: odd column
-            d[c * DW_G_WORDS] = (code >> 1) == 0u ? h : 0u;
-            d[c * DW_G_WORDS + 7] = (code >> 1) == 1u ? h : 0u;
+            const unsigned long long slot = shl64_clamped(bf16_bits(v[c]), 16u * code);
+            d[c * DW_G_WORDS] = (uint32_t)slot;
+            d[c * DW_G_WORDS + 7] = (uint32_t)(slot >> 32);
           }
         }
       }
@@ -351,9 +353,12 @@ __global__ void __launch_bounds__(256) conv1_bwd_tc(GradStepArgs a, WorkerTable 
         const float v[4] = {gr[k].x, gr[k].y, gr[k].z, gr[k].w};
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
+          // the BF16 value shifted left by 16 bits per decision lands in the half-word of the window position that
+          // won: low word = row 2py (even, odd column), high word = row 2py + 1; decision 4 shifts it out entirely
           const uint32_t code = (cr[k] >> (8 * c)) & 0xFFu;
-          d[c * C1B_A_WORDS] = bf16_pair(code == 0 ? v[c] : 0.f, code == 1 ? v[c] : 0.f);
-          d[c * C1B_A_WORDS + 14] = bf16_pair(code == 2 ? v[c] : 0.f, code == 3 ? v[c] : 0.f);
+          const unsigned long long slot = shl64_clamped(bf16_bits(v[c]), 16u * code);
+          d[c * C1B_A_WORDS] = (uint32_t)slot;
+          d[c * C1B_A_WORDS + 14] = (uint32_t)(slot >> 32);
         }
       }
     }
