@@ -282,22 +282,23 @@ __global__ void __launch_bounds__(DW_THREADS, 1) conv2_dw_tc(GradStepArgs a, Wor
 // ------------------------------------------------------------------------------------------------
 constexpr int C1B_SPB = 16;
 constexpr int C1B_A_WORDS = 396;       // 392 position pairs per channel + 4: 396 = 12 (mod 32 banks)
-constexpr int C1B_X_WORDS = 15 * 32;   // bordered 30 x 32 image as bf16 pairs
+constexpr int C1B_ROW = 42;            // elements per row of the bordered image: 21 words, so that the three filter rows
+constexpr int C1B_X_WORDS = 656;       // and the two copies (656 = 16 mod 32 words apart) fall into different banks
 constexpr int C1B_ITEMS = (4 * 196 + 255) / 256;   // (channel quad, position) items per thread
 constexpr int C1B_KSTEPS = 7;                       // k-steps per warp: ceil(49 / 8)
 __global__ void __launch_bounds__(256) conv1_bwd_tc(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks) {
   __shared__ __align__(16) uint32_t da1w[16 * C1B_A_WORDS];
-  __shared__ __align__(16) uint32_t xw[2][C1B_X_WORDS + 16];   // copy 1 is shifted by one element
+  __shared__ __align__(16) uint32_t xw[2][C1B_X_WORDS];   // bordered 30 x 42 image as bf16 pairs; copy 1 is shifted by one element
   __shared__ float red[8][16][17];
   uint16_t* xh0 = reinterpret_cast<uint16_t*>(xw[0]);
   const int s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-  for (int idx = tid; idx < 2 * (C1B_X_WORDS + 16); idx += 256) (&xw[0][0])[idx] = 0u;
+  for (int idx = tid; idx < 2 * C1B_X_WORDS; idx += 256) (&xw[0][0])[idx] = 0u;
   for (int idx = tid; idx < 16 * C1B_A_WORDS; idx += 256) da1w[idx] = 0u;
   // this lane's B columns: tile 0 column g = tap g; tile 1 column 0 = tap 8, column 1 = ones
   const int ky0 = g / 3, kx0 = g - ky0 * 3;                  // tap g (g < 8)
   const int copy0 = kx0 & 1;
-  const int off0 = ky0 * 32 + kx0 - copy0;                   // element offset of tap g in its copy (even)
-  const int off8 = 2 * 32 + 2;                               // tap 8 = (2, 2) in copy 0
+  const int off0 = ky0 * C1B_ROW + kx0 - copy0;                   // element offset of tap g in its copy (even)
+  const int off8 = 2 * C1B_ROW + 2;                               // tap 8 = (2, 2) in copy 0
   float acc[2][4];
 #pragma unroll
   for (int n = 0; n < 2; ++n)
@@ -314,7 +315,7 @@ __global__ void __launch_bounds__(256) conv1_bwd_tc(GradStepArgs a, WorkerTable 
   for (int i7 = 0; i7 < C1B_KSTEPS; ++i7) {
     const int j0 = (warp + 8 * i7) * 8 + t, j1 = j0 + 4;
     const int y0 = j0 / 14, x0 = 2 * (j0 - y0 * 14), y1 = j1 / 14, x1 = 2 * (j1 - y1 * 14);
-    const int e0 = y0 * 32 + x0, e1 = y1 * 32 + x1;         // bordered element (y, x) of tap (0, 0)
+    const int e0 = y0 * C1B_ROW + x0, e1 = y1 * C1B_ROW + x1;         // bordered element (y, x) of tap (0, 0)
     xo[i7][0] = (e0 + off0) >> 1; xo[i7][1] = (e1 + off0) >> 1; xo[i7][2] = (e0 + off8) >> 1; xo[i7][3] = (e1 + off8) >> 1;
   }
 
@@ -334,9 +335,9 @@ __global__ void __launch_bounds__(256) conv1_bwd_tc(GradStepArgs a, WorkerTable 
   for (int i = i0; i < i1; ++i) {
     __syncthreads();                        // the previous sample's products are done with shared memory
     if (tid < 196) {
-      // pixels 4 tid .. 4 tid + 3 of row yy; element (yy, xx) sits at el = (yy + 1) * 32 + xx + 1 of copy 0 and at
+      // pixels 4 tid .. 4 tid + 3 of row yy; element (yy, xx) sits at el = (yy + 1) * C1B_ROW + xx + 1 of copy 0 and at
       // el - 1 of copy 1, so the four are two aligned words of copy 1 and half, whole, half a word of copy 0
-      const int yy = tid / 7, xx = 4 * (tid - yy * 7), el = (yy + 1) * 32 + xx + 1;
+      const int yy = tid / 7, xx = 4 * (tid - yy * 7), el = (yy + 1) * C1B_ROW + xx + 1;
       const uint32_t h01 = bf16_pair(xr.x, xr.y), h23 = bf16_pair(xr.z, xr.w);
       xw[1][(el - 1) >> 1] = h01;
       xw[1][((el - 1) >> 1) + 1] = h23;

@@ -3,7 +3,8 @@ import numpy as np
 import pytest
 
 from paper_2406_05546_b200 import synth
-from tests.parity import TOL_FP32, TOL_TENSOR, assert_argmax_valid, assert_params_close
+from tests.parity import (TOL_FP32, TOL_TENSOR, assert_argmax_valid, assert_params_close,
+                          assert_params_close_up_to_unit_flips)
 
 pytestmark = pytest.mark.gpu
 
@@ -52,6 +53,11 @@ def _run_and_compare(W, b, lags=None, n_versions=1, step=3, drop_p=0.25, worker_
     thetas = [versions[s.version] for s in snaps]
     og, ol, oa, oz = cnn.workers_grad_step(thetas, ids, x, y, SEED, step, drop_p, precision=precision)
     for w in range(W):
+        if precision and W * b > 500:     # several hundred thousand ReLU decisions: see the helper's docstring
+            flipped = assert_params_close_up_to_unit_flips(grads[w, :ps.P], og[w], tol, 2, f"gradient of worker {w}")
+            if flipped.size:
+                print(f"worker {w}: hidden units decided differently near zero: {flipped}")
+            continue
         errs = assert_params_close(grads[w, :ps.P], og[w], tol, f"gradient of worker {w}")
         if precision and w == 0:
             print("tensor-path relative errors:", {k: f"{v:.1e}" for k, v in errs.items()})
@@ -81,12 +87,15 @@ def test_stale_snapshots_grouped_over_three_versions():
 
 @pytest.mark.parametrize("W,b,kw", [(2, 8, {}), (3, 5, {"worker_ids": [11, 4, 200]}), (2, 150, {}),
                                      (5, 6, {"lags": [2, 0, 1, 2, 0], "n_versions": 3}), (1, 1, {}),
-                                     (2, 4, {"drop_p": 0.0})])
-def test_tf32_tensor_core_path(W, b, kw):
+                                     (2, 4, {"drop_p": 0.0}),
+                                     # 777 rows over two weight versions: the persistent convolution kernels take
+                                     # ranges of several rows that cross worker boundaries inside a version group
+                                     (7, 111, {"lags": [1, 0, 1, 1, 0, 0, 1], "n_versions": 2})])
+def test_tensor_core_path(W, b, kw):
     _run_and_compare(W, b, precision=2, **kw)
 
 
-def test_tf32_repeatable_bit_for_bit():
+def test_tensor_core_path_repeatable_bit_for_bit():
     a = _run_and_compare(3, 9, precision=2)
     b = _run_and_compare(3, 9, precision=2)
     assert (a == b).all()
@@ -166,3 +175,44 @@ def test_argument_errors():
         srv.ps_pull_snapshot(0, lag=1)
     assert e.value.name == "PS_ERR_VERSION_EVICTED"
     srv.close()
+
+
+@pytest.mark.parametrize("precision,W,b", [(0, 3, 4), (0, 9, 5), (2, 9, 5), (2, 8, 16)])
+def test_tick_from_host_buffers_matches_the_oracle(precision, W, b):
+    """ps_tick_host: inputs copied in by worker chunks (four when there are eight workers or more), snapshots
+    with lags, grad step into reserved slots, enqueue, sync apply, losses and labels copied out."""
+    from oracle import cnn, ps as ops
+    import torch
+    from paper_2406_05546_b200 import ps
+    tol = TOL_TENSOR if precision else TOL_FP32
+    theta0 = synth.init_params(seed=1, bias_scale=0.05)
+    srv = ps.ParameterServer(theta0, max_workers=W, max_batch=b, ring_depth=2, queue_slots=W, dropout_p=0.25,
+                             precision=precision)
+    o = ops.OraclePS(theta0, ring_depth=2)
+    # one async update first, so that lag 1 reads different weights than lag 0
+    g = np.zeros((1, ps.P_PAD), dtype=np.float32)
+    g[0, :ps.P] = synth.random_gradients(1, seed=61, scale=2.0)[0]
+    srv.ps_enqueue([0], [0], 0, grads_dev=torch.from_numpy(g).cuda())
+    srv.ps_apply(ps.ASYNC, 0.01)
+    o.enqueue(g[:, :ps.P], [0], [0], 0)
+    o.apply(ops.ASYNC, 0.01)
+    rng = np.random.default_rng(11)
+    x = rng.random((W, b, 28, 28), dtype=np.float32)
+    y = rng.integers(0, 10, (W, b)).astype(np.int32)
+    lags = [(w * 3) % 2 for w in range(W)]
+    am = np.zeros((W, b), dtype=np.int32)
+    loss, res = srv.ps_tick_host(x, y, SEED, 5, ps.SYNC, 0.01, lags=lags, argmax_host=am)
+    theta, version = srv.ps_export_params()
+    srv.ps_stats()
+    srv.close()
+    thetas = [o.pull_snapshot(w, l)[1] for w, l in enumerate(lags)]
+    og, ol, oa, oz = cnn.workers_grad_step(thetas, list(range(W)), x, y, SEED, 5, 0.25, precision=precision)
+    o.enqueue(og.astype(np.float32), range(W), [1 - l for l in lags], 5)
+    o.apply(ops.SYNC, 0.01)
+    assert res["applied"] == W and version == res["new_version"] == 2
+    np.testing.assert_allclose(loss, ol, rtol=3e-3 if precision else 1e-5, atol=1e-6)
+    assert_argmax_valid(am, oz, tol if precision else 10 * TOL_FP32)
+    assert_params_close(theta, o.head(), tol, "parameters after the tick")
+    # the tick moves the head by lr * mean gradient: compare that step too, which the parameters' size would hide
+    before = o.ring[1].astype(np.float64)
+    assert_params_close(theta - before, o.head() - before, max(tol, 10 * TOL_FP32), "the tick's update")
