@@ -32,7 +32,7 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int m, int n) {     // fp32 ac
 
 constexpr int F_NBUF = 4;             // shared-memory tile buffers of the forward kernel (copies run four tiles ahead)
 struct Pipe {
-  uint64_t a_full[F_NBUF], a_empty[F_NBUF], acc_full[2], acc_empty[2], raw_full[2], raw_empty[2];
+  uint64_t a_full[F_NBUF], a_empty[F_NBUF], acc_full[2], acc_empty[2], raw_full[4], raw_empty[4];
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -45,8 +45,10 @@ __device__ __forceinline__ void pipe_init(Pipe* p, int a_full_arrivals, int acc_
   for (int i = 0; i < 2; ++i) {
     mbar_init(&p->acc_full[i], 1);
     mbar_init(&p->acc_empty[i], acc_empty_arrivals);
+  }
+  for (int i = 0; i < 4; ++i) {
     mbar_init(&p->raw_full[i], 1);
-    mbar_init(&p->raw_empty[i], LOADERS / 32);
+    mbar_init(&p->raw_empty[i], LOADERS / 64);
   }
   p->abort_flag = 0;
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -209,14 +211,15 @@ constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // staging stores of 
 constexpr int X_BUF_BYTES = 4 * X_PLANE_BYTES;             // four planes of eight output channels
 constexpr int X_W_BYTES = 12 * 48 * 16;                    // [filter row ky][k chunk oc/8][column = kx*16 + ic][8 bf16]
 constexpr int X_RAW_BYTES = FLAT * 4 + FLAT;                // one sample's pooled gradients (fp32) and pooling decisions (bytes)
-constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + 2 * X_RAW_BYTES + sizeof(Pipe) + 128;
+constexpr int X_RAW_SLOTS = 4;
+constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + X_RAW_SLOTS * X_RAW_BYTES + sizeof(Pipe) + 128;
 
 __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, GroupTable gt, Workspace ws, int range_len) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint16_t* bufs = reinterpret_cast<uint16_t*>(smem);
   uint16_t* Wk = reinterpret_cast<uint16_t*>(smem + 2 * X_BUF_BYTES);
   uint8_t* raw = smem + 2 * X_BUF_BYTES + X_W_BYTES;        // two raw staging slots filled by bulk copies
-  Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * X_BUF_BYTES + X_W_BYTES + 2 * X_RAW_BYTES);
+  Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * X_BUF_BYTES + X_W_BYTES + X_RAW_SLOTS * X_RAW_BYTES);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int grp, r_begin, r_end;
   if (!locate_row_range(gt, a.b, range_len, blockIdx.x, grp, r_begin, r_end)) return;
@@ -228,7 +231,7 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
     Wk[(((tap / 3) * 4 + (oc >> 3)) * 48 + (tap % 3) * 16 + ic) * 8 + (oc & 7)] = bf16_bits(theta[OFF_C2W + idx]);
   }
   for (int idx = tid; idx < 2 * X_BUF_BYTES / 16; idx += THREADS) reinterpret_cast<float4*>(smem)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (tid == 0) pipe_init(pipe, LOADERS / 32, 4);
+  if (tid == 0) pipe_init(pipe, LOADERS / 64, 4);
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&pipe->tmem_base)), "r"(256) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -266,35 +269,37 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
       }
     }
   } else if (warp <= LOADERS / 32) {
-    const int lt = tid - 32;
-    constexpr int X_ITEMS = (4 * 49 + LOADERS - 1) / LOADERS;      // (channel octet, position) items per thread
-    // The pooled gradients and decisions of a sample arrive in a raw slot by two bulk copies issued two
-    // tiles ahead, so no global-memory latency sits in this loop.
+    // Two groups of four staging warps: group g builds the tiles t = g, g + 2, ... into plane buffer g, so two
+    // tiles are being staged at any time (a tile's staging is a chain of dependent shared-memory accesses, bound
+    // by latency rather than by throughput).  The pooled gradients and decisions of a sample arrive in one of
+    // four raw slots by two bulk copies issued by the group's first thread, two of the group's tiles ahead.
+    const int grp_w = (warp - 1) >> 2, lt = (tid - 32) & 127;
+    constexpr int X_ITEMS = (4 * 49 + 127) / 128;                  // (channel octet, position) items per thread
     auto fetch_raw = [&](int t) {
       const int64_t row = r_begin + t;
-      uint8_t* slot = raw + (t & 1) * X_RAW_BYTES;
-      mbar_expect_tx(&pipe->raw_full[t & 1], X_RAW_BYTES);
-      bulk_load(slot, ws.dp2 + row * FLAT, FLAT * 4, &pipe->raw_full[t & 1]);
-      bulk_load(slot + FLAT * 4, ws.code2 + row * FLAT, FLAT, &pipe->raw_full[t & 1]);
+      uint8_t* slot = raw + (t & 3) * X_RAW_BYTES;
+      mbar_expect_tx(&pipe->raw_full[t & 3], X_RAW_BYTES);
+      bulk_load(slot, ws.dp2 + row * FLAT, FLAT * 4, &pipe->raw_full[t & 3]);
+      bulk_load(slot + FLAT * 4, ws.code2 + row * FLAT, FLAT, &pipe->raw_full[t & 3]);
     };
-    if (lt == 0) { fetch_raw(0); if (n_tiles > 1) fetch_raw(1); }
-    for (int t = 0; t < n_tiles; ++t) {
-      const int buf = t & 1;
+    if (lt == 0) { if (grp_w < n_tiles) fetch_raw(grp_w); if (grp_w + 2 < n_tiles) fetch_raw(grp_w + 2); }
+    for (int t = grp_w; t < n_tiles; t += 2) {
+      const int buf = t & 1, slot_i = t & 3;
       // every staging warp waits and reports on its own (no block-level barrier among them)
-      bool ok = mbar_wait(&pipe->raw_full[buf], (t >> 1) & 1);
+      bool ok = mbar_wait(&pipe->raw_full[slot_i], (t >> 2) & 1);
       if (ok && t >= 2) ok = mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1);
       if (!__all_sync(0xffffffffu, ok) || pipe->abort_flag) { pipe->abort_flag = 1; break; }
       uint16_t* dst = bufs + buf * (X_BUF_BYTES / 2);
-      const float* rg = reinterpret_cast<const float*>(raw + buf * X_RAW_BYTES);
-      const uint8_t* rc = raw + buf * X_RAW_BYTES + FLAT * 4;
-      // Item e = lt + 256 k is (octet of output channels e / 49, pooled position e % 49).  The raw slot holds
+      const float* rg = reinterpret_cast<const float*>(raw + slot_i * X_RAW_BYTES);
+      const uint8_t* rc = raw + slot_i * X_RAW_BYTES + FLAT * 4;
+      // Item e = lt + 128 k is (octet of output channels e / 49, pooled position e % 49).  The raw slot holds
       // the gradients and the decisions as [channel quad][position][4 channels], so an item is two 16-byte and
       // two 4-byte loads.  Its eight gradients become four BF16 pairs once; for each of the four positions of
       // the window the pairs are masked by "this position won" and stored as the position's 16-byte row, which
       // also clears the losers.
 #pragma unroll
       for (int k = 0; k < X_ITEMS; ++k) {
-        const int e = lt + k * LOADERS;
+        const int e = lt + k * 128;
         if (e < 4 * 49) {
           const int o8 = e / 49, p = e - o8 * 49, py = p / 7, px = p - py * 7;
           const float4 va = reinterpret_cast<const float4*>(rg)[(2 * o8) * 49 + p], vb = reinterpret_cast<const float4*>(rg)[(2 * o8 + 1) * 49 + p];
@@ -314,11 +319,11 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
       }
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) { mbar_arrive(&pipe->a_full[buf]); mbar_arrive(&pipe->raw_empty[buf]); }
-      // the raw slot is refilled once every staging warp has read it
-      if (lt == 0 && t + 2 < n_tiles) {
-        if (!mbar_wait(&pipe->raw_empty[buf], (t >> 1) & 1)) { pipe->abort_flag = 1; break; }
-        fetch_raw(t + 2);
+      if (lane == 0) { mbar_arrive(&pipe->a_full[buf]); mbar_arrive(&pipe->raw_empty[slot_i]); }
+      // the raw slot is refilled once every warp of the group has read it
+      if (lt == 0 && t + 4 < n_tiles) {
+        if (!mbar_wait(&pipe->raw_empty[slot_i], (t >> 2) & 1)) { pipe->abort_flag = 1; break; }
+        fetch_raw(t + 4);
       }
     }
   } else {
