@@ -1,0 +1,266 @@
+// Filter and bias gradient of the second convolution on the fifth-generation tensor cores (BF16 operands,
+// fp32 accumulation in tensor memory; values only, no decision depends on them).
+//
+//   dW[oc][ic][ky][kx] = sum over samples and positions of g2[oc][y][x] * p1pad[ic][y + ky][x + kx]
+//
+// with g2 the gradient at the convolution's output (the pooled gradient put back at the pooling winners) and
+// p1pad the zero-bordered 16x16 input.  The contraction runs over positions, so both operands are needed with
+// the position index contiguous ("k-major": core matrices of 8 rows x 8 positions).  With q = (y + ky) * 16 + x
+// as the contraction index, one MMA per image row q / 16 computes
+//
+//   D[(kx, ic)][(ky, oc)] += A[(kx, ic)][q] * B[(ky, oc)][q],   A[(kx, ic)][q] = p1pad[ic][q + kx],
+//                                                                B[(ky, oc)][q] = g2[oc][q - 16 ky]
+//
+// i.e. M = 48 (+ one row of ones, whose products are the bias gradient; the tile is M = 64, the other rows
+// are never read), N = 96, K = 16: sixteen MMAs per sample, accumulated over all samples of a worker.
+// The staging warps build both operands: A by transposing 8 x 8 blocks of the BF16 input planes (one
+// ldmatrix.trans + stmatrix pair per four blocks; the three kx copies differ in the rows addressed), B from the
+// pooled gradient and the pooling decisions, written three times, one image row apart, for the three ky.
+// One CTA per SM walks over a contiguous range of rows (sorted worker, sample); where the range passes from one
+// worker to the next, and at its end, the accumulator is written out as a partial sum that a later kernel adds
+// in a fixed order.  Every mbarrier wait is bounded.
+#include "device_common.cuh"
+#include "kernels.h"
+#include "tc5_common.cuh"
+
+namespace psk {
+
+namespace {
+
+constexpr int W5_LOAD_WARPS = 16;                       // two groups of eight: group g stages samples n = g, g + 2, ...
+constexpr int W5_THREADS = 32 * (1 + W5_LOAD_WARPS + 4);   // warp 0: MMA issue and tensor memory; the last four warps write out
+constexpr int W5_CHUNKS = 32;                           // 8-position chunks of the 256 contraction indices of a sample
+constexpr int W5_GROUP_BYTES = W5_CHUNKS * 128;         // one group of 8 operand rows: 32 core matrices of 128 bytes
+constexpr int W5_A_GROUPS = 7;                          // (kx, channel octet) x 6, then the group whose first row is all ones
+constexpr int W5_B_GROUPS = 12;                         // (ky, channel octet)
+constexpr int W5_A_BYTES = W5_A_GROUPS * W5_GROUP_BYTES;     // 28,672
+constexpr int W5_STAGE_BYTES = W5_A_BYTES + W5_B_GROUPS * W5_GROUP_BYTES;   // 77,824; the A descriptor of M = 64 spans 8
+                                                        // groups from the stage's start (the eighth is B's first: rows never read)
+constexpr int W5_RAW_P1 = P1_PLANE_ELEMS * 4, W5_RAW_DP2 = FLAT * 4, W5_RAW_CODE = FLAT;
+constexpr int W5_RAW_BYTES = W5_RAW_P1 + W5_RAW_DP2 + W5_RAW_CODE;          // 16,032
+constexpr int W5_RAW_SLOT = (W5_RAW_BYTES + 127) / 128 * 128;
+constexpr int W5_NRAW = 4;                              // raw input slots: each group's copies run two of its samples ahead
+constexpr int W5_SMEM = 2 * W5_STAGE_BYTES + W5_NRAW * W5_RAW_SLOT + 256 + 128;
+constexpr int W5_TMEM_COLS = 128;                       // 96 accumulator columns
+static_assert(8 * W5_GROUP_BYTES <= W5_STAGE_BYTES, "the 64-row A operand must stay inside its stage");
+static_assert(W5_SMEM <= 227 * 1024, "shared memory");
+
+__host__ __device__ constexpr uint32_t w5_idesc(int m, int n) {     // fp32 accumulate, BF16 x BF16, both k-contiguous
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void stmatrix_x4(uint32_t addr, const uint32_t (&r)[4]) {
+  asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};"
+               ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+}
+
+struct W5Bars {
+  uint64_t op_full[2], op_empty[2], raw_full[W5_NRAW], raw_empty[W5_NRAW], acc_full, acc_empty;
+  uint32_t tmem_base;
+  volatile uint32_t abort_flag;
+};
+
+// Rows (sorted worker, sample) are split into gridDim.x contiguous ranges of seg_len.  Partial sums of worker s go
+// to part2[s][range index - first range of s].
+__global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, WorkerTable wt, Workspace ws, int seg_len, int slots) {
+  extern __shared__ __align__(1024) uint8_t sm[];
+  uint8_t* raw = sm + 2 * W5_STAGE_BYTES;
+  W5Bars* bars = reinterpret_cast<W5Bars*>(raw + W5_NRAW * W5_RAW_SLOT);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int total = a.W * a.b;
+  const int r0 = blockIdx.x * seg_len, r1 = min(r0 + seg_len, total), n_samples = r1 - r0;
+
+  // operand stages start as zeros (B: borders and rows that a ky copy never reaches); the ones row of A is
+  // written once: row 0 of group 6, i.e. the first 16 bytes of each of its core matrices
+  for (int i = tid; i < 2 * W5_STAGE_BYTES / 16; i += W5_THREADS) reinterpret_cast<uint4*>(sm)[i] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+  for (int i = tid; i < 2 * W5_CHUNKS; i += W5_THREADS)
+    *reinterpret_cast<uint4*>(sm + (i / W5_CHUNKS) * W5_STAGE_BYTES + 6 * W5_GROUP_BYTES + (i % W5_CHUNKS) * 128) =
+        make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+  if (tid == 0) {
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->op_full[i], W5_LOAD_WARPS / 2); mbar_init(&bars->op_empty[i], 1); }
+    for (int i = 0; i < W5_NRAW; ++i) { mbar_init(&bars->raw_full[i], 1); mbar_init(&bars->raw_empty[i], W5_LOAD_WARPS / 2); }
+    mbar_init(&bars->acc_full, 1);
+    mbar_init(&bars->acc_empty, 4);
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)), "r"(W5_TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_proxy_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+
+  if (warp == 0) {
+    // ---------------- MMA issue
+    if (lane == 0) {
+      constexpr uint32_t idesc = w5_idesc(64, 96);
+      int writes = 0;
+      bool fresh = true;                       // the next MMA starts a new sum
+      for (int n = 0; n < n_samples; ++n) {
+        const int st = n & 1;
+        if (!mbar_wait(&bars->op_full[st], (n >> 1) & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
+        tc_fence_after();
+        const uint32_t a_lo = plain_desc_lo(smem_u32(sm) + st * W5_STAGE_BYTES, 128);
+        const uint32_t b_lo = plain_desc_lo(smem_u32(sm) + st * W5_STAGE_BYTES + W5_A_BYTES, 128);
+#pragma unroll
+        for (int ks = 0; ks < 16; ++ks)        // contraction indices 16 ks .. 16 ks + 15: two chunks of 128 bytes
+          umma_f16_split(tmem, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), idesc,
+                         (ks == 0 && fresh) ? 0u : 1u);
+        fresh = false;
+        umma_commit(&bars->op_empty[st]);
+        const int row = r0 + n;
+        if (row + 1 == r1 || (row + 1) % a.b == 0) {
+          // last row of the range or of a worker: hand the sum to the write-out warps and wait until they have read it
+          umma_commit(&bars->acc_full);
+          if (!mbar_wait(&bars->acc_empty, writes & 1)) { bars->abort_flag = 1; break; }
+          tc_fence_after();
+          ++writes;
+          fresh = true;
+        }
+      }
+    }
+  } else if (warp <= W5_LOAD_WARPS) {
+    // ---------------- staging: group g (eight warps) builds the operands of samples n = g, g + 2, ... in stage g
+    const int grp = (warp - 1) >> 3, gw = (warp - 1) & 7, gt_ = gw * 32 + lane;      // thread index inside the group
+    auto issue = [&](int n) {            // one thread: the three input rows of sample r0 + n
+      const int64_t row = r0 + n;
+      uint8_t* dst = raw + (n & 3) * W5_RAW_SLOT;
+      uint64_t* bar = &bars->raw_full[n & 3];
+      mbar_expect_tx(bar, W5_RAW_BYTES);
+      bulk_load(dst, ws.p1 + row * P1_PLANE_ELEMS, W5_RAW_P1, bar);
+      bulk_load(dst + W5_RAW_P1, ws.dp2 + row * FLAT, W5_RAW_DP2, bar);
+      bulk_load(dst + W5_RAW_P1 + W5_RAW_DP2, ws.code2 + row * FLAT, W5_RAW_CODE, bar);
+    };
+    if (gt_ == 0) { if (grp < n_samples) issue(grp); if (grp + 2 < n_samples) issue(grp + 2); }
+    for (int n = grp; n < n_samples; n += 2) {
+      const int slot = n & 3;
+      bool ok = mbar_wait(&bars->raw_full[slot], (n >> 2) & 1);
+      if (ok && n >= 2) ok = mbar_wait(&bars->op_empty[grp], ((n >> 1) - 1) & 1);
+      if (!__all_sync(0xffffffffu, ok) || bars->abort_flag) { bars->abort_flag = 1; break; }
+      const uint8_t* rp1 = raw + slot * W5_RAW_SLOT;
+      const float* rdp2f = reinterpret_cast<const float*>(rp1 + W5_RAW_P1);
+      const uint8_t* rcode8 = rp1 + W5_RAW_P1 + W5_RAW_DP2;
+      uint8_t* stage = sm + grp * W5_STAGE_BYTES;
+      // A: 6 groups x 32 chunks = 192 blocks of 8 positions x 8 channels, transposed four at a time.  Operation o of
+      // the 48 covers chunks 4 (o % 8) .. + 3 of group o / 8 = (kx, channel octet).  Lane l addresses row l % 8 of
+      // block l / 8: on the way in the input plane's row of position 8 chunk + row + kx (plane rows keep even and
+      // odd columns apart; positions past the end read the all-zero row 0), on the way out the core matrix's row.
+#pragma unroll
+      for (int o = gw; o < 48; o += 8) {
+        const int g = o >> 3, kx = g >> 1, oct = g & 1, chunk = 4 * (o & 7) + (lane >> 3);
+        const int i = 8 * chunk + (lane & 7) + kx;
+        const int prow = i < 256 ? (i & ~15) + ((i & 1) << 3) + ((i & 15) >> 1) : 0;
+        uint32_t r[4];
+        ldmatrix_x4_trans(r, smem_u32(rp1 + oct * 4096 + prow * 16));
+        stmatrix_x4(smem_u32(stage + g * W5_GROUP_BYTES + chunk * 128 + (lane & 7) * 16), r);
+      }
+      // B: a warp takes (octet of output channels, pooled row py, half of the pooled columns) and a lane one channel of
+      // the octet and one pooled column of the four: its words then fall into 32 different banks.  Every pooled entry
+      // owns the four positions of its window: shifted left by 16 bits per decision, the BF16 gradient lands in the
+      // half-word of the winner (low word: image row 2py, high word: row 2py + 1; decision 4 shifts it out), the other
+      // three are cleared.  The pair of columns (2px, 2px + 1) is one word of a core-matrix row; the three ky copies
+      // lie one image row (two chunks) apart, image rows 2py and 2py + 1 likewise.
+#pragma unroll
+      for (int k = 0; k < 7; ++k) {
+        const int wi = gw * 7 + k, oct = wi / 14, rem = wi - oct * 14, py = rem >> 1, pxhi = rem & 1;
+        const int rr = lane >> 2, pl = lane & 3, px = 4 * pxhi + pl;
+        if (px < 7) {
+          const int oc = 8 * oct + rr, e = ((oc >> 2) * 49 + py * 7 + px) * 4 + (oc & 3);
+          const uint32_t code = rcode8[e];
+          const unsigned long long slot64 = shl64_clamped(bf16_bits(rdp2f[e]), 16u * code);
+          uint32_t* d = reinterpret_cast<uint32_t*>(stage + W5_A_BYTES + oct * W5_GROUP_BYTES + (4 * py + pxhi) * 128 + rr * 16) + pl;
+#pragma unroll
+          for (int ky = 0; ky < 3; ++ky) {
+            uint32_t* dk = d + ky * ((4 * W5_GROUP_BYTES + 256) / 4);          // copy ky: four groups on, image row 2py + ky
+            dk[0] = (uint32_t)slot64;
+            dk[64] = (uint32_t)(slot64 >> 32);                               // image row 2py + 1 + ky
+          }
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&bars->op_full[grp]); mbar_arrive(&bars->raw_empty[slot]); }
+      if (gt_ == 0 && n + 4 < n_samples) {
+        if (!mbar_wait(&bars->raw_empty[slot], (n >> 2) & 1)) { bars->abort_flag = 1; break; }
+        issue(n + 4);
+      }
+    }
+  } else {
+    // ---------------- write-out: a warp reads the accumulator lanes 32 (warp % 4) .. + 31.  An accumulator of 64 rows
+    // keeps rows 16 w .. 16 w + 15 in the first sixteen lanes of quarter w.
+    const int quarter = warp & 3;
+    int writes = 0;
+    for (int row = r0; row < r1; ++row) {
+      if (!(row + 1 == r1 || (row + 1) % a.b == 0)) continue;
+      if (!mbar_wait(&bars->acc_full, writes & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
+      tc_fence_after();
+      const int s = row / a.b;
+      float* part = ws.part2 + ((int64_t)s * slots + (blockIdx.x - (s * a.b) / seg_len)) * C2_GRAD;
+      const int rr = lane < 16 ? quarter * 16 + lane : 64;   // accumulator row: (kx, ic) for rr < 48, the ones row at 48
+#pragma unroll
+      for (int cb = 0; cb < 6; ++cb) {                 // 16 columns at a time: ky = cb / 2, oc = 16 (cb % 2) + j
+        uint32_t v[16];
+        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cb * 16), v);
+        tmem_ld_wait();
+        const int ky = cb >> 1;
+        if (rr < 48) {
+          const int kx = rr >> 4, ic = rr & 15;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) part[((16 * (cb & 1) + j) * 16 + ic) * 9 + ky * 3 + kx] = __uint_as_float(v[j]);
+        } else if (rr == 48 && ky == 0) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) part[4608 + 16 * (cb & 1) + j] = __uint_as_float(v[j]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->acc_empty);
+      ++writes;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(W5_TMEM_COLS) : "memory");
+  }
+  if (tid == 0 && bars->abort_flag) {
+    atomicOr(ws.status, STATUS_WAIT_TIMEOUT);
+    for (int k = 0; k < 1000; ++k) __nanosleep(1000);   // let copies already issued land before the CTA ends
+  }
+}
+
+}  // namespace
+
+#define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
+
+int configure_dw5_kernels() {
+  return cudaFuncSetAttribute(conv2_dw_tc5, cudaFuncAttributeMaxDynamicSharedMemorySize, W5_SMEM) == cudaSuccess ? 0 : -1;
+}
+
+// Returns the number of partial-sum slots reserved per worker (the stride of part2) and, in *seg_len, the length
+// of a CTA's range of rows: worker s owns one partial sum per range that meets its rows.
+int launch_conv2_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof,
+                        int* seg_len) {
+  const int total = a.W * a.b;
+  int grid = total / 16;                  // a range is at least 16 rows long (bounds the partial sums per worker)
+  if (grid > g_sm_count) grid = g_sm_count;
+  if (grid < 1) grid = 1;
+  const int len = (total + grid - 1) / grid;
+  grid = (total + len - 1) / len;
+  const int slots = (a.b - 1) / len + 2;
+  TIMED(K_CONV2_DW, (conv2_dw_tc5<<<grid, W5_THREADS, W5_SMEM, st>>>(a, wt, ws, len, slots)));
+  *seg_len = len;
+  return slots;
+}
+
+}  // namespace psk

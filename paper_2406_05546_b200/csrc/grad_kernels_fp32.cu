@@ -585,7 +585,7 @@ __global__ void __launch_bounds__(256) conv1_bwd(GradStepArgs a, WorkerTable wt,
 }
 
 // ---- sums the per-block partial gradients in block order, finishes the loss and zeroes the padding.
-// part2 holds n_chunks2 slots per worker; all of them are summed when seg_len == 0, otherwise four for every
+// part2 holds n_chunks2 slots per worker; all of them are summed when seg_len == 0, otherwise one for every
 // range of seg_len rows that meets the worker's b rows (the tensor-core filter-gradient kernel's layout).
 // A worker's outputs are numbered conv2 (4640), conv1 (160), output layer (5642), loss, padding; a block takes
 // RED_PER_BLOCK of them.
@@ -596,7 +596,7 @@ __global__ void __launch_bounds__(256) conv_grad_reduce(GradStepArgs a, WorkerTa
                                                         int seg_len) {
   const int s = blockIdx.x, b = a.b;
   float* grad = wt.grad[s];
-  const int used2 = seg_len > 0 ? 4 * ((s * b + b - 1) / seg_len - (s * b) / seg_len + 1) : n_chunks2;
+  const int used2 = seg_len > 0 ? (s * b + b - 1) / seg_len - (s * b) / seg_len + 1 : n_chunks2;
   for (int v = blockIdx.y * RED_PER_BLOCK + threadIdx.x; v < min(RED_OUTPUTS, ((int)blockIdx.y + 1) * RED_PER_BLOCK); v += 256) {
     int o = v;
     if (o < C2_GRAD) {
@@ -687,7 +687,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     if (n < 0) return -1;
     launches += n;
     if (side.s2) { cudaEventRecord(side.fork2, st); cudaStreamWaitEvent(s2, side.fork2, 0); }
-    n_chunks2 = launch_conv2_dw_tc(a, wt, ws, s2, prof, &seg_len);
+    n_chunks2 = launch_conv2_dw_tc5(a, wt, ws, s2, prof, &seg_len);
     if (side.s2) cudaEventRecord(side.join2, s2);
     launch_conv2_dx_tc5(a, wt, gt, ws, st, prof);
     const int n_chunks1t = launch_conv1_bwd_tc(a, wt, ws, st, prof);

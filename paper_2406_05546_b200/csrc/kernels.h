@@ -140,12 +140,13 @@ int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, ui
 int configure_grad_kernels();
 int configure_tc_kernels();
 int launch_conv1_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof);
-int launch_conv2_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof,
-                       int* seg_len);
 extern int g_sm_count;   // SMs of the current device, set by configure_tc5_kernels
 int configure_tc5_kernels();
 int configure_conv5_kernels();
 int configure_conv1_kernels();
+int configure_dw5_kernels();
+int launch_conv2_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof,
+                        int* seg_len);
 int launch_conv1_fwd_planes(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                             cudaStream_t st, Profiler* prof);
 void launch_conv2_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
