@@ -12,7 +12,8 @@
 //                                                                B[(ky, oc)][q] = g2[oc][q - 16 ky]
 //
 // i.e. M = 48 (+ one row of ones, whose products are the bias gradient; the tile is M = 64, the other rows
-// are never read), N = 96, K = 16: sixteen MMAs per sample, accumulated over all samples of a worker.
+// are never read), N = 96, K = 16: fourteen MMAs per sample (the input's two border rows contribute nothing),
+// accumulated over all samples of a worker.
 // The staging warps build both operands: A by transposing 8 x 8 blocks of the BF16 input planes (one
 // ldmatrix.trans + stmatrix pair per four blocks; the three kx copies differ in the rows addressed), B from the
 // pooled gradient and the pooling decisions, written three times, one image row apart, for the three ky.
@@ -111,10 +112,12 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
         tc_fence_after();
         const uint32_t a_lo = plain_desc_lo(smem_u32(sm) + st * W5_STAGE_BYTES, 128);
         const uint32_t b_lo = plain_desc_lo(smem_u32(sm) + st * W5_STAGE_BYTES + W5_A_BYTES, 128);
+        // contraction indices 16 ks .. 16 ks + 15 (image row ks of the bordered input): two chunks of 128 bytes.
+        // Rows 0 and 15 are the input's zero border, so their products vanish and are not issued.
 #pragma unroll
-        for (int ks = 0; ks < 16; ++ks)        // contraction indices 16 ks .. 16 ks + 15: two chunks of 128 bytes
+        for (int ks = 1; ks < 15; ++ks)
           umma_f16_split(tmem, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), idesc,
-                         (ks == 0 && fresh) ? 0u : 1u);
+                         (ks == 1 && fresh) ? 0u : 1u);
         fresh = false;
         umma_commit(&bars->op_empty[st]);
         const int row = r0 + n;
@@ -216,7 +219,7 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
           const int kx = rr >> 4, ic = rr & 15;
 #pragma unroll
           for (int j = 0; j < 16; ++j) part[((16 * (cb & 1) + j) * 16 + ic) * 9 + ky * 3 + kx] = __uint_as_float(v[j]);
-        } else if (rr == 48 && ky == 0) {
+        } else if (rr == 48 && ky == 1) {     // the ones row against the ky = 1 copy, whose rows 1..14 are all issued
 #pragma unroll
           for (int j = 0; j < 16; ++j) part[4608 + 16 * (cb & 1) + j] = __uint_as_float(v[j]);
         }
