@@ -307,10 +307,10 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
 #pragma unroll
       for (int c = 1; c < NCLS; ++c)
         if (z[u][c] > zmax) { zmax = z[u][c]; am = c; }
-      float se = 0.f;
+      float ez[NCLS], se = 0.f;
 #pragma unroll
-      for (int c = 0; c < NCLS; ++c) se += expf(z[u][c] - zmax);
-      const float lse = zmax + logf(se);
+      for (int c = 0; c < NCLS; ++c) { ez[c] = expf(z[u][c] - zmax); se += ez[c]; }
+      const float lse = zmax + logf(se), inv_se = 1.0f / se;
       int label = a.y[(int64_t)src * a.b + i];
       if (label < 0 || label >= NCLS) {
         if (lane == 0) atomicOr(ws.status, STATUS_BAD_LABEL);
@@ -320,7 +320,7 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
 #pragma unroll
       for (int c = 0; c < NCLS; ++c) {
         if (c == label) zy = z[u][c];
-        dz[u][c] = (expf(z[u][c] - lse) - (c == label ? 1.f : 0.f)) * inv_b;
+        dz[u][c] = (ez[c] * inv_se - (c == label ? 1.f : 0.f)) * inv_b;     // softmax from the exponentials already taken
       }
       loss_acc += lse - zy;
       if (lane == 0) a.argmax[(int64_t)src * a.b + i] = am;
