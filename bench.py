@@ -34,8 +34,8 @@ N_BATCH_BUFFERS = 8
 REPLAY_TRAFFIC_PER_GRADIENT = 2.654663e9 / 816
 # dram bytes (read + written) per sample of the grad-step kernels, from one ncu capture of a reduced case
 # (W=128, b=64: 8,192 samples; traffic grows in proportion to the samples); None = not captured since the kernel changed
-KERNEL_TRAFFIC_PER_SAMPLE = {"conv2_dw": None, "conv1_fwd": 7551, "conv2_bwd": None, "fc1_dw": 51747, "conv2_fwd": 9645,
-                             "fc1_dx": 2766, "fc1_fwd": 6842, "fc2_fwd_bwd": 2060, "conv1_bwd": None}
+KERNEL_TRAFFIC_PER_SAMPLE = {"conv2_dw": 16603, "conv1_fwd": 7685, "conv2_bwd": 13688, "fc1_dw": 51717, "conv2_fwd": 9668,
+                             "fc1_dx": 2744, "fc1_fwd": 6782, "fc2_fwd_bwd": 2060, "conv1_bwd": 19293}
 
 
 def measured_peaks():
