@@ -154,8 +154,6 @@ __global__ void __launch_bounds__(256) conv1_bwd_tc(GradStepArgs a, WorkerTable 
 
 #define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
 
-int configure_tc_kernels() { return 0; }
-
 int launch_conv1_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof) {
   const int chunks = (a.b + C1B_SPB - 1) / C1B_SPB;
   TIMED(K_CONV1_BWD, (conv1_bwd_tc<<<dim3(chunks, a.W), 256, 0, st>>>(a, wt, ws, chunks)));

@@ -138,7 +138,6 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
 int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, uint32_t thresh,
                         uint8_t* keep, cudaStream_t st, Profiler* prof);
 int configure_grad_kernels();
-int configure_tc_kernels();
 int launch_conv1_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof);
 extern int g_sm_count;   // SMs of the current device, set by configure_tc5_kernels
 int configure_tc5_kernels();
@@ -159,16 +158,6 @@ int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupT
                       cudaStream_t st, Profiler* prof);
 int launch_fc1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                       cudaStream_t st, Profiler* prof);
-void launch_fc1_fwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
-                       cudaStream_t st, Profiler* prof);
-void launch_fc1_dx_tc(const GradStepArgs& a, const GroupTable& gt, const Workspace& ws, cudaStream_t st,
-                      Profiler* prof);
-void launch_conv2_fwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
-                         cudaStream_t st, Profiler* prof);
-int launch_conv2_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
-                        cudaStream_t st, Profiler* prof, bool with_dx);
-void launch_fc1_dw_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st,
-                      Profiler* prof);   // one-time function attributes (dynamic shared memory sizes)
 
 // Part B.
 struct SumApplyArgs {

@@ -242,7 +242,7 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
   x->ckpt_version.assign(x->ckpt_buf.size(), 0);
   double t = std::floor((double)cfg->dropout_p * 4294967296.0);
   x->drop_thresh = t <= 0.0 ? 0u : (t >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)t);
-  if (psk::configure_grad_kernels() != 0 || psk::configure_tc_kernels() != 0 || psk::configure_tc5_kernels() != 0 || psk::configure_conv5_kernels() != 0 || psk::configure_conv1_kernels() != 0 || psk::configure_dw5_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
+  if (psk::configure_grad_kernels() != 0 || psk::configure_tc5_kernels() != 0 || psk::configure_conv5_kernels() != 0 || psk::configure_conv1_kernels() != 0 || psk::configure_dw5_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
   if (cfg->precision != PS_FP32) {
     // two side streams let independent branches of the backward pass overlap (they allocate no device memory)
     bool ok = cudaStreamCreateWithFlags(&x->side.s1, cudaStreamNonBlocking) == cudaSuccess &&
