@@ -28,7 +28,8 @@ namespace psk {
 
 namespace {
 
-constexpr int W5_LOAD_WARPS = 16;                       // two groups of eight: group g stages samples n = g, g + 2, ...
+constexpr int W5_LOAD_WARPS = 16;                       // two groups: group g stages samples n = g, g + 2, ...
+constexpr int W5_GW = W5_LOAD_WARPS / 2;                // warps per group
 constexpr int W5_THREADS = 32 * (1 + W5_LOAD_WARPS + 4);   // warp 0: MMA issue and tensor memory; the last four warps write out
 constexpr int W5_CHUNKS = 32;                           // 8-position chunks of the 256 contraction indices of a sample
 constexpr int W5_GROUP_BYTES = W5_CHUNKS * 128;         // one group of 8 operand rows: 32 core matrices of 128 bytes
@@ -132,8 +133,8 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       }
     }
   } else if (warp <= W5_LOAD_WARPS) {
-    // ---------------- staging: group g (eight warps) builds the operands of samples n = g, g + 2, ... in stage g
-    const int grp = (warp - 1) >> 3, gw = (warp - 1) & 7, gt_ = gw * 32 + lane;      // thread index inside the group
+    // ---------------- staging: group g (W5_GW warps) builds the operands of samples n = g, g + 2, ... in stage g
+    const int grp = (warp - 1) / W5_GW, gw = (warp - 1) - grp * W5_GW, gt_ = gw * 32 + lane;      // thread index inside the group
     auto issue = [&](int n) {            // one thread: the three input rows of sample r0 + n
       const int64_t row = r0 + n;
       uint8_t* dst = raw + (n & 3) * W5_RAW_SLOT;
@@ -158,7 +159,7 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       // block l / 8: on the way in the input plane's row of position 8 chunk + row + kx (plane rows keep even and
       // odd columns apart; positions past the end read the all-zero row 0), on the way out the core matrix's row.
 #pragma unroll
-      for (int o = gw; o < 48; o += 8) {
+      for (int o = gw; o < 48; o += W5_GW) {
         const int g = o >> 3, kx = g >> 1, oct = g & 1, chunk = 4 * (o & 7) + (lane >> 3);
         const int i = 8 * chunk + (lane & 7) + kx;
         const int prow = i < 256 ? (i & ~15) + ((i & 1) << 3) + ((i & 15) >> 1) : 0;
@@ -173,8 +174,8 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       // three are cleared.  The pair of columns (2px, 2px + 1) is one word of a core-matrix row; the three ky copies
       // lie one image row (two chunks) apart, image rows 2py and 2py + 1 likewise.
 #pragma unroll
-      for (int k = 0; k < 7; ++k) {
-        const int wi = gw * 7 + k, oct = wi / 14, rem = wi - oct * 14, py = rem >> 1, pxhi = rem & 1;
+      for (int wi = gw; wi < 56; wi += W5_GW) {
+        const int oct = wi / 14, rem = wi - oct * 14, py = rem >> 1, pxhi = rem & 1;
         const int rr = lane >> 2, pl = lane & 3, px = 4 * pxhi + pl;
         if (px < 7) {
           const int oc = 8 * oct + rr, e = ((oc >> 2) * 49 + py * 7 + px) * 4 + (oc & 3);
