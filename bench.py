@@ -252,12 +252,18 @@ def main():
     hy = [torch.from_numpy(py[synth.batch_rows(t, W, b, px.shape[0])]).pin_memory() for t in range(2)]
     loss_host = torch.empty(W, dtype=torch.float32).pin_memory()
     e2e_steps = max(3, min(args.steps, 50))
+    # Two ticks are kept in flight (ps_tick_host_submit / ps_tick_host_wait): the copy of the next tick's inputs runs
+    # while the current tick computes.  Every timed step still copies its own inputs in and its losses out.
+    loss_bufs = [loss_host, torch.empty(W, dtype=torch.float32).pin_memory()]
     for t in range(3):
         srv.ps_tick_host(hx[t % 2], hy[t % 2], DROP_SEED, 10_000 + t, ps.REPLAY, LR, loss_host=loss_host)
     barrier()
     t0 = time.perf_counter()
-    for t in range(e2e_steps):
-        srv.ps_tick_host(hx[t % 2], hy[t % 2], DROP_SEED, 20_000 + t, ps.REPLAY, LR, loss_host=loss_host)
+    srv.ps_tick_host_submit(hx[0], hy[0], DROP_SEED, 20_000, ps.REPLAY, LR, loss_host=loss_bufs[0])
+    for t in range(1, e2e_steps):
+        srv.ps_tick_host_submit(hx[t % 2], hy[t % 2], DROP_SEED, 20_000 + t, ps.REPLAY, LR, loss_host=loss_bufs[t % 2])
+        srv.ps_tick_host_wait()
+    srv.ps_tick_host_wait()
     barrier()
     e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3)
     h2d = W * b * 784 * 4 + W * b * 4

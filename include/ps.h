@@ -233,6 +233,21 @@ int32_t ps_tick_host(ps_ctx* ctx, int32_t W, int32_t b, const int32_t* lags, con
                      float lr, float scale, const int32_t* order, float* loss_host,
                      int32_t* argmax_host, ps_apply_result* out);
 
+/* The same tick without waiting for it: ps_tick_host_submit enqueues the copies and all the work of a tick and
+ * returns; ps_tick_host_wait blocks until the oldest submitted tick has finished (its losses and labels are then in
+ * the host buffers given at submit) and returns its apply result.  Up to two ticks may be in flight, so the
+ * host-to-device copy of the next tick's inputs (on a copy stream of the library's own) runs while the current
+ * tick computes; on the device the ticks still run one after the other: snapshots, versions and the queue are
+ * exactly those of back-to-back ps_tick_host calls (the paper's workers likewise fetch their next batch while the
+ * server works).  x_host, y_host, loss_host and argmax_host must stay valid and untouched until the matching wait.
+ * Errors: PS_ERR_BAD_ARG when two ticks are already in flight (submit) or none is (wait); otherwise as ps_tick_host.
+ * Other calls on the context are allowed between submit and wait only if they do not depend on that tick. */
+int32_t ps_tick_host_submit(ps_ctx* ctx, int32_t W, int32_t b, const int32_t* lags, const float* x_host,
+                            const int32_t* y_host, uint64_t seed, uint64_t step, int32_t apply_mode,
+                            float lr, float scale, const int32_t* order, float* loss_host,
+                            int32_t* argmax_host);
+int32_t ps_tick_host_wait(ps_ctx* ctx, ps_apply_result* out);
+
 /* Per-kernel timing for measurement (no counterpart in the paper's method; it serves the roofline
  * report).  ps_profile(ctx, 1) clears the totals and from then on brackets every kernel launch with
  * two CUDA events on the context's stream (and runs the branches of the backward pass one after the

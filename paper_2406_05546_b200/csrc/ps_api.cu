@@ -57,7 +57,7 @@ struct ps_ctx {
   float* partial;
   float* queue;
   psk::Workspace ws;
-  float* x_stage; int32_t* y_stage; float* loss_stage; int32_t* argmax_stage;
+  float* x_stage[2]; int32_t* y_stage[2]; float* loss_stage[2]; int32_t* argmax_stage[2];   // two sets: two ticks may be in flight
   uint32_t* status_dev;
   // pinned
   std::vector<float*> ckpt_buf;
@@ -80,7 +80,10 @@ struct ps_ctx {
   int prep_n = 0;
   // ps_tick_host copies its inputs in on a stream of its own, chunk by chunk, while earlier chunks compute
   cudaStream_t copy_st = nullptr;
-  cudaEvent_t copy_ev[8] = {nullptr};
+  cudaEvent_t copy_ev[8] = {nullptr};          // [set][chunk]
+  cudaEvent_t stage_free[2] = {nullptr, nullptr}, tick_done[2] = {nullptr, nullptr};
+  struct { bool used = false; ps_apply_result res = {0, 0, 0, 0}; } inflight[2];
+  uint64_t ticks_submitted = 0, ticks_waited = 0;
   double prof_ms[psk::K_COUNT] = {0};
   int64_t prof_n[psk::K_COUNT] = {0};
 };
@@ -154,17 +157,20 @@ void layout(ps_ctx* x, const ps_config& c, void* arena, void* pinned, uint64_t* 
     ws.w1r = a.take<float>(groups * psk::HID * psk::FLAT * 4);
     ws.w1tr = a.take<float>(groups * psk::HID * psk::FLAT * 4);
   }
-  float* x_stage = a.take<float>(rows * PS_IMAGE_PIXELS * 4);
-  int32_t* y_stage = a.take<int32_t>(rows * 4);
-  float* loss_stage = a.take<float>((uint64_t)c.max_workers * 4);
-  int32_t* argmax_stage = a.take<int32_t>(rows * 4);
+  float* x_stage[2]; int32_t* y_stage[2]; float* loss_stage[2]; int32_t* argmax_stage[2];
+  for (int k = 0; k < 2; ++k) {
+    x_stage[k] = a.take<float>(rows * PS_IMAGE_PIXELS * 4);
+    y_stage[k] = a.take<int32_t>(rows * 4);
+    loss_stage[k] = a.take<float>((uint64_t)c.max_workers * 4);
+    argmax_stage[k] = a.take<int32_t>(rows * 4);
+  }
   Carver h(pinned);
   for (int i = 0; i < c.ckpt_slots; ++i) { float* p = h.take<float>(VEC_BYTES); if (x) x->ckpt_buf.push_back(p); }
   float* io_stage = h.take<float>(VEC_BYTES);
   uint32_t* status_host = h.take<uint32_t>(ALIGN);
   if (x) {
     x->partial = partial; x->queue = queue; x->ws = ws; x->status_dev = ws.status;
-    x->x_stage = x_stage; x->y_stage = y_stage; x->loss_stage = loss_stage; x->argmax_stage = argmax_stage;
+    for (int k = 0; k < 2; ++k) { x->x_stage[k] = x_stage[k]; x->y_stage[k] = y_stage[k]; x->loss_stage[k] = loss_stage[k]; x->argmax_stage[k] = argmax_stage[k]; }
     x->io_stage = io_stage; x->status_host = status_host;
   }
   if (arena_bytes) *arena_bytes = align_up(a.off);
@@ -254,6 +260,8 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
   {
     bool ok = cudaStreamCreateWithFlags(&x->copy_st, cudaStreamNonBlocking) == cudaSuccess;
     for (auto& ev : x->copy_ev) ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
+    for (auto& ev : x->stage_free) ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
+    for (auto& ev : x->tick_done) ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { delete x; return fail(PS_ERR_CUDA, "copy stream set-up failed: %s", cudaGetErrorString(cudaGetLastError())); }
   }
   std::memcpy(x->io_stage, init_params_host, sizeof(float) * PS_PARAM_COUNT);
@@ -279,6 +287,8 @@ int32_t ps_destroy(ps_ctx* x) {
   for (cudaEvent_t ev : {x->side.fork1, x->side.join1, x->side.fork2, x->side.join2}) if (ev) cudaEventDestroy(ev);
   if (x->copy_st) { cudaStreamSynchronize(x->copy_st); cudaStreamDestroy(x->copy_st); }
   for (cudaEvent_t ev : x->copy_ev) if (ev) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : x->stage_free) if (ev) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : x->tick_done) if (ev) cudaEventDestroy(ev);
   delete x;
   if (e != cudaSuccess) return cuda_fail(e, "ps_destroy");
   return PS_OK;
@@ -651,11 +661,13 @@ int32_t ps_profile_read(ps_ctx* x, int32_t kernel, const char** name, double* to
   return PS_OK;
 }
 
-int32_t ps_tick_host(ps_ctx* x, int32_t W, int32_t b, const int32_t* lags, const float* x_host, const int32_t* y_host,
-                     uint64_t seed, uint64_t step, int32_t apply_mode, float lr, float scale, const int32_t* order,
-                     float* loss_host, int32_t* argmax_host, ps_apply_result* out) {
+int32_t ps_tick_host_submit(ps_ctx* x, int32_t W, int32_t b, const int32_t* lags, const float* x_host, const int32_t* y_host,
+                            uint64_t seed, uint64_t step, int32_t apply_mode, float lr, float scale, const int32_t* order,
+                            float* loss_host, int32_t* argmax_host) {
   if (!x || !x_host || !y_host || !loss_host) return fail(PS_ERR_BAD_ARG, "NULL argument");
   if (W < 1 || W > x->cfg.max_workers || b < 1 || b > x->cfg.max_batch) return fail(PS_ERR_BAD_ARG, "W or b out of range");
+  const int set = (int)(x->ticks_submitted & 1);
+  if (x->inflight[set].used) return fail(PS_ERR_BAD_ARG, "two ticks are already in flight: call ps_tick_host_wait first");
   ps_snapshot snaps[PS_MAX_WORKERS];
   int32_t ids[PS_MAX_WORKERS];
   int64_t slots[PS_MAX_WORKERS];
@@ -669,27 +681,32 @@ int32_t ps_tick_host(ps_ctx* x, int32_t W, int32_t b, const int32_t* lags, const
   int32_t rc = ps_queue_reserve(x, W, slots);
   if (rc != PS_OK) return rc;
   const size_t rows = (size_t)W * b;
+  float* xs = x->x_stage[set];
+  int32_t* ys = x->y_stage[set];
   // The inputs go in on the copy stream in up to four chunks of workers; the grad step of a chunk starts as soon as
-  // its chunk has landed, so most of the host-to-device copy hides behind the computation of earlier chunks.
-  // (The staging buffers are free: the previous call synchronised the context's stream before it returned.)
+  // its chunk has landed, so most of the host-to-device copy hides behind the computation of earlier chunks, and the
+  // copies of this tick behind the previous tick's work.  This staging set was last read by the tick before the
+  // previous one; the copy stream waits for that tick's grad step.
+  if (x->ticks_submitted >= 2) CUDA_TRY(cudaStreamWaitEvent(x->copy_st, x->stage_free[set], 0));
   const int n_chunks = W >= 8 ? 4 : 1, per = (W + n_chunks - 1) / n_chunks;
   for (int c = 0; c < n_chunks; ++c) {
     const int w0 = c * per, w1 = std::min(W, w0 + per);
     if (w0 >= w1) break;
     const size_t r0 = (size_t)w0 * b, nr = (size_t)(w1 - w0) * b;
-    CUDA_TRY(cudaMemcpyAsync(x->x_stage + r0 * PS_IMAGE_PIXELS, x_host + r0 * PS_IMAGE_PIXELS, nr * PS_IMAGE_PIXELS * sizeof(float), cudaMemcpyHostToDevice, x->copy_st));
-    CUDA_TRY(cudaMemcpyAsync(x->y_stage + r0, y_host + r0, nr * sizeof(int32_t), cudaMemcpyHostToDevice, x->copy_st));
-    CUDA_TRY(cudaEventRecord(x->copy_ev[c], x->copy_st));
+    CUDA_TRY(cudaMemcpyAsync(xs + r0 * PS_IMAGE_PIXELS, x_host + r0 * PS_IMAGE_PIXELS, nr * PS_IMAGE_PIXELS * sizeof(float), cudaMemcpyHostToDevice, x->copy_st));
+    CUDA_TRY(cudaMemcpyAsync(ys + r0, y_host + r0, nr * sizeof(int32_t), cudaMemcpyHostToDevice, x->copy_st));
+    CUDA_TRY(cudaEventRecord(x->copy_ev[4 * set + c], x->copy_st));
   }
   for (int c = 0; c < n_chunks; ++c) {
     const int w0 = c * per, w1 = std::min(W, w0 + per);
     if (w0 >= w1) break;
     const size_t r0 = (size_t)w0 * b;
-    CUDA_TRY(cudaStreamWaitEvent(x->st, x->copy_ev[c], 0));
-    rc = workers_grad_step(x, w1 - w0, b, snaps + w0, ids + w0, x->x_stage + r0 * PS_IMAGE_PIXELS, x->y_stage + r0, seed, step,
-                           slots + w0, nullptr, x->loss_stage + w0, x->argmax_stage + r0);
+    CUDA_TRY(cudaStreamWaitEvent(x->st, x->copy_ev[4 * set + c], 0));
+    rc = workers_grad_step(x, w1 - w0, b, snaps + w0, ids + w0, xs + r0 * PS_IMAGE_PIXELS, ys + r0, seed, step,
+                           slots + w0, nullptr, x->loss_stage[set] + w0, x->argmax_stage[set] + r0);
     if (rc != PS_OK) { cudaStreamSynchronize(x->copy_st); return rc; }
   }
+  CUDA_TRY(cudaEventRecord(x->stage_free[set], x->st));
   rc = ps_enqueue(x, W, slots, nullptr, ids, bases, step);
   if (rc != PS_OK) return rc;
   ps_apply_result res = {0, x->version, 0, 0};
@@ -697,11 +714,33 @@ int32_t ps_tick_host(ps_ctx* x, int32_t W, int32_t b, const int32_t* lags, const
     rc = ps_apply(x, (ps_mode)apply_mode, lr, scale, order, &res);
     if (rc != PS_OK) return rc;
   }
-  CUDA_TRY(cudaMemcpyAsync(loss_host, x->loss_stage, (size_t)W * sizeof(float), cudaMemcpyDeviceToHost, x->st));
-  if (argmax_host) CUDA_TRY(cudaMemcpyAsync(argmax_host, x->argmax_stage, rows * sizeof(int32_t), cudaMemcpyDeviceToHost, x->st));
-  CUDA_TRY(cudaStreamSynchronize(x->st));
-  if (out) *out = res;
+  CUDA_TRY(cudaMemcpyAsync(loss_host, x->loss_stage[set], (size_t)W * sizeof(float), cudaMemcpyDeviceToHost, x->st));
+  if (argmax_host) CUDA_TRY(cudaMemcpyAsync(argmax_host, x->argmax_stage[set], rows * sizeof(int32_t), cudaMemcpyDeviceToHost, x->st));
+  CUDA_TRY(cudaEventRecord(x->tick_done[set], x->st));
+  x->inflight[set].used = true;
+  x->inflight[set].res = res;
+  x->ticks_submitted++;
   return PS_OK;
+}
+
+int32_t ps_tick_host_wait(ps_ctx* x, ps_apply_result* out) {
+  if (!x) return fail(PS_ERR_BAD_ARG, "ctx is NULL");
+  const int set = (int)(x->ticks_waited & 1);
+  if (x->ticks_waited == x->ticks_submitted || !x->inflight[set].used) return fail(PS_ERR_BAD_ARG, "no tick is in flight");
+  CUDA_TRY(cudaEventSynchronize(x->tick_done[set]));
+  if (out) *out = x->inflight[set].res;
+  x->inflight[set].used = false;
+  x->ticks_waited++;
+  return PS_OK;
+}
+
+int32_t ps_tick_host(ps_ctx* x, int32_t W, int32_t b, const int32_t* lags, const float* x_host, const int32_t* y_host,
+                     uint64_t seed, uint64_t step, int32_t apply_mode, float lr, float scale, const int32_t* order,
+                     float* loss_host, int32_t* argmax_host, ps_apply_result* out) {
+  if (x && x->ticks_waited != x->ticks_submitted) return fail(PS_ERR_BAD_ARG, "a submitted tick is still in flight: call ps_tick_host_wait first");
+  int32_t rc = ps_tick_host_submit(x, W, b, lags, x_host, y_host, seed, step, apply_mode, lr, scale, order, loss_host, argmax_host);
+  if (rc != PS_OK) return rc;
+  return ps_tick_host_wait(x, out);
 }
 
 }  // extern "C"

@@ -23,6 +23,7 @@ ERRORS = {-1: "PS_ERR_BAD_ARG", -2: "PS_ERR_DOWN", -3: "PS_ERR_QUEUE_FULL", -4: 
 EXPORTS = ["ps_query_bytes", "ps_create", "ps_destroy", "ps_pull_snapshot", "ps_queue_reserve", "ps_slot_ptr",
            "workers_grad_step", "ps_dropout_mask", "ps_enqueue", "ps_apply", "ps_checkpoint", "ps_restore", "ps_replicate",
            "ps_kill", "ps_failover", "ps_import_params", "ps_export_params", "ps_stats", "ps_tick_host",
+           "ps_tick_host_submit", "ps_tick_host_wait",
            "ps_profile", "ps_profile_read", "ps_last_error", "ps_replay_sum_static", "ps_replay_sum_static_error"]
 
 
@@ -88,6 +89,8 @@ def load(path=None):
         "ps_export_params": [vp, i32, vp, C.POINTER(u64)],
         "ps_stats": [vp, C.POINTER(Stats)],
         "ps_tick_host": [vp, i32, i32, vp, vp, vp, u64, u64, i32, f32, f32, vp, vp, vp, C.POINTER(ApplyResult)],
+        "ps_tick_host_submit": [vp, i32, i32, vp, vp, vp, u64, u64, i32, f32, f32, vp, vp, vp],
+        "ps_tick_host_wait": [vp, C.POINTER(ApplyResult)],
     }
     sig["ps_profile"] = [vp, i32]
     sig["ps_profile_read"] = [vp, i32, C.POINTER(C.c_char_p), C.POINTER(C.c_double), C.POINTER(i64)]
@@ -292,6 +295,29 @@ class ParameterServer:
                                           ptr(argmax_host) if argmax_host is not None else None, C.byref(res)))
         return loss_host, {"applied": res.applied, "new_version": res.new_version,
                            "checkpointed": res.checkpointed, "replicated": res.replicated}
+
+    def ps_tick_host_submit(self, x_host, y_host, seed, step, apply_mode, lr, scale=1.0, lags=None, order=None,
+                            loss_host=None, argmax_host=None):
+        """Enqueues a whole tick and returns at once; the buffers must stay alive until ps_tick_host_wait."""
+        W, b = int(y_host.shape[0]), int(y_host.shape[1])
+        ptr = lambda t: t.data_ptr() if hasattr(t, "data_ptr") else t.ctypes.data
+        if loss_host is None:
+            loss_host = np.zeros(W, dtype=np.float32)
+        lg = None if lags is None else np.ascontiguousarray(lags, dtype=np.int32)
+        o = None if order is None else np.ascontiguousarray(order, dtype=np.int32)
+        self._check(self.lib.ps_tick_host_submit(self.ctx, W, b, _np_ptr(lg), ptr(x_host), ptr(y_host), int(seed), int(step),
+                                                 int(apply_mode), float(lr), float(scale), _np_ptr(o), ptr(loss_host),
+                                                 ptr(argmax_host) if argmax_host is not None else None))
+        self._inflight = getattr(self, "_inflight", []) + [(x_host, y_host, loss_host, argmax_host, lg, o)]
+        return loss_host
+
+    def ps_tick_host_wait(self):
+        res = ApplyResult()
+        self._check(self.lib.ps_tick_host_wait(self.ctx, C.byref(res)))
+        if getattr(self, "_inflight", None):
+            self._inflight.pop(0)
+        return {"applied": res.applied, "new_version": res.new_version,
+                "checkpointed": res.checkpointed, "replicated": res.replicated}
 
     def ps_profile(self, enable):
         self._check(self.lib.ps_profile(self.ctx, int(bool(enable))))

@@ -216,3 +216,42 @@ def test_tick_from_host_buffers_matches_the_oracle(precision, W, b):
     # the tick moves the head by lr * mean gradient: compare that step too, which the parameters' size would hide
     before = o.ring[1].astype(np.float64)
     assert_params_close(theta - before, o.head() - before, max(tol, 10 * TOL_FP32), "the tick's update")
+
+
+@pytest.mark.parametrize("precision", [0, 2])
+def test_pipelined_ticks_equal_sequential_ticks(precision):
+    """Two ticks in flight (ps_tick_host_submit / ps_tick_host_wait) leave the same weights, losses, labels and
+    versions, bit for bit, as the same ticks run one by one through ps_tick_host."""
+    import torch
+    from paper_2406_05546_b200 import ps
+    W, b, T = 9, 6, 5
+    theta0 = synth.init_params(seed=1, bias_scale=0.05)
+    rng = np.random.default_rng(3)
+    xs = [torch.from_numpy(rng.random((W, b, 28, 28), dtype=np.float32)).pin_memory() for _ in range(T)]
+    ys = [torch.from_numpy(rng.integers(0, 10, (W, b)).astype(np.int32)).pin_memory() for _ in range(T)]
+    out = []
+    for pipelined in (False, True):
+        srv = ps.ParameterServer(theta0, max_workers=W, max_batch=b, ring_depth=2, queue_slots=W, precision=precision)
+        loss = [np.zeros(W, dtype=np.float32) for _ in range(T)]
+        am = [np.zeros((W, b), dtype=np.int32) for _ in range(T)]
+        results = []
+        if pipelined:
+            srv.ps_tick_host_submit(xs[0], ys[0], SEED, 0, ps.SYNC, 0.01, loss_host=loss[0], argmax_host=am[0])
+            for t in range(1, T):
+                srv.ps_tick_host_submit(xs[t], ys[t], SEED, t, ps.SYNC, 0.01, loss_host=loss[t], argmax_host=am[t])
+                results.append(srv.ps_tick_host_wait())
+            with pytest.raises(ps.PSError):          # the synchronous form refuses to run while a tick is in flight
+                srv.ps_tick_host(xs[0], ys[0], SEED, 99, ps.SYNC, 0.01)
+            results.append(srv.ps_tick_host_wait())
+            with pytest.raises(ps.PSError):
+                srv.ps_tick_host_wait()
+        else:
+            for t in range(T):
+                results.append(srv.ps_tick_host(xs[t], ys[t], SEED, t, ps.SYNC, 0.01, loss_host=loss[t], argmax_host=am[t])[1])
+        theta, version = srv.ps_export_params()
+        srv.ps_stats()
+        srv.close()
+        out.append((theta, version, np.stack(loss), np.stack(am), [r["new_version"] for r in results]))
+    a, p = out
+    assert a[1] == p[1] == T and a[4] == p[4] == list(range(1, T + 1))
+    assert (a[0] == p[0]).all() and (a[2] == p[2]).all() and (a[3] == p[3]).all()
