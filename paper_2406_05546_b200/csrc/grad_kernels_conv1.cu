@@ -19,22 +19,6 @@ namespace psk {
 
 namespace {
 
-typedef unsigned long long u64;
-__device__ __forceinline__ u64 pack2(float lo, float hi) {
-  u64 r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-// Two independent single-rounded fp32 multiply-adds in one instruction.
-__device__ __forceinline__ u64 ffma2(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-
 constexpr int C1_THREADS = 224;
 constexpr int C1_SPB = 8;                                // samples per block, taken two at a time
 constexpr int C1_BOX_W = 36, C1_BOX_H = 30;              // image box: columns -4..31 (a 16-byte aligned start), rows -1..28

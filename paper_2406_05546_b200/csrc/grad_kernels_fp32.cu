@@ -250,8 +250,11 @@ __device__ __forceinline__ float warp_sum(float v) {
 // warp at a time; then thread = hidden unit sums its outputs over the block's samples in sample order, several
 // loads in flight.  The block's sums (and its share of the loss) are partial results added later in block order.
 constexpr int FC2_THREADS = 512;
+constexpr int DZ_CHUNK = 128;      // samples whose logits gradients are held in shared memory at a time
+constexpr int W2T_PITCH = 12;      // 48-byte rows: 16-byte loads of consecutive rows fall on distinct banks
 __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
-  __shared__ float w2[NCLS][HID];
+  __shared__ __align__(16) float w2t[HID][W2T_PITCH];     // w2t[j][c] = W2[c][j]; the two pad columns are zero
+  __shared__ __align__(16) float dzs[DZ_CHUNK][W2T_PITCH];   // logits gradients of a chunk of samples
   __shared__ float b2[NCLS];
   __shared__ float warp_loss[FC2_THREADS / 32];
   const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -259,7 +262,8 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
   const int src = wt.src[s];
   const int per = ((a.b + FC2_SPLIT - 1) / FC2_SPLIT + 1) & ~1;          // samples per block, even
   const int i_lo = min(a.b, (int)blockIdx.y * per), i_hi = min(a.b, i_lo + per);
-  for (int t = tid; t < NCLS * HID; t += FC2_THREADS) (&w2[0][0])[t] = theta[OFF_F2W + t];
+  for (int t = tid; t < NCLS * HID; t += FC2_THREADS) w2t[t % HID][t / HID] = theta[OFF_F2W + t];
+  w2t[tid][NCLS] = w2t[tid][NCLS + 1] = 0.f;
   if (tid < NCLS) b2[tid] = theta[OFF_F2B + tid];
   __syncthreads();
   const float scale = 1.0f / (1.0f - a.drop_p);
@@ -272,25 +276,37 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
     // registers of a 512-thread block, so their address is made to look pass-dependent
     uint32_t opaque_zero;
     asm volatile("mov.u32 %0, 0;" : "=r"(opaque_zero));
-    const float (*w2p)[HID] = reinterpret_cast<const float (*)[HID]>(&w2[0][0] + opaque_zero);
+    const float4* w2p = reinterpret_cast<const float4*>(&w2t[0][0] + opaque_zero);
     const int64_t row0 = (int64_t)s * a.b + i0, row1 = two ? row0 + 1 : row0;
+    // the labels are asked for now: by the time the softmax needs them they have arrived
+    const int lab[2] = {a.y[(int64_t)src * a.b + i0], a.y[(int64_t)src * a.b + (two ? i0 + 1 : i0)]};
     float dv[2][16];
 #pragma unroll
     for (int t = 0; t < 16; ++t) {
       dv[0][t] = ws.d[row0 * HID + lane + 32 * t];
       dv[1][t] = ws.d[row1 * HID + lane + 32 * t];
     }
-    float z[2][NCLS];
+    // classes in pairs, one packed multiply-add per pair: zp[u][k] = logits 2k and 2k + 1 of sample u
+    u64 zp[2][NCLS / 2];
 #pragma unroll
-    for (int c = 0; c < NCLS; ++c) z[0][c] = z[1][c] = 0.f;
+    for (int k = 0; k < NCLS / 2; ++k) zp[0][k] = zp[1][k] = 0ull;
 #pragma unroll
     for (int t = 0; t < 16; ++t) {
+      const float4* wr = w2p + (lane + 32 * t) * (W2T_PITCH / 4);
+      const float4 q0 = wr[0], q1 = wr[1], q2 = wr[2];
+      const u64 wk[NCLS / 2] = {pack2(q0.x, q0.y), pack2(q0.z, q0.w), pack2(q1.x, q1.y), pack2(q1.z, q1.w), pack2(q2.x, q2.y)};
+      const u64 d0 = pack2(dv[0][t], dv[0][t]), d1 = pack2(dv[1][t], dv[1][t]);
 #pragma unroll
-      for (int c = 0; c < NCLS; ++c) {
-        const float wv = w2p[c][lane + 32 * t];
-        z[0][c] = fmaf(wv, dv[0][t], z[0][c]);
-        z[1][c] = fmaf(wv, dv[1][t], z[1][c]);
+      for (int k = 0; k < NCLS / 2; ++k) {
+        zp[0][k] = ffma2(wk[k], d0, zp[0][k]);
+        zp[1][k] = ffma2(wk[k], d1, zp[1][k]);
       }
+    }
+    float z[2][NCLS];
+#pragma unroll
+    for (int k = 0; k < NCLS / 2; ++k) {
+      unpack2(zp[0][k], z[0][2 * k], z[0][2 * k + 1]);
+      unpack2(zp[1][k], z[1][2 * k], z[1][2 * k + 1]);
     }
 #pragma unroll
     for (int c = 0; c < NCLS; ++c) {
@@ -311,7 +327,7 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
 #pragma unroll
       for (int c = 0; c < NCLS; ++c) { ez[c] = expf(z[u][c] - zmax); se += ez[c]; }
       const float lse = zmax + logf(se), inv_se = 1.0f / se;
-      int label = a.y[(int64_t)src * a.b + i];
+      int label = lab[u];
       if (label < 0 || label >= NCLS) {
         if (lane == 0) atomicOr(ws.status, STATUS_BAD_LABEL);
         label = 0;
@@ -337,23 +353,36 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
       for (int c = 0; c < NCLS; ++c) dz[1][c] = 0.f;
     }
     asm volatile("mov.u32 %0, 0;" : "=r"(opaque_zero));    // second read of the weights, as above
-    w2p = reinterpret_cast<const float (*)[HID]>(&w2[0][0] + opaque_zero);
+    w2p = reinterpret_cast<const float4*>(&w2t[0][0] + opaque_zero);
     uint32_t live0 = 0u, live1 = 0u;                         // which of the lane's 16 units passed ReLU and dropout
 #pragma unroll
     for (int t = 0; t < 16; ++t) {
       live0 |= (dv[0][t] > 0.f ? 1u : 0u) << t;
       live1 |= (dv[1][t] > 0.f ? 1u : 0u) << t;
     }
+    u64 dzk[2][NCLS / 2];
+#pragma unroll
+    for (int k = 0; k < NCLS / 2; ++k) {
+      dzk[0][k] = pack2(dz[0][2 * k], dz[0][2 * k + 1]);
+      dzk[1][k] = pack2(dz[1][2 * k], dz[1][2 * k + 1]);
+    }
 #pragma unroll 2
     for (int t = 0; t < 16; ++t) {
       const int j = lane + 32 * t;
-      float dd0 = 0.f, dd1 = 0.f;
+      const float4* wr = w2p + j * (W2T_PITCH / 4);
+      const float4 q0 = wr[0], q1 = wr[1], q2 = wr[2];
+      const u64 wk[NCLS / 2] = {pack2(q0.x, q0.y), pack2(q0.z, q0.w), pack2(q1.x, q1.y), pack2(q1.z, q1.w), pack2(q2.x, q2.y)};
+      // even classes accumulate in the low half, odd classes in the high half; the halves are added at the end
+      u64 e0 = 0ull, e1 = 0ull;
 #pragma unroll
-      for (int c = 0; c < NCLS; ++c) {
-        const float wv = w2p[c][j];
-        dd0 = fmaf(wv, dz[0][c], dd0);
-        dd1 = fmaf(wv, dz[1][c], dd1);
+      for (int k = 0; k < NCLS / 2; ++k) {
+        e0 = ffma2(wk[k], dzk[0][k], e0);
+        e1 = ffma2(wk[k], dzk[1][k], e1);
       }
+      float lo0, hi0, lo1, hi1;
+      unpack2(e0, lo0, hi0);
+      unpack2(e1, lo1, hi1);
+      const float dd0 = lo0 + hi0, dd1 = lo1 + hi1;
       float v0 = (live0 >> t) & 1u ? dd0 * scale : 0.f, v1 = (live1 >> t) & 1u ? dd1 * scale : 0.f;
       if (a.precision != 0) { v0 = round_tf32(v0); v1 = round_tf32(v1); }   // they feed tensor-core products only
       ws.da1[row0 * HID + j] = v0;
@@ -375,18 +404,35 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
   const float* dzp = ws.dz + (int64_t)s * a.b * DZ_STRIDE;
   const float* dp = ws.d + (int64_t)s * a.b * HID + j;
   const float* da1p = ws.da1 + (int64_t)s * a.b * HID + j;
-#pragma unroll 4
-  for (int i = i_lo; i < i_hi; ++i) {
-    const float dval = dp[(int64_t)i * HID];
-    const float4 z0 = *reinterpret_cast<const float4*>(dzp + i * DZ_STRIDE);
-    const float4 z1 = *reinterpret_cast<const float4*>(dzp + i * DZ_STRIDE + 4);
-    const float2 z2 = *reinterpret_cast<const float2*>(dzp + i * DZ_STRIDE + 8);
-    const float dzv[NCLS] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w, z2.x, z2.y};
+  u64 gwk[NCLS / 2];
 #pragma unroll
-    for (int c = 0; c < NCLS; ++c) gw[c] = fmaf(dzv[c], dval, gw[c]);
-    gb1 += da1p[(int64_t)i * HID];
-    if (j < NCLS) gb2 += dzp[i * DZ_STRIDE + j];
+  for (int k = 0; k < NCLS / 2; ++k) gwk[k] = 0ull;
+  // The logits gradients of DZ_CHUNK samples at a time are brought into shared memory, where every thread reads
+  // them as broadcasts; what is left per sample is two loads from global memory, many of them in flight.
+  for (int c0 = i_lo; c0 < i_hi; c0 += DZ_CHUNK) {
+    const int n = min(DZ_CHUNK, i_hi - c0);
+    __syncthreads();
+    for (int t = tid; t < n * (W2T_PITCH / 4); t += FC2_THREADS) {
+      const int i = t / (W2T_PITCH / 4), q = t - i * (W2T_PITCH / 4);
+      reinterpret_cast<float4*>(&dzs[i][0])[q] = *reinterpret_cast<const float4*>(dzp + (c0 + i) * DZ_STRIDE + 4 * q);
+    }
+    __syncthreads();
+#pragma unroll 16
+    for (int i = 0; i < n; ++i) {
+      const float dval = dp[(int64_t)(c0 + i) * HID];
+      const float4* zr = reinterpret_cast<const float4*>(&dzs[i][0]);
+      const float4 z0 = zr[0], z1 = zr[1], z2 = zr[2];
+      const u64 dzk[NCLS / 2] = {pack2(z0.x, z0.y), pack2(z0.z, z0.w), pack2(z1.x, z1.y), pack2(z1.z, z1.w), pack2(z2.x, z2.y)};
+      const u64 dd = pack2(dval, dval);
+#pragma unroll
+      for (int k = 0; k < NCLS / 2; ++k) gwk[k] = ffma2(dzk[k], dd, gwk[k]);
+      gb1 += da1p[(int64_t)(c0 + i) * HID];
+    }
+    if (j < NCLS)
+      for (int i = 0; i < n; ++i) gb2 += dzs[i][j];
   }
+#pragma unroll
+  for (int k = 0; k < NCLS / 2; ++k) unpack2(gwk[k], gw[2 * k], gw[2 * k + 1]);
 #pragma unroll
   for (int c = 0; c < NCLS; ++c) part[c * HID + j] = gw[c];
   part[NCLS * HID + j] = gb1;
