@@ -238,18 +238,13 @@ __global__ void __launch_bounds__(256) fc1_fwd(GradStepArgs a, WorkerTable wt, G
   }
 }
 
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
 // ---- fc2 forward, softmax cross-entropy, argmax, and the backward pass down to the gradient with
 // respect to fc1's pre-activation; then the worker's fc2 weight/bias and fc1 bias gradients.
-// FC2_SPLIT blocks of 16 warps per worker, each with its share of the worker's samples: first two samples per
-// warp at a time; then thread = hidden unit sums its outputs over the block's samples in sample order, several
+// FC2_SPLIT blocks of 16 warps per worker, each with its share of the worker's samples: first four samples per
+// warp at a time; then thread = hidden unit sums its outputs over the block's samples in sample order, many
 // loads in flight.  The block's sums (and its share of the loss) are partial results added later in block order.
 constexpr int FC2_THREADS = 512;
+constexpr int FC2_NS = 4;          // samples per warp and pass
 constexpr int DZ_CHUNK = 128;      // samples whose logits gradients are held in shared memory at a time
 constexpr int W2T_PITCH = 12;      // 48-byte rows: 16-byte loads of consecutive rows fall on distinct banks
 __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, WorkerTable wt, GroupTable gt, Workspace ws) {
@@ -269,125 +264,150 @@ __global__ void __launch_bounds__(FC2_THREADS, 1) fc2_fwd_bwd(GradStepArgs a, Wo
   const float scale = 1.0f / (1.0f - a.drop_p);
   const float inv_b = 1.0f / (float)a.b;
   float loss_acc = 0.f;
-  // two samples per warp and pass, so that every weight read from shared memory is used twice
-  for (int i0 = i_lo + 2 * warp; i0 < i_hi; i0 += 2 * (FC2_THREADS / 32)) {
-    const bool two = i0 + 1 < i_hi;                      // warp-uniform
+  // Four samples per warp and pass, so that every weight read from shared memory is used four times.  A lane owns
+  // the 16 hidden units lane + 32 t.
+  const bool hi16 = lane & 16, hi8 = lane & 8, hi4 = lane & 4;
+  const int my_u = lane >> 3, sub = lane & 7;          // after the reduction a lane works for sample my_u of the pass
+  for (int i0 = i_lo + FC2_NS * warp; i0 < i_hi; i0 += FC2_NS * (FC2_THREADS / 32)) {
+    const int n_s = min(FC2_NS, i_hi - i0);              // warp-uniform
+    const bool mine = my_u < n_s;
     // the weights are re-read from shared memory on every pass: 160 of them per lane would not fit in the
     // registers of a 512-thread block, so their address is made to look pass-dependent
     uint32_t opaque_zero;
     asm volatile("mov.u32 %0, 0;" : "=r"(opaque_zero));
     const float4* w2p = reinterpret_cast<const float4*>(&w2t[0][0] + opaque_zero);
-    const int64_t row0 = (int64_t)s * a.b + i0, row1 = two ? row0 + 1 : row0;
-    // the labels are asked for now: by the time the softmax needs them they have arrived
-    const int lab[2] = {a.y[(int64_t)src * a.b + i0], a.y[(int64_t)src * a.b + (two ? i0 + 1 : i0)]};
-    float dv[2][16];
-#pragma unroll
-    for (int t = 0; t < 16; ++t) {
-      dv[0][t] = ws.d[row0 * HID + lane + 32 * t];
-      dv[1][t] = ws.d[row1 * HID + lane + 32 * t];
-    }
+    const int64_t row0 = (int64_t)s * a.b + i0;
+    // the label is asked for now: by the time the softmax needs it, it has arrived
+    int label = a.y[(int64_t)src * a.b + i0 + (mine ? my_u : 0)];
     // classes in pairs, one packed multiply-add per pair: zp[u][k] = logits 2k and 2k + 1 of sample u
-    u64 zp[2][NCLS / 2];
+    u64 zp[FC2_NS][NCLS / 2];
+    uint32_t live[FC2_NS];                               // which of the lane's 16 units passed ReLU and dropout
 #pragma unroll
-    for (int k = 0; k < NCLS / 2; ++k) zp[0][k] = zp[1][k] = 0ull;
+    for (int u = 0; u < FC2_NS; ++u) {
+      live[u] = 0u;
 #pragma unroll
-    for (int t = 0; t < 16; ++t) {
-      const float4* wr = w2p + (lane + 32 * t) * (W2T_PITCH / 4);
-      const float4 q0 = wr[0], q1 = wr[1], q2 = wr[2];
-      const u64 wk[NCLS / 2] = {pack2(q0.x, q0.y), pack2(q0.z, q0.w), pack2(q1.x, q1.y), pack2(q1.z, q1.w), pack2(q2.x, q2.y)};
-      const u64 d0 = pack2(dv[0][t], dv[0][t]), d1 = pack2(dv[1][t], dv[1][t]);
+      for (int k = 0; k < NCLS / 2; ++k) zp[u][k] = 0ull;
+    }
 #pragma unroll
-      for (int k = 0; k < NCLS / 2; ++k) {
-        zp[0][k] = ffma2(wk[k], d0, zp[0][k]);
-        zp[1][k] = ffma2(wk[k], d1, zp[1][k]);
+    for (int h = 0; h < 2; ++h) {                        // the units in two halves, to bound the registers
+      float dv[FC2_NS][8];
+#pragma unroll
+      for (int u = 0; u < FC2_NS; ++u)
+#pragma unroll
+        for (int t = 0; t < 8; ++t) dv[u][t] = ws.d[(row0 + (u < n_s ? u : 0)) * HID + lane + 32 * (8 * h + t)];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        const float4* wr = w2p + (lane + 32 * (8 * h + t)) * (W2T_PITCH / 4);
+        const float4 q0 = wr[0], q1 = wr[1], q2 = wr[2];
+        const u64 wk[NCLS / 2] = {pack2(q0.x, q0.y), pack2(q0.z, q0.w), pack2(q1.x, q1.y), pack2(q1.z, q1.w), pack2(q2.x, q2.y)};
+#pragma unroll
+        for (int u = 0; u < FC2_NS; ++u) {
+          live[u] |= (dv[u][t] > 0.f ? 1u : 0u) << (8 * h + t);
+          const u64 du = pack2(dv[u][t], dv[u][t]);
+#pragma unroll
+          for (int k = 0; k < NCLS / 2; ++k) zp[u][k] = ffma2(wk[k], du, zp[u][k]);
+        }
       }
     }
-    float z[2][NCLS];
+    // Sum over the lanes.  Each exchange halves what a lane goes on with: after the first two a lane holds the ten
+    // partial logits of sample lane / 8 only, after the third five of them; two plain exchanges finish the sums and a
+    // last one brings the two halves of the classes together.
+    float v[FC2_NS * NCLS];
+#pragma unroll
+    for (int u = 0; u < FC2_NS; ++u)
+#pragma unroll
+      for (int k = 0; k < NCLS / 2; ++k) unpack2(zp[u][k], v[u * NCLS + 2 * k], v[u * NCLS + 2 * k + 1]);
+    float w20[2 * NCLS], x10[NCLS], y5[NCLS / 2], z[NCLS];
+#pragma unroll
+    for (int k = 0; k < 2 * NCLS; ++k) {
+      const float keep = hi16 ? v[2 * NCLS + k] : v[k], send = hi16 ? v[k] : v[2 * NCLS + k];
+      w20[k] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+#pragma unroll
+    for (int k = 0; k < NCLS; ++k) {
+      const float keep = hi8 ? w20[NCLS + k] : w20[k], send = hi8 ? w20[k] : w20[NCLS + k];
+      x10[k] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
 #pragma unroll
     for (int k = 0; k < NCLS / 2; ++k) {
-      unpack2(zp[0][k], z[0][2 * k], z[0][2 * k + 1]);
-      unpack2(zp[1][k], z[1][2 * k], z[1][2 * k + 1]);
+      const float keep = hi4 ? x10[NCLS / 2 + k] : x10[k], send = hi4 ? x10[k] : x10[NCLS / 2 + k];
+      y5[k] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+      y5[k] += __shfl_xor_sync(0xffffffffu, y5[k], 2);
+      y5[k] += __shfl_xor_sync(0xffffffffu, y5[k], 1);
     }
 #pragma unroll
-    for (int c = 0; c < NCLS; ++c) {
-      z[0][c] = warp_sum(z[0][c]) + b2[c];
-      z[1][c] = warp_sum(z[1][c]) + b2[c];
+    for (int k = 0; k < NCLS / 2; ++k) {
+      const float other = __shfl_xor_sync(0xffffffffu, y5[k], 4);
+      z[k] = (hi4 ? other : y5[k]) + b2[k];
+      z[NCLS / 2 + k] = (hi4 ? y5[k] : other) + b2[NCLS / 2 + k];
     }
-    float dz[2][NCLS];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      if (u == 1 && !two) continue;
-      const int i = i0 + u;
-      float zmax = z[u][0];
+    // softmax, loss and logits gradient of the lane's sample (the eight lanes of a sample do the same work)
+    float dzl[NCLS];
+    {
+      float zmax = z[0];
       int am = 0;
 #pragma unroll
       for (int c = 1; c < NCLS; ++c)
-        if (z[u][c] > zmax) { zmax = z[u][c]; am = c; }
+        if (z[c] > zmax) { zmax = z[c]; am = c; }
       float ez[NCLS], se = 0.f;
 #pragma unroll
-      for (int c = 0; c < NCLS; ++c) { ez[c] = expf(z[u][c] - zmax); se += ez[c]; }
+      for (int c = 0; c < NCLS; ++c) { ez[c] = expf(z[c] - zmax); se += ez[c]; }
       const float lse = zmax + logf(se), inv_se = 1.0f / se;
-      int label = lab[u];
       if (label < 0 || label >= NCLS) {
-        if (lane == 0) atomicOr(ws.status, STATUS_BAD_LABEL);
+        if (mine && sub == 0) atomicOr(ws.status, STATUS_BAD_LABEL);
         label = 0;
       }
       float zy = 0.f;
 #pragma unroll
       for (int c = 0; c < NCLS; ++c) {
-        if (c == label) zy = z[u][c];
-        dz[u][c] = (ez[c] * inv_se - (c == label ? 1.f : 0.f)) * inv_b;     // softmax from the exponentials already taken
+        if (c == label) zy = z[c];
+        const float g = (ez[c] * inv_se - (c == label ? 1.f : 0.f)) * inv_b;     // softmax from the exponentials already taken
+        dzl[c] = mine ? g : 0.f;
       }
-      loss_acc += lse - zy;
-      if (lane == 0) a.argmax[(int64_t)src * a.b + i] = am;
-      if (lane < DZ_STRIDE) {
-        float v = 0.f;
+      if (mine) {
+        loss_acc += lse - zy;
+        if (sub == 0) a.argmax[(int64_t)src * a.b + i0 + my_u] = am;
+        float e0 = 0.f, e1 = 0.f;                          // lane sub of a sample stores elements 2 sub and 2 sub + 1 of its padded row
 #pragma unroll
-        for (int c = 0; c < NCLS; ++c)
-          if (lane == c) v = dz[u][c];
-        ws.dz[(row0 + u) * DZ_STRIDE + lane] = v;
+        for (int m = 0; m < NCLS / 2; ++m)
+          if (sub == m) { e0 = dzl[2 * m]; e1 = dzl[2 * m + 1]; }
+        *reinterpret_cast<float2*>(ws.dz + (row0 + my_u) * DZ_STRIDE + 2 * sub) = make_float2(e0, e1);
       }
     }
-    if (!two) {
+    // every lane needs the logits gradients of all four samples, as class pairs
+    u64 dzk[FC2_NS][NCLS / 2];
 #pragma unroll
-      for (int c = 0; c < NCLS; ++c) dz[1][c] = 0.f;
-    }
+    for (int u = 0; u < FC2_NS; ++u)
+#pragma unroll
+      for (int k = 0; k < NCLS / 2; ++k)
+        dzk[u][k] = pack2(__shfl_sync(0xffffffffu, dzl[2 * k], 8 * u), __shfl_sync(0xffffffffu, dzl[2 * k + 1], 8 * u));
     asm volatile("mov.u32 %0, 0;" : "=r"(opaque_zero));    // second read of the weights, as above
     w2p = reinterpret_cast<const float4*>(&w2t[0][0] + opaque_zero);
-    uint32_t live0 = 0u, live1 = 0u;                         // which of the lane's 16 units passed ReLU and dropout
-#pragma unroll
-    for (int t = 0; t < 16; ++t) {
-      live0 |= (dv[0][t] > 0.f ? 1u : 0u) << t;
-      live1 |= (dv[1][t] > 0.f ? 1u : 0u) << t;
-    }
-    u64 dzk[2][NCLS / 2];
-#pragma unroll
-    for (int k = 0; k < NCLS / 2; ++k) {
-      dzk[0][k] = pack2(dz[0][2 * k], dz[0][2 * k + 1]);
-      dzk[1][k] = pack2(dz[1][2 * k], dz[1][2 * k + 1]);
-    }
 #pragma unroll 2
     for (int t = 0; t < 16; ++t) {
       const int j = lane + 32 * t;
       const float4* wr = w2p + j * (W2T_PITCH / 4);
       const float4 q0 = wr[0], q1 = wr[1], q2 = wr[2];
       const u64 wk[NCLS / 2] = {pack2(q0.x, q0.y), pack2(q0.z, q0.w), pack2(q1.x, q1.y), pack2(q1.z, q1.w), pack2(q2.x, q2.y)};
-      // even classes accumulate in the low half, odd classes in the high half; the halves are added at the end
-      u64 e0 = 0ull, e1 = 0ull;
 #pragma unroll
-      for (int k = 0; k < NCLS / 2; ++k) {
-        e0 = ffma2(wk[k], dzk[0][k], e0);
-        e1 = ffma2(wk[k], dzk[1][k], e1);
+      for (int u = 0; u < FC2_NS; ++u) {
+        // even classes accumulate in the low half, odd classes in the high half; the halves are added at the end
+        u64 e = 0ull;
+#pragma unroll
+        for (int k = 0; k < NCLS / 2; ++k) e = ffma2(wk[k], dzk[u][k], e);
+        float lo, hi;
+        unpack2(e, lo, hi);
+        float o = (live[u] >> t) & 1u ? (lo + hi) * scale : 0.f;
+        if (a.precision != 0) o = round_tf32(o);             // it feeds tensor-core products only
+        if (u < n_s) ws.da1[(row0 + u) * HID + j] = o;
       }
-      float lo0, hi0, lo1, hi1;
-      unpack2(e0, lo0, hi0);
-      unpack2(e1, lo1, hi1);
-      const float dd0 = lo0 + hi0, dd1 = lo1 + hi1;
-      float v0 = (live0 >> t) & 1u ? dd0 * scale : 0.f, v1 = (live1 >> t) & 1u ? dd1 * scale : 0.f;
-      if (a.precision != 0) { v0 = round_tf32(v0); v1 = round_tf32(v1); }   // they feed tensor-core products only
-      ws.da1[row0 * HID + j] = v0;
-      if (two) ws.da1[row1 * HID + j] = v1;
     }
+  }
+  {
+    // the eight lanes of a sample hold the same loss: one of each, in lane order
+    const float l0 = __shfl_sync(0xffffffffu, loss_acc, 0), l1 = __shfl_sync(0xffffffffu, loss_acc, 8);
+    const float l2 = __shfl_sync(0xffffffffu, loss_acc, 16), l3 = __shfl_sync(0xffffffffu, loss_acc, 24);
+    loss_acc = (l0 + l1) + (l2 + l3);
   }
   if (lane == 0) warp_loss[warp] = loss_acc;
   __syncthreads();   // also makes this block's dz / da1 stores visible to all of its threads
