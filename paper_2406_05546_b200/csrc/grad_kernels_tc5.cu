@@ -30,8 +30,8 @@ constexpr int MAX_STAGES = 4;
 constexpr int EPI_ROW_FLOATS = 36;                       // 32 columns + 4 of padding: conflict-free both ways
 constexpr int EPI_WARP_BYTES = 32 * EPI_ROW_FLOATS * 4;  // per epilogue warp: a 32 x 32 block being transposed
 __host__ __device__ constexpr int stage_bytes(int bn) { return A_BYTES + bn * BK * 4; }
-__host__ __device__ constexpr int gemm_smem_bytes(int bn, int stages) {
-  return stages * stage_bytes(bn) + 1024 /* alignment slack */ + 256 /* barriers */ + 4 * EPI_WARP_BYTES;
+__host__ __device__ constexpr int gemm_smem_bytes(int bn, int stages, int epi_warps) {
+  return stages * stage_bytes(bn) + 1024 /* alignment slack */ + 256 /* barriers */ + epi_warps * EPI_WARP_BYTES;
 }
 
 // Shared-memory matrix descriptor, k-contiguous operand, 128-byte swizzle: rows are 128 bytes apart,
@@ -76,6 +76,11 @@ struct GemmMaps {
 };
 
 enum { EPI_FC1_FWD = 0, EPI_STORE = 1 };
+// Epilogue warps: the plain-store products are bound by getting the accumulator out to global memory, so two warps
+// share each quarter of the accumulator rows and take alternate 32-column blocks; the forward product's epilogue
+// keeps one warp per quarter (its registers and shared memory leave no room for more).
+__host__ __device__ constexpr int epi_warps(int epi) { return epi == EPI_STORE ? 8 : 4; }
+__host__ __device__ constexpr int gemm_threads(int epi) { return 64 + 32 * epi_warps(epi); }
 
 struct GemmArgs {
   int K;            // reduction length (columns beyond it are zero-filled by TMA)
@@ -88,9 +93,8 @@ struct GemmArgs {
 };
 
 // Persistent kernel: one CTA per SM walks over output tiles (columns fastest, so that neighbouring CTAs
-// share their A rows in L2).  192 threads: warp 0 = TMA producer, warp 1 = tensor-memory owner and MMA
-// issuer, warps 2..5 = epilogue (each reads the 32 accumulator lanes of its quarter, quarter = warp index
-// mod 4).  The accumulator is double-buffered in tensor memory (2 x BN columns), so the epilogue of one
+// share their A rows in L2).  Warp 0 = TMA producer, warp 1 = tensor-memory owner and MMA issuer, warps 2.. =
+// epilogue (each reads the 32 accumulator lanes of its quarter, quarter = warp index mod 4).  The accumulator is double-buffered in tensor memory (2 x BN columns), so the epilogue of one
 // tile (tensor memory -> registers -> global) overlaps the loads and MMAs of the next.
 // BN = tile columns: 256 for the 512-wide forward product, 224 = 1568/7 for the other two.
 struct TileCoord { int grp, m0, m_end, n0, z; };
@@ -112,7 +116,7 @@ __device__ __forceinline__ bool decode_tile(int t, const GemmArgs& ga, const Gro
 }
 
 template <int EPI, int BN, bool MN = false>
-__global__ void __launch_bounds__(192, 1) tc5_gemm(const __grid_constant__ GemmMaps maps, GemmArgs ga, GradStepArgs a,
+__global__ void __launch_bounds__(gemm_threads(EPI), 1) tc5_gemm(const __grid_constant__ GemmMaps maps, GemmArgs ga, GradStepArgs a,
                                                    WorkerTable wt, GroupTable gt, Workspace ws) {
   constexpr int STAGES = MAX_STAGES;
   constexpr int B_BYTES = BN * BK * 4, STAGE_BYTES = A_BYTES + B_BYTES;
@@ -134,7 +138,7 @@ __global__ void __launch_bounds__(192, 1) tc5_gemm(const __grid_constant__ GemmM
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], epi_warps(EPI)); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -228,7 +232,7 @@ __global__ void __launch_bounds__(192, 1) tc5_gemm(const __grid_constant__ GemmM
       if (EPI == EPI_FC1_FWD && row_ok) { s_w = m_lane / a.b; smp = m_lane - s_w * a.b; }
       const float* bias = gt.theta[c.grp] + OFF_F1B;
 #pragma unroll 1
-      for (int ch = 0; ch < BN / 32; ++ch) {
+      for (int ch = (warp - 2) >> 2; ch < BN / 32; ch += epi_warps(EPI) / 4) {
         const int n = c.n0 + ch * 32;
         if (n >= ga.N) break;                    // warp-uniform
         uint32_t r[32];
@@ -360,9 +364,9 @@ int configure_tc5_kernels() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_sm_count <= 0) return -1;
-  cudaError_t e = cudaFuncSetAttribute(tc5_gemm<EPI_FC1_FWD, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(256, MAX_STAGES));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES));
+  cudaError_t e = cudaFuncSetAttribute(tc5_gemm<EPI_FC1_FWD, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(256, MAX_STAGES, epi_warps(EPI_FC1_FWD)));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES, epi_warps(EPI_STORE)));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES, epi_warps(EPI_STORE)));
   return e == cudaSuccess ? 0 : -1;
 }
 
@@ -378,7 +382,7 @@ int launch_fc1_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const Group
   const int mt = group_tiles(gt, a.b, BM);
   GemmArgs ga{FLAT, HID, HID, 0, ws.d, HID / 256, (HID / 256) * mt};
   const int grid = ga.n_tiles < g_sm_count ? ga.n_tiles : g_sm_count;
-  TIMED(K_FC1_FWD, (tc5_gemm<EPI_FC1_FWD, 256><<<grid, 192, gemm_smem_bytes(256, MAX_STAGES), st>>>(maps, ga, a, wt, gt, ws)));
+  TIMED(K_FC1_FWD, (tc5_gemm<EPI_FC1_FWD, 256><<<grid, gemm_threads(EPI_FC1_FWD), gemm_smem_bytes(256, MAX_STAGES, epi_warps(EPI_FC1_FWD)), st>>>(maps, ga, a, wt, gt, ws)));
   return a.skip_prep_w1 ? 1 : 2;
 }
 
@@ -392,7 +396,7 @@ int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupT
   const int mt = group_tiles(gt, a.b, BM);
   GemmArgs ga{HID, FLAT, FLAT, 0, ws.dp2, FLAT / 224, (FLAT / 224) * mt};
   const int grid = ga.n_tiles < g_sm_count ? ga.n_tiles : g_sm_count;
-  TIMED(K_FC1_DX, (tc5_gemm<EPI_STORE, 224><<<grid, 192, gemm_smem_bytes(224, MAX_STAGES), st>>>(maps, ga, a, wt, gt, ws)));
+  TIMED(K_FC1_DX, (tc5_gemm<EPI_STORE, 224><<<grid, gemm_threads(EPI_STORE), gemm_smem_bytes(224, MAX_STAGES, epi_warps(EPI_STORE)), st>>>(maps, ga, a, wt, gt, ws)));
   return 1;
 }
 
@@ -403,7 +407,7 @@ int launch_fc1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupT
   if (!make_map_mn(&maps.b[0], ws.p2, FLAT, a.b, a.W, 224 / 32)) return -1;
   GemmArgs ga{a.b, FLAT, FLAT, 1, nullptr, FLAT / 224, (FLAT / 224) * (HID / BM) * a.W};
   const int grid = ga.n_tiles < g_sm_count ? ga.n_tiles : g_sm_count;
-  TIMED(K_FC1_DW, (tc5_gemm<EPI_STORE, 224, true><<<grid, 192, gemm_smem_bytes(224, MAX_STAGES), st>>>(maps, ga, a, wt, gt, ws)));
+  TIMED(K_FC1_DW, (tc5_gemm<EPI_STORE, 224, true><<<grid, gemm_threads(EPI_STORE), gemm_smem_bytes(224, MAX_STAGES, epi_warps(EPI_STORE)), st>>>(maps, ga, a, wt, gt, ws)));
   return 1;
 }
 
