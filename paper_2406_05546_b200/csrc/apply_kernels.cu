@@ -143,7 +143,7 @@ int launch_sum_apply(const SumApplyArgs& a, cudaStream_t st, Profiler* prof) {
   float4* tout = reinterpret_cast<float4*>(a.theta_out);
   float4* rep = reinterpret_cast<float4*>(a.replica);
   int n_split = 1;
-  if (a.K > 48 && a.max_split > 1) {
+  if (a.K > 160 && a.max_split > 1) {
     int64_t want = (a.K + 31) / 32;
     n_split = (int)(want < a.max_split ? want : a.max_split);
   }
