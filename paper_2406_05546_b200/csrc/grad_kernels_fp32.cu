@@ -722,7 +722,8 @@ int configure_grad_kernels() {
   return e == cudaSuccess ? 0 : -1;
 }
 
-// Launch order of one grad step.  On the tensor-core path the backward pass forks: once the output
+// Launch order of one grad step.  On the tensor-core path the copies of the dense layer's weights are made on a
+// side stream while the convolutions run, and the backward pass forks: once the output
 // layer's backward has produced da1, the dense layer's per-worker weight gradient (bound by its 3.2 MB
 // per worker of writes) runs on a side stream next to the input-gradient chain, and once dp2 exists the
 // second convolution's filter gradient runs on another side stream next to its input gradient and the
@@ -736,14 +737,21 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
   const int n_chunks1b = (a.b + CONV1B_SPB - 1) / CONV1B_SPB;
   int launches = 0, n_chunks2 = n_chunks, seg_len = 0;
   if (tc) {
+    cudaStream_t s1 = side.s1 ? side.s1 : st, s2 = side.s2 ? side.s2 : st;
+    // the copies of W1 are not needed before the dense layer: they are made next to the convolutions
+    if (!a.skip_prep_w1) {
+      if (side.s1) { cudaEventRecord(side.fork1, st); cudaStreamWaitEvent(s1, side.fork1, 0); }
+      launches += launch_prep_w1(gt, ws, s1, prof);
+      if (side.s1) cudaEventRecord(side.join1, s1);
+    }
     if (launch_conv1_fwd_planes(a, wt, gt, ws, st, prof) < 0) return -1;
     launch_conv2_fwd_tc5(a, wt, gt, ws, st, prof);
+    if (!a.skip_prep_w1 && side.s1) cudaStreamWaitEvent(st, side.join1, 0);
     int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof);
     if (n < 0) return -1;
     launches += 2 + n;
     TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<dim3(a.W, FC2_SPLIT), FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
     launches += 1;
-    cudaStream_t s1 = side.s1 ? side.s1 : st, s2 = side.s2 ? side.s2 : st;
     if (side.s1) { cudaEventRecord(side.fork1, st); cudaStreamWaitEvent(s1, side.fork1, 0); }
     n = launch_fc1_dw_tc5(a, wt, gt, ws, s1, prof);
     if (n < 0) return -1;

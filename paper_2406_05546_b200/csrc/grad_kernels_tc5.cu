@@ -370,10 +370,15 @@ int configure_tc5_kernels() {
   return e == cudaSuccess ? 0 : -1;
 }
 
-// Rounded / transposed copies of W1 for every weight group of this call, then the forward product.
+// Rounded / transposed copies of W1 for every weight group of this call.
+int launch_prep_w1(const GroupTable& gt, const Workspace& ws, cudaStream_t st, Profiler* prof) {
+  TIMED(K_PREP_W1, (prep_w1<<<dim3(FLAT / 32, HID / 32, gt.n_groups), 256, 0, st>>>(gt, ws.w1r, ws.w1tr)));
+  return 1;
+}
+
+// The forward product; the copies of W1 must be in place.
 int launch_fc1_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                        cudaStream_t st, Profiler* prof) {
-  if (!a.skip_prep_w1) TIMED(K_PREP_W1, (prep_w1<<<dim3(FLAT / 32, HID / 32, gt.n_groups), 256, 0, st>>>(gt, ws.w1r, ws.w1tr)));
   GemmMaps maps;
   const uint64_t rows = (uint64_t)a.W * a.b;
   if (!make_map(&maps.a, ws.p2, FLAT, rows, 1, FLAT, rows * FLAT, BM)) return -1;
@@ -383,7 +388,7 @@ int launch_fc1_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const Group
   GemmArgs ga{FLAT, HID, HID, 0, ws.d, HID / 256, (HID / 256) * mt};
   const int grid = ga.n_tiles < g_sm_count ? ga.n_tiles : g_sm_count;
   TIMED(K_FC1_FWD, (tc5_gemm<EPI_FC1_FWD, 256><<<grid, gemm_threads(EPI_FC1_FWD), gemm_smem_bytes(256, MAX_STAGES, epi_warps(EPI_FC1_FWD)), st>>>(maps, ga, a, wt, gt, ws)));
-  return a.skip_prep_w1 ? 1 : 2;
+  return 1;
 }
 
 int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,

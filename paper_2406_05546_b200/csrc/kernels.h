@@ -152,6 +152,7 @@ void launch_conv2_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const Gr
                           cudaStream_t st, Profiler* prof);
 void launch_conv2_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                          cudaStream_t st, Profiler* prof);
+int launch_prep_w1(const GroupTable& gt, const Workspace& ws, cudaStream_t st, Profiler* prof);
 int launch_fc1_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                        cudaStream_t st, Profiler* prof);
 int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
