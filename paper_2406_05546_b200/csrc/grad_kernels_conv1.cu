@@ -19,21 +19,26 @@ namespace psk {
 
 namespace {
 
-constexpr int C1_THREADS = 224;
-constexpr int C1_SPB = 8;                                // samples per block, taken two at a time
+constexpr int C1_SPS = 1;                                // samples per step
+constexpr int C1_THREADS = 112 * C1_SPS;
+constexpr int C1_BLOCKS_PER_SM = 6 / C1_SPS;
+constexpr int C1_SPB = 8;                                // samples per block, taken C1_SPS at a time
 constexpr int C1_BOX_W = 36, C1_BOX_H = 30;              // image box: columns -4..31 (a 16-byte aligned start), rows -1..28
 constexpr int C1_BOX_BYTES = C1_BOX_W * C1_BOX_H * 4;    // 4320
 constexpr int C1_IMG_SLOT = 4352;                        // box padded to a multiple of 128 bytes
-constexpr int C1_IN_BYTES = 2 * C1_IMG_SLOT;             // two images per step
+constexpr int C1_IN_BYTES = C1_SPS * C1_IMG_SLOT;        // the images of a step
 constexpr int C1_PLANES_BYTES = P1_PLANE_ELEMS * 4;      // 8192 per sample
-constexpr int C1_OUT_BYTES = 2 * C1_PLANES_BYTES + 2 * P1_ELEMS;   // two samples: planes, then decisions
+constexpr int C1_OUT_BYTES = C1_SPS * (C1_PLANES_BYTES + P1_ELEMS);   // a step's samples: planes, then decisions
 constexpr int C1_STAGES = 2;
 constexpr int C1_SMEM = C1_STAGES * C1_IN_BYTES + 2 * C1_OUT_BYTES + 64 + 128;
 
-// Work items of a step = (sample of the pair, pooled position, group of four channels): 2 * 196 * 4 = 1568
-// = 7 per thread.  Thread tid takes channel group tid & 3 and the pooled positions (tid >> 2) + 56 k of the
-// two samples laid end to end; 56 = four rows of 14, so its column is fixed and its row advances by four.
-__global__ void __launch_bounds__(C1_THREADS, 3) conv1_fwd_planes(const __grid_constant__ CUtensorMap xmap, GradStepArgs a,
+// Work items of a step = (sample, pooled position, group of four channels): C1_SPS * 196 * 4 = 7 per thread.
+// Thread tid takes channel group tid & 3 and the pooled positions (tid >> 2) + 28 C1_SPS k of the step's samples
+// laid end to end; 28 = two rows of 14, so its column is fixed and its row advances by 2 C1_SPS.  Small blocks
+// (one sample per step, six blocks per SM) keep the blocks' phases apart: the barrier of a step lines up the
+// multiply-add phases of all warps of a block, and with few large blocks the FMA pipe idles while all of them
+// pool and store.
+__global__ void __launch_bounds__(C1_THREADS, C1_BLOCKS_PER_SM) conv1_fwd_planes(const __grid_constant__ CUtensorMap xmap, GradStepArgs a,
                                                                   WorkerTable wt, GroupTable gt, Workspace ws) {
   extern __shared__ __align__(128) uint8_t sm[];
   const float* in = reinterpret_cast<const float*>(sm);
@@ -41,7 +46,7 @@ __global__ void __launch_bounds__(C1_THREADS, 3) conv1_fwd_planes(const __grid_c
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + C1_STAGES * C1_IN_BYTES + 2 * C1_OUT_BYTES);
   const int s = blockIdx.y, tid = threadIdx.x, cg = tid & 3;
   const int i0 = blockIdx.x * C1_SPB, i1 = min(i0 + C1_SPB, a.b);
-  const int n_steps = (i1 - i0 + 1) / 2;
+  const int n_steps = (i1 - i0 + C1_SPS - 1) / C1_SPS;
   const float* theta = group_theta(wt, gt, s);
   if (tid == 0) {
     for (int k = 0; k < C1_STAGES; ++k) mbar_init(&full[k], 1);
@@ -60,11 +65,11 @@ __global__ void __launch_bounds__(C1_THREADS, 3) conv1_fwd_planes(const __grid_c
   __syncthreads();
   const int64_t src_row0 = (int64_t)wt.src[s] * a.b + i0;     // the caller's image index of the block's first sample
   auto issue = [&](int st) {     // thread 0: the images of step st
-    const int n_s = min(2, i1 - (i0 + 2 * st));
+    const int n_s = min(C1_SPS, i1 - (i0 + C1_SPS * st));
     uint64_t* bar = &full[st % C1_STAGES];
     mbar_expect_tx(bar, n_s * C1_BOX_BYTES);
     for (int k = 0; k < n_s; ++k)
-      tma_load_3d(sm + (st % C1_STAGES) * C1_IN_BYTES + k * C1_IMG_SLOT, &xmap, bar, -4, -1, (int)(src_row0 + 2 * st + k));
+      tma_load_3d(sm + (st % C1_STAGES) * C1_IN_BYTES + k * C1_IMG_SLOT, &xmap, bar, -4, -1, (int)(src_row0 + C1_SPS * st + k));
   };
   if (tid == 0)
     for (int st = 0; st < C1_STAGES && st < n_steps; ++st) issue(st);
@@ -72,13 +77,13 @@ __global__ void __launch_bounds__(C1_THREADS, 3) conv1_fwd_planes(const __grid_c
   const int X = px + 1, col_row = (X & 1) * 8 + (X >> 1);
   bool ok = true;
   for (int st = 0; st < n_steps && ok; ++st) {
-    const int n_s = min(2, i1 - (i0 + 2 * st));
+    const int n_s = min(C1_SPS, i1 - (i0 + C1_SPS * st));
     if (!mbar_wait(&full[st % C1_STAGES], (st / C1_STAGES) & 1)) { ok = false; break; }
     const float* img = in + (st % C1_STAGES) * (C1_IN_BYTES / 4);
     uint8_t* ob = outb + (st & 1) * C1_OUT_BYTES;
 #pragma unroll 1
     for (int k = 0; k < 7; ++k) {
-      const int R = py0 + 4 * k, sp = R >= 14 ? 1 : 0, py = R - 14 * sp;
+      const int R = py0 + 2 * C1_SPS * k, sp = R / 14, py = R - 14 * sp;
       if (sp >= n_s) break;
       // image row 2 py - 1 is box row 2 py, image column 2 px - 1 is box column 2 px + 3
       const float* src = img + sp * (C1_IMG_SLOT / 4) + (2 * py) * C1_BOX_W + 2 * px + 3;
@@ -122,15 +127,15 @@ __global__ void __launch_bounds__(C1_THREADS, 3) conv1_fwd_planes(const __grid_c
       const int row = (py + 1) * 16 + col_row, pos = py * 14 + px;
       *reinterpret_cast<uint2*>(ob + sp * C1_PLANES_BYTES + (cg >> 1) * (C1_PLANES_BYTES / 2) + row * 16 + (cg & 1) * 8) =
           make_uint2(bf16_pair(best[0], best[1]), bf16_pair(best[2], best[3]));
-      *reinterpret_cast<uint32_t*>(ob + 2 * C1_PLANES_BYTES + sp * P1_ELEMS + cg * 784 + pos * 4) = codes;
+      *reinterpret_cast<uint32_t*>(ob + C1_SPS * C1_PLANES_BYTES + sp * P1_ELEMS + cg * 784 + pos * 4) = codes;
     }
     fence_proxy_async_smem();
     if (tid == 0) bulk_wait_read0();      // the previous step's copies have read their buffer, which the next step overwrites
     __syncthreads();
     if (tid == 0) {
-      const int64_t row0 = (int64_t)s * a.b + i0 + 2 * st;
+      const int64_t row0 = (int64_t)s * a.b + i0 + C1_SPS * st;
       bulk_store(reinterpret_cast<uint8_t*>(ws.p1) + row0 * C1_PLANES_BYTES, ob, n_s * C1_PLANES_BYTES);
-      bulk_store(ws.code1 + row0 * P1_ELEMS, ob + 2 * C1_PLANES_BYTES, n_s * P1_ELEMS);
+      bulk_store(ws.code1 + row0 * P1_ELEMS, ob + C1_SPS * C1_PLANES_BYTES, n_s * P1_ELEMS);
       bulk_commit();
       if (st + C1_STAGES < n_steps) issue(st + C1_STAGES);
     }
