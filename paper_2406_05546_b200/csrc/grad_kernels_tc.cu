@@ -31,7 +31,7 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
 // warp's k-steps and their shared-memory offsets are fixed, so they are worked out once); their accumulators
 // persist over the block's samples and are combined in a fixed order at the end.
 // ------------------------------------------------------------------------------------------------
-constexpr int C1B_SPB = 16;
+constexpr int C1B_SPB = 8;
 constexpr int C1B_A_WORDS = 396;       // 392 position pairs per channel + 4: 396 = 12 (mod 32 banks)
 constexpr int C1B_ROW = 42;            // elements per row of the bordered image: 21 words, so that the three filter rows
 constexpr int C1B_X_WORDS = 656;       // and the two copies (656 = 16 mod 32 words apart) fall into different banks
