@@ -22,7 +22,7 @@ namespace {
 constexpr int C1_SPS = 1;                                // samples per step
 constexpr int C1_THREADS = 112 * C1_SPS;
 constexpr int C1_BLOCKS_PER_SM = 6 / C1_SPS;
-constexpr int C1_SPB = 8;                                // samples per block, taken C1_SPS at a time
+constexpr int C1_SPB = 4;                                // samples per block, taken C1_SPS at a time
 constexpr int C1_BOX_W = 36, C1_BOX_H = 30;              // image box: columns -4..31 (a 16-byte aligned start), rows -1..28
 constexpr int C1_BOX_BYTES = C1_BOX_W * C1_BOX_H * 4;    // 4320
 constexpr int C1_IMG_SLOT = 4352;                        // box padded to a multiple of 128 bytes
