@@ -244,6 +244,20 @@ static void conv3x3_bwd_x(const double* dout, int cout, int hw, const double* w,
             }
 }
 
+/* Optional per-sample intermediates of the exact (double) pass, for tests that ask how far a decision
+ * is from flipping.  Nothing here is new arithmetic: every array is a value the step computes anyway.
+ * Any pointer may be NULL. */
+typedef struct {
+    double* p1;      /* [b][16][14][14] pooled output of the first convolution (the second one's input)        */
+    double* a2;      /* [b][32][14][14] pre-activations of the second convolution                               */
+    double* p2;      /* [b][1568]       pooled output of the second convolution, channel-major flatten          */
+    double* u;       /* [b][512]        pre-activations of the 512-unit layer                                   */
+    double* dh;      /* [b][512]        gradient of the mean loss w.r.t. the layer's output AFTER its ReLU,     */
+                     /*                 dropout applied: a unit that is on contributes dh * p2 to its row       */
+    int32_t* code2;  /* [b][1568]       pooling decision of the second convolution that was used (0..3, 4 dead) */
+    int32_t* on;     /* [b][512]        ReLU decision of the 512-unit layer that was used                       */
+} oracle_diag;
+
 /*
  * One worker's gradient step in double precision.
  *   theta  [P]          parameters (canonical layout)
@@ -263,11 +277,12 @@ static void conv3x3_bwd_x(const double* dout, int cout, int hw, const double* w,
  *   loss                mean over the batch of logsumexp(z) - z[y]
  *   argmax [b]          lowest index of the maximal logit
  *   logits [b][10]
+ *   diag                optional intermediates of the exact pass (see oracle_diag), or NULL
  * Returns 0, or -1 on a bad argument (label out of range, b <= 0).
  */
-int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t* y, int32_t b,
-                             const uint8_t* keep, double drop_p, int32_t precision, double* grad,
-                             double* loss, int32_t* argmax, double* logits) {
+int32_t oracle_grad_step_f64_diag(const double* theta, const double* x, const int32_t* y, int32_t b,
+                                  const uint8_t* keep, double drop_p, int32_t precision, double* grad,
+                                  double* loss, int32_t* argmax, double* logits, const oracle_diag* diag) {
     if (b <= 0 || !theta || !x || !y || !grad) return -1;
     for (int i = 0; i < b; ++i)
         if (y[i] < 0 || y[i] >= NCLS) return -1;
@@ -309,6 +324,12 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
             for (size_t k = 0; k < np2; ++k) p2q[k] = round_operand((double)(float)p2q[k], dense_rounding(precision));
         }
         pool_apply(a2, i2, C2, H1, p2); /* p2 is already the channel-major flatten */
+        if (diag) {
+            if (diag->p1) memcpy(diag->p1 + (size_t)i * np1, p1, sizeof(double) * np1);
+            if (diag->a2) memcpy(diag->a2 + (size_t)i * na2, a2, sizeof(double) * na2);
+            if (diag->p2) memcpy(diag->p2 + (size_t)i * np2, p2, sizeof(double) * np2);
+            if (diag->code2) for (size_t k = 0; k < np2; ++k) diag->code2[(size_t)i * np2 + k] = i2[k];
+        }
         for (int j = 0; j < HID; ++j) {
             double s = f1b[j];
             for (int k = 0; k < FLAT; ++k) s += f1w[(size_t)j * FLAT + k] * p2[k];
@@ -350,6 +371,9 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
             int kept = keep ? keep[(size_t)i * HID + j] : 1;
             double dh = kept ? s * scale : 0.0;
             du[j] = on[j] ? dh : 0.0;
+            if (diag && diag->dh) diag->dh[(size_t)i * HID + j] = dh;
+            if (diag && diag->u) diag->u[(size_t)i * HID + j] = u[j];
+            if (diag && diag->on) diag->on[(size_t)i * HID + j] = on[j];
         }
         memset(dp2, 0, sizeof(double) * np2);
         for (int j = 0; j < HID; ++j) {
@@ -371,6 +395,12 @@ int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t
     free(a1); free(da1); free(p1); free(dp1); free(a2); free(da2); free(p2); free(dp2);
     free(i1); free(i2); free(p1q); free(a2q); free(p2q);
     return 0;
+}
+
+int32_t oracle_grad_step_f64(const double* theta, const double* x, const int32_t* y, int32_t b,
+                             const uint8_t* keep, double drop_p, int32_t precision, double* grad,
+                             double* loss, int32_t* argmax, double* logits) {
+    return oracle_grad_step_f64_diag(theta, x, y, b, keep, drop_p, precision, grad, loss, argmax, logits, NULL);
 }
 
 /*

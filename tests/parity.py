@@ -27,13 +27,16 @@ def assert_params_close(got, ref, tol, what=""):
     return errs
 
 
-def assert_params_close_up_to_unit_flips(got, ref, tol, max_units, what=""):
-    """As assert_params_close, except that up to max_units of the 512 hidden units may be off in fc1.w / fc1.b.
-    A hidden unit whose pre-activation lies within rounding distance of zero in some sample can be switched on by
-    one side and off by the other (both take the decision on TF32 products, but sum them in different orders);
-    that moves the unit's row of fc1.w and its fc1.b entry by that sample's contribution and nothing else by
-    more than the tolerance.  With hundreds of thousands of such decisions per call a flip is expected now and
-    then, so large cases use this check; the flagged units are returned."""
+def assert_params_close_up_to_unit_flips(got, ref, tol, theta, diag, what=""):
+    """As assert_params_close, except that a row of fc1.w (with its fc1.b entry) may differ from the reference by
+    ReLU decisions of that hidden unit that came out the other way, under two conditions that are both checked:
+    (1) only samples in which the unit's exact pre-activation lies within the operand-rounding bound of zero
+    (tests/margins.py) may have flipped, and (2) the difference of the row must equal, within the tolerance, the
+    signed sum of exactly those samples' contributions dh[i, j] * p2[i, :] (found by least squares over the
+    candidate samples, coefficients rounded to -1 / 0 / +1).  A row that is off for any other reason fails.
+    `theta` are the worker's weights and `diag` the oracle's intermediates of the same pass that produced `ref`.
+    Every other tensor must be within the tolerance.  Returns the list of (unit, [(sample, sign), ...])."""
+    from tests import margins
     errs = tensor_rel_errors(got, ref)
     lay = {name: (off, shape) for name, off, shape in synth.layout()}
     off_w, shape_w = lay["fc1.w"]
@@ -43,12 +46,27 @@ def assert_params_close_up_to_unit_flips(got, ref, tol, max_units, what=""):
     rw = np.asarray(ref[off_w:off_w + n], dtype=np.float64).reshape(shape_w)
     gb = np.asarray(got[off_b:off_b + shape_w[0]], dtype=np.float64)
     rb = np.asarray(ref[off_b:off_b + shape_w[0]], dtype=np.float64)
-    unit_err = np.maximum(np.abs(gw - rw).max(axis=1) / np.abs(rw).max(), np.abs(gb - rb) / np.abs(rb).max())
+    w_scale, b_scale = np.abs(rw).max(), np.abs(rb).max()
+    unit_err = np.maximum(np.abs(gw - rw).max(axis=1) / w_scale, np.abs(gb - rb) / b_scale)
     flagged = np.where(unit_err > tol)[0]
-    assert flagged.size <= max_units, f"{what}: {flagged.size} hidden units off by more than {tol}: {flagged[:10]}"
+    explained = []
+    if flagged.size:
+        m = margins.decision_margins(theta, diag)
+        for j in flagged:
+            cand = np.where(m["relu_uncertain"][:, j])[0]
+            assert cand.size, f"{what}: hidden unit {j} is off by {unit_err[j]:.2e} and no sample has it near zero"
+            contrib = margins.unit_contributions(diag, j)
+            # bias column rescaled so that one absolute tolerance serves the whole row
+            k = w_scale / b_scale
+            contrib[:, -1] *= k
+            diff = np.concatenate([gw[j] - rw[j], [(gb[j] - rb[j]) * k]])
+            flips = margins.explain_row_by_flips(diff, contrib, cand, tol * w_scale)
+            assert flips, (f"{what}: hidden unit {j} is off by {unit_err[j]:.2e} and no set of near-zero samples "
+                           f"({cand.tolist()}) explains the difference of its row")
+            explained.append((int(j), flips))
     bad = {k: v for k, v in errs.items() if not v <= tol and k not in ("fc1.w", "fc1.b")}
     assert not bad, f"{what}: relative error above {tol}: {bad} (all: {errs})"
-    return flagged
+    return explained
 
 
 def assert_argmax_valid(got, ref_logits, tol):

@@ -4,7 +4,7 @@ import pytest
 
 from paper_2406_05546_b200 import synth
 from tests.parity import (TOL_FP32, TOL_TENSOR, assert_argmax_valid, assert_params_close,
-                          assert_params_close_up_to_unit_flips)
+                          assert_params_close_up_to_unit_flips, tensor_rel_errors)
 
 pytestmark = pytest.mark.gpu
 
@@ -53,15 +53,21 @@ def _run_and_compare(W, b, lags=None, n_versions=1, step=3, drop_p=0.25, worker_
     thetas = [versions[s.version] for s in snaps]
     og, ol, oa, oz = cnn.workers_grad_step(thetas, ids, x, y, SEED, step, drop_p, precision=precision)
     for w in range(W):
-        if precision and W * b > 500:     # several hundred thousand ReLU decisions: see the helper's docstring
-            flipped = assert_params_close_up_to_unit_flips(grads[w, :ps.P], og[w], tol, 2, f"gradient of worker {w}")
-            if flipped.size:
-                print(f"worker {w}: hidden units decided differently near zero: {flipped}")
+        assert (grads[w, ps.P:] == 0).all()
+        if precision and W * b > 500:
+            # several hundred thousand ReLU decisions: a hidden unit within rounding distance of zero may come out the
+            # other way; the helper admits that, and only that (see its docstring), so the oracle's intermediates of
+            # this worker are needed whenever a row is off
+            errs = tensor_rel_errors(grads[w, :ps.P], og[w])
+            if max(errs.values()) > tol:
+                g1, _, _, _, diag = cnn.worker_grad_step_diag(thetas[w], ids[w], x[w], y[w], SEED, step, drop_p, precision)
+                assert np.array_equal(g1, og[w])
+                flips = assert_params_close_up_to_unit_flips(grads[w, :ps.P], og[w], tol, thetas[w], diag, f"gradient of worker {w}")
+                print(f"worker {w}: hidden units decided differently within the rounding bound of zero: {flips}")
             continue
         errs = assert_params_close(grads[w, :ps.P], og[w], tol, f"gradient of worker {w}")
         if precision and w == 0:
             print("tensor-path relative errors:", {k: f"{v:.1e}" for k, v in errs.items()})
-        assert (grads[w, ps.P:] == 0).all()
     np.testing.assert_allclose(loss.cpu().numpy(), ol, rtol=3e-3 if precision else 1e-5, atol=1e-6)
     assert_argmax_valid(am.cpu().numpy(), oz, tol)
     srv.close()
@@ -99,6 +105,55 @@ def test_tensor_core_path_repeatable_bit_for_bit():
     a = _run_and_compare(3, 9, precision=2)
     b = _run_and_compare(3, 9, precision=2)
     assert (a == b).all()
+
+
+@pytest.mark.parametrize("W,b", [(2, 8), (3, 40)])
+def test_tensor_core_path_against_the_plain_definition(W, b):
+    """The tensor-core path against the oracle with EVERY decision taken on exact values (precision 0): what the
+    benchmarked path's error is against the definition, and that it comes from decisions inside the
+    operand-rounding bound and from nothing else.
+      - output layer: within the tolerance as it stands (a ReLU that flips at zero changes no forward value);
+      - 512-unit layer: every row is within the tolerance after removing the contributions of samples whose exact
+        pre-activation is inside the bound (least-squares explanation, coefficients -1 / 0 / +1);
+      - convolutions: pooling winners inside the bound re-route gradient between neighbouring positions; their
+        error is reported and must not exceed what the oracle itself shows between exact and rounded decisions
+        plus the tolerance (every such difference lies inside the bound: tests/test_margins.py)."""
+    from oracle import cnn
+    import torch
+    from paper_2406_05546_b200 import ps
+    from tests import margins
+    torch_, ps_, srv, theta0 = _setup(W, b, 1, 0.25, 2)
+    rng = np.random.default_rng(21)
+    x = rng.random((W, b, 28, 28), dtype=np.float32)
+    y = rng.integers(0, 10, (W, b)).astype(np.int32)
+    snaps = [srv.ps_pull_snapshot(w) for w in range(W)]
+    gd = torch.full((W, ps.P_PAD), float("nan"), device="cuda")
+    srv.workers_grad_step(snaps, list(range(W)), torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(), SEED, 4, grads_dev=gd)
+    srv.ps_stats()
+    grads = gd.cpu().numpy()
+    srv.close()
+    n_flips = n_pool_unc = n_relu_unc = 0
+    for w in range(W):
+        g0, _, _, _, d0 = cnn.worker_grad_step_diag(theta0, w, x[w], y[w], SEED, 4, 0.25, precision=0)
+        g2 = cnn.worker_grad_step_diag(theta0, w, x[w], y[w], SEED, 4, 0.25, precision=2)[0]
+        m = margins.decision_margins(theta0, d0)
+        n_pool_unc += int(m["pool_uncertain"].sum()); n_relu_unc += int(m["relu_uncertain"].sum())
+        e_kernel = tensor_rel_errors(grads[w, :ps.P], g0)
+        e_oracle = tensor_rel_errors(g2, g0)
+        print(f"worker {w}: kernel vs exact decisions", {k: f"{v:.1e}" for k, v in e_kernel.items()})
+        print(f"worker {w}: oracle with rounded decisions vs exact decisions", {k: f"{v:.1e}" for k, v in e_oracle.items()})
+        for name in ("fc2.w", "fc2.b"):
+            assert e_kernel[name] <= TOL_TENSOR, (name, e_kernel[name])
+        for name in ("conv1.w", "conv1.b", "conv2.w", "conv2.b"):
+            assert e_kernel[name] <= e_oracle[name] + TOL_TENSOR, (name, e_kernel[name], e_oracle[name])
+        # the 512-unit layer, row by row: got = exact-decision gradient + flips of samples inside the bound.  The
+        # convolution tensors are excluded from this call's tolerance check by comparing them in a copy.
+        probe = g0.copy()
+        probe[4800:808128] = grads[w, 4800:808128]
+        flips = assert_params_close_up_to_unit_flips(probe, g0, TOL_TENSOR, theta0, d0, f"worker {w} vs exact decisions")
+        n_flips += sum(len(f) for _, f in flips)
+    print(f"{n_flips} ReLU decisions of the 512-unit layer differ from the exact ones; all inside the bound "
+          f"({n_relu_unc} of {W * b * 512} decisions are; pooling: {n_pool_unc} of {W * b * 1568})")
 
 
 def test_no_dropout():
