@@ -151,25 +151,34 @@ class OraclePS:
         return self.version
 
     def replicate(self):
+        """One replication event.  The frontend hands its weights to the next live server and waits for that
+        server's acknowledgement only (the relaxed consistency of the chain design); the hop from that server to
+        the one behind it completes with the following event.  So after an event the first live server behind the
+        frontend holds the frontend's version, the second what the first held before, and so on: a server further
+        down the chain holds more outdated weights, as the design section says of the tertiary server."""
         live = [r for r in self.replicas if r["alive"]]
         if not live:
             raise PSError(NO_REPLICA, "no live replica")
-        for r in live:
-            r["version"] = self.version
-            r["theta"] = self.head().copy()
+        for i in range(len(live) - 1, 0, -1):
+            live[i]["version"] = live[i - 1]["version"]
+            live[i]["theta"] = live[i - 1]["theta"]
+        live[0]["version"] = self.version
+        live[0]["theta"] = self.head().copy()
         return self.version
 
     def kill(self, server=0):
-        """server 0 = the current frontend; i >= 1 = the i-th server behind it."""
+        """server 0 = the current frontend; i >= 1 = the i-th LIVE server behind it (a dead server has left the
+        chain: the one behind it watches the next live one in front of it instead)."""
         if server == 0:
             self.up = False
             if not self.external_store:
                 self.ring = {}
                 self.queue = []
         else:
-            if server - 1 >= len(self.replicas):
+            live = [r for r in self.replicas if r["alive"]]
+            if server < 0 or server - 1 >= len(live):
                 raise PSError(BAD_ARG, "no such server")
-            self.replicas[server - 1]["alive"] = False
+            live[server - 1]["alive"] = False
 
     def restore(self):
         """Resurrected server: latest checkpoint (stateful) or the surviving store (stateless)."""

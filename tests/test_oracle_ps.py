@@ -232,3 +232,94 @@ def test_queue_capacity():
     with pytest.raises(ops.PSError) as e:
         s.enqueue(g, [0, 1], [0, 0], 1)
     assert e.value.code == ops.QUEUE_FULL
+
+
+def _steps(s, n, seed0, W=2):
+    for t in range(n):
+        s.enqueue(_small_grads(W, seed=seed0 + t), range(W), [s.version] * W, t)
+        s.apply(ops.SYNC, 0.01)
+
+
+def test_chain_of_three_tertiary_holds_older_weights_and_survives_a_double_failure():
+    # Design, chain replication: the frontend waits for the next server only, so the server behind that one is one
+    # replication event behind; when frontend and secondary both fail, the tertiary recovers with older weights.
+    theta = synth.init_params(1)
+    R = 2
+    s = ops.OraclePS(theta, chain_len=3, replicate_every=R)
+    hist = {0: theta.copy()}
+    for t in range(5):
+        _steps(s, 1, 40 + t)
+        hist[s.version] = s.head().copy()
+        first = (s.version // R) * R
+        assert s.replicas[0]["version"] == first
+        assert s.replicas[1]["version"] == max(first - R, 0)
+        assert (s.replicas[0]["theta"] == hist[first]).all() and (s.replicas[1]["theta"] == hist[max(first - R, 0)]).all()
+    assert s.version == 5
+    s.kill(0)
+    s.kill(1)                                   # the secondary dies too
+    assert s.failover() == 2                    # the tertiary takes over, one event (R versions) behind the secondary's 4
+    assert (s.head() == hist[2]).all() and s.oldest_version() == 2 and s.replicas == []
+    _steps(s, 1, 60)                            # training goes on without a replica
+    assert s.version == 3
+    s.kill(0)
+    with pytest.raises(ops.PSError) as e:
+        s.failover()
+    assert e.value.code == ops.NO_REPLICA
+
+
+def test_killing_a_server_behind_the_frontend_shortens_the_chain():
+    theta = synth.init_params(1)
+    s = ops.OraclePS(theta, chain_len=4, replicate_every=1)
+    _steps(s, 3, 70)
+    assert [r["version"] for r in s.replicas] == [3, 2, 1]
+    s.kill(2)                                   # the second live server behind the frontend
+    assert [r["alive"] for r in s.replicas] == [True, False, True]
+    _steps(s, 1, 80)
+    # the dead server is skipped: the last one now follows the first, and the dead one keeps what it had
+    assert [r["version"] for r in s.replicas] == [4, 2, 3]
+    s.kill(2)                                   # now the second LIVE one is the last server
+    assert [r["alive"] for r in s.replicas] == [True, False, False]
+    with pytest.raises(ops.PSError) as e:
+        s.kill(2)
+    assert e.value.code == ops.BAD_ARG
+    s.kill(1)
+    s.kill(0)
+    with pytest.raises(ops.PSError) as e:
+        s.failover()
+    assert e.value.code == ops.NO_REPLICA
+    # failover skips dead servers in front of the first live one
+    s = ops.OraclePS(theta, chain_len=3, replicate_every=1)
+    _steps(s, 2, 90)
+    th1 = s.replicas[1]["theta"].copy()
+    s.kill(1); s.kill(0)
+    assert s.failover() == 1 and (s.head() == th1).all() and s.replicas == []
+
+
+def test_periodic_replication_rolls_back_to_the_last_replicated_version():
+    # R > 1: updates since the last replication event are lost with the frontend
+    theta = synth.init_params(1)
+    s = ops.OraclePS(theta, chain_len=2, replicate_every=4)
+    seen = {}
+    for t in range(7):
+        _steps(s, 1, 100 + t)
+        seen[s.version] = s.head().copy()
+    assert s.version == 7 and s.replicas[0]["version"] == 4
+    s.kill(0)
+    assert s.failover() == 4 and (s.head() == seen[4]).all()
+    _steps(s, 1, 200)
+    assert s.version == 5 and not (s.head() == seen[5]).all()      # a different fifth update than the lost one
+
+
+def test_checkpoint_slots_keep_the_most_recent_ones():
+    theta = synth.init_params(1)
+    s = ops.OraclePS(theta, ckpt_every=2, ckpt_slots=3)
+    kept = {}
+    for t in range(9):
+        _steps(s, 1, 300 + t)
+        if s.version % 2 == 0:
+            kept[s.version] = s.head().copy()
+    assert [v for v, _ in s.ckpts] == [4, 6, 8]                     # 2 was overwritten by 8
+    for v, th in s.ckpts:
+        assert (th == kept[v]).all()
+    s.kill(0)
+    assert s.restore() == 8 and (s.head() == kept[8]).all()
