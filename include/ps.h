@@ -81,7 +81,10 @@ typedef struct {
   int32_t  ckpt_every;       /* checkpoint when version % ckpt_every == 0; 0 = never          */
   int32_t  ckpt_slots;       /* pinned host checkpoint slots (oldest overwritten); >= 0       */
   int32_t  chain_len;        /* servers in the chain; 1 = no replica                           */
-  int32_t  replicate_every;  /* R: mirror versions with version % R == 0 to the replicas      */
+  int32_t  replicate_every;  /* R: versions with version % R == 0 are replication events: the next live server
+                              * receives that version; each server further down the chain holds what the one
+                              * in front of it held one event earlier (the frontend waits for the next server
+                              * only: design section on chain replication, relaxed consistency)              */
   int32_t  external_store;   /* 1 = stateless server: weights and queue survive ps_kill()     */
   int32_t  precision;        /* PS_FP32 | PS_TF32 | PS_BF16                                    */
   float    dropout_p;        /* dropout rate of the 512-unit layer, 0 <= p < 1                 */
@@ -103,11 +106,11 @@ int32_t ps_query_bytes(const ps_config* cfg, uint64_t* arena_bytes, uint64_t* pi
 int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** out);
 int32_t ps_destroy(ps_ctx* ctx);   /* synchronises the stream; frees host state only */
 
-/* ---- worker side (paper: the stateless_worker pseudo-code; "workers pull ... weights") ------ */
+/* ---- worker side (paper: the worker loop of the stateless-server pseudo-code figure) -------- */
 
 typedef struct { uint64_t version; const float* dev_ptr; } ps_snapshot;
 
-/* The worker's "get weights": version head - lag (lag 0 = latest).  No bytes move: dev_ptr is
+/* The worker's weight fetch (first step of the worker loop): version head - lag (lag 0 = latest).  No bytes move: dev_ptr is
  * borrowed from the version ring and stays valid until ring_depth further versions have been
  * produced or the server is killed/restored.  While a stateless server is down the stored
  * weights can still be pulled.  Errors: PS_ERR_DOWN, PS_ERR_VERSION_EVICTED, PS_ERR_BAD_ARG. */
@@ -121,7 +124,7 @@ int32_t ps_queue_reserve(ps_ctx* ctx, int32_t n, int64_t* slot_ids);
 /* Device address of a queue slot (PS_PARAM_STRIDE floats), borrowed. */
 int32_t ps_slot_ptr(ps_ctx* ctx, int64_t slot_id, float** dev_ptr_out);
 
-/* The worker's gradient computation ("trainer.apply(latest_weights)" in the pseudo-code) for W
+/* The worker's gradient computation (the training call of the pseudo-code figure's worker loop) for W
  * workers of batch b at once.  Worker w uses weights snaps[w].dev_ptr (workers sharing a pointer
  * are processed as one group), images x_dev[w] and labels y_dev[w], and the dropout mask of
  * Philox4x32-10 keyed by (seed, worker_ids[w], step): element (sample i, unit j) uses counter
@@ -147,7 +150,7 @@ int32_t workers_grad_step(ps_ctx* ctx, int32_t W, int32_t b, const ps_snapshot* 
 int32_t ps_dropout_mask(ps_ctx* ctx, uint64_t seed, int32_t worker_id, uint64_t step, int32_t b,
                         uint8_t* keep_dev);
 
-/* The worker's "append gradient": commits n gradients with their metadata.  With slot_ids (the
+/* The worker's gradient append (last step of the worker loop): commits n gradients with their metadata.  With slot_ids (the
  * slots of the current reservation, in order) nothing is copied; with slot_ids == NULL the rows
  * of grads_dev ([n][PS_PARAM_STRIDE], dev) are copied into the next n slots.  All enqueue calls
  * between two applies must carry the same n (it is the per-tick worker count that PS_REPLAY
@@ -165,10 +168,10 @@ typedef struct {
 } ps_apply_result;
 
 /* One server step over the whole queue (K gradients), which is then emptied.
- *   PS_SYNC   ("applies all updates ... at once"):      theta <- theta - lr*scale/K      * sum g ; version+1
+ *   PS_SYNC   (synchronous training, implementation section): theta <- theta - lr*scale/K * sum g ; version+1
  *   PS_REPLAY (stateless step: get all gradients, apply, put): theta - lr*scale/W_tick * sum g ; version+1
  *             where W_tick is the n of the enqueue calls (one tick's replay equals the sync step)
- *   PS_ASYNC  ("as soon as it receives any worker gradient"): for k in order: theta <- theta - lr*scale*g_k,
+ *   PS_ASYNC  (asynchronous training: one update per arriving gradient): for k in order: theta <- theta - lr*scale*g_k,
  *             version+1 each; the last ring_depth versions stay readable by stale workers
  * order (host, [K]) is a permutation of the queue positions giving the arrival order for
  * PS_ASYNC (NULL = FIFO); the other modes sum, so they ignore it.  Versions that are multiples of
@@ -177,25 +180,27 @@ typedef struct {
 int32_t ps_apply(ps_ctx* ctx, ps_mode mode, float lr, float scale, const int32_t* order,
                  ps_apply_result* out);
 
-/* "saves a checkpoint of parameters to persistent storage": copies the head weights and version
- * into the next pinned host slot (stream-ordered device-to-host copy). */
+/* The periodic save of the parameters to persistent storage (design section on checkpointing): copies the
+ * head weights and version into the next pinned host slot (stream-ordered device-to-host copy); when all slots
+ * are in use the oldest checkpoint is overwritten. */
 int32_t ps_checkpoint(ps_ctx* ctx, uint64_t* version_out);
 
-/* Resurrects the server.  Stateful: "look for the latest checkpoint ... and continue from that
- * older state": weights and version are the checkpoint's, the queue is empty, only that version
+/* Resurrects the server.  Stateful (design section on checkpointing: a restarted server resumes from its latest
+ * checkpoint): weights and version are the checkpoint's, the queue is empty, only that version
  * is retained.  Stateless: the store survived, nothing is rolled back.  PS_ERR_NO_CHECKPOINT. */
 int32_t ps_restore(ps_ctx* ctx, uint64_t* version_out);
 
-/* Explicit head -> replica copy (the periodic replication step on its own). PS_ERR_NO_REPLICA. */
+/* One replication event on its own: the head's weights go to the next live server, and what each server held
+ * moves one server further down the chain (see ps_config.replicate_every). PS_ERR_NO_REPLICA. */
 int32_t ps_replicate(ps_ctx* ctx, uint64_t* version_out);
 
-/* Host-side failure injection: server 0 is the current frontend, i >= 1 the i-th server behind
- * it.  Killing a stateful frontend loses its weights, retained versions and queue; no device
+/* Host-side failure injection: server 0 is the current frontend, i >= 1 the i-th LIVE server behind
+ * it (a dead server has left the chain).  Killing a stateful frontend loses its weights, retained versions and queue; no device
  * fault is provoked. */
 int32_t ps_kill(ps_ctx* ctx, int32_t server);
 
-/* The next live server of the chain becomes the frontend with the weights it has "warm in
- * memory" (its last mirrored version); the queue is empty.  PS_ERR_NO_REPLICA. */
+/* The next live server of the chain becomes the frontend with the weights it already holds in memory (the
+ * version it last received); the queue is empty.  PS_ERR_NO_REPLICA. */
 int32_t ps_failover(ps_ctx* ctx, uint64_t* version_out);
 
 /* Replaces the head weights (host, canonical order) without changing the version; used to load a
@@ -248,6 +253,15 @@ int32_t ps_tick_host_submit(ps_ctx* ctx, int32_t W, int32_t b, const int32_t* la
                             int32_t* argmax_host);
 int32_t ps_tick_host_wait(ps_ctx* ctx, ps_apply_result* out);
 
+/* Exercises the give-up path of the library's bounded waits without disturbing anything (no counterpart in the
+ * paper's method; it serves failure detection).  Every wait of the tensor-core kernels on a barrier has a cycle
+ * limit; when it runs out the kernel sets bit 1 of the status word, releases what it holds and returns, and
+ * ps_stats() then reports PS_ERR_DEVICE_STATUS.  This call launches, on the context's stream, one warp that waits on
+ * a barrier of its own at which nobody arrives, for at most limit_cycles SM clock cycles (1..2e9; 20,000 is about
+ * 10 microseconds), and then does exactly that.  Nothing else is touched; the context stays usable, but its status
+ * word keeps the bit until the context is destroyed. */
+int32_t ps_selftest_wait_timeout(ps_ctx* ctx, int64_t limit_cycles);
+
 /* Per-kernel timing for measurement (no counterpart in the paper's method; it serves the roofline
  * report).  ps_profile(ctx, 1) clears the totals and from then on brackets every kernel launch with
  * two CUDA events on the context's stream (and runs the branches of the backward pass one after the
@@ -272,12 +286,17 @@ int32_t ps_profile_read(ps_ctx* ctx, int32_t kernel, const char** name, double* 
  * enqueued on `stream` (a cudaStream_t, NULL = legacy default stream) of the current device.
  *
  * The partial sums are kept in a fixed array inside the library image: PS_STATIC_REPLAY_SPLITS
- * vectors of PS_PARAM_STRIDE floats, about 13 MB, resident on every GPU that loads the library
- * for as long as the process lives.  The entry point calls no allocator, CUDA's or anyone
- * else's.  The first call on each device looks up that array's device address; make that first
- * call before starting any stream capture.  All calls on a device share the one array and it is
- * not cleared between calls (each call overwrites every element it later reads), so two calls
- * whose kernels may overlap on the GPU, e.g. on different streams, race: serialise them.
+ * vectors of PS_PARAM_STRIDE floats, about 13 MB per GPU, held until the process exits.  The entry
+ * point calls no allocator, CUDA's or anyone else's.
+ *
+ * The first call on each device is a set-up call: it looks up the array's device address, and because
+ * CUDA loads a library's device code lazily, that lookup is also the moment the driver sets the array
+ * up on that device (13 MB; it can take as long as an allocation would, and on a device whose memory is
+ * all taken it fails: PS_ERR_CUDA with a text that says so).  So make one warm-up call per device at
+ * start-up, before the application's pool takes the memory and before any stream capture; later calls
+ * only launch two kernels.  All calls on a device share the one array and it is not cleared between
+ * calls (each call overwrites every element it later reads), so two calls whose kernels may overlap on
+ * the GPU, e.g. on different streams, race: serialise them.
  * ps_replay_sum_static_error() returns the text of the calling thread's last failure here. */
 #define PS_STATIC_REPLAY_SPLITS 4
 #define PS_STATIC_REPLAY_MAX_GRADIENTS 65536

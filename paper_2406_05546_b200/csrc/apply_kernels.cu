@@ -46,9 +46,10 @@ __device__ __forceinline__ float4 column_sum(const float4* __restrict__ q, int64
 
 // theta_out = theta_in - coef * sum_k g_k, whole queue in one pass (small K).
 __global__ void __launch_bounds__(TPB) sum_apply_direct(const float4* __restrict__ queue, int64_t K,
-                                                        const float4* __restrict__ theta_in,
-                                                        float4* __restrict__ theta_out,
+                                                        const float4* theta_in, float4* theta_out,
                                                         float4* __restrict__ replica, float coef) {
+  // theta_in and theta_out may be the same buffer (a ring of depth one): each thread reads its column before it
+  // writes it, and the two pointers carry no no-alias promise
   int col = blockIdx.x * TPB + threadIdx.x;
   if (col >= P_VEC4) return;
   float4 s = column_sum(queue + col, 0, K);
@@ -73,8 +74,7 @@ __global__ void __launch_bounds__(TPB) sum_partial(const float4* __restrict__ qu
 
 // Stage 2: sums the partials in slot order and applies the update.
 __global__ void __launch_bounds__(TPB) sum_finish(const float4* __restrict__ partial, int n_split,
-                                                  const float4* __restrict__ theta_in,
-                                                  float4* __restrict__ theta_out,
+                                                  const float4* theta_in, float4* theta_out,   // may alias (see above)
                                                   float4* __restrict__ replica, float coef) {
   int col = blockIdx.x * TPB + threadIdx.x;
   if (col >= P_VEC4) return;
@@ -111,7 +111,8 @@ __global__ void __launch_bounds__(TPB) async_apply(AsyncApplyArgs a, AsyncOrder 
           int slot = (int)((a.v0 + (uint64_t)k + 1) % (uint64_t)a.ring_depth);
           reinterpret_cast<float4*>(a.ring[slot])[col] = t;
         }
-        if (k == a.mirror_k) reinterpret_cast<float4*>(a.replica)[col] = t;
+        for (int m = 0; m < a.n_mirror; ++m)
+          if (k == a.mirror_k[m]) reinterpret_cast<float4*>(a.replica[m])[col] = t;
       }
     }
   }

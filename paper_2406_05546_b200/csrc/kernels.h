@@ -13,6 +13,7 @@ constexpr int P_VEC4 = P_PAD / 4;      // 203,328 float4 columns
 constexpr int MAX_WORKERS = 256;
 constexpr int MAX_RING = 16;
 constexpr int MAX_GROUPS = 16;
+constexpr int MAX_CHAIN = 8;           // servers in a replication chain, the frontend included
 
 constexpr int OFF_C1W = 0, OFF_C1B = 144, OFF_C2W = 160, OFF_C2B = 4768;
 constexpr int OFF_F1W = 4800, OFF_F1B = 807616, OFF_F2W = 808128, OFF_F2B = 813248;
@@ -183,12 +184,16 @@ struct AsyncApplyArgs {
   int ring_depth;
   uint64_t v0;              // version of theta_in; version v0+k+1 is stored in ring[(v0+k+1) % depth]
   int first_stored;         // only k >= first_stored are stored (the last ring_depth versions)
-  int mirror_k;             // k whose result is also written to replica, or -1
-  float* replica;
+  int n_mirror;             // chain-replication stores of this segment (at most one per server behind the frontend)
+  int mirror_k[MAX_CHAIN];  // k whose result is also written to replica[m]
+  float* replica[MAX_CHAIN];
   float coef;               // lr*scale
 };
 int launch_async_apply(const AsyncApplyArgs& a, const AsyncOrder& ord, cudaStream_t st, Profiler* prof);
 
 int launch_copy_rows(float* dst, const float* src, int64_t rows, cudaStream_t st, Profiler* prof);
+
+// One warp waits on a barrier nobody arrives at, for at most limit_cycles, then sets STATUS_WAIT_TIMEOUT in *status.
+int launch_wait_timeout_probe(uint32_t* status, long long limit_cycles, cudaStream_t st);
 
 }  // namespace psk

@@ -204,17 +204,28 @@ int32_t do_checkpoint(ps_ctx* x) {
   return PS_OK;
 }
 
-// Copies the first live replica's fresh contents to the other live replicas (chains longer than 2).
-int32_t propagate_chain(ps_ctx* x, uint64_t version) {
-  Replica* first = first_live(x);
-  if (!first) return PS_OK;
-  first->version = version;
-  for (auto& r : x->replicas) {
-    if (!r.alive || &r == first) continue;
-    CUDA_TRY(cudaMemcpyAsync(r.buf, first->buf, VEC_BYTES, cudaMemcpyDeviceToDevice, x->st));
-    r.version = version;
+// Chain replication with relaxed consistency (paper, design section on chain-replicated servers): at a replication
+// event the frontend hands its weights to the next live server and waits for that server only; the hop to the server
+// behind it completes with the following event.  After `events` events the i-th live server behind the frontend
+// (i = 0 first) therefore holds the version replicated i events before the latest one.  This routine does the part
+// that moves existing contents down the chain, on the stream and BEFORE the kernel (or copy) that writes the
+// newest versions: server i takes what server i - events held.  Servers i < events are written by the caller, which
+// sets their versions with set_replica_versions().
+int32_t shift_chain(ps_ctx* x, int events) {
+  std::vector<Replica*> live;
+  for (auto& r : x->replicas) if (r.alive) live.push_back(&r);
+  for (int i = (int)live.size() - 1; i >= events; --i) {
+    CUDA_TRY(cudaMemcpyAsync(live[i]->buf, live[i - events]->buf, VEC_BYTES, cudaMemcpyDeviceToDevice, x->st));
+    live[i]->version = live[i - events]->version;
   }
   return PS_OK;
+}
+
+// The live servers behind the frontend, nearest first.
+std::vector<Replica*> live_chain(ps_ctx* x) {
+  std::vector<Replica*> live;
+  for (auto& r : x->replicas) if (r.alive) live.push_back(&r);
+  return live;
 }
 
 }  // namespace
@@ -425,10 +436,12 @@ int32_t ps_replicate(ps_ctx* x, uint64_t* version_out) {
   if (!x->up || x->weights_lost) return fail(PS_ERR_DOWN, "server is down");
   Replica* r = first_live(x);
   if (!r) return fail(PS_ERR_NO_REPLICA, "no live replica");
+  int32_t rc = shift_chain(x, 1);
+  if (rc != PS_OK) return rc;
   CUDA_TRY(cudaMemcpyAsync(r->buf, head(x), VEC_BYTES, cudaMemcpyDeviceToDevice, x->st));
-  int32_t rc = propagate_chain(x, x->version);
-  if (rc == PS_OK && version_out) *version_out = x->version;
-  return rc;
+  r->version = x->version;
+  if (version_out) *version_out = x->version;
+  return PS_OK;
 }
 
 int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* order, ps_apply_result* out) {
@@ -455,6 +468,7 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
     a.theta_in = head(x);
     a.theta_out = x->ring[(x->version + 1) % depth];
     const bool mirror = rep && ((x->version + 1) % R == 0);
+    if (mirror) { int32_t rc = shift_chain(x, 1); if (rc != PS_OK) return rc; }
     a.replica = mirror ? rep->buf : nullptr;
     a.coef = lr * scale / (float)(mode == PS_SYNC ? K : (int64_t)x->w_tick);
     a.partial = x->partial; a.max_split = MAX_SPLIT;
@@ -464,7 +478,7 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
     x->version += 1;
     x->weights_epoch++;
     advance_oldest(x);
-    if (mirror) { int32_t rc = propagate_chain(x, x->version); if (rc != PS_OK) return rc; res.replicated = 1; }
+    if (mirror) { rep->version = x->version; res.replicated = 1; }
     if (x->cfg.ckpt_every > 0 && x->version % (uint64_t)x->cfg.ckpt_every == 0) {
       int32_t rc = do_checkpoint(x); if (rc != PS_OK) return rc; res.checkpointed = 1;
     }
@@ -485,15 +499,24 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
       for (int i = 0; i < psk::MAX_RING; ++i) a.ring[i] = i < x->cfg.ring_depth ? x->ring[i] : nullptr;
       a.ring_depth = x->cfg.ring_depth; a.v0 = x->version;
       a.first_stored = (int)std::max<int64_t>(0, seg - (int64_t)depth);
-      a.mirror_k = -1; a.replica = nullptr; a.coef = lr * scale;
-      uint64_t mirrored = 0;
+      a.n_mirror = 0; a.coef = lr * scale;
       if (rep) {
-        uint64_t last = (x->version + (uint64_t)seg) / R * R;
-        if (last > x->version) {
-          a.mirror_k = (int)(last - x->version - 1);
-          a.replica = rep->buf;
-          mirrored = last;
-          res.replicated += (int32_t)((x->version + (uint64_t)seg) / R - x->version / R);
+        // replication events inside this segment: versions that are multiples of R.  The i-th live server behind
+        // the frontend receives the version of the i-th latest event if that version is produced here; what the
+        // servers further down receive comes from the servers in front of them (shift_chain, before the launch).
+        const uint64_t last = (x->version + (uint64_t)seg) / R * R;
+        const int events = (int)((x->version + (uint64_t)seg) / R - x->version / R);
+        if (events > 0) {
+          int32_t rc = shift_chain(x, events); if (rc != PS_OK) return rc;
+          std::vector<Replica*> live = live_chain(x);
+          for (int i = 0; i < (int)live.size() && i < events; ++i) {
+            const uint64_t v = last - (uint64_t)i * R;
+            a.mirror_k[a.n_mirror] = (int)(v - x->version - 1);
+            a.replica[a.n_mirror] = live[i]->buf;
+            ++a.n_mirror;
+            live[i]->version = v;
+          }
+          res.replicated += events;
         }
       }
       for (int64_t u = 0; u < seg; ++u) ord.slot[u] = order ? order[pos + u] : (int32_t)(pos + u);
@@ -503,7 +526,6 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
       x->version += (uint64_t)seg;
       x->weights_epoch++;
       advance_oldest(x);
-      if (mirrored) { int32_t rc = propagate_chain(x, mirrored); if (rc != PS_OK) return rc; }
       if (x->cfg.ckpt_every > 0 && x->version % (uint64_t)x->cfg.ckpt_every == 0) {
         int32_t rc = do_checkpoint(x); if (rc != PS_OK) return rc; res.checkpointed += 1;
       }
@@ -638,6 +660,15 @@ int32_t ps_stats(ps_ctx* x, ps_stats_t* out) {
   out->last_ckpt_version = x->ckpt_order.empty() ? 0 : x->ckpt_version[x->ckpt_order.back()];
   out->kernel_launches = x->launches;
   if (out->device_status != 0) return fail(PS_ERR_DEVICE_STATUS, "device status 0x%x (bit 0: label outside 0..9; bit 1: a bounded wait in a tensor-core kernel gave up)", out->device_status);
+  return PS_OK;
+}
+
+int32_t ps_selftest_wait_timeout(ps_ctx* x, int64_t limit_cycles) {
+  if (!x) return fail(PS_ERR_BAD_ARG, "ctx is NULL");
+  if (limit_cycles < 1 || limit_cycles > 2000000000ll) return fail(PS_ERR_BAD_ARG, "limit_cycles must be 1..2e9");
+  int n = psk::launch_wait_timeout_probe(x->status_dev, (long long)limit_cycles, x->st);
+  if (n < 0) return cuda_fail(cudaGetLastError(), "probe launch");
+  x->launches += n;
   return PS_OK;
 }
 

@@ -31,7 +31,7 @@ static __device__ __align__(256) float g_static_partials[(size_t)SPLITS * psk::P
 // once per device and remembered here.
 float* g_partials_addr[MAX_DEVICES] = {nullptr};
 std::mutex g_setup_mutex;
-thread_local char g_static_err[256] = "";
+thread_local char g_static_err[320] = "";
 
 __device__ __forceinline__ void add4(float4& a, const float4& b) {
   a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
@@ -69,8 +69,8 @@ __global__ void __launch_bounds__(TPB) static_partial(const float4* __restrict__
 }
 
 __global__ void __launch_bounds__(TPB) static_finish(const float4* __restrict__ partial,
-                                                     const float4* __restrict__ theta_in,
-                                                     float4* __restrict__ theta_out, float coef) {
+                                                     const float4* theta_in, float4* theta_out,   // may be one buffer
+                                                     float coef) {
   const int col = blockIdx.x * TPB + threadIdx.x;
   if (col >= psk::P_VEC4) return;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -111,7 +111,15 @@ int32_t ps_replay_sum_static(const float* queue_dev, int64_t K, const float* the
     std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (!g_partials_addr[dev]) {
       void* p = nullptr;
+      // With lazy module loading (the CUDA 12 default) this lookup is what brings the array into being on this
+      // device: the driver reserves its 13 MB now.  A device whose memory is already taken fails here, not later.
       e = cudaGetSymbolAddress(&p, g_static_partials);
+      if (e == cudaErrorMemoryAllocation) {
+        cudaGetLastError();
+        return static_fail(PS_ERR_CUDA, "the first call on this device could not place the library's 13 MB scratch array: "
+                                        "the device is out of memory.  Make one warm-up call at start-up, before the "
+                                        "application's pool takes the memory");
+      }
       if (e != cudaSuccess) return static_fail(PS_ERR_CUDA, "cudaGetSymbolAddress: ", cudaGetErrorString(e));
       g_partials_addr[dev] = static_cast<float*>(p);
     }

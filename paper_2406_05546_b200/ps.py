@@ -24,7 +24,7 @@ EXPORTS = ["ps_query_bytes", "ps_create", "ps_destroy", "ps_pull_snapshot", "ps_
            "workers_grad_step", "ps_dropout_mask", "ps_enqueue", "ps_apply", "ps_checkpoint", "ps_restore", "ps_replicate",
            "ps_kill", "ps_failover", "ps_import_params", "ps_export_params", "ps_stats", "ps_tick_host",
            "ps_tick_host_submit", "ps_tick_host_wait",
-           "ps_profile", "ps_profile_read", "ps_last_error", "ps_replay_sum_static", "ps_replay_sum_static_error"]
+           "ps_profile", "ps_profile_read", "ps_selftest_wait_timeout", "ps_last_error", "ps_replay_sum_static", "ps_replay_sum_static_error"]
 
 
 class PSError(RuntimeError):
@@ -93,6 +93,7 @@ def load(path=None):
         "ps_tick_host_wait": [vp, C.POINTER(ApplyResult)],
     }
     sig["ps_profile"] = [vp, i32]
+    sig["ps_selftest_wait_timeout"] = [vp, i64]
     sig["ps_profile_read"] = [vp, i32, C.POINTER(C.c_char_p), C.POINTER(C.c_double), C.POINTER(i64)]
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -318,6 +319,9 @@ class ParameterServer:
             self._inflight.pop(0)
         return {"applied": res.applied, "new_version": res.new_version,
                 "checkpointed": res.checkpointed, "replicated": res.replicated}
+
+    def ps_selftest_wait_timeout(self, limit_cycles=20000):
+        self._check(self.lib.ps_selftest_wait_timeout(self.ctx, int(limit_cycles)))
 
     def ps_profile(self, enable):
         self._check(self.lib.ps_profile(self.ctx, int(bool(enable))))

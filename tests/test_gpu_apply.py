@@ -241,3 +241,165 @@ def test_async_checkpoint_mid_apply_and_errors():
         g.ps_apply(ps.ASYNC, 0.01, order=[0, 0, 1, 2, 3, 4, 5, 6])
     assert e.value.name == "PS_ERR_BAD_ARG"
     g.close()
+
+
+def _steps(o, g, ops, ps, n, seed0, W=2, mode=None):
+    for t in range(n):
+        _both_enqueue(o, g, synth.random_gradients(W, seed=seed0 + t), step=t)
+        assert o.apply(ops.SYNC if mode is None else mode, 0.01) == g.ps_apply(ps.SYNC if mode is None else mode, 0.01)
+
+
+def _chain_matches(o, g, what):
+    live = [r for r in o.replicas if r["alive"]]
+    assert g.ps_stats()["live_replicas"] == len(live)
+    for i, r in enumerate(live):
+        th, v = g.ps_export_params(-(i + 1))
+        assert v == r["version"], (what, i)
+        assert_params_close(th, r["theta"], TOL_APPLY, f"{what}: server {i + 1} behind the frontend")
+
+
+def test_chain_of_three_double_failure():
+    """Frontend and secondary die; the tertiary, one replication event behind, takes over (design section on chain
+    replication).  Sync and async applies, R = 2."""
+    for mode_name in ("SYNC", "ASYNC"):
+        ops, ps, o, g = _pair(queue_slots=8, ring_depth=4, chain_len=3, replicate_every=2)
+        mode_o, mode_g = getattr(ops, mode_name), getattr(ps, mode_name)
+        for t in range(5):
+            W = 1 if mode_name == "SYNC" else [1, 3, 2, 1, 2][t]
+            _both_enqueue(o, g, synth.random_gradients(W, seed=40 + t), step=t)
+            assert o.apply(mode_o, 0.01) == g.ps_apply(mode_g, 0.01)
+            _chain_matches(o, g, f"{mode_name} step {t}")
+        o.kill(0); g.ps_kill(0)
+        o.kill(1); g.ps_kill(1)
+        v = o.failover()
+        assert g.ps_failover() == v and o.replicas == []
+        th, vg = g.ps_export_params()
+        assert vg == v
+        assert_params_close(th, o.head(), TOL_APPLY, "tertiary's weights")
+        st = g.ps_stats()
+        assert st["live_replicas"] == 0 and st["version"] == st["oldest_version"] == v and st["up"] == 1
+        _steps(o, g, ops, ps, 1, 60)
+        assert_params_close(g.ps_export_params()[0], o.head(), TOL_APPLY, "after the double failure")
+        g.ps_kill(0)
+        with pytest.raises(ps.PSError) as e:
+            g.ps_failover()
+        assert e.value.name == "PS_ERR_NO_REPLICA"
+        g.close()
+
+
+def test_async_segment_with_many_replication_events_fills_the_chain():
+    # R = 1 and a 20-gradient ordered apply: 20 events in one launch; the servers behind the frontend end up with the
+    # last, the one before last and the one before that
+    ops, ps, o, g = _pair(queue_slots=32, ring_depth=9, chain_len=4, replicate_every=1, max_workers=32)
+    for tick, K in enumerate([20, 2, 1]):
+        grads = synth.random_gradients(K, seed=70 + tick)
+        _both_enqueue(o, g, grads, step=tick)
+        order = synth.arrival_order(tick, K)
+        assert o.apply(ops.ASYNC, 0.01, order=order) == g.ps_apply(ps.ASYNC, 0.01, order=order)
+        assert [r["version"] for r in o.replicas] == [o.version, o.version - 1, o.version - 2]
+        _chain_matches(o, g, f"tick {tick}")
+    g.close()
+
+
+def test_killing_a_server_behind_the_frontend():
+    ops, ps, o, g = _pair(queue_slots=4, chain_len=4, replicate_every=1)
+    _steps(o, g, ops, ps, 3, 70)
+    o.kill(2); g.ps_kill(2)
+    _steps(o, g, ops, ps, 1, 80)
+    assert [r["version"] for r in o.replicas if r["alive"]] == [4, 3]
+    _chain_matches(o, g, "after the middle server died")
+    o.kill(2); g.ps_kill(2)
+    with pytest.raises(ps.PSError) as e:
+        g.ps_kill(2)
+    assert e.value.name == "PS_ERR_BAD_ARG"
+    with pytest.raises(ops.PSError):
+        o.kill(2)
+    _steps(o, g, ops, ps, 1, 90)
+    _chain_matches(o, g, "one server left behind the frontend")
+    g.close()
+    # failover skips dead servers in front of the first live one
+    ops, ps, o, g = _pair(queue_slots=4, chain_len=3, replicate_every=1)
+    _steps(o, g, ops, ps, 2, 90)
+    for srv in (1, 0):
+        o.kill(srv); g.ps_kill(srv)
+    assert o.failover() == g.ps_failover() == 1
+    assert_params_close(g.ps_export_params()[0], o.head(), TOL_APPLY, "the last server's weights")
+    g.close()
+
+
+def test_periodic_replication_rollback_to_last_replicated_version():
+    ops, ps, o, g = _pair(queue_slots=4, chain_len=2, replicate_every=4)
+    _steps(o, g, ops, ps, 7, 100)
+    o.kill(0); g.ps_kill(0)
+    assert o.failover() == g.ps_failover() == 4
+    assert_params_close(g.ps_export_params()[0], o.head(), TOL_APPLY, "rolled back to version 4")
+    _steps(o, g, ops, ps, 2, 200)
+    assert g.ps_stats()["version"] == o.version == 6
+    assert_params_close(g.ps_export_params()[0], o.head(), TOL_APPLY, "after the rollback")
+    g.close()
+
+
+def test_checkpoint_slots_keep_the_most_recent_ones():
+    ops, ps, o, g = _pair(queue_slots=4, ckpt_every=2, ckpt_slots=3)
+    heads = {}
+    for t in range(9):
+        _steps(o, g, ops, ps, 1, 300 + t)
+        heads[o.version] = g.ps_export_params()[0]
+    assert [v for v, _ in o.ckpts] == [4, 6, 8]
+    st = g.ps_stats()
+    assert st["checkpoints"] == 3 and st["last_ckpt_version"] == 8
+    for j, v in enumerate([8, 6, 4]):
+        th, vg = g.ps_export_params(1000 + j)
+        assert vg == v and (th == heads[v]).all()
+    with pytest.raises(ps.PSError) as e:
+        g.ps_export_params(1003)
+    assert e.value.name == "PS_ERR_NO_CHECKPOINT"
+    o.kill(0); g.ps_kill(0)
+    assert o.restore() == g.ps_restore() == 8
+    assert (g.ps_export_params()[0] == heads[8]).all()
+    g.close()
+
+
+@pytest.mark.parametrize("K", [5, 300])
+def test_apply_in_place_with_a_ring_of_depth_one(K):
+    # ring_depth 1 (the benchmark's configuration): the new head overwrites the old one in the same buffer
+    ops, ps, o, g = _pair(queue_slots=K, ring_depth=1, external_store=True, max_workers=8)
+    grads = synth.random_gradients(K, seed=11)
+    o.enqueue(grads, range(K), [0] * K, 0)
+    g.ps_enqueue(list(range(K)), [0] * K, 0, grads_dev=_pad(grads))
+    assert o.apply(ops.REPLAY, 0.01, scale=1.0 / 8) == g.ps_apply(ps.REPLAY, 0.01, scale=1.0 / 8)
+    assert_params_close(g.ps_export_params()[0], o.head(), TOL_APPLY, "in-place apply")
+    g.close()
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_nothing_hangs():
+    """The give-up path of the tensor-core kernels' waits: a probe kernel waits about 10 microseconds on a barrier
+    nobody arrives at, records the time-out in the status word and returns; ps_stats reports it; the device and a
+    fresh context work as before."""
+    import torch
+    ops, ps, o, g = _pair(queue_slots=4)
+    assert g.ps_stats()["device_status"] == 0
+    g.ps_selftest_wait_timeout(20000)
+    with pytest.raises(ps.PSError) as e:
+        g.ps_stats()
+    assert e.value.name == "PS_ERR_DEVICE_STATUS"
+    assert g.ps_stats(check=False)["device_status"] == 2
+    with pytest.raises(ps.PSError) as e:
+        g.ps_selftest_wait_timeout(0)
+    assert e.value.name == "PS_ERR_BAD_ARG"
+    # the context still computes (its status word keeps the flag) ...
+    _both_enqueue(o, g, synth.random_gradients(2, seed=1))
+    assert o.apply(ops.SYNC, 0.01) == g.ps_apply(ps.SYNC, 0.01)
+    assert_params_close(g.ps_export_params()[0], o.head(), TOL_APPLY, "apply after the probe")
+    g.close()
+    # ... and a fresh context runs a tensor-core tick with a clean status
+    theta = synth.init_params(1)
+    srv = ps.ParameterServer(theta, max_workers=2, max_batch=4, queue_slots=2, precision=ps.BF16)
+    rng = np.random.default_rng(0)
+    x = rng.random((2, 4, 28, 28), dtype=np.float32)
+    y = rng.integers(0, 10, (2, 4)).astype(np.int32)
+    loss, res = srv.ps_tick_host(x, y, 0x5EED, 0, ps.SYNC, 0.01)
+    st = srv.ps_stats()
+    assert st["device_status"] == 0 and st["version"] == 1 and np.isfinite(loss).all()
+    srv.close()
+    torch.cuda.synchronize()

@@ -177,3 +177,183 @@ def test_full_size_replay_of_25600_gradients_on_sampled_columns():
     assert np.abs(step_g - step_o).max() <= 2e-3 * np.abs(step_o).max()
     assert (th != theta).mean() > 0.99      # the whole vector moved, not only the sampled columns
     srv.close()
+
+
+# ---- configurations 2, 3 and 4 at their stated sizes: one whole tick, every worker against the oracle -------------
+
+def _advance_both(srv, o, n, seed0, mode_g, mode_o, scale=2.0):
+    """n server updates from seeded synthetic gradients on both sides (no CNN involved), one gradient each."""
+    import torch
+    from paper_2406_05546_b200 import ps
+    for k in range(n):
+        g = np.zeros((1, ps.P_PAD), dtype=np.float32)
+        g[0, :ps.P] = synth.random_gradients(1, seed=seed0 + k, scale=scale)[0]
+        srv.ps_enqueue([0], [o.version], 0, grads_dev=torch.from_numpy(g).cuda())
+        o.enqueue(g[:, :ps.P], [0], [o.version], 0)
+        assert srv.ps_apply(mode_g, 0.01) == o.apply(mode_o, 0.01)
+
+
+def _full_size_tick(n, precision, t, srv, o, lags=None):
+    """Grad step of every worker of configuration n at tick t into reserved slots, on the GPU and on the oracle (each
+    side from its own weights and its own gradients), enqueue on both.  Returns (schedule, gpu gradients, oracle
+    gradients, slots)."""
+    import torch
+    from oracle import cnn
+    from paper_2406_05546_b200 import ps
+    from tests.parity import assert_params_close_up_to_unit_flips, tensor_rel_errors
+    s = schedules.config(n)
+    tol = TOL_TENSOR if precision else TOL_FP32
+    px, py = synth.image_pool(synth.POOL_IMAGES, seed=0)
+    x, y = synth.tick_batch(px, py, t, s.W, s.b)
+    lags = [0] * s.W if lags is None else [int(l) for l in lags]
+    ids = list(range(s.W))
+    snaps = [srv.ps_pull_snapshot(w, lags[w]) for w in range(s.W)]
+    pulled = [o.pull_snapshot(w, lags[w]) for w in range(s.W)]
+    assert [sn.version for sn in snaps] == [v for v, _ in pulled]
+    slots = srv.ps_queue_reserve(s.W)
+    loss, am = srv.workers_grad_step(snaps, ids, torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(), s.seed, t,
+                                     slot_ids=slots)
+    srv.ps_stats()
+    gg = torch.stack([srv.slot_tensor(sl) for sl in slots]).cpu().numpy()
+    og, ol, oa, oz = cnn.workers_grad_step([th for _, th in pulled], ids, x, y, s.seed, t, s.dropout_p, precision=precision)
+    n_flipped = 0
+    for w in range(s.W):
+        assert (gg[w, ps.P:] == 0).all()
+        errs = tensor_rel_errors(gg[w, :ps.P], og[w])
+        if precision and max(errs.values()) > tol:
+            diag = cnn.worker_grad_step_diag(pulled[w][1], w, x[w], y[w], s.seed, t, s.dropout_p, precision)[4]
+            n_flipped += len(assert_params_close_up_to_unit_flips(gg[w, :ps.P], og[w], tol, pulled[w][1], diag,
+                                                                  f"config {n} worker {w}"))
+        else:
+            assert_params_close(gg[w, :ps.P], og[w], tol, f"config {n} worker {w}")
+    if n_flipped:
+        print(f"config {n}: {n_flipped} hidden units decided differently within the rounding bound of zero")
+    np.testing.assert_allclose(loss.cpu().numpy(), ol, rtol=3e-3 if precision else 1e-5, atol=1e-6)
+    assert_argmax_valid(am.cpu().numpy(), oz, tol)
+    srv.ps_enqueue(ids, [sn.version for sn in snaps], t, slot_ids=slots)
+    o.enqueue(og.astype(np.float32), ids, [v for v, _ in pulled], t)
+    return s, gg, og, slots
+
+
+def _assert_update_close(th_g, th_o, before, tol, what):
+    """Parameters within the apply tolerance, and the step taken (which the parameters' size would hide) within the
+    gradient tolerance, per tensor."""
+    assert_params_close(th_g, th_o, 1e-5, what)
+    assert_params_close(th_g.astype(np.float64) - before, th_o.astype(np.float64) - before, tol, what + " (the step)")
+
+
+@pytest.mark.parametrize("precision", [0, 2])
+def test_full_size_config2_tick_checkpoint_and_rollback(precision):
+    """W=8 x b=64, sync server with a checkpoint every 25 updates: the tick that produces version 25 at full size,
+    the checkpoint it triggers, a kill, and the restore from that checkpoint, byte for byte."""
+    from paper_2406_05546_b200 import harness, ps
+    s = schedules.config(2)
+    theta = synth.init_params(1)
+    srv = harness.make_server(s, theta, precision=precision)
+    o = oracle_driver.make_oracle(s, theta)
+    _advance_both(srv, o, 24, 500, ps.SYNC, schedules.SYNC, scale=0.05)
+    before = o.head().astype(np.float64)
+    _full_size_tick(2, precision, 24, srv, o)
+    rg, ro = srv.ps_apply(ps.SYNC, s.lr), o.apply(schedules.SYNC, s.lr)
+    assert rg == ro and rg["new_version"] == 25 and rg["checkpointed"] == 1 and rg["applied"] == 8
+    head, v = srv.ps_export_params()
+    _assert_update_close(head, o.head(), before, max(TOL_TENSOR if precision else TOL_FP32, 1e-3), "config 2 sync step")
+    ck, vc = srv.ps_export_params(1000)
+    assert vc == 25 and (ck == head).all()
+    _advance_both(srv, o, 3, 600, ps.SYNC, schedules.SYNC, scale=0.05)      # versions 26..28 are lost with the server
+    srv.ps_kill(); o.kill()
+    with pytest.raises(ps.PSError):
+        srv.ps_pull_snapshot(0)
+    assert srv.ps_restore() == o.restore() == 25
+    th, v = srv.ps_export_params()
+    assert v == 25 and (th == ck).all()
+    st = srv.ps_stats()
+    assert st["queue_len"] == 0 and st["oldest_version"] == 25 and st["last_ckpt_version"] == 25
+    srv.close()
+
+
+@pytest.mark.parametrize("precision", [0, 2])
+def test_full_size_config3_tick_and_replay_of_1600_gradients(precision):
+    """W=16 x b=64, stateless server: one full-size tick (every worker against the oracle, replay of one tick = the
+    sync step), then the 100-tick outage: 1,600 buffered gradients (5.2 GB) replayed in one pass, compared with the
+    oracle on sampled parameter columns."""
+    import torch
+    from oracle import ps as ops
+    from paper_2406_05546_b200 import harness, ps
+    s = schedules.config(3)
+    theta = synth.init_params(1)
+    srv = harness.make_server(s, theta, precision=precision)
+    o = oracle_driver.make_oracle(s, theta)
+    before = theta.astype(np.float64)
+    _full_size_tick(3, precision, 0, srv, o)
+    rg, ro = srv.ps_apply(ps.REPLAY, s.lr), o.apply(ops.REPLAY, s.lr)
+    assert rg == ro and rg["applied"] == 16 and rg["new_version"] == 1
+    head1, _ = srv.ps_export_params()
+    _assert_update_close(head1, o.head(), before, max(TOL_TENSOR if precision else TOL_FP32, 1e-3), "config 3 tick")
+    # the outage: the stored weights stay readable, 100 ticks x 16 gradients pile up
+    srv.ps_kill(); o.kill()
+    assert srv.ps_pull_snapshot(0).version == o.pull_snapshot(0)[0] == 1
+    K = s.W * (s.recover_at - s.kill_at)
+    cols = np.sort(np.random.default_rng(2).choice(ps.P, size=512, replace=False))
+    cols_d = torch.from_numpy(cols).cuda()
+    oc = ops.OraclePS(o.head()[cols], external_store=True)
+    oc.kill()
+    gen = torch.Generator(device="cuda").manual_seed(6)
+    block = torch.empty((s.W, ps.P_PAD), device="cuda")
+    for t in range(s.recover_at - s.kill_at):
+        block.normal_(0.0, 0.01, generator=gen)
+        block[:, ps.P:] = 0
+        srv.ps_enqueue(list(range(s.W)), [1] * s.W, t, grads_dev=block)
+        oc.enqueue(block[:, cols_d].cpu().numpy(), range(s.W), [1] * s.W, t)
+    assert srv.ps_stats()["queue_len"] == K == 1600
+    srv.ps_restore(); oc.restore()
+    rg = srv.ps_apply(ps.REPLAY, s.lr, scale=0.25)
+    roc = oc.apply(ops.REPLAY, s.lr, scale=0.25)
+    assert rg["applied"] == roc["applied"] == K and rg["new_version"] == 2
+    th = srv.ps_export_params()[0]
+    step_g = th[cols].astype(np.float64) - head1[cols]
+    step_o = oc.head().astype(np.float64) - head1[cols]
+    assert np.abs(th[cols] - oc.head()).max() <= 1e-6 * np.abs(theta).max()
+    assert np.abs(step_g - step_o).max() <= 1e-3 * np.abs(step_o).max()
+    assert (th != head1).mean() > 0.99
+    srv.close()
+
+
+@pytest.mark.parametrize("precision", [0, 2])
+def test_full_size_config4_tick_nine_versions_ordered_apply_and_mirror(precision):
+    """W=64 x b=32, async server with a ring of 9 versions and a mirrored replica: the workers read nine distinct
+    snapshots (seeded lags 0..8), every worker's gradient is checked against the oracle, then the 64 gradients are
+    applied one by one in seeded arrival order, every update mirrored; every retained version and the replica are
+    compared with the oracle's, and the failover that follows."""
+    import torch
+    from paper_2406_05546_b200 import harness, ps
+    s = schedules.config(4)
+    theta = synth.init_params(1)
+    srv = harness.make_server(s, theta, precision=precision)
+    o = oracle_driver.make_oracle(s, theta)
+    _advance_both(srv, o, 12, 700, ps.ASYNC, schedules.ASYNC)          # versions 4..12 retained, all different
+    t = 5
+    lags = synth.lags(t, s.W, s.max_lag)
+    assert sorted(set(lags.tolist())) == list(range(9))
+    before = o.head().astype(np.float64)
+    _full_size_tick(4, precision, t, srv, o, lags=lags)
+    order = synth.arrival_order(t, s.W)
+    rg, ro = srv.ps_apply(ps.ASYNC, s.lr, order=order), o.apply(schedules.ASYNC, s.lr, order=order)
+    assert rg == ro and rg["applied"] == 64 and rg["new_version"] == 76 and rg["replicated"] == 64
+    st = srv.ps_stats()
+    assert st["version"] == 76 and st["oldest_version"] == o.oldest_version() == 68 and st["replica_version"] == 76
+    tol_step = max(TOL_TENSOR if precision else TOL_FP32, 1e-3)
+    for lag in range(9):
+        sn = srv.ps_pull_snapshot(0, lag)
+        v, th_o = o.pull_snapshot(0, lag)
+        assert sn.version == v == 76 - lag
+        off = sn.dev_ptr - srv.arena.data_ptr()
+        th_g = srv.arena[off:off + ps.P * 4].view(torch.float32).cpu().numpy()
+        _assert_update_close(th_g, th_o, before, tol_step, f"config 4 version {v}")
+    head, _ = srv.ps_export_params(0)
+    rep, rv = srv.ps_export_params(-1)
+    assert rv == 76 and (rep == head).all()
+    srv.ps_kill(); o.kill()
+    assert srv.ps_failover() == o.failover() == 76
+    assert (srv.ps_export_params()[0] == head).all()
+    srv.close()
