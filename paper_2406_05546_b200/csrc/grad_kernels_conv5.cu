@@ -352,10 +352,11 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
           const float left = __shfl_up_sync(0xffffffffu, __uint_as_float(e2[ic]), 1);
           v[ic] = (__uint_as_float(e1[ic]) + right) + (x == 0 ? 0.f : left);
         }
-        if (y < 14 && x < 14) {      // dp1 of a sample is [channel quad][position][4 channels]: a warp writes 448 contiguous bytes
-          float4* out = reinterpret_cast<float4*>(ws.dp1 + row * P1_ELEMS) + (y * 14 + x);
+        if (y < 14 && x < 14) {      // dp1 of a sample is [channel quad][position][4 channels] in BF16 (its only reader
+          // multiplies in BF16): a warp writes 224 contiguous bytes per quad; a row keeps its fp32-sized pitch
+          uint2* out = reinterpret_cast<uint2*>(ws.dp1 + row * P1_ELEMS) + (y * 14 + x);
 #pragma unroll
-          for (int q = 0; q < 4; ++q) out[q * 196] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+          for (int q = 0; q < 4; ++q) out[q * 196] = make_uint2(bf16_pair(v[4 * q], v[4 * q + 1]), bf16_pair(v[4 * q + 2], v[4 * q + 3]));
         }
       }
       tc_fence_before();

@@ -658,11 +658,13 @@ __global__ void __launch_bounds__(256) conv1_bwd(GradStepArgs a, WorkerTable wt,
 constexpr int RED_PER_BLOCK = 1024;
 constexpr int RED_OUTPUTS = C2_GRAD + C1_GRAD + (NCLS * HID + HID + NCLS) + 1 + (P_PAD - P);
 constexpr int RED_BLOCKS = (RED_OUTPUTS + RED_PER_BLOCK - 1) / RED_PER_BLOCK;
-__global__ void __launch_bounds__(256) conv_grad_reduce(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks, int n_chunks2,
-                                                        int seg_len) {
+__global__ void __launch_bounds__(256) conv_grad_reduce(GradStepArgs a, WorkerTable wt, Workspace ws, int n_chunks, int seg_len1,
+                                                        int n_chunks2, int seg_len) {
   const int s = blockIdx.x, b = a.b;
   float* grad = wt.grad[s];
   const int used2 = seg_len > 0 ? (s * b + b - 1) / seg_len - (s * b) / seg_len + 1 : n_chunks2;
+  // part1 likewise: all n_chunks slots, or four (one per window element) for every range of seg_len1 rows
+  const int used1 = seg_len1 > 0 ? 4 * ((s * b + b - 1) / seg_len1 - (s * b) / seg_len1 + 1) : n_chunks;
   for (int v = blockIdx.y * RED_PER_BLOCK + threadIdx.x; v < min(RED_OUTPUTS, ((int)blockIdx.y + 1) * RED_PER_BLOCK); v += 256) {
     int o = v;
     if (o < C2_GRAD) {
@@ -674,7 +676,7 @@ __global__ void __launch_bounds__(256) conv_grad_reduce(GradStepArgs a, WorkerTa
     o -= C2_GRAD;
     if (o < C1_GRAD) {
       float t = 0.f;
-      for (int c = 0; c < n_chunks; ++c) t += ws.part1[((int64_t)s * n_chunks + c) * C1_GRAD + o];
+      for (int c = 0; c < used1; ++c) t += ws.part1[((int64_t)s * n_chunks + c) * C1_GRAD + o];
       grad[OFF_C1W + o] = t;
       continue;
     }
@@ -764,10 +766,12 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     n_chunks2 = launch_conv2_dw_tc5(a, wt, ws, s2, prof, &seg_len);
     if (side.s2) cudaEventRecord(side.join2, s2);
     launch_conv2_dx_tc5(a, wt, gt, ws, st, prof);
-    const int n_chunks1t = launch_conv1_bwd_tc(a, wt, ws, st, prof);
+    int seg_len1 = 0;
+    const int n_chunks1t = launch_conv1_dw_tc5(a, wt, ws, st, prof, &seg_len1);
+    if (n_chunks1t < 0) return -1;
     if (side.s1) cudaStreamWaitEvent(st, side.join1, 0);
     if (side.s2) cudaStreamWaitEvent(st, side.join2, 0);
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1t, n_chunks2, seg_len)));
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1t, seg_len1, n_chunks2, seg_len)));
     launches += 4;
   } else {
     TIMED(K_CONV1_FWD, (conv1_fwd<<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
@@ -778,7 +782,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
     TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
     TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks1b, a.W), 256, 0, st>>>(a, wt, ws, n_chunks1b)));
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1b, n_chunks2, 0)));
+    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1b, 0, n_chunks2, 0)));
     launches = 9;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;

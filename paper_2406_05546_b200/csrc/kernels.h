@@ -104,9 +104,9 @@ struct Workspace {
   float* da1;      // [rows][512]         gradient w.r.t. fc1 pre-activation
   float* dz;       // [rows][16]          gradient w.r.t. logits (10 used)
   float* dp2;      // [rows][1568]        gradient w.r.t. p2
-  float* dp1;      // [rows][3136]        gradient w.r.t. p1; [16][196] (FP32 path) or [4 channel quads][196][4] (tensor-core path)
+  float* dp1;      // [rows][3136]        gradient w.r.t. p1; [16][196] fp32 (FP32 path) or [4 channel quads][196][4] BF16 in the first half of the row (tensor-core path)
   float* part2;    // [W][chunks][4640]   per-block partial conv2 weight/bias gradients
-  float* part1;    // [W][chunks][160]    per-block partial conv1 weight/bias gradients
+  float* part1;    // [W][4 chunks][160]  per-block partial conv1 weight/bias gradients (tensor-core path: four per range, one per window element)
   float* partf;    // [W][FC2_SPLIT][FC_PART] per-block partial output-layer gradients and loss sums
   float* w1r;      // [groups][512][1568] TF32-rounded fc1 weights of each weight group of the call
   float* w1tr;     // [groups][1568][512] and their transpose
@@ -139,12 +139,14 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
 int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, uint32_t thresh,
                         uint8_t* keep, cudaStream_t st, Profiler* prof);
 int configure_grad_kernels();
-int launch_conv1_bwd_tc(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof);
 extern int g_sm_count;   // SMs of the current device, set by configure_tc5_kernels
 int configure_tc5_kernels();
 int configure_conv5_kernels();
 int configure_conv1_kernels();
 int configure_dw5_kernels();
+int configure_c1d5_kernels();
+int launch_conv1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof,
+                        int* seg_len);
 int launch_conv2_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof,
                         int* seg_len);
 int launch_conv1_fwd_planes(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,

@@ -148,7 +148,7 @@ void layout(ps_ctx* x, const ps_config& c, void* arena, void* pinned, uint64_t* 
   ws.dp2 = a.take<float>(rows * psk::FLAT * 4);
   ws.dp1 = a.take<float>(rows * psk::P1_ELEMS * 4);
   ws.part2 = a.take<float>((uint64_t)c.max_workers * chunks * psk::C2_GRAD * 4);
-  ws.part1 = a.take<float>((uint64_t)c.max_workers * chunks * psk::C1_GRAD * 4);
+  ws.part1 = a.take<float>((uint64_t)c.max_workers * 4 * chunks * psk::C1_GRAD * 4);
   ws.partf = a.take<float>((uint64_t)c.max_workers * psk::FC2_SPLIT * psk::FC_PART * 4);
   ws.status = a.take<uint32_t>(ALIGN);
   ws.w1r = ws.w1tr = nullptr;
@@ -259,7 +259,7 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
   x->ckpt_version.assign(x->ckpt_buf.size(), 0);
   double t = std::floor((double)cfg->dropout_p * 4294967296.0);
   x->drop_thresh = t <= 0.0 ? 0u : (t >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)t);
-  if (psk::configure_grad_kernels() != 0 || psk::configure_tc5_kernels() != 0 || psk::configure_conv5_kernels() != 0 || psk::configure_conv1_kernels() != 0 || psk::configure_dw5_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
+  if (psk::configure_grad_kernels() != 0 || psk::configure_tc5_kernels() != 0 || psk::configure_conv5_kernels() != 0 || psk::configure_conv1_kernels() != 0 || psk::configure_dw5_kernels() != 0 || psk::configure_c1d5_kernels() != 0) { delete x; return fail(PS_ERR_CUDA, "kernel configuration failed: %s", cudaGetErrorString(cudaGetLastError())); }
   if (cfg->precision != PS_FP32) {
     // two side streams let independent branches of the backward pass overlap (they allocate no device memory)
     bool ok = cudaStreamCreateWithFlags(&x->side.s1, cudaStreamNonBlocking) == cudaSuccess &&

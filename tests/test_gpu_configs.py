@@ -236,9 +236,9 @@ def _full_size_tick(n, precision, t, srv, o, lags=None):
 
 
 def _assert_update_close(th_g, th_o, before, tol, what):
-    """Parameters within the apply tolerance, and the step taken (which the parameters' size would hide) within the
-    gradient tolerance, per tensor."""
-    assert_params_close(th_g, th_o, 1e-5, what)
+    """Parameters and the step taken (which the parameters' size would hide) within the path's tolerance, per tensor
+    (biases start at zero, so for them the two are the same check)."""
+    assert_params_close(th_g, th_o, tol, what)
     assert_params_close(th_g.astype(np.float64) - before, th_o.astype(np.float64) - before, tol, what + " (the step)")
 
 
@@ -311,10 +311,11 @@ def test_full_size_config3_tick_and_replay_of_1600_gradients(precision):
     roc = oc.apply(ops.REPLAY, s.lr, scale=0.25)
     assert rg["applied"] == roc["applied"] == K and rg["new_version"] == 2
     th = srv.ps_export_params()[0]
+    # each side replays from its own version-1 weights (they differ by the tick's tolerance): compare the steps
     step_g = th[cols].astype(np.float64) - head1[cols]
-    step_o = oc.head().astype(np.float64) - head1[cols]
-    assert np.abs(th[cols] - oc.head()).max() <= 1e-6 * np.abs(theta).max()
-    assert np.abs(step_g - step_o).max() <= 1e-3 * np.abs(step_o).max()
+    step_o = oc.head().astype(np.float64) - o.head()[cols]
+    assert np.abs(step_o).max() > 1e-4
+    assert np.abs(step_g - step_o).max() <= 1e-3 * np.abs(step_o).max() + 1.2e-7 * np.abs(theta).max()
     assert (th != head1).mean() > 0.99
     srv.close()
 
