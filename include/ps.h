@@ -144,6 +144,15 @@ int32_t workers_grad_step(ps_ctx* ctx, int32_t W, int32_t b, const ps_snapshot* 
                           uint64_t seed, uint64_t step, const int64_t* slot_ids, float* grads_dev,
                           float* loss_dev, int32_t* argmax_dev);
 
+/* Evaluation pass (paper, implementation section: the metric exporter reports accuracy and loss while training):
+ * the forward pass only, without dropout (every unit kept, nothing rescaled), of W groups of b samples, group w
+ * against weights snaps[w].dev_ptr.  Same inputs and layouts as workers_grad_step.  loss_dev [W] receives the mean
+ * cross-entropy of each group, argmax_dev [W][b] the lowest index of the largest logit, correct_dev [W] the number of
+ * samples of the group whose argmax equals the label (all dev, written).  No gradient is produced and the queue is
+ * not touched.  Errors as workers_grad_step. */
+int32_t workers_eval(ps_ctx* ctx, int32_t W, int32_t b, const ps_snapshot* snaps, const float* x_dev,
+                     const int32_t* y_dev, float* loss_dev, int32_t* argmax_dev, int32_t* correct_dev);
+
 /* The dropout keep mask (1 = kept) the grad step uses for one worker: same generator, keying and
  * threshold as workers_grad_step (model endnote: 25 % dropout; rate from ps_config.dropout_p).
  * keep_dev (dev, [b][512] bytes) is written on the context's stream. */
@@ -179,6 +188,19 @@ typedef struct {
  * the same pass.  K = 0 is a no-op.  Errors: PS_ERR_DOWN, PS_ERR_BAD_ARG. */
 int32_t ps_apply(ps_ctx* ctx, ps_mode mode, float lr, float scale, const int32_t* order,
                  ps_apply_result* out);
+
+/* ps_apply with the treatments of stale gradients that the paper's design section names, in its closing remarks on the
+ * stateless server, as alternatives to a smaller learning rate for many pending gradients (gradient clipping, an
+ * adaptive learning rate).  Readings taken here:
+ *   clip_norm c > 0        every queued gradient g is scaled by min(1, c / ||g||_2) (clipping by global norm, per
+ *                          gradient); costs one extra pass over the queue that takes the norms;
+ *   staleness_alpha a > 0  gradient k is scaled by 1 / (1 + a * tau_k), tau_k = the version its update is applied to
+ *                          (the head for PS_SYNC / PS_REPLAY, head + j for the j-th gradient of PS_ASYNC) minus the
+ *                          base_version given at ps_enqueue.  A base version newer than that is PS_ERR_BAD_ARG.
+ * 0 switches a treatment off; with both off the call is ps_apply.  Everything else (modes, order, checkpoints,
+ * replication, result) is as in ps_apply. */
+int32_t ps_apply_stale(ps_ctx* ctx, ps_mode mode, float lr, float scale, const int32_t* order, float clip_norm,
+                       float staleness_alpha, ps_apply_result* out);
 
 /* The periodic save of the parameters to persistent storage (design section on checkpointing): copies the
  * head weights and version into the next pinned host slot (stream-ordered device-to-host copy); when all slots

@@ -143,6 +143,17 @@ def workers_grad_step(thetas, worker_ids, x, y, seed, step, drop_p=0.25, precisi
     return grads, loss, am, logits
 
 
+def workers_eval(thetas, x, y, precision=0):
+    """Evaluation pass (the paper's metric exporter: accuracy and loss while training): the forward pass of
+    workers_grad_step without dropout (every unit kept, no rescaling).  Returns (loss[W] f64, argmax[W,b] i32,
+    correct[W] i64 = samples whose argmax equals the label, logits[W,b,10] f64).  The gradient the C routine also
+    computes is not returned."""
+    W = len(thetas)
+    _, loss, am, logits = workers_grad_step(thetas, list(range(W)), x, y, 0, 0, drop_p=0.0, precision=precision)
+    correct = (am == np.asarray(y, dtype=np.int32)).sum(axis=1)
+    return loss, am, correct, logits
+
+
 def round_operand(v, precision):
     return float(lib().oracle_round_operand(float(v), int(precision)))
 

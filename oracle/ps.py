@@ -109,7 +109,18 @@ class OraclePS:
             self.replicate()
             result["replicated"] += 1
 
-    def apply(self, mode, lr, scale=1.0, order=None):
+    def apply(self, mode, lr, scale=1.0, order=None, clip_norm=None, staleness_alpha=0.0):
+        """One server step over the whole queue.
+
+        clip_norm and staleness_alpha are the two treatments of stale gradients that the design section's closing
+        remarks on the stateless server name as alternatives to a smaller learning rate (gradient clipping; an
+        adaptive, here staleness-dependent, learning rate).  Readings recorded in the design notes:
+          clip_norm c > 0:  every queued gradient is scaled by min(1, c / ||g||_2) (clipping by global norm, per
+                            gradient, norm taken in double);
+          staleness_alpha a >= 0:  gradient k is scaled by 1 / (1 + a * tau_k), tau_k = the version its update is
+                            applied to minus the version its worker had read (base_version): SYNC / REPLAY apply
+                            everything to the head, ASYNC applies the j-th gradient in arrival order to head + j.
+        With clip_norm None and alpha 0 every factor is exactly 1."""
         if not self.up:
             raise PSError(DOWN, "server is down")
         K = len(self.queue)
@@ -119,20 +130,41 @@ class OraclePS:
         idx = list(range(K)) if order is None else [int(o) for o in order]
         if sorted(idx) != list(range(K)):
             raise PSError(BAD_ARG, "order is not a permutation of the queue")
+        if clip_norm is not None and not clip_norm > 0:
+            raise PSError(BAD_ARG, "clip_norm must be positive")
+        if staleness_alpha < 0:
+            raise PSError(BAD_ARG, "staleness_alpha must be >= 0")
         lr = float(np.float32(lr))
         scale = float(np.float32(scale))
+        alpha = float(np.float32(staleness_alpha))
+        clip = None if clip_norm is None else float(np.float32(clip_norm))
+        v0 = self.version
+
+        def factor(k, applied_to):
+            f = 1.0
+            if clip is not None:
+                norm = float(np.sqrt(np.sum(self.queue[k]["g"].astype(np.float64) ** 2)))
+                if norm > clip:
+                    f *= clip / norm
+            if alpha > 0.0:
+                tau = applied_to - self.queue[k]["base_version"]
+                if tau < 0:
+                    raise PSError(BAD_ARG, "a gradient claims a base version newer than the weights it is applied to")
+                f /= 1.0 + alpha * tau
+            return f
+
         theta = self.head()
         if mode in (SYNC, REPLAY):
             total = np.zeros(self.P, dtype=np.float64)
             for k in idx:
-                total += self.queue[k]["g"].astype(np.float64)
+                total += factor(k, v0) * self.queue[k]["g"].astype(np.float64)
             div = K if mode == SYNC else self.w_tick
             new = (theta.astype(np.float64) - (lr * scale / div) * total).astype(np.float32)
             self._publish(new, result)
         elif mode == ASYNC:
-            for k in idx:
+            for j, k in enumerate(idx):
                 new = (theta.astype(np.float64)
-                       - (lr * scale) * self.queue[k]["g"].astype(np.float64)).astype(np.float32)
+                       - (lr * scale * factor(k, v0 + j)) * self.queue[k]["g"].astype(np.float64)).astype(np.float32)
                 self._publish(new, result)
                 theta = new
         else:

@@ -21,9 +21,15 @@ __device__ __forceinline__ void add4(float4& a, const float4& b) {
   a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
 }
 
+__device__ __forceinline__ void fma4(float c, const float4& v, float4& a) {
+  a.x = fmaf(c, v.x, a.x); a.y = fmaf(c, v.y, a.y); a.z = fmaf(c, v.z, a.z); a.w = fmaf(c, v.w, a.w);
+}
+
 // Sum of slots [k0, k1) of one float4 column, in a fixed order: eight interleaved running sums
-// (slot k goes to sum k mod 8 relative to k0), combined pairwise at the end.
-__device__ __forceinline__ float4 column_sum(const float4* __restrict__ q, int64_t k0, int64_t k1) {
+// (slot k goes to sum k mod 8 relative to k0), combined pairwise at the end.  With WEIGHTED every slot is
+// multiplied by its own factor coef_k[k] (the stale-gradient treatments) as it is added.
+template <bool WEIGHTED>
+__device__ __forceinline__ float4 column_sum(const float4* __restrict__ q, int64_t k0, int64_t k1, const float* __restrict__ coef_k) {
   float4 acc[8];
 #pragma unroll
   for (int u = 0; u < 8; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -33,26 +39,34 @@ __device__ __forceinline__ float4 column_sum(const float4* __restrict__ q, int64
 #pragma unroll
     for (int u = 0; u < 8; ++u) v[u] = ld_stream(q + (k + u) * (int64_t)P_VEC4);
 #pragma unroll
-    for (int u = 0; u < 8; ++u) add4(acc[u], v[u]);
+    for (int u = 0; u < 8; ++u) {
+      if (WEIGHTED) fma4(coef_k[k + u], v[u], acc[u]);
+      else add4(acc[u], v[u]);
+    }
   }
 #pragma unroll
   for (int u = 0; u < 7; ++u)
-    if (k + u < k1) add4(acc[u], ld_stream(q + (k + u) * (int64_t)P_VEC4));
+    if (k + u < k1) {
+      const float4 v = ld_stream(q + (k + u) * (int64_t)P_VEC4);
+      if (WEIGHTED) fma4(coef_k[k + u], v, acc[u]);
+      else add4(acc[u], v);
+    }
   add4(acc[0], acc[1]); add4(acc[2], acc[3]); add4(acc[4], acc[5]); add4(acc[6], acc[7]);
   add4(acc[0], acc[2]); add4(acc[4], acc[6]);
   add4(acc[0], acc[4]);
   return acc[0];
 }
 
-// theta_out = theta_in - coef * sum_k g_k, whole queue in one pass (small K).
+// theta_out = theta_in - coef * sum_k g_k (or - sum_k coef_k[k] g_k), whole queue in one pass (small K).
+template <bool WEIGHTED>
 __global__ void __launch_bounds__(TPB) sum_apply_direct(const float4* __restrict__ queue, int64_t K,
                                                         const float4* theta_in, float4* theta_out,
-                                                        float4* __restrict__ replica, float coef) {
+                                                        float4* __restrict__ replica, float coef, const float* __restrict__ coef_k) {
   // theta_in and theta_out may be the same buffer (a ring of depth one): each thread reads its column before it
   // writes it, and the two pointers carry no no-alias promise
   int col = blockIdx.x * TPB + threadIdx.x;
   if (col >= P_VEC4) return;
-  float4 s = column_sum(queue + col, 0, K);
+  float4 s = column_sum<WEIGHTED>(queue + col, 0, K, coef_k);
   float4 t = theta_in[col];
   t.x = fmaf(-coef, s.x, t.x); t.y = fmaf(-coef, s.y, t.y);
   t.z = fmaf(-coef, s.z, t.z); t.w = fmaf(-coef, s.w, t.w);
@@ -61,14 +75,15 @@ __global__ void __launch_bounds__(TPB) sum_apply_direct(const float4* __restrict
 }
 
 // Stage 1 of the long-queue reduction: block (x, y) sums slot range y of column block x.
+template <bool WEIGHTED>
 __global__ void __launch_bounds__(TPB) sum_partial(const float4* __restrict__ queue, int64_t K,
-                                                   int n_split, float4* __restrict__ partial) {
+                                                   int n_split, float4* __restrict__ partial, const float* __restrict__ coef_k) {
   int col = blockIdx.x * TPB + threadIdx.x;
   if (col >= P_VEC4) return;
   int s = blockIdx.y;
   int64_t per = (K + n_split - 1) / n_split;
   int64_t k0 = s * per, k1 = k0 + per < K ? k0 + per : K;
-  float4 acc = k0 < k1 ? column_sum(queue + col, k0, k1) : make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 acc = k0 < k1 ? column_sum<WEIGHTED>(queue + col, k0, k1, coef_k) : make_float4(0.f, 0.f, 0.f, 0.f);
   partial[(int64_t)s * P_VEC4 + col] = acc;
 }
 
@@ -105,8 +120,9 @@ __global__ void __launch_bounds__(TPB) async_apply(AsyncApplyArgs a, AsyncOrder 
     for (int u = 0; u < U; ++u) {
       int k = k0 + u;
       if (k < a.K) {
-        t.x = fmaf(-a.coef, g[u].x, t.x); t.y = fmaf(-a.coef, g[u].y, t.y);
-        t.z = fmaf(-a.coef, g[u].z, t.z); t.w = fmaf(-a.coef, g[u].w, t.w);
+        const float c = a.coef_k ? a.coef_k[ord.slot[k]] : a.coef;
+        t.x = fmaf(-c, g[u].x, t.x); t.y = fmaf(-c, g[u].y, t.y);
+        t.z = fmaf(-c, g[u].z, t.z); t.w = fmaf(-c, g[u].w, t.w);
         if (k >= a.first_stored) {
           int slot = (int)((a.v0 + (uint64_t)k + 1) % (uint64_t)a.ring_depth);
           reinterpret_cast<float4*>(a.ring[slot])[col] = t;
@@ -126,6 +142,50 @@ __global__ void __launch_bounds__(TPB) copy_rows(float4* __restrict__ dst, const
   for (; i < n_vec; i += stride) dst[i] = src[i];
 }
 
+// ---- clipping by global norm ------------------------------------------------------------------------------------
+// Block (c, k) sums the squares of chunk c of gradient k: every thread over its float4 columns in four interleaved
+// sums, then lanes and warps in a fixed order.
+constexpr int NORM_VEC = P_VEC4 / NORM_CHUNKS;      // 25,416 float4 columns per chunk
+static_assert(NORM_VEC * NORM_CHUNKS == P_VEC4, "chunks tile the vector");
+__global__ void __launch_bounds__(TPB) sq_norm_partial(const float4* __restrict__ queue, float* __restrict__ norm_part) {
+  __shared__ float warp_sum[TPB / 32];
+  const int64_t k = blockIdx.y;
+  const float4* g = queue + k * (int64_t)P_VEC4 + (int64_t)blockIdx.x * NORM_VEC;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  int i = threadIdx.x;
+  for (; i + 3 * TPB < NORM_VEC; i += 4 * TPB) {
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = g[i + u * TPB];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) acc[u] = fmaf(v[u].x, v[u].x, fmaf(v[u].y, v[u].y, fmaf(v[u].z, v[u].z, fmaf(v[u].w, v[u].w, acc[u]))));
+  }
+  for (; i < NORM_VEC; i += TPB) {
+    const float4 v = g[i];
+    acc[0] = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, fmaf(v.w, v.w, acc[0]))));
+  }
+  float t = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = t;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < TPB / 32; ++w) s += warp_sum[w];
+    norm_part[k * NORM_CHUNKS + blockIdx.x] = s;
+  }
+}
+
+__global__ void __launch_bounds__(TPB) clip_coef_finish(const float* __restrict__ norm_part, int64_t K, float clip, float* __restrict__ coef_k) {
+  const int64_t k = (int64_t)blockIdx.x * TPB + threadIdx.x;
+  if (k >= K) return;
+  float n2 = 0.f;
+#pragma unroll
+  for (int c = 0; c < NORM_CHUNKS; ++c) n2 += norm_part[k * NORM_CHUNKS + c];
+  coef_k[k] *= fminf(1.0f, clip / sqrtf(n2));      // a zero gradient keeps its factor (clip / 0 = inf)
+}
+
 }  // namespace
 
 #define TIMED(id, launch) do { if (prof) prof->begin(id, st); launch; if (prof) prof->end(st); } while (0)
@@ -134,7 +194,7 @@ const char* kernel_name(int id) {
   static const char* names[K_COUNT] = {
       "conv1_fwd", "conv2_fwd", "fc1_fwd", "fc2_fwd_bwd", "fc1_dw", "fc1_dx", "conv2_bwd", "conv1_bwd",
       "conv_grad_reduce", "sum_apply_direct", "sum_partial", "sum_finish", "async_apply", "copy_rows",
-      "dropout_mask", "conv2_dw", "prep_w1"};
+      "dropout_mask", "conv2_dw", "prep_w1", "sq_norm_partial", "clip_coef_finish", "eval_finish"};
   return id >= 0 && id < K_COUNT ? names[id] : "?";
 }
 
@@ -149,16 +209,26 @@ int launch_sum_apply(const SumApplyArgs& a, cudaStream_t st, Profiler* prof) {
     n_split = (int)(want < a.max_split ? want : a.max_split);
   }
   int launches = 0;
+  const float* ck = a.coef_k;
+  const float coef = ck ? 1.0f : a.coef;      // the per-gradient factors already carry the learning rate
   if (n_split <= 1) {
-    TIMED(K_SUM_APPLY_DIRECT, (sum_apply_direct<<<COL_BLOCKS, TPB, 0, st>>>(q, a.K, tin, tout, rep, a.coef)));
+    if (ck) TIMED(K_SUM_APPLY_DIRECT, (sum_apply_direct<true><<<COL_BLOCKS, TPB, 0, st>>>(q, a.K, tin, tout, rep, coef, ck)));
+    else TIMED(K_SUM_APPLY_DIRECT, (sum_apply_direct<false><<<COL_BLOCKS, TPB, 0, st>>>(q, a.K, tin, tout, rep, coef, nullptr)));
     launches = 1;
   } else {
     float4* part = reinterpret_cast<float4*>(a.partial);
-    TIMED(K_SUM_PARTIAL, (sum_partial<<<dim3(COL_BLOCKS, n_split), TPB, 0, st>>>(q, a.K, n_split, part)));
-    TIMED(K_SUM_FINISH, (sum_finish<<<COL_BLOCKS, TPB, 0, st>>>(part, n_split, tin, tout, rep, a.coef)));
+    if (ck) TIMED(K_SUM_PARTIAL, (sum_partial<true><<<dim3(COL_BLOCKS, n_split), TPB, 0, st>>>(q, a.K, n_split, part, ck)));
+    else TIMED(K_SUM_PARTIAL, (sum_partial<false><<<dim3(COL_BLOCKS, n_split), TPB, 0, st>>>(q, a.K, n_split, part, nullptr)));
+    TIMED(K_SUM_FINISH, (sum_finish<<<COL_BLOCKS, TPB, 0, st>>>(part, n_split, tin, tout, rep, coef)));
     launches = 2;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;
+}
+
+int launch_clip_factors(const float* queue, int64_t K, float clip, float* coef_k, float* norm_part, cudaStream_t st, Profiler* prof) {
+  TIMED(K_SQ_NORM, (sq_norm_partial<<<dim3(NORM_CHUNKS, (unsigned)K), TPB, 0, st>>>(reinterpret_cast<const float4*>(queue), norm_part)));
+  TIMED(K_COEF_FINISH, (clip_coef_finish<<<(unsigned)((K + TPB - 1) / TPB), TPB, 0, st>>>(norm_part, K, clip, coef_k)));
+  return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
 
 int launch_async_apply(const AsyncApplyArgs& a, const AsyncOrder& ord, cudaStream_t st, Profiler* prof) {

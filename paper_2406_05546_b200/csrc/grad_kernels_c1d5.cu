@@ -47,7 +47,9 @@ constexpr int D1_RAW_G = P1_ELEMS * 2, D1_RAW_CODE = P1_ELEMS;
 constexpr int D1_RAW_SLOT = (D1_RAW_X + D1_RAW_G + D1_RAW_CODE + 127) / 128 * 128;     // 13,824
 constexpr int D1_NRAW = 4;                               // raw input slots: each group's copies run two of its samples ahead
 constexpr int D1_SMEM = 2 * D1_STAGE_BYTES + D1_NRAW * D1_RAW_SLOT + 256 + 128;
-constexpr int D1_TMEM_COLS = 32;                         // 24 accumulator columns
+constexpr int D1_NACC = 4;                               // accumulators used in turn: an MMA that adds to the sum of the one before
+                                                         // it waits for that one to finish, and these MMAs are short
+constexpr int D1_TMEM_COLS = 32 * D1_NACC;               // 24 accumulator columns each, 32 apart
 constexpr int D1_KSTEPS = D1_CHUNKS / 2;                 // 13
 static_assert(D1_SMEM <= 227 * 1024, "shared memory");
 static_assert(D1_GT == 256, "the item split below assumes 256 threads per group");
@@ -62,10 +64,10 @@ struct D1Bars {
   volatile uint32_t abort_flag;
 };
 
-// Top bit of byte k set iff byte k of `codes` (each 0..4) equals w.
-__device__ __forceinline__ uint32_t eq_flags(uint32_t codes, uint32_t w) {
-  return ~((codes ^ (0x01010101u * w)) + 0x7F7F7F7Fu) & 0x80808080u;
-}
+// The decisions arrive as one byte per (channel, position) holding 1 << winner (0 = no gradient).  Shifting a word of
+// four such bytes left by 7 - w brings "the winner is w" into the top bit of every byte, which is the only bit the
+// sign-replicating byte permute below looks at.
+__device__ __forceinline__ uint32_t win_flags(uint32_t onehot, int w) { return onehot << (7 - w); }
 
 // Rows (sorted worker, sample) are split into gridDim.x contiguous ranges of seg_len.  Partial sums of worker s go
 // to part1[s][4 (range index - first range of s) + window element].
@@ -118,8 +120,8 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_const
         // contraction indices 16 ks .. 16 ks + 15: two core matrices, 2 x 144 bytes further along every row group
 #pragma unroll
         for (int ks = 0; ks < D1_KSTEPS; ++ks)
-          umma_f16_split(tmem, a_lo + ks * (2 * D1_CHUNK_PITCH / 16), plain_desc_hi(D1_GROUP_BYTES), b_lo + ks * (2 * D1_CHUNK_PITCH / 16),
-                         plain_desc_hi(D1_GROUP_BYTES), idesc, (ks == 0 && fresh) ? 0u : 1u);
+          umma_f16_split(tmem + (ks % D1_NACC) * 32, a_lo + ks * (2 * D1_CHUNK_PITCH / 16), plain_desc_hi(D1_GROUP_BYTES),
+                         b_lo + ks * (2 * D1_CHUNK_PITCH / 16), plain_desc_hi(D1_GROUP_BYTES), idesc, (ks < D1_NACC && fresh) ? 0u : 1u);
         fresh = false;
         umma_commit(&bars->op_empty[st]);
         const int row = r0 + n;
@@ -152,11 +154,19 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_const
     const int a_src = (aq * 196 + 8 * ac + 4 * ah);                       // (quad, first position) in units of one position's 4 channels
     const int a_dst = ((aq >> 1)) * D1_GROUP_BYTES + ac * D1_CHUNK_PITCH + ((aq & 1) * 4) * 16 + ah * 8;   // window element 0, channel 0 of the quad
     // B items of this thread: shift bn = (sy, sx) and chunks bc0 = gt_ / 16 and bc0 + 16 (the latter for bc0 < 9;
-    // chunk 24 holds positions 192..195 only).  Word offsets of the eight positions' window origins in the image box
-    // (box row 2 py + sy is image row 2 py + sy - 1, box column 2 px + sx + 3 is image column 2 px + sx - 1).
+    // chunk 24 holds positions 192..195 only).  The word offsets of the sixteen elements in the image box are fixed
+    // for the whole kernel (box row 2 py + sy is image row 2 py + sy - 1, box column 2 px + sx + 3 is image column
+    // 2 px + sx - 1) and are worked out once.
     const int bn = gt_ & 15, sy = bn >> 2, sx = bn & 3, bc0 = gt_ >> 4;
-    const int b_base = sy * D1_BOX_W + sx + 3;
     const int b_dst = (bn >> 3) * D1_GROUP_BYTES + (bn & 7) * 16;
+    int b_off[2][8];                     // word 0 of the box is outside the image (always zero): positions past 195 read it
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int p = 8 * (bc0 + 16 * h) + j, py = p / 14, px = p - 14 * py;
+        b_off[h][j] = p < 196 ? sy * D1_BOX_W + sx + 3 + 2 * py * D1_BOX_W + 2 * px : 0;
+      }
 
     if (gt_ == 0) { if (grp < n_samples) issue(grp); if (grp + 2 < n_samples) issue(grp + 2); }
     for (int n = grp; n < n_samples; n += 2) {
@@ -180,7 +190,7 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_const
                                   {prmt(g01.y, g01.w, 0x7632u), prmt(g23.y, g23.w, 0x7632u)}};
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
-          const uint32_t e0 = eq_flags(cd.x, w), e1 = eq_flags(cd.y, w), e2 = eq_flags(cd.z, w), e3 = eq_flags(cd.w, w);
+          const uint32_t e0 = win_flags(cd.x, w), e1 = win_flags(cd.y, w), e2 = win_flags(cd.z, w), e3 = win_flags(cd.w, w);
           uint8_t* d = stage + a_dst + w * (2 * D1_GROUP_BYTES);
           // channel c: half-word masks from the top bits of byte c of the two positions' flags
           *reinterpret_cast<uint2*>(d) = make_uint2(v[0][0] & prmt(e0, e1, 0xCC88u), v[0][1] & prmt(e2, e3, 0xCC88u));
@@ -195,10 +205,7 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_const
         if (bc < 25) {
           float xv[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int p = 8 * bc + j, py = p / 14, px = p - 14 * py;
-            xv[j] = p < 196 ? img[b_base + 2 * py * D1_BOX_W + 2 * px] : 0.f;
-          }
+          for (int j = 0; j < 8; ++j) xv[j] = img[b_off[h][j]];
           *reinterpret_cast<uint4*>(stage + D1_A_BYTES + b_dst + bc * D1_CHUNK_PITCH) =
               make_uint4(bf16_pair(xv[0], xv[1]), bf16_pair(xv[2], xv[3]), bf16_pair(xv[4], xv[5]), bf16_pair(xv[6], xv[7]));
         }
@@ -222,10 +229,19 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_const
       if (!(row + 1 == r1 || (row + 1) % a.b == 0)) continue;
       if (!mbar_wait(&bars->acc_full, writes & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
       tc_fence_after();
-      uint32_t v0[16], v1[16];
-      tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16), v0);
-      tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + 16u, v1);      // columns 16..31: 16 = bias, 17..23 zero rows, 24..31 unused
-      tmem_ld_wait();
+      float v0[16], vb = 0.f;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v0[j] = 0.f;
+#pragma unroll
+      for (int acc = 0; acc < D1_NACC; ++acc) {      // the accumulators are added in a fixed order
+        uint32_t t0[16], t1[16];
+        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 32), t0);
+        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 32 + 16), t1);      // column 16 = bias, 17..23 zero rows, 24..31 unused
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v0[j] += __uint_as_float(t0[j]);
+        vb += __uint_as_float(t1[0]);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->acc_empty);
@@ -237,9 +253,9 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_const
         for (int w = 0; w < 4; ++w)
           if (w == quarter) {
 #pragma unroll
-            for (int tap = 0; tap < 9; ++tap) part[lane * 9 + tap] = __uint_as_float(v0[((w >> 1) + tap / 3) * 4 + (w & 1) + tap % 3]);
+            for (int tap = 0; tap < 9; ++tap) part[lane * 9 + tap] = v0[((w >> 1) + tap / 3) * 4 + (w & 1) + tap % 3];
           }
-        part[144 + lane] = __uint_as_float(v1[0]);
+        part[144 + lane] = vb;
       }
       ++writes;
     }

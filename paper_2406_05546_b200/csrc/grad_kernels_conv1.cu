@@ -9,7 +9,8 @@
 //   - results are collected in shared memory in exactly the layout the second convolution's kernels
 //     copy from (two planes of eight BF16 channels, one 16-byte row per position of a zero-bordered
 //     16x16 grid with even and odd columns apart) and leave by bulk copies, 8 KB per sample; the
-//     pooling decisions leave the same way, one byte per element as [channel quad][position][4 channels].
+//     pooling decisions leave the same way, one byte per element (1 << winner, 0 = no gradient) as
+//     [channel quad][position][4 channels].
 // Every wait on an mbarrier is bounded.
 #include "device_common.cuh"
 #include "kernels.h"
@@ -113,8 +114,8 @@ __global__ void __launch_bounds__(C1_THREADS, C1_BLOCKS_PER_SM) conv1_fwd_planes
       for (int cp = 0; cp < 2; ++cp)
 #pragma unroll
         for (int j = 0; j < 4; ++j) unpack2(acc[cp][j], v[2 * cp][j], v[2 * cp + 1][j]);
-      // ReLU then max = max then ReLU; the winner is the first window element that reaches the maximum, and an
-      // element whose maximum is not positive passes no gradient (code 4)
+      // ReLU then max = max then ReLU; the winner is the first window element that reaches the maximum (stored as the
+      // byte 1 << winner), and an element whose maximum is not positive passes no gradient (byte 0)
       float best[4];
       uint32_t codes = 0;
 #pragma unroll
@@ -122,7 +123,7 @@ __global__ void __launch_bounds__(C1_THREADS, C1_BLOCKS_PER_SM) conv1_fwd_planes
         const float m = fmaxf(fmaxf(v[c][0], v[c][1]), fmaxf(v[c][2], v[c][3]));
         const uint32_t bi = v[c][0] == m ? 0u : (v[c][1] == m ? 1u : (v[c][2] == m ? 2u : 3u));
         best[c] = fmaxf(m, 0.f);
-        codes |= (m > 0.f ? bi : 4u) << (8 * c);
+        codes |= (m > 0.f ? (1u << bi) : 0u) << (8 * c);      // one bit per window element: the filter-gradient kernel shifts it into a mask
       }
       const int row = (py + 1) * 16 + col_row, pos = py * 14 + px;
       *reinterpret_cast<uint2*>(ob + sp * C1_PLANES_BYTES + (cg >> 1) * (C1_PLANES_BYTES / 2) + row * 16 + (cg & 1) * 8) =

@@ -66,10 +66,53 @@ constexpr int F_THREADS = 320;
 constexpr int F_PLANE_ROWS = 2 * 256 + 32;                 // two stacked 16x16 images + overrun of the padding rows
 constexpr int F_PLANE_BYTES = F_PLANE_ROWS * 16;           // 8704
 constexpr int F_BUF_BYTES = 2 * F_PLANE_BYTES;             // two planes of eight channels
-constexpr int F_W_BYTES = 18 * 32 * 16;                    // [k chunk = tap*2 + ic/8][oc][8 bf16]
+// One MMA per input SHIFT instead of one per (window element, tap).  Window element (jy, jx) and tap (ky, kx) read the
+// input plane shifted by (sy, sx) = (jy + ky, jx + kx), sixteen shifts in all, and a shift serves every (window
+// element, tap) pair that adds up to it: the products of one shifted plane with the filters of all those taps land
+// side by side in the accumulator columns [window element][channel] when the weight operand stacks the taps' filters
+// in that column order.  A shift whose window elements are not adjacent in the column order takes two MMAs, so a
+// tile costs 20 MMAs (N = 128, 64 or 32) instead of 36 of N = 32; an MMA of M = 128, K = 16 is bound by reading
+// its 4 KB position operand from shared memory whatever N is.  The host lists the MMAs (FoldTable).
+constexpr int F_OPS = 20;
+constexpr int F_W_BLOCKS = 36;                             // 32-row blocks of the stacked weight operand (1,152 rows)
+constexpr int F_W_ROWS = 32 * F_W_BLOCKS;
+constexpr int F_W_BYTES = 2 * F_W_ROWS * 16;               // [channel octet][row][8 bf16]
 constexpr int F_SMEM = F_NBUF * F_BUF_BYTES + F_W_BYTES + 32 * 4 + sizeof(Pipe) + 128;
+static_assert(2 * F_SMEM <= 227 * 1024, "two CTAs per SM");
 
-__global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, GroupTable gt, Workspace ws, int range_len) {
+struct FoldTable {
+  int32_t a_off[F_OPS];        // start of the shifted plane, in 16-byte rows
+  int32_t d_col[F_OPS];        // first accumulator column
+  int32_t b_row[F_OPS];        // first row of the op's block of the weight operand
+  uint32_t idesc[F_OPS];       // instruction descriptor (M = 128, the op's N)
+  uint8_t tap_of_block[F_W_BLOCKS];   // filter tap ky * 3 + kx whose 32 filters fill a 32-row block
+};
+
+FoldTable make_fold_table() {
+  FoldTable t;
+  int n_ops = 0, row = 0;
+  auto add = [&](int sy, int sx, int jy0, int ny, int jx0, int nx) {       // window elements [jy0, jy0 + ny) x [jx0, jx0 + nx)
+    t.a_off[n_ops] = sy * 16 + (sx & 1) * 8 + (sx >> 1);
+    t.d_col[n_ops] = (2 * jy0 + jx0) * 32;
+    t.b_row[n_ops] = row;
+    t.idesc[n_ops] = idesc_bf16(128, 32 * ny * nx);
+    for (int jy = jy0; jy < jy0 + ny; ++jy)
+      for (int jx = jx0; jx < jx0 + nx; ++jx) { t.tap_of_block[row / 32] = (uint8_t)((sy - jy) * 3 + (sx - jx)); row += 32; }
+    ++n_ops;
+  };
+  for (int pass = 0; pass < 2; ++pass)          // the op that covers all 128 columns comes first: it starts the sums
+    for (int sy = 0; sy < 4; ++sy)
+      for (int sx = 0; sx < 4; ++sx) {
+        if ((pass == 0) != (sy == 1 && sx == 1)) continue;
+        const int jy0 = sy == 3 ? 1 : 0, ny = (sy == 0 || sy == 3) ? 1 : 2;
+        const int jx0 = sx == 3 ? 1 : 0, nx = (sx == 0 || sx == 3) ? 1 : 2;
+        if (nx == 2) add(sy, sx, jy0, ny, jx0, 2);                       // columns of consecutive window elements
+        else for (int jy = jy0; jy < jy0 + ny; ++jy) add(sy, sx, jy, 1, jx0, 1);
+      }
+  return t;      // n_ops == F_OPS and row == F_W_ROWS by construction (checked where the table is made)
+}
+
+__global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, GroupTable gt, Workspace ws, int range_len, const __grid_constant__ FoldTable fold) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint16_t* Wk = reinterpret_cast<uint16_t*>(smem + F_NBUF * F_BUF_BYTES);
   float* bias = reinterpret_cast<float*>(smem + F_NBUF * F_BUF_BYTES + F_W_BYTES);
@@ -81,9 +124,10 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Gr
   const float* theta = gt.theta[grp];
   const int n_tiles = (r_end - r_begin + 1) / 2;
 
-  for (int idx = tid; idx < 4608; idx += F_THREADS) {
-    int oc = idx / 144, rem = idx - oc * 144, ic = rem / 9, tap = rem - ic * 9;
-    Wk[((tap * 2 + (ic >> 3)) * 32 + oc) * 8 + (ic & 7)] = bf16_bits(theta[OFF_C2W + idx]);
+  // the stacked weight operand: block rb holds the 32 filters of tap fold.tap_of_block[rb], one row per output channel
+  for (int idx = tid; idx < F_W_BLOCKS * 512; idx += F_THREADS) {
+    const int rb = idx >> 9, oc = (idx >> 4) & 31, ic = idx & 15;
+    Wk[((ic >> 3) * F_W_ROWS + rb * 32 + oc) * 8 + (ic & 7)] = bf16_bits(theta[OFF_C2W + (oc * 16 + ic) * 9 + fold.tap_of_block[rb]]);
   }
   if (tid < 32) bias[tid] = theta[OFF_C2B + tid];
   // rows never written by a copy (the overrun of the padding rows, a missing second sample) only feed
@@ -102,30 +146,20 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Gr
 
   if (warp == 0) {
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(128, 32);
-      const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), 512);
+      const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), F_W_ROWS * 16);
       for (int t = 0; t < n_tiles; ++t) {
         const int buf = t % F_NBUF, ab = t & 1;
         if (!mbar_wait(&pipe->a_full[buf], (t / F_NBUF) & 1)) { pipe->abort_flag = 1; break; }
         if (t >= 2 && !mbar_wait(&pipe->acc_empty[ab], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
         if (pipe->abort_flag) break;
         tc_fence_after();
-        // 36 MMAs (one per window element and tap: K = 16 channels), fully unrolled: every descriptor is a
-        // per-tile base plus a compile-time constant
+        // 20 MMAs, one or two per input shift (K = 16 channels); every descriptor is a per-tile base plus a table entry
         const uint32_t a_lo = plain_desc_lo(smem_u32(smem) + buf * F_BUF_BYTES, F_PLANE_BYTES);
         const uint32_t d_tmem = tmem + ab * 128;
-        // (taps outermost: consecutive MMAs go to the four different accumulators)
 #pragma unroll
-        for (int tap = 0; tap < 9; ++tap) {
-          const int ky = tap / 3, kx = tap - ky * 3;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int jy = j >> 1, jx = j & 1, sx = jx + kx;
-            const int row_off = (jy + ky) * 16 + (sx & 1) * 8 + (sx >> 1);     // in 16-byte rows
-            umma_f16_split(d_tmem + j * 32, a_lo + row_off, plain_desc_hi(512), w_lo + (tap * 2) * (512 / 16),
-                           plain_desc_hi(128), idesc, tap ? 1u : 0u);
-          }
-        }
+        for (int op = 0; op < F_OPS; ++op)
+          umma_f16_split(d_tmem + fold.d_col[op], a_lo + fold.a_off[op], plain_desc_hi(512), w_lo + fold.b_row[op],
+                         plain_desc_hi(128), fold.idesc[op], op ? 1u : 0u);
         umma_commit(&pipe->a_empty[buf]);
         umma_commit(&pipe->acc_full[ab]);
       }
@@ -388,9 +422,10 @@ int configure_conv5_kernels() {
 
 void launch_conv2_fwd_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
                           cudaStream_t st, Profiler* prof) {
+  static const FoldTable fold = make_fold_table();
   int len;
   const int n = plan_row_ranges(gt, a.b, 2 * g_sm_count, 2, &len);      // two CTAs per SM, tiles of two samples
-  TIMED(K_CONV2_FWD, (conv2_fwd_tc5<<<n, F_THREADS, F_SMEM, st>>>(a, gt, ws, len)));
+  TIMED(K_CONV2_FWD, (conv2_fwd_tc5<<<n, F_THREADS, F_SMEM, st>>>(a, gt, ws, len, fold)));
 }
 
 void launch_conv2_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,

@@ -43,7 +43,9 @@ constexpr int W5_RAW_BYTES = W5_RAW_P1 + W5_RAW_DP2 + W5_RAW_CODE;          // 1
 constexpr int W5_RAW_SLOT = (W5_RAW_BYTES + 127) / 128 * 128;
 constexpr int W5_NRAW = 4;                              // raw input slots: each group's copies run two of its samples ahead
 constexpr int W5_SMEM = 2 * W5_STAGE_BYTES + W5_NRAW * W5_RAW_SLOT + 256 + 128;
-constexpr int W5_TMEM_COLS = 128;                       // 96 accumulator columns
+constexpr int W5_NACC = 4;                              // accumulators used in turn (an MMA that adds to the sum of the one before it
+                                                        // waits for that one to finish); they are added up at write-out
+constexpr int W5_TMEM_COLS = 512;                       // W5_NACC x 96 accumulator columns
 static_assert(8 * W5_GROUP_BYTES <= W5_STAGE_BYTES, "the 64-row A operand must stay inside its stage");
 static_assert(W5_SMEM <= 227 * 1024, "shared memory");
 
@@ -117,8 +119,8 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
         // Rows 0 and 15 are the input's zero border, so their products vanish and are not issued.
 #pragma unroll
         for (int ks = 1; ks < 15; ++ks)
-          umma_f16_split(tmem, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), idesc,
-                         (ks == 1 && fresh) ? 0u : 1u);
+          umma_f16_split(tmem + ((ks - 1) % W5_NACC) * 96, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo + ks * 16,
+                         plain_desc_hi(W5_GROUP_BYTES), idesc, (ks - 1 < W5_NACC && fresh) ? 0u : 1u);
         fresh = false;
         umma_commit(&bars->op_empty[st]);
         const int row = r0 + n;
@@ -212,17 +214,25 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       const int rr = lane < 16 ? quarter * 16 + lane : 64;   // accumulator row: (kx, ic) for rr < 48, the ones row at 48
 #pragma unroll
       for (int cb = 0; cb < 6; ++cb) {                 // 16 columns at a time: ky = cb / 2, oc = 16 (cb % 2) + j
-        uint32_t v[16];
-        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cb * 16), v);
-        tmem_ld_wait();
+        float v[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] = 0.f;
+#pragma unroll
+        for (int acc = 0; acc < W5_NACC; ++acc) {       // fixed order
+          uint32_t t[16];
+          tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 96 + cb * 16), t);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] += __uint_as_float(t[j]);
+        }
         const int ky = cb >> 1;
         if (rr < 48) {
           const int kx = rr >> 4, ic = rr & 15;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) part[((16 * (cb & 1) + j) * 16 + ic) * 9 + ky * 3 + kx] = __uint_as_float(v[j]);
+          for (int j = 0; j < 16; ++j) part[((16 * (cb & 1) + j) * 16 + ic) * 9 + ky * 3 + kx] = v[j];
         } else if (rr == 48 && ky == 1) {     // the ones row against the ky = 1 copy, whose rows 1..14 are all issued
 #pragma unroll
-          for (int j = 0; j < 16; ++j) part[4608 + 16 * (cb & 1) + j] = __uint_as_float(v[j]);
+          for (int j = 0; j < 16; ++j) part[4608 + 16 * (cb & 1) + j] = v[j];
         }
       }
       tc_fence_before();

@@ -696,6 +696,29 @@ __global__ void __launch_bounds__(256) conv_grad_reduce(GradStepArgs a, WorkerTa
   }
 }
 
+// ---- evaluation: per worker, the mean loss from the output-layer kernel's partial sums and the number of samples
+// whose predicted label equals the given one (an integer count, summed in a fixed order).
+__global__ void __launch_bounds__(128) eval_finish(GradStepArgs a, WorkerTable wt, Workspace ws, int32_t* __restrict__ correct) {
+  __shared__ int warp_hits[4];
+  const int s = blockIdx.x, src = wt.src[s];
+  int hits = 0;
+  for (int i = threadIdx.x; i < a.b; i += 128) {
+    const int64_t r = (int64_t)src * a.b + i;
+    hits += a.argmax[r] == a.y[r] ? 1 : 0;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) hits += __shfl_xor_sync(0xffffffffu, hits, o);
+  if ((threadIdx.x & 31) == 0) warp_hits[threadIdx.x >> 5] = hits;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    correct[src] = warp_hits[0] + warp_hits[1] + warp_hits[2] + warp_hits[3];
+    float t = 0.f;
+#pragma unroll
+    for (int c = 0; c < FC2_SPLIT; ++c) t += ws.partf[((int64_t)s * FC2_SPLIT + c) * FC_PART + NCLS * HID + HID + NCLS];
+    a.loss[src] = t * (1.0f / (float)a.b);
+  }
+}
+
 // ---- the keep mask on its own: thread e/4 draws the four words of elements 4*(e/4) .. +3.
 __global__ void __launch_bounds__(256) dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int n_quads,
                                                     uint32_t thresh, uchar4* __restrict__ keep) {
@@ -722,6 +745,33 @@ int configure_grad_kernels() {
   cudaError_t e = cudaFuncSetAttribute(conv2_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)(C2B_SMEM_FLOATS * sizeof(float)));
   return e == cudaSuccess ? 0 : -1;
+}
+
+// Evaluation pass: the forward kernels of the grad step with the dropout switched off (the output-layer kernel also
+// produces backward quantities into the workspace; nothing reads them), then the per-worker loss and hit count.
+int launch_eval(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws, int32_t* correct,
+                cudaStream_t st, Profiler* prof) {
+  const int n_chunks = (a.b + CONV_SPB - 1) / CONV_SPB;
+  const int mt = group_tiles(gt, a.b, 64);
+  int launches = 0;
+  if (a.precision != 0) {
+    if (!a.skip_prep_w1) launches += launch_prep_w1(gt, ws, st, prof);
+    if (launch_conv1_fwd_planes(a, wt, gt, ws, st, prof) < 0) return -1;
+    launch_conv2_fwd_tc5(a, wt, gt, ws, st, prof);
+    const int n = launch_fc1_fwd_tc5(a, wt, gt, ws, st, prof);
+    if (n < 0) return -1;
+    launches += 2 + n;
+  } else {
+    const int n_chunks1 = (a.b + CONV1_SPB - 1) / CONV1_SPB;
+    TIMED(K_CONV1_FWD, (conv1_fwd<<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
+    TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
+    launches += 3;
+  }
+  TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<dim3(a.W, FC2_SPLIT), FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
+  TIMED(K_EVAL_FINISH, (eval_finish<<<a.W, 128, 0, st>>>(a, wt, ws, correct)));
+  launches += 2;
+  return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 // Launch order of one grad step.  On the tensor-core path the copies of the dense layer's weights are made on a

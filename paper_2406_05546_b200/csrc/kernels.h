@@ -37,7 +37,7 @@ constexpr uint32_t STATUS_WAIT_TIMEOUT = 2u;   // a bounded barrier wait in a te
 enum KernelId {
   K_CONV1_FWD = 0, K_CONV2_FWD, K_FC1_FWD, K_FC2_FWD_BWD, K_FC1_DW, K_FC1_DX, K_CONV2_BWD, K_CONV1_BWD,
   K_CONV_GRAD_REDUCE, K_SUM_APPLY_DIRECT, K_SUM_PARTIAL, K_SUM_FINISH, K_ASYNC_APPLY, K_COPY_ROWS,
-  K_DROPOUT_MASK, K_CONV2_DW, K_PREP_W1, K_COUNT
+  K_DROPOUT_MASK, K_CONV2_DW, K_PREP_W1, K_SQ_NORM, K_COEF_FINISH, K_EVAL_FINISH, K_COUNT
 };
 const char* kernel_name(int id);
 
@@ -97,7 +97,8 @@ struct GroupTable {
 // Activation workspace carved from the arena (rows = sorted worker * b + sample).
 struct Workspace {
   float* p1;       // conv1 -> ReLU -> pool: [rows][16][14][14] fp32 (FP32 path) or [rows][2 planes][256][8] BF16 (tensor-core path)
-  uint8_t* code1;  // [rows][3136]        pool-1 argmax 0..3, 4 = no gradient (max <= 0); [16][196] (FP32 path) or [4 channel quads][196][4] (tensor-core path)
+  uint8_t* code1;  // [rows][3136]        pool-1 decisions. FP32 path: [16][196], argmax 0..3, 4 = no gradient (max <= 0); tensor-core path:
+                   //                     [4 channel quads][196][4], the byte 1 << argmax, 0 = no gradient
   float* p2;       // [rows][1568]        conv2 -> ReLU -> pool, channel-major flatten
   uint8_t* code2;  // [rows][1568]
   float* d;        // [rows][512]         fc1 -> ReLU -> dropout (scaled)
@@ -173,6 +174,7 @@ struct SumApplyArgs {
   float coef;               // lr*scale/divisor
   float* partial;           // [max_split][P_PAD] scratch
   int max_split;
+  const float* coef_k;      // per-gradient factors [K] that replace coef (the stale-gradient treatments), or nullptr
 };
 int launch_sum_apply(const SumApplyArgs& a, cudaStream_t st, Profiler* prof);
 
@@ -190,10 +192,20 @@ struct AsyncApplyArgs {
   int mirror_k[MAX_CHAIN];  // k whose result is also written to replica[m]
   float* replica[MAX_CHAIN];
   float coef;               // lr*scale
+  const float* coef_k;      // per-gradient factors indexed by queue slot that replace coef, or nullptr
 };
 int launch_async_apply(const AsyncApplyArgs& a, const AsyncOrder& ord, cudaStream_t st, Profiler* prof);
 
 int launch_copy_rows(float* dst, const float* src, int64_t rows, cudaStream_t st, Profiler* prof);
+
+// Clipping by global norm: coef_k[k] *= min(1, clip / ||queue[k]||_2) for k < K.  norm_part: [K][NORM_CHUNKS] scratch.
+constexpr int NORM_CHUNKS = 8;
+int launch_clip_factors(const float* queue, int64_t K, float clip, float* coef_k, float* norm_part, cudaStream_t st, Profiler* prof);
+
+// Evaluation pass: forward only, no dropout; loss [W] mean cross-entropy, argmax [W][b], correct [W] = samples whose
+// argmax equals the label.  Returns the number of kernels launched or -1.
+int launch_eval(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws, int32_t* correct,
+                cudaStream_t st, Profiler* prof);
 
 // One warp waits on a barrier nobody arrives at, for at most limit_cycles, then sets STATUS_WAIT_TIMEOUT in *status.
 int launch_wait_timeout_probe(uint32_t* status, long long limit_cycles, cudaStream_t st);

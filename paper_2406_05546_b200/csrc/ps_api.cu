@@ -56,6 +56,9 @@ struct ps_ctx {
   std::vector<Replica> replicas;
   float* partial;
   float* queue;
+  float* coef_dev;                      // [queue_slots] per-gradient factors of a treated apply
+  float* norm_part;                     // [queue_slots][NORM_CHUNKS] partial sums of squares
+  cudaEvent_t coef_uploaded = nullptr;  // the staged factors have left coef_host
   psk::Workspace ws;
   float* x_stage[2]; int32_t* y_stage[2]; float* loss_stage[2]; int32_t* argmax_stage[2];   // two sets: two ticks may be in flight
   uint32_t* status_dev;
@@ -64,6 +67,7 @@ struct ps_ctx {
   std::vector<uint64_t> ckpt_version;   // parallel to ckpt_buf
   std::vector<int> ckpt_order;          // slot indices, oldest first
   float* io_stage;
+  float* coef_host;                     // per-gradient factors of a treated apply, staged for upload
   uint32_t* status_host;
   // state
   uint64_t version = 0, oldest = 0;
@@ -136,6 +140,8 @@ void layout(ps_ctx* x, const ps_config& c, void* arena, void* pinned, uint64_t* 
   for (int i = 0; i + 1 < c.chain_len; ++i) { float* p = a.take<float>(VEC_BYTES); if (x) x->replicas.push_back({p, 0, true}); }
   float* partial = a.take<float>(VEC_BYTES * MAX_SPLIT);
   float* queue = a.take<float>(VEC_BYTES * (uint64_t)c.queue_slots);
+  float* coef_dev = a.take<float>((uint64_t)c.queue_slots * 4);
+  float* norm_part = a.take<float>((uint64_t)c.queue_slots * psk::NORM_CHUNKS * 4);
   psk::Workspace ws;
   const uint64_t p1_elems = c.precision != PS_FP32 ? psk::P1_PLANE_ELEMS : psk::P1_ELEMS;
   ws.p1 = a.take<float>(rows * p1_elems * 4);
@@ -167,9 +173,11 @@ void layout(ps_ctx* x, const ps_config& c, void* arena, void* pinned, uint64_t* 
   Carver h(pinned);
   for (int i = 0; i < c.ckpt_slots; ++i) { float* p = h.take<float>(VEC_BYTES); if (x) x->ckpt_buf.push_back(p); }
   float* io_stage = h.take<float>(VEC_BYTES);
+  float* coef_host = h.take<float>((uint64_t)c.queue_slots * 4);
   uint32_t* status_host = h.take<uint32_t>(ALIGN);
   if (x) {
     x->partial = partial; x->queue = queue; x->ws = ws; x->status_dev = ws.status;
+    x->coef_dev = coef_dev; x->norm_part = norm_part; x->coef_host = coef_host;
     for (int k = 0; k < 2; ++k) { x->x_stage[k] = x_stage[k]; x->y_stage[k] = y_stage[k]; x->loss_stage[k] = loss_stage[k]; x->argmax_stage[k] = argmax_stage[k]; }
     x->io_stage = io_stage; x->status_host = status_host;
   }
@@ -273,6 +281,7 @@ int32_t ps_create(const ps_config* cfg, const float* init_params_host, ps_ctx** 
     for (auto& ev : x->copy_ev) ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
     for (auto& ev : x->stage_free) ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
     for (auto& ev : x->tick_done) ok = ok && cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&x->coef_uploaded, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { delete x; return fail(PS_ERR_CUDA, "copy stream set-up failed: %s", cudaGetErrorString(cudaGetLastError())); }
   }
   std::memcpy(x->io_stage, init_params_host, sizeof(float) * PS_PARAM_COUNT);
@@ -300,6 +309,7 @@ int32_t ps_destroy(ps_ctx* x) {
   for (cudaEvent_t ev : x->copy_ev) if (ev) cudaEventDestroy(ev);
   for (cudaEvent_t ev : x->stage_free) if (ev) cudaEventDestroy(ev);
   for (cudaEvent_t ev : x->tick_done) if (ev) cudaEventDestroy(ev);
+  if (x->coef_uploaded) cudaEventDestroy(x->coef_uploaded);
   delete x;
   if (e != cudaSuccess) return cuda_fail(e, "ps_destroy");
   return PS_OK;
@@ -332,14 +342,10 @@ int32_t ps_slot_ptr(ps_ctx* x, int64_t slot_id, float** out) {
   return PS_OK;
 }
 
-int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* snaps, const int32_t* worker_ids,
-                          const float* x_dev, const int32_t* y_dev, uint64_t seed, uint64_t step,
-                          const int64_t* slot_ids, float* grads_dev, float* loss_dev, int32_t* argmax_dev) {
-  if (!x || !snaps || !worker_ids || !x_dev || !y_dev || !loss_dev || !argmax_dev) return fail(PS_ERR_BAD_ARG, "NULL argument");
-  if (W < 1 || W > x->cfg.max_workers || b < 1 || b > x->cfg.max_batch) return fail(PS_ERR_BAD_ARG, "W=%d, b=%d outside 1..%d, 1..%d", W, b, x->cfg.max_workers, x->cfg.max_batch);
-  if (!slot_ids && !grads_dev) return fail(PS_ERR_BAD_ARG, "neither slot_ids nor grads_dev given");
-  psk::GroupTable gt;
-  psk::WorkerTable wt;
+// Sorts the workers of a call by weight snapshot (workers sharing a pointer become one group) and fills the tables
+// the kernels take.  grad destinations: queue slots, rows of grads_dev, or none (evaluation).
+static int32_t build_tables(ps_ctx* x, int32_t W, const ps_snapshot* snaps, const int32_t* worker_ids, const int64_t* slot_ids,
+                            float* grads_dev, psk::WorkerTable& wt, psk::GroupTable& gt) {
   int group_of[PS_MAX_WORKERS];
   gt.n_groups = 0;
   for (int w = 0; w < W; ++w) {
@@ -362,31 +368,71 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
         if (id < x->queue_len || id >= x->queue_len + x->reserved) return fail(PS_ERR_BAD_ARG, "slot %lld is not reserved", (long long)id);
         wt.grad[s] = x->queue + id * (int64_t)psk::P_PAD;
       } else {
-        wt.grad[s] = grads_dev + (int64_t)w * psk::P_PAD;
+        wt.grad[s] = grads_dev ? grads_dev + (int64_t)w * psk::P_PAD : nullptr;
       }
-      wt.wid[s] = worker_ids[w];
+      wt.wid[s] = worker_ids ? worker_ids[w] : w;
       wt.src[s] = w;
       wt.group[s] = (int16_t)g;
       ++s;
     }
   }
   gt.first[gt.n_groups] = W;
+  if (x->cfg.precision != PS_FP32 && gt.n_groups > std::min(x->cfg.max_workers, x->cfg.ring_depth))
+    return fail(PS_ERR_BAD_ARG, "%d distinct snapshots but the tensor-core workspace holds ring_depth = %d", gt.n_groups, x->cfg.ring_depth);
+  return PS_OK;
+}
+
+// The rounded / transposed copies of the dense-layer weights are reused while the same snapshots hold the same weights.
+static int prep_is_current(ps_ctx* x, const psk::GroupTable& gt) {
+  bool same = x->prep_epoch == x->weights_epoch && x->prep_n == gt.n_groups;
+  for (int g = 0; g < gt.n_groups && same; ++g) same = x->prep_theta[g] == gt.theta[g];
+  return same ? 1 : 0;
+}
+static void prep_done(ps_ctx* x, const psk::GroupTable& gt) {
+  x->prep_epoch = x->weights_epoch; x->prep_n = gt.n_groups;
+  for (int g = 0; g < gt.n_groups; ++g) x->prep_theta[g] = gt.theta[g];
+}
+
+int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* snaps, const int32_t* worker_ids,
+                          const float* x_dev, const int32_t* y_dev, uint64_t seed, uint64_t step,
+                          const int64_t* slot_ids, float* grads_dev, float* loss_dev, int32_t* argmax_dev) {
+  if (!x || !snaps || !worker_ids || !x_dev || !y_dev || !loss_dev || !argmax_dev) return fail(PS_ERR_BAD_ARG, "NULL argument");
+  if (W < 1 || W > x->cfg.max_workers || b < 1 || b > x->cfg.max_batch) return fail(PS_ERR_BAD_ARG, "W=%d, b=%d outside 1..%d, 1..%d", W, b, x->cfg.max_workers, x->cfg.max_batch);
+  if (!slot_ids && !grads_dev) return fail(PS_ERR_BAD_ARG, "neither slot_ids nor grads_dev given");
+  psk::GroupTable gt;
+  psk::WorkerTable wt;
+  int32_t rc = build_tables(x, W, snaps, worker_ids, slot_ids, grads_dev, wt, gt);
+  if (rc != PS_OK) return rc;
   psk::GradStepArgs a;
   a.W = W; a.b = b; a.x = x_dev; a.y = y_dev; a.loss = loss_dev; a.argmax = argmax_dev;
   a.seed = seed; a.step = step; a.drop_p = x->cfg.dropout_p; a.drop_thresh = x->drop_thresh;
   a.precision = x->cfg.precision;
   if (a.precision != PS_FP32 && ((uintptr_t)x_dev & 15) != 0) return fail(PS_ERR_BAD_ARG, "x_dev must be 16-byte aligned on the tensor-core path");
-  if (a.precision != PS_FP32 && gt.n_groups > std::min(x->cfg.max_workers, x->cfg.ring_depth))
-    return fail(PS_ERR_BAD_ARG, "%d distinct snapshots but the tensor-core workspace holds ring_depth = %d", gt.n_groups, x->cfg.ring_depth);
-  // the rounded / transposed copies of the dense-layer weights are reused while the same snapshots hold the same weights
-  a.skip_prep_w1 = x->prep_epoch == x->weights_epoch && x->prep_n == gt.n_groups;
-  for (int g = 0; g < gt.n_groups && a.skip_prep_w1; ++g) a.skip_prep_w1 = x->prep_theta[g] == gt.theta[g];
+  a.skip_prep_w1 = prep_is_current(x, gt);
   int n = psk::launch_grad_step(a, wt, gt, x->ws, x->st, x->prof.on ? psk::SideStreams() : x->side, &x->prof);
-  if (n >= 0 && a.precision != PS_FP32) {
-    x->prep_epoch = x->weights_epoch; x->prep_n = gt.n_groups;
-    for (int g = 0; g < gt.n_groups; ++g) x->prep_theta[g] = gt.theta[g];
-  }
+  if (n >= 0 && a.precision != PS_FP32) prep_done(x, gt);
   if (n < 0) return cuda_fail(cudaGetLastError(), "grad step launch");
+  x->launches += n;
+  return PS_OK;
+}
+
+int32_t workers_eval(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* snaps, const float* x_dev, const int32_t* y_dev,
+                     float* loss_dev, int32_t* argmax_dev, int32_t* correct_dev) {
+  if (!x || !snaps || !x_dev || !y_dev || !loss_dev || !argmax_dev || !correct_dev) return fail(PS_ERR_BAD_ARG, "NULL argument");
+  if (W < 1 || W > x->cfg.max_workers || b < 1 || b > x->cfg.max_batch) return fail(PS_ERR_BAD_ARG, "W=%d, b=%d outside 1..%d, 1..%d", W, b, x->cfg.max_workers, x->cfg.max_batch);
+  psk::GroupTable gt;
+  psk::WorkerTable wt;
+  int32_t rc = build_tables(x, W, snaps, nullptr, nullptr, nullptr, wt, gt);
+  if (rc != PS_OK) return rc;
+  psk::GradStepArgs a;
+  a.W = W; a.b = b; a.x = x_dev; a.y = y_dev; a.loss = loss_dev; a.argmax = argmax_dev;
+  a.seed = 0; a.step = 0; a.drop_p = 0.f; a.drop_thresh = 0u;      // inference: nothing is dropped, nothing rescaled
+  a.precision = x->cfg.precision;
+  if (a.precision != PS_FP32 && ((uintptr_t)x_dev & 15) != 0) return fail(PS_ERR_BAD_ARG, "x_dev must be 16-byte aligned on the tensor-core path");
+  a.skip_prep_w1 = prep_is_current(x, gt);
+  int n = psk::launch_eval(a, wt, gt, x->ws, correct_dev, x->st, &x->prof);
+  if (n >= 0 && a.precision != PS_FP32) prep_done(x, gt);
+  if (n < 0) return cuda_fail(cudaGetLastError(), "evaluation launch");
   x->launches += n;
   return PS_OK;
 }
@@ -444,7 +490,11 @@ int32_t ps_replicate(ps_ctx* x, uint64_t* version_out) {
   return PS_OK;
 }
 
-int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* order, ps_apply_result* out) {
+// One server step.  clip_norm > 0 and / or staleness_alpha > 0 switch the stale-gradient treatments on: every queued
+// gradient then gets a factor of its own (learning rate included), staged on the host, uploaded, and, for clipping,
+// multiplied on the device by min(1, clip_norm / ||g||) after one pass over the queue that takes the norms.
+static int32_t apply_impl(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* order, float clip_norm,
+                          float staleness_alpha, ps_apply_result* out) {
   if (!x) return fail(PS_ERR_BAD_ARG, "ctx is NULL");
   if (!x->up || x->weights_lost) return fail(PS_ERR_DOWN, "server is down");
   if (mode != PS_SYNC && mode != PS_ASYNC && mode != PS_REPLAY) return fail(PS_ERR_BAD_ARG, "unknown mode %d", (int)mode);
@@ -457,6 +507,31 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
     for (int64_t k = 0; k < K; ++k) {
       if (order[k] < 0 || order[k] >= K || seen[(size_t)order[k]]) return fail(PS_ERR_BAD_ARG, "order is not a permutation of the queue");
       seen[(size_t)order[k]] = 1;
+    }
+  }
+  const bool treated = clip_norm > 0.f || staleness_alpha > 0.f;
+  if (treated) {
+    // factor of the gradient in queue slot k: the step size of its mode times 1 / (1 + alpha * staleness), where the
+    // staleness is the version the update is applied to minus the version the worker had read
+    const double step = mode == PS_ASYNC ? (double)lr * (double)scale
+                                         : (double)lr * (double)scale / (double)(mode == PS_SYNC ? K : (int64_t)x->w_tick);
+    CUDA_TRY(cudaEventSynchronize(x->coef_uploaded));      // an earlier treated apply has read the staging buffer
+    for (int64_t j = 0; j < K; ++j) {
+      const int64_t k = (mode == PS_ASYNC && order) ? order[j] : j;
+      const uint64_t applied_to = x->version + (mode == PS_ASYNC ? (uint64_t)j : 0u);
+      const uint64_t base = x->meta[(size_t)k].base_version;
+      if (staleness_alpha > 0.f && base > applied_to)
+        return fail(PS_ERR_BAD_ARG, "gradient %lld claims base version %llu, newer than the version %llu it is applied to",
+                    (long long)k, (unsigned long long)base, (unsigned long long)applied_to);
+      const double tau = staleness_alpha > 0.f ? (double)(applied_to - base) : 0.0;
+      x->coef_host[k] = (float)(step / (1.0 + (double)staleness_alpha * tau));
+    }
+    CUDA_TRY(cudaMemcpyAsync(x->coef_dev, x->coef_host, (size_t)K * sizeof(float), cudaMemcpyHostToDevice, x->st));
+    CUDA_TRY(cudaEventRecord(x->coef_uploaded, x->st));
+    if (clip_norm > 0.f) {
+      int n = psk::launch_clip_factors(x->queue, K, clip_norm, x->coef_dev, x->norm_part, x->st, &x->prof);
+      if (n < 0) return cuda_fail(cudaGetLastError(), "clipping launch");
+      x->launches += n;
     }
   }
   const uint64_t depth = (uint64_t)x->cfg.ring_depth;
@@ -472,6 +547,7 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
     a.replica = mirror ? rep->buf : nullptr;
     a.coef = lr * scale / (float)(mode == PS_SYNC ? K : (int64_t)x->w_tick);
     a.partial = x->partial; a.max_split = MAX_SPLIT;
+    a.coef_k = treated ? x->coef_dev : nullptr;
     int n = psk::launch_sum_apply(a, x->st, &x->prof);
     if (n < 0) return cuda_fail(cudaGetLastError(), "apply launch");
     x->launches += n;
@@ -500,6 +576,7 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
       a.ring_depth = x->cfg.ring_depth; a.v0 = x->version;
       a.first_stored = (int)std::max<int64_t>(0, seg - (int64_t)depth);
       a.n_mirror = 0; a.coef = lr * scale;
+      a.coef_k = treated ? x->coef_dev : nullptr;
       if (rep) {
         // replication events inside this segment: versions that are multiples of R.  The i-th live server behind
         // the frontend receives the version of the i-th latest event if that version is produced here; what the
@@ -539,6 +616,16 @@ int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* 
   res.new_version = x->version;
   if (out) *out = res;
   return PS_OK;
+}
+
+int32_t ps_apply(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* order, ps_apply_result* out) {
+  return apply_impl(x, mode, lr, scale, order, 0.f, 0.f, out);
+}
+
+int32_t ps_apply_stale(ps_ctx* x, ps_mode mode, float lr, float scale, const int32_t* order, float clip_norm,
+                       float staleness_alpha, ps_apply_result* out) {
+  if (!(clip_norm >= 0.f) || !(staleness_alpha >= 0.f)) return fail(PS_ERR_BAD_ARG, "clip_norm and staleness_alpha must be >= 0");
+  return apply_impl(x, mode, lr, scale, order, clip_norm, staleness_alpha, out);
 }
 
 int32_t ps_kill(ps_ctx* x, int32_t server) {

@@ -21,7 +21,7 @@ ERRORS = {-1: "PS_ERR_BAD_ARG", -2: "PS_ERR_DOWN", -3: "PS_ERR_QUEUE_FULL", -4: 
           -8: "PS_ERR_CUDA", -9: "PS_ERR_DEVICE_STATUS"}
 
 EXPORTS = ["ps_query_bytes", "ps_create", "ps_destroy", "ps_pull_snapshot", "ps_queue_reserve", "ps_slot_ptr",
-           "workers_grad_step", "ps_dropout_mask", "ps_enqueue", "ps_apply", "ps_checkpoint", "ps_restore", "ps_replicate",
+           "workers_grad_step", "workers_eval", "ps_dropout_mask", "ps_enqueue", "ps_apply", "ps_apply_stale", "ps_checkpoint", "ps_restore", "ps_replicate",
            "ps_kill", "ps_failover", "ps_import_params", "ps_export_params", "ps_stats", "ps_tick_host",
            "ps_tick_host_submit", "ps_tick_host_wait",
            "ps_profile", "ps_profile_read", "ps_selftest_wait_timeout", "ps_last_error", "ps_replay_sum_static", "ps_replay_sum_static_error"]
@@ -77,6 +77,8 @@ def load(path=None):
         "ps_queue_reserve": [vp, i32, vp],
         "ps_slot_ptr": [vp, i64, C.POINTER(vp)],
         "workers_grad_step": [vp, i32, i32, vp, vp, vp, vp, u64, u64, vp, vp, vp, vp],
+        "workers_eval": [vp, i32, i32, vp, vp, vp, vp, vp, vp],
+        "ps_apply_stale": [vp, i32, f32, f32, vp, f32, f32, C.POINTER(ApplyResult)],
         "ps_dropout_mask": [vp, u64, i32, u64, i32, vp],
         "ps_enqueue": [vp, i32, vp, vp, vp, vp, u64],
         "ps_apply": [vp, i32, f32, f32, vp, C.POINTER(ApplyResult)],
@@ -219,6 +221,20 @@ class ParameterServer:
             loss_dev.data_ptr(), argmax_dev.data_ptr()))
         return loss_dev, argmax_dev
 
+    def workers_eval(self, snaps, x_dev, y_dev):
+        """Forward pass without dropout.  Returns (loss_dev [W], argmax_dev [W,b], correct_dev [W])."""
+        torch = self._torch
+        W, b = int(y_dev.shape[0]), int(y_dev.shape[1])
+        assert x_dev.is_cuda and x_dev.dtype == torch.float32 and x_dev.is_contiguous() and x_dev.numel() == W * b * 784
+        assert y_dev.is_cuda and y_dev.dtype == torch.int32 and y_dev.is_contiguous()
+        arr = (Snapshot * W)(*snaps)
+        loss = torch.empty(W, dtype=torch.float32, device="cuda")
+        am = torch.empty((W, b), dtype=torch.int32, device="cuda")
+        correct = torch.empty(W, dtype=torch.int32, device="cuda")
+        self._check(self.lib.workers_eval(self.ctx, W, b, C.cast(arr, C.c_void_p), x_dev.data_ptr(), y_dev.data_ptr(),
+                                          loss.data_ptr(), am.data_ptr(), correct.data_ptr()))
+        return loss, am, correct
+
     def ps_dropout_mask(self, seed, worker_id, step, b):
         keep = self._torch.empty((b, 512), dtype=self._torch.uint8, device="cuda")
         self._check(self.lib.ps_dropout_mask(self.ctx, int(seed), int(worker_id), int(step), int(b), keep.data_ptr()))
@@ -240,6 +256,14 @@ class ParameterServer:
         res = ApplyResult()
         o = None if order is None else np.ascontiguousarray(order, dtype=np.int32)
         self._check(self.lib.ps_apply(self.ctx, int(mode), float(lr), float(scale), _np_ptr(o), C.byref(res)))
+        return {"applied": res.applied, "new_version": res.new_version, "checkpointed": res.checkpointed,
+                "replicated": res.replicated}
+
+    def ps_apply_stale(self, mode, lr, scale=1.0, order=None, clip_norm=0.0, staleness_alpha=0.0):
+        res = ApplyResult()
+        o = None if order is None else np.ascontiguousarray(order, dtype=np.int32)
+        self._check(self.lib.ps_apply_stale(self.ctx, int(mode), float(lr), float(scale), _np_ptr(o), float(clip_norm),
+                                            float(staleness_alpha), C.byref(res)))
         return {"applied": res.applied, "new_version": res.new_version, "checkpointed": res.checkpointed,
                 "replicated": res.replicated}
 

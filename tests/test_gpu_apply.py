@@ -403,3 +403,72 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_nothing_hangs():
     assert st["device_status"] == 0 and st["version"] == 1 and np.isfinite(loss).all()
     srv.close()
     torch.cuda.synchronize()
+
+
+# ---- treatments of stale gradients ------------------------------------------------------------------------------------
+
+def _known_norm_grads(norms, seed):
+    rng = np.random.default_rng(seed)
+    g = synth.random_gradients(len(norms), seed=seed)
+    for k, nrm in enumerate(norms):
+        g[k] *= np.float32(nrm / np.linalg.norm(g[k].astype(np.float64)))
+    return g
+
+
+@pytest.mark.parametrize("mode_name,K", [("SYNC", 6), ("REPLAY", 300), ("ASYNC", 9)])
+def test_clipping_by_global_norm(mode_name, K):
+    ops, ps, o, g = _pair(queue_slots=max(K, 8), ring_depth=3, external_store=(mode_name == "REPLAY"), max_workers=64)
+    norms = np.random.default_rng(K).uniform(0.2, 5.0, size=K)
+    norms[0], norms[-1] = 0.01, 50.0
+    grads = _known_norm_grads(norms, seed=K)
+    _both_enqueue(o, g, grads)
+    order = synth.arrival_order(0, K) if mode_name == "ASYNC" else None
+    ro = o.apply(getattr(ops, mode_name), 0.01, order=order, clip_norm=1.0)
+    rg = g.ps_apply_stale(getattr(ps, mode_name), 0.01, order=order, clip_norm=1.0)
+    assert ro == rg
+    theta0 = synth.init_params(seed=1, bias_scale=0.05)
+    th = g.ps_export_params()[0]
+    assert_params_close(th, o.head(), TOL_APPLY, f"clipped {mode_name}")
+    step_o, step_g = o.head().astype(np.float64) - theta0, th.astype(np.float64) - theta0
+    assert np.abs(step_g - step_o).max() <= 2e-3 * np.abs(step_o).max()
+    # and the clipping did something: the plain step is far from this one
+    _, _, o2, _g2 = _pair(queue_slots=max(K, 8), ring_depth=3, external_store=(mode_name == "REPLAY"), max_workers=64)
+    o2.enqueue(grads, range(K), [0] * K, 0)
+    o2.apply(getattr(ops, mode_name), 0.01, order=order)
+    assert np.abs((o2.head().astype(np.float64) - theta0) - step_o).max() > 0.1 * np.abs(step_o).max()
+    _g2.close(); g.close()
+
+
+@pytest.mark.parametrize("mode_name", ["SYNC", "REPLAY", "ASYNC"])
+def test_staleness_scaled_learning_rate(mode_name):
+    ops, ps, o, g = _pair(queue_slots=16, ring_depth=9, external_store=(mode_name == "REPLAY"), max_workers=16)
+    _steps(o, g, ops, ps, 5, 800)                           # head is version 5
+    K = 8
+    grads = synth.random_gradients(K, seed=33)
+    base = [5, 0, 3, 5, 1, 4, 2, 0]
+    _both_enqueue(o, g, grads, step=9, base=base)
+    order = synth.arrival_order(2, K) if mode_name == "ASYNC" else None
+    before = o.head().astype(np.float64)
+    ro = o.apply(getattr(ops, mode_name), 0.01, order=order, staleness_alpha=0.5, clip_norm=3.0)
+    rg = g.ps_apply_stale(getattr(ps, mode_name), 0.01, order=order, staleness_alpha=0.5, clip_norm=3.0)
+    assert ro == rg
+    th = g.ps_export_params()[0]
+    assert_params_close(th, o.head(), TOL_APPLY, f"staleness-scaled {mode_name}")
+    step_o, step_g = o.head().astype(np.float64) - before, th.astype(np.float64) - before
+    assert np.abs(step_g - step_o).max() <= 2e-3 * np.abs(step_o).max()
+    # both treatments off is the plain apply, bit for bit
+    _both_enqueue(o, g, grads, step=10)
+    h0 = g.ps_export_params()[0]
+    rg = g.ps_apply_stale(getattr(ps, mode_name), 0.01, order=order)
+    plain = g.ps_export_params()[0]
+    _, _, _, g2 = _pair(queue_slots=16, ring_depth=9, external_store=(mode_name == "REPLAY"), max_workers=16)
+    g2.ps_import_params(h0)
+    g2.ps_enqueue(list(range(K)), [0] * K, 10, grads_dev=_pad(grads))
+    g2.ps_apply(getattr(ps, mode_name), 0.01, order=order)
+    assert (g2.ps_export_params()[0] == plain).all()
+    # a base version from the future is refused
+    g.ps_enqueue([0], [10 ** 6], 11, grads_dev=_pad(grads[:1]))
+    with pytest.raises(ps.PSError) as e:
+        g.ps_apply_stale(getattr(ps, mode_name), 0.01, staleness_alpha=0.5)
+    assert e.value.name == "PS_ERR_BAD_ARG"
+    g2.close(); g.close()

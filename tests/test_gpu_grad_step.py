@@ -310,3 +310,36 @@ def test_pipelined_ticks_equal_sequential_ticks(precision):
     a, p = out
     assert a[1] == p[1] == T and a[4] == p[4] == list(range(1, T + 1))
     assert (a[0] == p[0]).all() and (a[2] == p[2]).all() and (a[3] == p[3]).all()
+
+
+@pytest.mark.parametrize("precision,W,b,lags", [(0, 3, 17, None), (2, 3, 17, None), (2, 4, 150, [1, 0, 0, 1]), (0, 1, 1, None)])
+def test_evaluation_pass_matches_the_oracle(precision, W, b, lags):
+    """workers_eval: forward only, no dropout; loss, labels and the count of correct labels per group."""
+    from oracle import cnn
+    n_versions = 2 if lags else 1
+    torch, ps, srv, theta0 = _setup(W, b, n_versions, 0.25, precision)      # the context's dropout rate must not matter
+    versions = {0: theta0}
+    if lags:
+        g = np.zeros((1, ps.P_PAD), dtype=np.float32)
+        g[0, :ps.P] = synth.random_gradients(1, seed=51, scale=2.0)[0]
+        srv.ps_enqueue([0], [0], 0, grads_dev=torch.from_numpy(g).cuda())
+        srv.ps_apply(ps.ASYNC, 0.01)
+        versions[1] = srv.ps_export_params(0)[0]
+    rng = np.random.default_rng(8)
+    x = rng.random((W, b, 28, 28), dtype=np.float32)
+    y = rng.integers(0, 10, (W, b)).astype(np.int32)
+    snaps = [srv.ps_pull_snapshot(w, lags[w] if lags else 0) for w in range(W)]
+    before = srv.ps_stats()
+    loss, am, correct = srv.workers_eval(snaps, torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda())
+    after = srv.ps_stats()
+    assert after["queue_len"] == before["queue_len"] == 0 and after["version"] == before["version"]
+    ol, oa, oc, oz = cnn.workers_eval([versions[s.version] for s in snaps], x, y, precision=precision)
+    tol = TOL_TENSOR if precision else TOL_FP32
+    np.testing.assert_allclose(loss.cpu().numpy(), ol, rtol=3e-3 if precision else 1e-5, atol=1e-6)
+    am = am.cpu().numpy()
+    n_amb = assert_argmax_valid(am, oz, tol)
+    # the count is exact given the labels the kernel chose; it equals the oracle's where no row is ambiguous
+    assert (correct.cpu().numpy() == (am == y).sum(axis=1)).all()
+    if n_amb == 0:
+        assert (correct.cpu().numpy() == oc).all()
+    srv.close()

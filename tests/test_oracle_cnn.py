@@ -279,3 +279,35 @@ def test_reduced_precision_decisions_against_a_torch_restatement(precision):
     # the case is a discriminating one: these decisions differ from the exact ones and from the other mode's
     for other in {0, 1, 2} - {precision}:
         assert (cnn.grad_step_f64(theta, x, y, keep, 0.25, precision=other)[0] != g).sum() > 1000
+
+
+# ---- evaluation pass ------------------------------------------------------------------------------------------------
+
+def test_evaluation_pass_is_the_forward_pass_without_dropout():
+    import torch
+    rng = np.random.default_rng(5)
+    W, b = 2, 6
+    theta = synth.init_params(seed=1, bias_scale=0.05)
+    x = rng.random((W, b, 28, 28), dtype=np.float32)
+    y = rng.integers(0, 10, (W, b)).astype(np.int32)
+    loss, am, correct, logits = cnn.workers_eval([theta] * W, x, y)
+    # the same network in torch (float64), no dropout layer at all
+    t = torch.tensor(theta.astype(np.float64))
+    seg = lambda name: t[cnn.TENSORS[name][0]:cnn.TENSORS[name][0] + int(np.prod(cnn.TENSORS[name][1]))].reshape(cnn.TENSORS[name][1])
+    F = torch.nn.functional
+    for w in range(W):
+        h = torch.tensor(x[w].astype(np.float64)).reshape(b, 1, 28, 28)
+        h = F.max_pool2d(F.relu(F.conv2d(h, seg("conv1.w"), seg("conv1.b"), padding=1)), 2)
+        h = F.max_pool2d(F.relu(F.conv2d(h, seg("conv2.w"), seg("conv2.b"), padding=1)), 2)
+        h = F.relu(F.linear(h.flatten(1), seg("fc1.w"), seg("fc1.b")))
+        z = F.linear(h, seg("fc2.w"), seg("fc2.b"))
+        assert np.abs(z.numpy() - logits[w]).max() < 1e-11
+        assert abs(float(F.cross_entropy(z, torch.tensor(y[w].astype(np.int64)))) - loss[w]) < 1e-12
+        assert (z.argmax(1).numpy() == am[w]).all()
+        assert correct[w] == int((z.argmax(1).numpy() == y[w]).sum())
+    # with dropout the logits differ: the evaluation pass really switched it off
+    _, _, _, z_train = cnn.workers_grad_step([theta] * W, [0, 1], x, y, 7, 0, 0.25)
+    assert np.abs(z_train - logits).max() > 1e-3
+    # zero weights: every logit is zero, the loss is ln 10, the predicted class is 0
+    l0, a0, c0, _ = cnn.workers_eval([np.zeros(cnn.P, dtype=np.float32)], x[:1], y[:1])
+    assert abs(l0[0] - np.log(10.0)) < 1e-12 and (a0 == 0).all() and c0[0] == int((y[0] == 0).sum())

@@ -323,3 +323,83 @@ def test_checkpoint_slots_keep_the_most_recent_ones():
         assert (th == kept[v]).all()
     s.kill(0)
     assert s.restore() == 8 and (s.head() == kept[8]).all()
+
+
+# ---- treatments of stale gradients (design section, closing remarks on the stateless server) ----------------------
+
+def _unit_grads(norms, P=P, seed=0):
+    """Gradients of exactly known Euclidean norm: a few +-1 entries scaled."""
+    rng = np.random.default_rng(seed)
+    out = np.zeros((len(norms), P), dtype=np.float32)
+    for k, nrm in enumerate(norms):
+        pos = rng.choice(P, size=16, replace=False)
+        out[k, pos] = np.float32(nrm / 4.0) * rng.choice([-1.0, 1.0], size=16).astype(np.float32)   # sqrt(16) = 4
+    return out
+
+
+def test_clipping_by_global_norm_closed_form():
+    theta = synth.init_params(1)
+    norms = [0.5, 2.0, 8.0, 1.0]           # powers of two: every scaled entry is exact in fp32
+    g = _unit_grads(norms)
+    s = ops.OraclePS(theta, external_store=True)
+    s.enqueue(g, range(4), [0] * 4, 0)
+    s.apply(ops.REPLAY, 0.5, clip_norm=1.0)
+    clipped = np.stack([g[k].astype(np.float64) * min(1.0, 1.0 / norms[k]) for k in range(4)])
+    expect = (theta.astype(np.float64) - 0.5 / 4 * clipped.sum(0)).astype(np.float32)
+    assert (s.head() == expect).all()
+    for k in range(4):                      # what was applied has norm min(norm, c)
+        assert abs(np.linalg.norm(clipped[k]) - min(norms[k], 1.0)) < 1e-12
+    # a bound above every norm changes nothing, bit for bit
+    a = ops.OraclePS(theta, external_store=True); a.enqueue(g, range(4), [0] * 4, 0); a.apply(ops.REPLAY, 0.5, clip_norm=100.0)
+    b = ops.OraclePS(theta, external_store=True); b.enqueue(g, range(4), [0] * 4, 0); b.apply(ops.REPLAY, 0.5)
+    assert (a.head() == b.head()).all()
+    with pytest.raises(ops.PSError):
+        a.enqueue(g, range(4), [1] * 4, 0); a.apply(ops.REPLAY, 0.5, clip_norm=0.0)
+
+
+def test_staleness_scaling_closed_forms():
+    theta = synth.init_params(1)
+    g = _small_grads(6, seed=12)
+    lr32 = np.float64(np.float32(0.01))
+    # replay after an outage: every queued gradient was computed on the stored version, so they are all equally stale
+    # and the treatment is a plain learning-rate scale of 1 / (1 + alpha * tau)
+    s = ops.OraclePS(theta, external_store=True)
+    _steps(s, 3, 400)                                   # head is version 3
+    s.enqueue(g, range(6), [1] * 6, 0)                  # read at version 1: tau = 2
+    t = ops.OraclePS(s.head(), external_store=True)
+    t.enqueue(g, range(6), [0] * 6, 0)
+    s.apply(ops.REPLAY, 0.01, staleness_alpha=0.5)
+    t.apply(ops.REPLAY, 0.01, scale=0.5)                # 1 / (1 + 0.5 * 2)
+    assert (s.head() == t.head()).all()
+    # alpha = 0 is the plain step
+    a = ops.OraclePS(theta); a.enqueue(g, range(6), [0] * 6, 0); a.apply(ops.SYNC, 0.01, staleness_alpha=0.0)
+    b = ops.OraclePS(theta); b.enqueue(g, range(6), [0] * 6, 0); b.apply(ops.SYNC, 0.01)
+    assert (a.head() == b.head()).all()
+    # async: the j-th update in arrival order is applied to version v0 + j; mixed base versions
+    s = ops.OraclePS(theta, ring_depth=4)
+    _steps(s, 2, 500)                                   # v0 = 2
+    base = [2, 0, 1, 2, 0, 1]
+    order = [4, 1, 0, 5, 2, 3]
+    s.enqueue(g, range(6), base, 0)
+    run = s.head().astype(np.float64)
+    v0 = s.version
+    s.apply(ops.ASYNC, 0.01, order=order, staleness_alpha=0.25)
+    for j, k in enumerate(order):
+        run = (run - lr32 / (1.0 + np.float64(0.25) * (v0 + j - base[k])) * g[k].astype(np.float64)).astype(np.float32).astype(np.float64)
+    assert (s.head() == run.astype(np.float32)).all() and s.version == v0 + 6
+    # a base version from the future is refused
+    s.enqueue(g[:1], [0], [s.version + 1], 0)
+    with pytest.raises(ops.PSError):
+        s.apply(ops.SYNC, 0.01, staleness_alpha=0.1)
+
+
+def test_clipping_and_staleness_compose():
+    theta = synth.init_params(1)
+    g = _unit_grads([4.0, 0.25], seed=3)
+    s = ops.OraclePS(theta)
+    _steps(s, 4, 600)
+    th0 = s.head().astype(np.float64)
+    s.enqueue(g, [0, 1], [4, 2], 0)                     # tau = 0 and 2
+    s.apply(ops.SYNC, 1.0, clip_norm=1.0, staleness_alpha=1.0)
+    expect = th0 - 1.0 / 2 * (g[0].astype(np.float64) * 0.25 * 1.0 + g[1].astype(np.float64) * 1.0 / 3.0)
+    assert np.abs(s.head() - expect).max() <= 2.0 ** -24 * max(1.0, np.abs(expect).max())
