@@ -11,16 +11,23 @@
 //       Xs[(sy, sx)][p] = x[2 py + sy - 1][2 px + sx - 1]   (sy, sx = 0..3: the sixteen stride-2 shifts of the image)
 //   dW[oc][ky][kx]      = sum over w of T[(w, oc)][(wy + ky, wx + kx)],    db[oc] = sum over w, p of G_w[oc][p]
 //
-// i.e. per sample one product of M = 64, N = 24 (sixteen shifts, a row of ones whose products are the bias gradient,
-// seven rows of zeros), K = 208 (196 positions, padded): thirteen tcgen05 MMAs of K = 16, accumulated in tensor
-// memory over all samples of a worker.  Both operands have the position index contiguous (core matrices of 8 rows x
-// 8 positions); the 128-byte core matrices of a row group lie 144 bytes apart, so that threads that fill consecutive
-// core matrices store to different shared-memory banks.
+// Per sample that is a product of 64 x 24 (sixteen shifts, a row of ones whose products are the bias gradient, seven
+// rows of zeros) over K = 208 (196 positions, padded).  A tcgen05 MMA costs some forty to sixty cycles however small
+// it is, so two samples of a worker share every MMA: their row blocks are stacked (M = 128) and their shift blocks
+// too (N = 48); the two diagonal blocks of the 128 x 48 product are the two samples' sums, the off-diagonal blocks
+// are never read.  Thirteen MMAs of K = 16 per pair, accumulated in tensor memory over all pairs of a worker; a
+// worker's odd last sample runs as a pair whose second shift block is zero.
+// Both operands have the position index contiguous (core matrices of 8 rows x 8 positions); the 128-byte core
+// matrices of a row group lie 144 bytes apart, so that threads that fill consecutive core matrices store to
+// different shared-memory banks.
 // One CTA per SM walks over a contiguous range of rows (sorted worker, sample); where the range passes from one
-// worker to the next, and at its end, the accumulator is written out as a partial sum that a later kernel adds in a
-// fixed order.  The images arrive by TMA tile loads whose box starts outside the image (zero border for free), the
-// pooled gradients (BF16, as the second convolution's input-gradient kernel stores them) and the decisions by bulk
-// copies, two samples ahead.  Every mbarrier wait is bounded.
+// worker to the next, and at its end, the accumulator is written out as partial sums that a later kernel adds in a
+// fixed order.  Two groups of eight warps build the operands, one sample of the pair each; a sample's inputs (image,
+// pooled gradients in BF16 as the second convolution's input-gradient kernel stores them, pooling decisions) arrive
+// by bulk copies issued by a warp of their own into five raw slots used in turn, i.e. two to three pairs ahead.
+// What bounds the kernel is shared-memory traffic: per pair the tensor core reads 73 KB of operands (three quarters
+// of the row operand are the zeros of the window elements that did not win), the staging warps write 66 KB and the
+// copies 25 KB.  Every mbarrier wait is bounded.
 #include "device_common.cuh"
 #include "kernels.h"
 #include "tc5_common.cuh"
@@ -29,28 +36,29 @@ namespace psk {
 
 namespace {
 
-constexpr int D1_LOAD_WARPS = 16;                        // two groups: group g stages samples n = g, g + 2, ...
+constexpr int D1_LOAD_WARPS = 16;                        // two groups: group h stages sample h of every pair
 constexpr int D1_GW = D1_LOAD_WARPS / 2;                 // warps per group
 constexpr int D1_GT = 32 * D1_GW;                        // threads per group
-constexpr int D1_THREADS = 32 * (1 + D1_LOAD_WARPS + 4); // warp 0: MMA issue and tensor memory; the last four warps write out
+constexpr int D1_THREADS = 32 * (1 + D1_LOAD_WARPS + 4 + 1); // warp 0: MMA issue and tensor memory; then the staging warps, four
+                                                            // write-out warps, and the warp that issues the loads
 constexpr int D1_CHUNKS = 26;                            // 8-position chunks of the 208 contraction indices of a sample
 constexpr int D1_CHUNK_PITCH = 144;                      // bytes from one core matrix of a row group to the next
 constexpr int D1_GROUP_BYTES = D1_CHUNKS * D1_CHUNK_PITCH;   // 3,744: one group of 8 operand rows
-constexpr int D1_A_GROUPS = 8;                           // (window element, channel octet)
-constexpr int D1_B_GROUPS = 3;                           // shifts 0..7, shifts 8..15, ones row + zero rows
+constexpr int D1_A_GROUPS = 16;                          // (sample of the pair, window element, channel octet)
+constexpr int D1_B_GROUPS = 6;                           // per sample: shifts 0..7, shifts 8..15, ones row + zero rows
 constexpr int D1_A_BYTES = D1_A_GROUPS * D1_GROUP_BYTES;
-constexpr int D1_STAGE_BYTES = ((D1_A_GROUPS + D1_B_GROUPS) * D1_GROUP_BYTES + 127) / 128 * 128;    // 41,216
-constexpr int D1_BOX_W = 36, D1_BOX_H = 30;              // image box: columns -4..31 (a 16-byte aligned start), rows -1..28
-constexpr int D1_BOX_BYTES = D1_BOX_W * D1_BOX_H * 4;    // 4,320
-constexpr int D1_RAW_X = 4352;                           // box padded to a multiple of 128 bytes
+constexpr int D1_STAGE_BYTES = ((D1_A_GROUPS + D1_B_GROUPS) * D1_GROUP_BYTES + 127) / 128 * 128;    // 82,432
+constexpr int D1_NSTAGE = 2;                             // operand stages (pair u -> stage u % 2)
+constexpr int D1_RAW_ZERO = 16;                          // a zero word at the start of a raw slot: what elements outside the image read
+constexpr int D1_RAW_X = IMG * IMG * 4;                  // 3,136: the image as it lies in memory
 constexpr int D1_RAW_G = P1_ELEMS * 2, D1_RAW_CODE = P1_ELEMS;
-constexpr int D1_RAW_SLOT = (D1_RAW_X + D1_RAW_G + D1_RAW_CODE + 127) / 128 * 128;     // 13,824
-constexpr int D1_NRAW = 4;                               // raw input slots: each group's copies run two of its samples ahead
-constexpr int D1_SMEM = 2 * D1_STAGE_BYTES + D1_NRAW * D1_RAW_SLOT + 256 + 128;
-constexpr int D1_NACC = 4;                               // accumulators used in turn: an MMA that adds to the sum of the one before
-                                                         // it waits for that one to finish, and these MMAs are short
-constexpr int D1_TMEM_COLS = 32 * D1_NACC;               // 24 accumulator columns each, 32 apart
+constexpr int D1_RAW_BYTES = D1_RAW_X + D1_RAW_G + D1_RAW_CODE;                        // 12,544 copied per sample
+constexpr int D1_RAW_SLOT = (D1_RAW_ZERO + D1_RAW_BYTES + 127) / 128 * 128;            // 12,672
+constexpr int D1_NRAW = 5;                               // raw input slots: the q-th sample of the range -> slot q % 5
+constexpr int D1_SMEM = D1_NSTAGE * D1_STAGE_BYTES + D1_NRAW * D1_RAW_SLOT + 256 + 128;
+constexpr int D1_TMEM_COLS = 64;                         // 48 accumulator columns
 constexpr int D1_KSTEPS = D1_CHUNKS / 2;                 // 13
+constexpr int D1_SUBSLOTS = 8;                           // partial sums per range: (sample of the pair, window element)
 static_assert(D1_SMEM <= 227 * 1024, "shared memory");
 static_assert(D1_GT == 256, "the item split below assumes 256 threads per group");
 
@@ -59,7 +67,7 @@ __host__ __device__ constexpr uint32_t d1_idesc(int m, int n) {     // fp32 accu
 }
 
 struct D1Bars {
-  uint64_t op_full[2], op_empty[2], raw_full[D1_NRAW], raw_empty[D1_NRAW], acc_full, acc_empty;
+  uint64_t op_full[D1_NSTAGE], op_empty[D1_NSTAGE], raw_full[D1_NRAW], raw_empty[D1_NRAW], acc_full, acc_empty;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -69,26 +77,34 @@ struct D1Bars {
 // sign-replicating byte permute below looks at.
 __device__ __forceinline__ uint32_t win_flags(uint32_t onehot, int w) { return onehot << (7 - w); }
 
+// The rows [row, r1) of a CTA are taken in units of two consecutive samples of one worker, or of one sample where a
+// worker's (or the range's) last sample has no partner.  After a unit with `flush` the accumulator is written out.
+struct D1Unit { int row, n; bool flush; };
+__device__ __forceinline__ bool d1_next_unit(int& row, int r1, int b, D1Unit& u) {
+  if (row >= r1) return false;
+  const int wend = (row / b + 1) * b;            // first row of the next worker
+  u.row = row;
+  u.n = (row + 1 < r1 && row + 1 < wend) ? 2 : 1;
+  row += u.n;
+  u.flush = row == r1 || row == wend;
+  return true;
+}
+
 // Rows (sorted worker, sample) are split into gridDim.x contiguous ranges of seg_len.  Partial sums of worker s go
-// to part1[s][4 (range index - first range of s) + window element].
-__global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_constant__ CUtensorMap xmap, GradStepArgs a, WorkerTable wt,
-                                                              Workspace ws, int seg_len, int slots) {
+// to part1[s][8 (range index - first range of s) + 4 (sample of the pair) + window element].
+__global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(GradStepArgs a, WorkerTable wt, Workspace ws, int seg_len, int slots) {
   extern __shared__ __align__(1024) uint8_t sm[];
-  uint8_t* raw = sm + 2 * D1_STAGE_BYTES;
+  uint8_t* raw = sm + D1_NSTAGE * D1_STAGE_BYTES;
   D1Bars* bars = reinterpret_cast<D1Bars*>(raw + D1_NRAW * D1_RAW_SLOT);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int total = a.W * a.b;
-  const int r0 = blockIdx.x * seg_len, r1 = min(r0 + seg_len, total), n_samples = r1 - r0;
+  const int r0 = blockIdx.x * seg_len, r1 = min(r0 + seg_len, total);
 
-  // Operand stages start as zeros: positions 196..207, the zero rows of B, and every entry of A that no sample's
-  // staging writes.  The ones row of B (row 0 of its third group) is written once.
-  for (int i = tid; i < 2 * D1_STAGE_BYTES / 16; i += D1_THREADS) reinterpret_cast<uint4*>(sm)[i] = make_uint4(0u, 0u, 0u, 0u);
-  __syncthreads();
-  for (int i = tid; i < 2 * D1_CHUNKS; i += D1_THREADS)
-    *reinterpret_cast<uint4*>(sm + (i / D1_CHUNKS) * D1_STAGE_BYTES + D1_A_BYTES + 2 * D1_GROUP_BYTES + (i % D1_CHUNKS) * D1_CHUNK_PITCH) =
-        make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
+  // Operand stages start as zeros: positions 196..207, the zero rows of B, and every entry that no staging writes.
+  for (int i = tid; i < D1_NSTAGE * D1_STAGE_BYTES / 16; i += D1_THREADS) reinterpret_cast<uint4*>(sm)[i] = make_uint4(0u, 0u, 0u, 0u);
+  if (tid < D1_NRAW) *reinterpret_cast<uint4*>(raw + tid * D1_RAW_SLOT) = make_uint4(0u, 0u, 0u, 0u);
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->op_full[i], D1_GW); mbar_init(&bars->op_empty[i], 1); }
+    for (int i = 0; i < D1_NSTAGE; ++i) { mbar_init(&bars->op_full[i], D1_LOAD_WARPS); mbar_init(&bars->op_empty[i], 1); }
     for (int i = 0; i < D1_NRAW; ++i) { mbar_init(&bars->raw_full[i], 1); mbar_init(&bars->raw_empty[i], D1_GW); }
     mbar_init(&bars->acc_full, 1);
     mbar_init(&bars->acc_empty, 4);
@@ -108,25 +124,25 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_const
   if (warp == 0) {
     // ---------------- MMA issue
     if (lane == 0) {
-      constexpr uint32_t idesc = d1_idesc(64, 24);
-      int writes = 0;
+      constexpr uint32_t idesc = d1_idesc(128, 48);
+      int writes = 0, row = r0;
       bool fresh = true;                       // the next MMA starts a new sum
-      for (int n = 0; n < n_samples; ++n) {
-        const int st = n & 1;
-        if (!mbar_wait(&bars->op_full[st], (n >> 1) & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
+      D1Unit un;
+      for (int u = 0; d1_next_unit(row, r1, a.b, un); ++u) {
+        const int st = u & 1;
+        if (!mbar_wait(&bars->op_full[st], (u >> 1) & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
         tc_fence_after();
         const uint32_t a_lo = plain_desc_lo(smem_u32(sm) + st * D1_STAGE_BYTES, D1_CHUNK_PITCH);
         const uint32_t b_lo = plain_desc_lo(smem_u32(sm) + st * D1_STAGE_BYTES + D1_A_BYTES, D1_CHUNK_PITCH);
         // contraction indices 16 ks .. 16 ks + 15: two core matrices, 2 x 144 bytes further along every row group
 #pragma unroll
         for (int ks = 0; ks < D1_KSTEPS; ++ks)
-          umma_f16_split(tmem + (ks % D1_NACC) * 32, a_lo + ks * (2 * D1_CHUNK_PITCH / 16), plain_desc_hi(D1_GROUP_BYTES),
-                         b_lo + ks * (2 * D1_CHUNK_PITCH / 16), plain_desc_hi(D1_GROUP_BYTES), idesc, (ks < D1_NACC && fresh) ? 0u : 1u);
+          umma_f16_split(tmem, a_lo + ks * (2 * D1_CHUNK_PITCH / 16), plain_desc_hi(D1_GROUP_BYTES), b_lo + ks * (2 * D1_CHUNK_PITCH / 16),
+                         plain_desc_hi(D1_GROUP_BYTES), idesc, (ks == 0 && fresh) ? 0u : 1u);
         fresh = false;
         umma_commit(&bars->op_empty[st]);
-        const int row = r0 + n;
-        if (row + 1 == r1 || (row + 1) % a.b == 0) {
-          // last row of the range or of a worker: hand the sum to the write-out warps and wait until they have read it
+        if (un.flush) {
+          // last rows of the range or of a worker: hand the sums to the write-out warps and wait until they have read them
           umma_commit(&bars->acc_full);
           if (!mbar_wait(&bars->acc_empty, writes & 1)) { bars->abort_flag = 1; break; }
           tc_fence_after();
@@ -136,53 +152,51 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_const
       }
     }
   } else if (warp <= D1_LOAD_WARPS) {
-    // ---------------- staging: group g (D1_GW warps) builds the operands of samples n = g, g + 2, ... in stage g
-    const int grp = (warp - 1) / D1_GW, gt_ = (warp - 1 - grp * D1_GW) * 32 + lane;      // thread index inside the group
-    auto issue = [&](int n) {            // one thread: the three inputs of sample r0 + n
-      const int row = r0 + n, s = row / a.b, i = row - s * a.b;
-      uint8_t* dst = raw + (n & 3) * D1_RAW_SLOT;
-      uint64_t* bar = &bars->raw_full[n & 3];
-      mbar_expect_tx(bar, D1_BOX_BYTES + D1_RAW_G + D1_RAW_CODE);
-      tma_load_3d(dst, &xmap, bar, -4, -1, wt.src[s] * a.b + i);
-      bulk_load(dst + D1_RAW_X, reinterpret_cast<const uint8_t*>(ws.dp1) + (int64_t)row * (P1_ELEMS * 4), D1_RAW_G, bar);
-      bulk_load(dst + D1_RAW_X + D1_RAW_G, ws.code1 + (int64_t)row * P1_ELEMS, D1_RAW_CODE, bar);
-    };
+    // ---------------- staging: group h (D1_GW warps) builds the operands of sample h of every pair
+    const int h = (warp - 1) / D1_GW, gt_ = (warp - 1 - h * D1_GW) * 32 + lane;      // thread index inside the group
     // A item of this thread: (channel quad aq, chunk ac, half ah) = four pooled positions of four channels.
     // 4 quads x (24 chunks x 2 halves + the first half of chunk 24) = 196 items; the other threads have none.
     const int aq = gt_ / 49, arem = gt_ - aq * 49, ac = arem >> 1, ah = arem & 1;
     const bool a_item = gt_ < 196;
     const int a_src = (aq * 196 + 8 * ac + 4 * ah);                       // (quad, first position) in units of one position's 4 channels
-    const int a_dst = ((aq >> 1)) * D1_GROUP_BYTES + ac * D1_CHUNK_PITCH + ((aq & 1) * 4) * 16 + ah * 8;   // window element 0, channel 0 of the quad
+    const int a_dst = (8 * h + (aq >> 1)) * D1_GROUP_BYTES + ac * D1_CHUNK_PITCH + ((aq & 1) * 4) * 16 + ah * 8;   // window element 0, channel 0 of the quad
     // B items of this thread: shift bn = (sy, sx) and chunks bc0 = gt_ / 16 and bc0 + 16 (the latter for bc0 < 9;
-    // chunk 24 holds positions 192..195 only).  The word offsets of the sixteen elements in the image box are fixed
-    // for the whole kernel (box row 2 py + sy is image row 2 py + sy - 1, box column 2 px + sx + 3 is image column
-    // 2 px + sx - 1) and are worked out once.
+    // chunk 24 holds positions 192..195 only); threads 0..24 also write the ones row's chunk gt_.  Where the sixteen
+    // elements lie in the raw slot is fixed for the whole kernel and worked out once: element (sy, sx) of pooled
+    // position (py, px) is image pixel (2 py + sy - 1, 2 px + sx - 1); a pixel outside the image, and a position past
+    // 195, reads the slot's zero word.
     const int bn = gt_ & 15, sy = bn >> 2, sx = bn & 3, bc0 = gt_ >> 4;
-    const int b_dst = (bn >> 3) * D1_GROUP_BYTES + (bn & 7) * 16;
-    int b_off[2][8];                     // word 0 of the box is outside the image (always zero): positions past 195 read it
+    const int b_dst = D1_A_BYTES + (3 * h + (bn >> 3)) * D1_GROUP_BYTES + (bn & 7) * 16;
+    const int ones_dst = D1_A_BYTES + (3 * h + 2) * D1_GROUP_BYTES + gt_ * D1_CHUNK_PITCH;
+    int b_off[2][8];
 #pragma unroll
-    for (int h = 0; h < 2; ++h)
+    for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        const int p = 8 * (bc0 + 16 * h) + j, py = p / 14, px = p - 14 * py;
-        b_off[h][j] = p < 196 ? sy * D1_BOX_W + sx + 3 + 2 * py * D1_BOX_W + 2 * px : 0;
+        const int p = 8 * (bc0 + 16 * hh) + j, py = p / 14, px = p - 14 * py;
+        const int iy = 2 * py + sy - 1, ix = 2 * px + sx - 1;
+        b_off[hh][j] = (p < 196 && iy >= 0 && iy < IMG && ix >= 0 && ix < IMG) ? D1_RAW_ZERO / 4 + iy * IMG + ix : 0;
       }
 
-    if (gt_ == 0) { if (grp < n_samples) issue(grp); if (grp + 2 < n_samples) issue(grp + 2); }
-    for (int n = grp; n < n_samples; n += 2) {
-      const int slot = n & 3;
-      bool ok = mbar_wait(&bars->raw_full[slot], (n >> 2) & 1);
-      if (ok && n >= 2) ok = mbar_wait(&bars->op_empty[grp], ((n >> 1) - 1) & 1);
+    int row = r0, q0 = 0;                            // q0: samples of the range before this unit
+    D1Unit un;
+    for (int u = 0; d1_next_unit(row, r1, a.b, un); q0 += un.n, ++u) {
+      const int st = u & 1, q = q0 + h, slot = q % D1_NRAW;      // this group's sample is the range's q-th: the (q / 5)-th use of its slot
+      const bool mine = h < un.n;                    // an odd last sample: group 1 only clears its shift block
+      bool ok = true;
+      if (mine) ok = mbar_wait(&bars->raw_full[slot], (q / D1_NRAW) & 1);
+      if (ok && u >= 2) ok = mbar_wait(&bars->op_empty[st], ((u >> 1) - 1) & 1);      // the MMAs of unit u - 2 have read the stage
       if (!__all_sync(0xffffffffu, ok) || bars->abort_flag) { bars->abort_flag = 1; break; }
       const uint8_t* rslot = raw + slot * D1_RAW_SLOT;
       const float* img = reinterpret_cast<const float*>(rslot);
-      uint8_t* stage = sm + grp * D1_STAGE_BYTES;
-      if (a_item) {
+      const uint8_t* rg = rslot + D1_RAW_ZERO + D1_RAW_X;
+      uint8_t* stage = sm + st * D1_STAGE_BYTES;
+      if (mine && a_item) {
         // four positions of four channels: the gradients as two 16-byte loads ([position][4 channels] BF16), the
         // decisions as one ([position][4 channels] bytes)
-        const uint4 g01 = reinterpret_cast<const uint4*>(rslot + D1_RAW_X)[a_src >> 1];          // positions 0, 1: {c0c1, c2c3, c0c1, c2c3}
-        const uint4 g23 = reinterpret_cast<const uint4*>(rslot + D1_RAW_X)[(a_src >> 1) + 1];
-        const uint4 cd = reinterpret_cast<const uint4*>(rslot + D1_RAW_X + D1_RAW_G)[a_src >> 2];
+        const uint4 g01 = reinterpret_cast<const uint4*>(rg)[a_src >> 1];          // positions 0, 1: {c0c1, c2c3, c0c1, c2c3}
+        const uint4 g23 = reinterpret_cast<const uint4*>(rg)[(a_src >> 1) + 1];
+        const uint4 cd = reinterpret_cast<const uint4*>(rg + D1_RAW_G)[a_src >> 2];
         // per channel, the position pairs (0, 1) and (2, 3) as one word each
         const uint32_t v[4][2] = {{prmt(g01.x, g01.z, 0x5410u), prmt(g23.x, g23.z, 0x5410u)},
                                   {prmt(g01.x, g01.z, 0x7632u), prmt(g23.x, g23.z, 0x7632u)},
@@ -200,63 +214,76 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(const __grid_const
         }
       }
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int bc = bc0 + 16 * h;
+      for (int hh = 0; hh < 2; ++hh) {
+        const int bc = bc0 + 16 * hh;
         if (bc < 25) {
-          float xv[8];
+          uint4 o = make_uint4(0u, 0u, 0u, 0u);        // no second sample: its shift block is zero, so whatever its row block
+          if (mine) {                                  // still holds from an earlier pair adds nothing
+            float xv[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) xv[j] = img[b_off[h][j]];
-          *reinterpret_cast<uint4*>(stage + D1_A_BYTES + b_dst + bc * D1_CHUNK_PITCH) =
-              make_uint4(bf16_pair(xv[0], xv[1]), bf16_pair(xv[2], xv[3]), bf16_pair(xv[4], xv[5]), bf16_pair(xv[6], xv[7]));
+            for (int j = 0; j < 8; ++j) xv[j] = img[b_off[hh][j]];
+            o = make_uint4(bf16_pair(xv[0], xv[1]), bf16_pair(xv[2], xv[3]), bf16_pair(xv[4], xv[5]), bf16_pair(xv[6], xv[7]));
+          }
+          *reinterpret_cast<uint4*>(stage + b_dst + bc * D1_CHUNK_PITCH) = o;
         }
+      }
+      if (gt_ < 25) {
+        const uint32_t one2 = mine ? 0x3F803F80u : 0u;                       // the ones row (bias gradient), zero likewise
+        *reinterpret_cast<uint4*>(stage + ones_dst) = gt_ < 24 ? make_uint4(one2, one2, one2, one2) : make_uint4(one2, one2, 0u, 0u);
       }
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) { mbar_arrive(&bars->op_full[grp]); mbar_arrive(&bars->raw_empty[slot]); }
-      if (gt_ == 0 && n + 4 < n_samples) {
-        if (!mbar_wait(&bars->raw_empty[slot], (n >> 2) & 1)) { bars->abort_flag = 1; break; }
-        issue(n + 4);
-      }
+      if (lane == 0) { mbar_arrive(&bars->op_full[st]); if (mine) mbar_arrive(&bars->raw_empty[slot]); }
+    }
+  } else if (warp == D1_LOAD_WARPS + 5) {
+    // ---------------- loads: one thread issues every sample's three bulk copies into the raw slots in turn; before a
+    // slot's k-th reuse it waits until the eight warps that staged the slot's previous sample have read it
+    if (lane == 0) {
+      int row = r0, q = 0;
+      D1Unit un;
+      bool ok = true;
+      while (ok && d1_next_unit(row, r1, a.b, un))
+        for (int h = 0; h < un.n; ++h, ++q) {
+          const int slot = q % D1_NRAW, use = q / D1_NRAW;
+          if (use > 0 && (!mbar_wait(&bars->raw_empty[slot], (use - 1) & 1) || bars->abort_flag)) { bars->abort_flag = 1; ok = false; break; }
+          const int r = un.row + h, s = r / a.b, i = r - s * a.b;
+          uint8_t* dst = raw + slot * D1_RAW_SLOT + D1_RAW_ZERO;
+          uint64_t* bar = &bars->raw_full[slot];
+          mbar_expect_tx(bar, D1_RAW_BYTES);
+          bulk_load(dst, a.x + ((int64_t)wt.src[s] * a.b + i) * (IMG * IMG), D1_RAW_X, bar);
+          bulk_load(dst + D1_RAW_X, reinterpret_cast<const uint8_t*>(ws.dp1) + (int64_t)r * (P1_ELEMS * 4), D1_RAW_G, bar);
+          bulk_load(dst + D1_RAW_X + D1_RAW_G, ws.code1 + (int64_t)r * P1_ELEMS, D1_RAW_CODE, bar);
+        }
     }
   } else {
-    // ---------------- write-out: a warp reads the accumulator lanes 32 (warp % 4) .. + 31.  An accumulator of 64 rows
-    // keeps rows 16 q .. 16 q + 15 in the first sixteen lanes of quarter q, so warp q holds window element q = (wy, wx)
-    // and lane oc < 16 one output channel.  Each warp writes its window element's share of the 160 sums to a partial
-    // slot of its own (the final reduction adds the four in a fixed order), so the warps exchange nothing.
-    const int quarter = warp & 3;
-    int writes = 0;
-    for (int row = r0; row < r1; ++row) {
-      if (!(row + 1 == r1 || (row + 1) % a.b == 0)) continue;
+    // ---------------- write-out: warp q reads the accumulator lanes 32 q .. 32 q + 31 = rows (sample q / 2 of the pair,
+    // window elements 2 (q % 2) and 2 (q % 2) + 1, 16 channels each); a sample's sums are in its own 24 columns.  Every
+    // (sample, window element) writes its share of the 160 sums to a partial slot of its own (the final reduction adds
+    // them in a fixed order), so the warps exchange nothing.
+    const int quarter = warp & 3, half = quarter >> 1, my_w = 2 * (quarter & 1) + (lane >> 4), oc = lane & 15;
+    int writes = 0, row = r0;
+    D1Unit un;
+    while (d1_next_unit(row, r1, a.b, un)) {
+      if (!un.flush) continue;
       if (!mbar_wait(&bars->acc_full, writes & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
       tc_fence_after();
-      float v0[16], vb = 0.f;
-#pragma unroll
-      for (int j = 0; j < 16; ++j) v0[j] = 0.f;
-#pragma unroll
-      for (int acc = 0; acc < D1_NACC; ++acc) {      // the accumulators are added in a fixed order
-        uint32_t t0[16], t1[16];
-        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 32), t0);
-        tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 32 + 16), t1);      // column 16 = bias, 17..23 zero rows, 24..31 unused
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 16; ++j) v0[j] += __uint_as_float(t0[j]);
-        vb += __uint_as_float(t1[0]);
-      }
+      uint32_t v0[16], v1[16];
+      tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(24 * half), v0);
+      tmem_ld16(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(24 * half + 16), v1);      // first column: the bias gradient
+      tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->acc_empty);
-      const int s = row / a.b;
-      float* part = ws.part1 + (((int64_t)s * slots + (blockIdx.x - (s * a.b) / seg_len)) * 4 + quarter) * C1_GRAD;
-      if (lane < 16) {
-        // dW[oc][ky][kx] takes shift (wy + ky, wx + kx) of this window element
+      const int s = un.row / a.b;
+      float* part = ws.part1 + (((int64_t)s * slots + (blockIdx.x - (s * a.b) / seg_len)) * D1_SUBSLOTS + 4 * half + my_w) * C1_GRAD;
+      // dW[oc][ky][kx] takes shift (wy + ky, wx + kx) of this window element
 #pragma unroll
-        for (int w = 0; w < 4; ++w)
-          if (w == quarter) {
+      for (int w = 0; w < 4; ++w)
+        if (w == my_w) {
 #pragma unroll
-            for (int tap = 0; tap < 9; ++tap) part[lane * 9 + tap] = v0[((w >> 1) + tap / 3) * 4 + (w & 1) + tap % 3];
-          }
-        part[144 + lane] = vb;
-      }
+          for (int tap = 0; tap < 9; ++tap) part[oc * 9 + tap] = __uint_as_float(v0[((w >> 1) + tap / 3) * 4 + (w & 1) + tap % 3]);
+        }
+      part[144 + oc] = __uint_as_float(v1[0]);
       ++writes;
     }
   }
@@ -280,15 +307,10 @@ int configure_c1d5_kernels() {
   return cudaFuncSetAttribute(conv1_dw_tc5, cudaFuncAttributeMaxDynamicSharedMemorySize, D1_SMEM) == cudaSuccess ? 0 : -1;
 }
 
-// Returns the number of partial-sum slots reserved per worker (the stride of part1: four per range), or -1;
-// *seg_len receives the length of a CTA's range of rows: worker s owns four partial sums per range that meets its rows.
+// Returns the number of partial-sum slots reserved per worker (the stride of part1: eight per range), or -1;
+// *seg_len receives the length of a CTA's range of rows: worker s owns eight partial sums per range that meets its rows.
 int launch_conv1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const Workspace& ws, cudaStream_t st, Profiler* prof,
                         int* seg_len) {
-  CUtensorMap xmap;
-  const uint64_t dims[3] = {IMG, IMG, (uint64_t)a.W * a.b};
-  const uint64_t strides[2] = {IMG * 4, IMG * IMG * 4};
-  const uint32_t box[3] = {D1_BOX_W, D1_BOX_H, 1};
-  if (!encode_tensor_map_f32(&xmap, a.x, 3, dims, strides, box)) return -1;
   const int total = a.W * a.b;
   int grid = total / 16;                  // a range is at least 16 rows long (bounds the partial sums per worker)
   if (grid > g_sm_count) grid = g_sm_count;
@@ -296,9 +318,9 @@ int launch_conv1_dw_tc5(const GradStepArgs& a, const WorkerTable& wt, const Work
   const int len = (total + grid - 1) / grid;
   grid = (total + len - 1) / len;
   const int slots = (a.b - 1) / len + 2;
-  TIMED(K_CONV1_BWD, (conv1_dw_tc5<<<grid, D1_THREADS, D1_SMEM, st>>>(xmap, a, wt, ws, len, slots)));
+  TIMED(K_CONV1_BWD, (conv1_dw_tc5<<<grid, D1_THREADS, D1_SMEM, st>>>(a, wt, ws, len, slots)));
   *seg_len = len;
-  return 4 * slots;
+  return D1_SUBSLOTS * slots;
 }
 
 }  // namespace psk

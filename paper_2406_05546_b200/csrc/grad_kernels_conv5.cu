@@ -124,12 +124,18 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Gr
   const float* theta = gt.theta[grp];
   const int n_tiles = (r_end - r_begin + 1) / 2;
 
-  // the stacked weight operand: block rb holds the 32 filters of tap fold.tap_of_block[rb], one row per output channel
+  // the filter bank comes in once with coalesced 16-byte loads (into the tile buffers, which are cleared afterwards) ...
+  float* wtmp = reinterpret_cast<float*>(smem);
+  for (int idx = tid; idx < 4608 / 4; idx += F_THREADS) reinterpret_cast<float4*>(wtmp)[idx] = reinterpret_cast<const float4*>(theta + OFF_C2W)[idx];
+  if (tid < 32) bias[tid] = theta[OFF_C2B + tid];
+  __syncthreads();
+  // ... and is laid out as the stacked weight operand: block rb holds the 32 filters of tap fold.tap_of_block[rb], one
+  // row per output channel
   for (int idx = tid; idx < F_W_BLOCKS * 512; idx += F_THREADS) {
     const int rb = idx >> 9, oc = (idx >> 4) & 31, ic = idx & 15;
-    Wk[((ic >> 3) * F_W_ROWS + rb * 32 + oc) * 8 + (ic & 7)] = bf16_bits(theta[OFF_C2W + (oc * 16 + ic) * 9 + fold.tap_of_block[rb]]);
+    Wk[((ic >> 3) * F_W_ROWS + rb * 32 + oc) * 8 + (ic & 7)] = bf16_bits(wtmp[(oc * 16 + ic) * 9 + fold.tap_of_block[rb]]);
   }
-  if (tid < 32) bias[tid] = theta[OFF_C2B + tid];
+  __syncthreads();
   // rows never written by a copy (the overrun of the padding rows, a missing second sample) only feed
   // results that are dropped; they are cleared once so that those results stay finite
   for (int idx = tid; idx < F_NBUF * F_BUF_BYTES / 16; idx += F_THREADS) reinterpret_cast<float4*>(smem)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);

@@ -43,9 +43,9 @@ constexpr int W5_RAW_BYTES = W5_RAW_P1 + W5_RAW_DP2 + W5_RAW_CODE;          // 1
 constexpr int W5_RAW_SLOT = (W5_RAW_BYTES + 127) / 128 * 128;
 constexpr int W5_NRAW = 4;                              // raw input slots: each group's copies run two of its samples ahead
 constexpr int W5_SMEM = 2 * W5_STAGE_BYTES + W5_NRAW * W5_RAW_SLOT + 256 + 128;
-constexpr int W5_NACC = 4;                              // accumulators used in turn (an MMA that adds to the sum of the one before it
-                                                        // waits for that one to finish); they are added up at write-out
-constexpr int W5_TMEM_COLS = 512;                       // W5_NACC x 96 accumulator columns
+constexpr int W5_NACC = 1;                              // accumulators used in turn and added up at write-out (measured: four instead of one
+                                                        // change nothing, so consecutive MMAs into one accumulator do not wait for each other)
+constexpr int W5_TMEM_COLS = 128;                       // W5_NACC x 96 accumulator columns, rounded up to a power of two
 static_assert(8 * W5_GROUP_BYTES <= W5_STAGE_BYTES, "the 64-row A operand must stay inside its stage");
 static_assert(W5_SMEM <= 227 * 1024, "shared memory");
 

@@ -663,8 +663,8 @@ __global__ void __launch_bounds__(256) conv_grad_reduce(GradStepArgs a, WorkerTa
   const int s = blockIdx.x, b = a.b;
   float* grad = wt.grad[s];
   const int used2 = seg_len > 0 ? (s * b + b - 1) / seg_len - (s * b) / seg_len + 1 : n_chunks2;
-  // part1 likewise: all n_chunks slots, or four (one per window element) for every range of seg_len1 rows
-  const int used1 = seg_len1 > 0 ? 4 * ((s * b + b - 1) / seg_len1 - (s * b) / seg_len1 + 1) : n_chunks;
+  // part1 likewise: all n_chunks slots, or eight (sample of a pair x window element) for every range of seg_len1 rows
+  const int used1 = seg_len1 > 0 ? 8 * ((s * b + b - 1) / seg_len1 - (s * b) / seg_len1 + 1) : n_chunks;
   for (int v = blockIdx.y * RED_PER_BLOCK + threadIdx.x; v < min(RED_OUTPUTS, ((int)blockIdx.y + 1) * RED_PER_BLOCK); v += 256) {
     int o = v;
     if (o < C2_GRAD) {

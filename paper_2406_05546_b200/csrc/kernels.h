@@ -107,7 +107,7 @@ struct Workspace {
   float* dp2;      // [rows][1568]        gradient w.r.t. p2
   float* dp1;      // [rows][3136]        gradient w.r.t. p1; [16][196] fp32 (FP32 path) or [4 channel quads][196][4] BF16 in the first half of the row (tensor-core path)
   float* part2;    // [W][chunks][4640]   per-block partial conv2 weight/bias gradients
-  float* part1;    // [W][4 chunks][160]  per-block partial conv1 weight/bias gradients (tensor-core path: four per range, one per window element)
+  float* part1;    // [W][8 chunks][160]  per-block partial conv1 weight/bias gradients (tensor-core path: eight per range, one per sample of a pair and window element)
   float* partf;    // [W][FC2_SPLIT][FC_PART] per-block partial output-layer gradients and loss sums
   float* w1r;      // [groups][512][1568] TF32-rounded fc1 weights of each weight group of the call
   float* w1tr;     // [groups][1568][512] and their transpose

@@ -154,7 +154,7 @@ void layout(ps_ctx* x, const ps_config& c, void* arena, void* pinned, uint64_t* 
   ws.dp2 = a.take<float>(rows * psk::FLAT * 4);
   ws.dp1 = a.take<float>(rows * psk::P1_ELEMS * 4);
   ws.part2 = a.take<float>((uint64_t)c.max_workers * chunks * psk::C2_GRAD * 4);
-  ws.part1 = a.take<float>((uint64_t)c.max_workers * 4 * chunks * psk::C1_GRAD * 4);
+  ws.part1 = a.take<float>((uint64_t)c.max_workers * 8 * chunks * psk::C1_GRAD * 4);
   ws.partf = a.take<float>((uint64_t)c.max_workers * psk::FC2_SPLIT * psk::FC_PART * 4);
   ws.status = a.take<uint32_t>(ALIGN);
   ws.w1r = ws.w1tr = nullptr;
