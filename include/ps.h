@@ -144,6 +144,19 @@ int32_t workers_grad_step(ps_ctx* ctx, int32_t W, int32_t b, const ps_snapshot* 
                           uint64_t seed, uint64_t step, const int64_t* slot_ids, float* grads_dev,
                           float* loss_dev, int32_t* argmax_dev);
 
+/* The worker step when the server is up and only the SUM of the workers' gradients is needed (paper, design section on
+ * the stateless server: one server step takes all gradients, applies them, stores the result; synchronous training:
+ * all updates of an iteration at once).  Every worker must hold the same snapshot (PS_ERR_BAD_ARG otherwise: stale
+ * readers and the outage window need the per-worker gradients of workers_grad_step).  Same inputs as
+ * workers_grad_step; instead of W gradient vectors one vector, grad_sum_dev (dev, PS_PARAM_STRIDE floats, 16-byte
+ * aligned, written, padding zero) = sum over the workers of each worker's gradient of its own mean loss.  The
+ * 512-unit layer's weight gradient, which dominates the bytes, is computed over groups of workers at once, so the W
+ * vectors of 3.2 MB are never written.  loss_dev / argmax_dev as in workers_grad_step.  Uses the context's reduction
+ * scratch: do not run it concurrently with an apply on another stream. */
+int32_t workers_grad_step_summed(ps_ctx* ctx, int32_t W, int32_t b, const ps_snapshot* snaps, const int32_t* worker_ids,
+                                 const float* x_dev, const int32_t* y_dev, uint64_t seed, uint64_t step,
+                                 float* grad_sum_dev, float* loss_dev, int32_t* argmax_dev);
+
 /* Evaluation pass (paper, implementation section: the metric exporter reports accuracy and loss while training):
  * the forward pass only, without dropout (every unit kept, nothing rescaled), of W groups of b samples, group w
  * against weights snaps[w].dev_ptr.  Same inputs and layouts as workers_grad_step.  loss_dev [W] receives the mean
@@ -201,6 +214,12 @@ int32_t ps_apply(ps_ctx* ctx, ps_mode mode, float lr, float scale, const int32_t
  * replication, result) is as in ps_apply. */
 int32_t ps_apply_stale(ps_ctx* ctx, ps_mode mode, float lr, float scale, const int32_t* order, float clip_norm,
                        float staleness_alpha, ps_apply_result* out);
+
+/* The synchronous server step from the sum that workers_grad_step_summed produces: theta <- theta - lr * scale / n_workers * grad_sum; version + 1;
+ * checkpoint and replication as in ps_apply(PS_SYNC), whose result it equals up to rounding when grad_sum is the sum
+ * of the n_workers queued gradients.  The queue must be empty (PS_ERR_BAD_ARG).  `applied` reports n_workers. */
+int32_t ps_apply_summed(ps_ctx* ctx, const float* grad_sum_dev, int32_t n_workers, float lr, float scale,
+                        ps_apply_result* out);
 
 /* The periodic save of the parameters to persistent storage (design section on checkpointing): copies the
  * head weights and version into the next pinned host slot (stream-ordered device-to-host copy); when all slots

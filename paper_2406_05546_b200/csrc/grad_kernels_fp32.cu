@@ -696,6 +696,70 @@ __global__ void __launch_bounds__(256) conv_grad_reduce(GradStepArgs a, WorkerTa
   }
 }
 
+// ---- the summed step's final reduction: ONE gradient vector, the sum over all workers (who share one weight
+// snapshot).  The 512-unit layer's weight gradient arrives as n_super partial vectors (one per group of workers whose
+// samples went through one product), every other tensor as the per-worker, per-block partial sums the per-worker
+// reduction also reads; everything is added in a fixed order (group after group, worker after worker, block after
+// block).  Blocks 0 .. FUSED_W1_BLOCKS - 1 take the float4 columns of the big tensor, the rest the small outputs.
+constexpr int FUSED_W1_VEC = HID * FLAT / 4;                                 // 200,704 float4
+constexpr int FUSED_W1_BLOCKS = (FUSED_W1_VEC + 255) / 256;                  // 784
+constexpr int FUSED_SMALL = C2_GRAD + C1_GRAD + (NCLS * HID + HID + NCLS) + (P_PAD - P);
+constexpr int FUSED_SMALL_BLOCKS = (FUSED_SMALL + 255) / 256;
+__global__ void __launch_bounds__(256) fused_finish(GradStepArgs a, WorkerTable wt, Workspace ws, const float* __restrict__ super_part,
+                                                    int n_super, float* __restrict__ grad_sum, int n_chunks, int seg_len1,
+                                                    int n_chunks2, int seg_len) {
+  const int b = a.b;
+  if (blockIdx.x < FUSED_W1_BLOCKS) {
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= FUSED_W1_VEC) return;
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int g = 0; g < n_super; ++g) {
+      const float4 v = reinterpret_cast<const float4*>(super_part + (int64_t)g * P_PAD + OFF_F1W)[i];
+      t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+    }
+    reinterpret_cast<float4*>(grad_sum + OFF_F1W)[i] = t;
+    return;
+  }
+  int o = (blockIdx.x - FUSED_W1_BLOCKS) * 256 + threadIdx.x;
+  if (o < a.W) {      // the per-worker losses ride along (W <= 256 fits the first block of this part)
+    float t = 0.f;
+#pragma unroll
+    for (int c = 0; c < FC2_SPLIT; ++c) t += ws.partf[((int64_t)o * FC2_SPLIT + c) * FC_PART + NCLS * HID + HID + NCLS];
+    a.loss[wt.src[o]] = t * (1.0f / (float)b);
+  }
+  if (o >= FUSED_SMALL) return;
+  float t = 0.f;
+  if (o < C2_GRAD) {
+    for (int s = 0; s < a.W; ++s) {
+      const int used2 = seg_len > 0 ? (s * b + b - 1) / seg_len - (s * b) / seg_len + 1 : n_chunks2;
+      for (int c = 0; c < used2; ++c) t += ws.part2[((int64_t)s * n_chunks2 + c) * C2_GRAD + o];
+    }
+    grad_sum[OFF_C2W + o] = t;
+    return;
+  }
+  o -= C2_GRAD;
+  if (o < C1_GRAD) {
+    for (int s = 0; s < a.W; ++s) {
+      const int used1 = seg_len1 > 0 ? 8 * ((s * b + b - 1) / seg_len1 - (s * b) / seg_len1 + 1) : n_chunks;
+      for (int c = 0; c < used1; ++c) t += ws.part1[((int64_t)s * n_chunks + c) * C1_GRAD + o];
+    }
+    grad_sum[OFF_C1W + o] = t;
+    return;
+  }
+  o -= C1_GRAD;
+  if (o < NCLS * HID + HID + NCLS) {
+    for (int s = 0; s < a.W; ++s)
+#pragma unroll
+      for (int c = 0; c < FC2_SPLIT; ++c) t += ws.partf[((int64_t)s * FC2_SPLIT + c) * FC_PART + o];
+    if (o < NCLS * HID) grad_sum[OFF_F2W + o] = t;
+    else if (o < NCLS * HID + HID) grad_sum[OFF_F1B + o - NCLS * HID] = t;
+    else grad_sum[OFF_F2B + o - NCLS * HID - HID] = t;
+    return;
+  }
+  o -= NCLS * HID + HID + NCLS;
+  grad_sum[P + o] = 0.f;
+}
+
 // ---- evaluation: per worker, the mean loss from the output-layer kernel's partial sums and the number of samples
 // whose predicted label equals the given one (an integer count, summed in a fixed order).
 __global__ void __launch_bounds__(128) eval_finish(GradStepArgs a, WorkerTable wt, Workspace ws, int32_t* __restrict__ correct) {
@@ -781,13 +845,23 @@ int launch_eval(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& 
 // second convolution's filter gradient runs on another side stream next to its input gradient and the
 // first convolution's backward.  Everything joins before the final reduction.
 int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
-                     cudaStream_t st, const SideStreams& side, Profiler* prof) {
+                     cudaStream_t st, const SideStreams& side, Profiler* prof, const SummedStep* sum) {
   const int n_chunks = (a.b + CONV_SPB - 1) / CONV_SPB;
   const int mt = group_tiles(gt, a.b, 64);
   const bool tc = a.precision != 0;
   const int n_chunks1 = (a.b + CONV1_SPB - 1) / CONV1_SPB;
   const int n_chunks1b = (a.b + CONV1B_SPB - 1) / CONV1B_SPB;
   int launches = 0, n_chunks2 = n_chunks, seg_len = 0;
+  // Summed step: the 512-unit layer's weight gradient is taken over groups of workers at once ("super-workers" of
+  // W / n_super workers: their samples are consecutive rows, so the product only sees a longer batch) and written to
+  // n_super partial vectors instead of one vector per worker.
+  GradStepArgs a_dw = a;
+  WorkerTable wt_dw = wt;
+  if (sum) {
+    a_dw.W = sum->n_super;
+    a_dw.b = a.b * (a.W / sum->n_super);
+    for (int g = 0; g < sum->n_super; ++g) wt_dw.grad[g] = sum->super_part + (int64_t)g * P_PAD;
+  }
   if (tc) {
     cudaStream_t s1 = side.s1 ? side.s1 : st, s2 = side.s2 ? side.s2 : st;
     // the copies of W1 are not needed before the dense layer: they are made next to the convolutions
@@ -805,7 +879,7 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<dim3(a.W, FC2_SPLIT), FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
     launches += 1;
     if (side.s1) { cudaEventRecord(side.fork1, st); cudaStreamWaitEvent(s1, side.fork1, 0); }
-    n = launch_fc1_dw_tc5(a, wt, gt, ws, s1, prof);
+    n = sum ? launch_fc1_dw_tc5(a_dw, wt_dw, gt, ws, s1, prof) : launch_fc1_dw_tc5(a, wt, gt, ws, s1, prof);
     if (n < 0) return -1;
     launches += n;
     if (side.s1) cudaEventRecord(side.join1, s1);
@@ -821,18 +895,21 @@ int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTa
     if (n_chunks1t < 0) return -1;
     if (side.s1) cudaStreamWaitEvent(st, side.join1, 0);
     if (side.s2) cudaStreamWaitEvent(st, side.join2, 0);
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1t, seg_len1, n_chunks2, seg_len)));
+    if (sum) TIMED(K_CONV_GRAD_REDUCE, (fused_finish<<<FUSED_W1_BLOCKS + FUSED_SMALL_BLOCKS, 256, 0, st>>>(a, wt, ws, sum->super_part, sum->n_super, sum->grad_sum, n_chunks1t, seg_len1, n_chunks2, seg_len)));
+    else TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1t, seg_len1, n_chunks2, seg_len)));
     launches += 4;
   } else {
     TIMED(K_CONV1_FWD, (conv1_fwd<<<dim3(n_chunks1, a.W), 224, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_CONV2_FWD, (conv2_fwd<<<dim3(n_chunks, a.W), 256, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_FC1_FWD, (fc1_fwd<<<dim3(HID / 64, mt), 256, 0, st>>>(a, wt, gt, ws)));
     TIMED(K_FC2_FWD_BWD, (fc2_fwd_bwd<<<dim3(a.W, FC2_SPLIT), FC2_THREADS, 0, st>>>(a, wt, gt, ws)));
-    TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
+    if (sum) TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a_dw.W), 256, 0, st>>>(a_dw, wt_dw, ws)));
+    else TIMED(K_FC1_DW, (fc1_dw<<<dim3((FLAT + 63) / 64, HID / 64, a.W), 256, 0, st>>>(a, wt, ws)));
     TIMED(K_FC1_DX, (fc1_dx<<<dim3((FLAT + 63) / 64, mt), 256, 0, st>>>(a, gt, ws)));
     TIMED(K_CONV2_BWD, (conv2_bwd<<<dim3(n_chunks, a.W), 256, C2B_SMEM_FLOATS * sizeof(float), st>>>(a, wt, gt, ws, n_chunks)));
     TIMED(K_CONV1_BWD, (conv1_bwd<<<dim3(n_chunks1b, a.W), 256, 0, st>>>(a, wt, ws, n_chunks1b)));
-    TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1b, 0, n_chunks2, 0)));
+    if (sum) TIMED(K_CONV_GRAD_REDUCE, (fused_finish<<<FUSED_W1_BLOCKS + FUSED_SMALL_BLOCKS, 256, 0, st>>>(a, wt, ws, sum->super_part, sum->n_super, sum->grad_sum, n_chunks1b, 0, n_chunks2, 0)));
+    else TIMED(K_CONV_GRAD_REDUCE, (conv_grad_reduce<<<dim3(a.W, RED_BLOCKS), 256, 0, st>>>(a, wt, ws, n_chunks1b, 0, n_chunks2, 0)));
     launches = 9;
   }
   return cudaGetLastError() == cudaSuccess ? launches : -1;

@@ -134,9 +134,17 @@ struct SideStreams {
   cudaEvent_t fork1 = nullptr, join1 = nullptr, fork2 = nullptr, join2 = nullptr;
 };
 
-// Part A. Returns the number of kernels launched, or -1 on a launch error.
+// The summed step (all workers on one snapshot, only the sum of their gradients wanted): where it goes and the scratch
+// for the partial sums of the 512-unit layer's weight gradient.
+struct SummedStep {
+  float* grad_sum;      // [P_PAD] the sum over workers
+  float* super_part;    // [n_super][P_PAD] scratch
+  int n_super;          // groups of W / n_super workers (a divisor of W, at most 16)
+};
+
+// Part A. Returns the number of kernels launched, or -1 on a launch error.  sum == nullptr: one gradient per worker.
 int launch_grad_step(const GradStepArgs& a, const WorkerTable& wt, const GroupTable& gt, const Workspace& ws,
-                     cudaStream_t st, const SideStreams& side, Profiler* prof);
+                     cudaStream_t st, const SideStreams& side, Profiler* prof, const SummedStep* sum = nullptr);
 int launch_dropout_mask(uint64_t seed, uint32_t worker, uint64_t step, int b, uint32_t thresh,
                         uint8_t* keep, cudaStream_t st, Profiler* prof);
 int configure_grad_kernels();

@@ -416,6 +416,71 @@ int32_t workers_grad_step(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* sn
   return PS_OK;
 }
 
+int32_t workers_grad_step_summed(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* snaps, const int32_t* worker_ids,
+                                 const float* x_dev, const int32_t* y_dev, uint64_t seed, uint64_t step, float* grad_sum_dev,
+                                 float* loss_dev, int32_t* argmax_dev) {
+  if (!x || !snaps || !worker_ids || !x_dev || !y_dev || !grad_sum_dev || !loss_dev || !argmax_dev) return fail(PS_ERR_BAD_ARG, "NULL argument");
+  if (W < 1 || W > x->cfg.max_workers || b < 1 || b > x->cfg.max_batch) return fail(PS_ERR_BAD_ARG, "W=%d, b=%d outside 1..%d, 1..%d", W, b, x->cfg.max_workers, x->cfg.max_batch);
+  if (((uintptr_t)grad_sum_dev & 15) != 0) return fail(PS_ERR_BAD_ARG, "grad_sum_dev must be 16-byte aligned");
+  psk::GroupTable gt;
+  psk::WorkerTable wt;
+  int32_t rc = build_tables(x, W, snaps, worker_ids, nullptr, nullptr, wt, gt);
+  if (rc != PS_OK) return rc;
+  if (gt.n_groups != 1) return fail(PS_ERR_BAD_ARG, "the summed step needs every worker on the same snapshot (%d distinct ones given)", gt.n_groups);
+  psk::GradStepArgs a;
+  a.W = W; a.b = b; a.x = x_dev; a.y = y_dev; a.loss = loss_dev; a.argmax = argmax_dev;
+  a.seed = seed; a.step = step; a.drop_p = x->cfg.dropout_p; a.drop_thresh = x->drop_thresh;
+  a.precision = x->cfg.precision;
+  if (a.precision != PS_FP32 && ((uintptr_t)x_dev & 15) != 0) return fail(PS_ERR_BAD_ARG, "x_dev must be 16-byte aligned on the tensor-core path");
+  a.skip_prep_w1 = prep_is_current(x, gt);
+  psk::SummedStep sum;
+  sum.grad_sum = grad_sum_dev;
+  sum.super_part = x->partial;          // the reduction scratch is free between applies
+  sum.n_super = 1;
+  for (int g = MAX_SPLIT; g >= 1; --g)
+    if (W % g == 0) { sum.n_super = g; break; }
+  int n = psk::launch_grad_step(a, wt, gt, x->ws, x->st, x->prof.on ? psk::SideStreams() : x->side, &x->prof, &sum);
+  if (n >= 0 && a.precision != PS_FP32) prep_done(x, gt);
+  if (n < 0) return cuda_fail(cudaGetLastError(), "summed grad step launch");
+  x->launches += n;
+  return PS_OK;
+}
+
+int32_t ps_apply_summed(ps_ctx* x, const float* grad_sum_dev, int32_t n_workers, float lr, float scale, ps_apply_result* out) {
+  if (!x || !grad_sum_dev || n_workers < 1) return fail(PS_ERR_BAD_ARG, "bad argument");
+  if (!x->up || x->weights_lost) return fail(PS_ERR_DOWN, "server is down");
+  if (x->queue_len != 0) return fail(PS_ERR_BAD_ARG, "the queue holds %lld gradients: apply them first", (long long)x->queue_len);
+  if (((uintptr_t)grad_sum_dev & 15) != 0) return fail(PS_ERR_BAD_ARG, "grad_sum_dev must be 16-byte aligned");
+  const uint64_t depth = (uint64_t)x->cfg.ring_depth, R = (uint64_t)x->cfg.replicate_every;
+  Replica* rep = first_live(x);
+  ps_apply_result res = {0, x->version, 0, 0};
+  psk::SumApplyArgs a;
+  a.queue = grad_sum_dev; a.K = 1;
+  a.theta_in = head(x);
+  a.theta_out = x->ring[(x->version + 1) % depth];
+  const bool mirror = rep && ((x->version + 1) % R == 0);
+  if (mirror) { int32_t rc = shift_chain(x, 1); if (rc != PS_OK) return rc; }
+  a.replica = mirror ? rep->buf : nullptr;
+  a.coef = lr * scale / (float)n_workers;
+  a.partial = x->partial; a.max_split = 1;
+  a.coef_k = nullptr;
+  int n = psk::launch_sum_apply(a, x->st, &x->prof);
+  if (n < 0) return cuda_fail(cudaGetLastError(), "apply launch");
+  x->launches += n;
+  x->version += 1;
+  x->weights_epoch++;
+  advance_oldest(x);
+  if (mirror) { rep->version = x->version; res.replicated = 1; }
+  if (x->cfg.ckpt_every > 0 && x->version % (uint64_t)x->cfg.ckpt_every == 0) {
+    int32_t rc = do_checkpoint(x); if (rc != PS_OK) return rc; res.checkpointed = 1;
+  }
+  x->applied_total += n_workers;
+  res.applied = n_workers;
+  res.new_version = x->version;
+  if (out) *out = res;
+  return PS_OK;
+}
+
 int32_t workers_eval(ps_ctx* x, int32_t W, int32_t b, const ps_snapshot* snaps, const float* x_dev, const int32_t* y_dev,
                      float* loss_dev, int32_t* argmax_dev, int32_t* correct_dev) {
   if (!x || !snaps || !x_dev || !y_dev || !loss_dev || !argmax_dev || !correct_dev) return fail(PS_ERR_BAD_ARG, "NULL argument");

@@ -21,7 +21,7 @@ ERRORS = {-1: "PS_ERR_BAD_ARG", -2: "PS_ERR_DOWN", -3: "PS_ERR_QUEUE_FULL", -4: 
           -8: "PS_ERR_CUDA", -9: "PS_ERR_DEVICE_STATUS"}
 
 EXPORTS = ["ps_query_bytes", "ps_create", "ps_destroy", "ps_pull_snapshot", "ps_queue_reserve", "ps_slot_ptr",
-           "workers_grad_step", "workers_eval", "ps_dropout_mask", "ps_enqueue", "ps_apply", "ps_apply_stale", "ps_checkpoint", "ps_restore", "ps_replicate",
+           "workers_grad_step", "workers_grad_step_summed", "ps_apply_summed", "workers_eval", "ps_dropout_mask", "ps_enqueue", "ps_apply", "ps_apply_stale", "ps_checkpoint", "ps_restore", "ps_replicate",
            "ps_kill", "ps_failover", "ps_import_params", "ps_export_params", "ps_stats", "ps_tick_host",
            "ps_tick_host_submit", "ps_tick_host_wait",
            "ps_profile", "ps_profile_read", "ps_selftest_wait_timeout", "ps_last_error", "ps_replay_sum_static", "ps_replay_sum_static_error"]
@@ -78,6 +78,8 @@ def load(path=None):
         "ps_slot_ptr": [vp, i64, C.POINTER(vp)],
         "workers_grad_step": [vp, i32, i32, vp, vp, vp, vp, u64, u64, vp, vp, vp, vp],
         "workers_eval": [vp, i32, i32, vp, vp, vp, vp, vp, vp],
+        "workers_grad_step_summed": [vp, i32, i32, vp, vp, vp, vp, u64, u64, vp, vp, vp],
+        "ps_apply_summed": [vp, vp, i32, f32, f32, C.POINTER(ApplyResult)],
         "ps_apply_stale": [vp, i32, f32, f32, vp, f32, f32, C.POINTER(ApplyResult)],
         "ps_dropout_mask": [vp, u64, i32, u64, i32, vp],
         "ps_enqueue": [vp, i32, vp, vp, vp, vp, u64],
@@ -220,6 +222,32 @@ class ParameterServer:
             int(seed), int(step), _np_ptr(sid), grads_dev.data_ptr() if grads_dev is not None else None,
             loss_dev.data_ptr(), argmax_dev.data_ptr()))
         return loss_dev, argmax_dev
+
+    def workers_grad_step_summed(self, snaps, worker_ids, x_dev, y_dev, seed, step, grad_sum_dev=None, loss_dev=None,
+                                 argmax_dev=None):
+        """All workers on one snapshot; returns (grad_sum_dev [P_PAD], loss_dev [W], argmax_dev [W,b])."""
+        torch = self._torch
+        W, b = int(y_dev.shape[0]), int(y_dev.shape[1])
+        assert x_dev.is_cuda and x_dev.dtype == torch.float32 and x_dev.is_contiguous() and x_dev.numel() == W * b * 784
+        assert y_dev.is_cuda and y_dev.dtype == torch.int32 and y_dev.is_contiguous()
+        arr = (Snapshot * W)(*snaps)
+        wid = np.ascontiguousarray(worker_ids, dtype=np.int32)
+        if grad_sum_dev is None:
+            grad_sum_dev = torch.empty(P_PAD, dtype=torch.float32, device="cuda")
+        if loss_dev is None:
+            loss_dev = torch.empty(W, dtype=torch.float32, device="cuda")
+        if argmax_dev is None:
+            argmax_dev = torch.empty((W, b), dtype=torch.int32, device="cuda")
+        self._check(self.lib.workers_grad_step_summed(
+            self.ctx, W, b, C.cast(arr, C.c_void_p), _np_ptr(wid), x_dev.data_ptr(), y_dev.data_ptr(), int(seed), int(step),
+            grad_sum_dev.data_ptr(), loss_dev.data_ptr(), argmax_dev.data_ptr()))
+        return grad_sum_dev, loss_dev, argmax_dev
+
+    def ps_apply_summed(self, grad_sum_dev, n_workers, lr, scale=1.0):
+        res = ApplyResult()
+        self._check(self.lib.ps_apply_summed(self.ctx, grad_sum_dev.data_ptr(), int(n_workers), float(lr), float(scale), C.byref(res)))
+        return {"applied": res.applied, "new_version": res.new_version, "checkpointed": res.checkpointed,
+                "replicated": res.replicated}
 
     def workers_eval(self, snaps, x_dev, y_dev):
         """Forward pass without dropout.  Returns (loss_dev [W], argmax_dev [W,b], correct_dev [W])."""

@@ -358,3 +358,37 @@ def test_full_size_config4_tick_nine_versions_ordered_apply_and_mirror(precision
     assert srv.ps_failover() == o.failover() == 76
     assert (srv.ps_export_params()[0] == head).all()
     srv.close()
+
+
+@pytest.mark.parametrize("precision", [0, 2])
+def test_full_size_config5_summed_tick(precision):
+    """W=128 x b=128 through the summed step (sixteen groups of eight workers in the 512-unit layer's weight gradient):
+    the one vector against the sum of all 128 oracle gradients, and the server step against the oracle's."""
+    import torch
+    from oracle import cnn, ps as ops
+    from paper_2406_05546_b200 import harness, ps
+    tol = TOL_TENSOR if precision else TOL_FP32
+    s = schedules.config(5)
+    px, py = synth.image_pool(synth.POOL_IMAGES, seed=0)
+    theta = synth.init_params(1)
+    srv = harness.make_server(s, theta, queue_slots=s.W, precision=precision)
+    t = 7
+    x, y = synth.tick_batch(px, py, t, s.W, s.b)
+    ids = list(range(s.W))
+    snaps = [srv.ps_pull_snapshot(w) for w in range(s.W)]
+    gsum, loss, am = srv.workers_grad_step_summed(snaps, ids, torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda(), s.seed, t)
+    srv.ps_stats()
+    og, ol, oa, oz = cnn.workers_grad_step([theta] * s.W, ids, x, y, s.seed, t, 0.25, precision=precision)
+    got = gsum.cpu().numpy()
+    assert (got[ps.P:] == 0).all()
+    # 2 million ReLU decisions: single units may flip near zero (see the per-worker tests); the sum over 128 workers
+    # dilutes one sample's contribution to a row far below the tolerance, so the plain check applies
+    assert_params_close(got[:ps.P], og.sum(axis=0), tol, "summed gradient at full size")
+    np.testing.assert_allclose(loss.cpu().numpy(), ol, rtol=3e-3 if precision else 1e-5, atol=1e-6)
+    assert_argmax_valid(am.cpu().numpy(), oz, tol)
+    o = ops.OraclePS(theta, external_store=True)
+    o.enqueue(og.astype(np.float32), ids, [0] * s.W, t)
+    assert o.apply(ops.REPLAY, s.lr) == srv.ps_apply_summed(gsum, s.W, s.lr)
+    th = srv.ps_export_params()[0]
+    _assert_update_close(th, o.head(), theta.astype(np.float64), max(tol, 1e-3), "summed tick")
+    srv.close()

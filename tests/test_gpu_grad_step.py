@@ -343,3 +343,64 @@ def test_evaluation_pass_matches_the_oracle(precision, W, b, lags):
     if n_amb == 0:
         assert (correct.cpu().numpy() == oc).all()
     srv.close()
+
+
+@pytest.mark.parametrize("precision,W,b", [(0, 3, 5), (0, 8, 9), (2, 2, 8), (2, 8, 24), (2, 17, 6), (2, 6, 70)])
+def test_summed_step_equals_the_sum_of_the_workers_gradients_and_the_sync_update(precision, W, b):
+    """workers_grad_step_summed + ps_apply_summed: the one vector equals the sum of the oracle's per-worker gradients,
+    and the update equals the oracle's synchronous step over those gradients (W = 17 has no divisor up to 16 but 1:
+    the whole batch goes through one product; W = 8: eight groups; W = 6: six)."""
+    from oracle import cnn, ps as ops
+    tol = TOL_TENSOR if precision else TOL_FP32
+    torch, ps, srv, theta0 = _setup(W, b, 1, 0.25, precision)
+    rng = np.random.default_rng(31)
+    x = rng.random((W, b, 28, 28), dtype=np.float32)
+    y = rng.integers(0, 10, (W, b)).astype(np.int32)
+    ids = [(5 * w + 2) % 251 for w in range(W)]
+    snaps = [srv.ps_pull_snapshot(w) for w in range(W)]
+    xd, yd = torch.from_numpy(x).cuda(), torch.from_numpy(y).cuda()
+    gsum = torch.full((ps.P_PAD,), float("nan"), device="cuda")
+    _, loss, am = srv.workers_grad_step_summed(snaps, ids, xd, yd, SEED, 6, grad_sum_dev=gsum)
+    srv.ps_stats()
+    og, ol, oa, oz = cnn.workers_grad_step([theta0] * W, ids, x, y, SEED, 6, 0.25, precision=precision)
+    got = gsum.cpu().numpy()
+    assert (got[ps.P:] == 0).all()
+    assert_params_close(got[:ps.P], og.sum(axis=0), tol, "summed gradient")
+    np.testing.assert_allclose(loss.cpu().numpy(), ol, rtol=3e-3 if precision else 1e-5, atol=1e-6)
+    assert_argmax_valid(am.cpu().numpy(), oz, tol)
+    # the per-worker path gives the same sum (another order of additions)
+    gd = torch.zeros((W, ps.P_PAD), device="cuda")
+    srv.workers_grad_step(snaps, ids, xd, yd, SEED, 6, grads_dev=gd)
+    assert_params_close(got[:ps.P], gd.sum(dim=0).cpu().numpy()[:ps.P], 1e-5 if precision == 0 else 1e-4, "summed vs per-worker path")
+    # the server step
+    o = ops.OraclePS(theta0)
+    o.enqueue(og.astype(np.float32), ids, [0] * W, 6)
+    ro = o.apply(ops.SYNC, 0.01)
+    rg = srv.ps_apply_summed(gsum, W, 0.01)
+    assert ro == rg
+    th, v = srv.ps_export_params()
+    assert v == 1
+    assert_params_close(th, o.head(), tol, "parameters after the summed step")
+    assert_params_close(th.astype(np.float64) - theta0, o.head().astype(np.float64) - theta0, max(tol, 1e-3), "the summed step's update")
+    # errors: stale readers need the per-worker path; a non-empty queue must be applied first
+    g = torch.zeros((1, ps.P_PAD), device="cuda")
+    srv.ps_enqueue([0], [1], 7, grads_dev=g)
+    with pytest.raises(ps.PSError) as e:
+        srv.ps_apply_summed(gsum, W, 0.01)
+    assert e.value.name == "PS_ERR_BAD_ARG"
+    srv.close()
+
+
+def test_summed_step_refuses_mixed_snapshots():
+    torch, ps, srv, theta0 = _setup(2, 4, 2, 0.25, 0)
+    g = np.zeros((1, ps.P_PAD), dtype=np.float32)
+    g[0, :ps.P] = synth.random_gradients(1, seed=52, scale=2.0)[0]
+    srv.ps_enqueue([0], [0], 0, grads_dev=torch.from_numpy(g).cuda())
+    srv.ps_apply(ps.ASYNC, 0.01)
+    snaps = [srv.ps_pull_snapshot(0, 0), srv.ps_pull_snapshot(1, 1)]
+    x = torch.zeros((2, 4, 28, 28), device="cuda")
+    y = torch.zeros((2, 4), dtype=torch.int32, device="cuda")
+    with pytest.raises(ps.PSError) as e:
+        srv.workers_grad_step_summed(snaps, [0, 1], x, y, SEED, 0)
+    assert e.value.name == "PS_ERR_BAD_ARG"
+    srv.close()
