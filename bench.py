@@ -375,6 +375,48 @@ def main():
     h2d = W * b * 784 * 4 + W * b * 4
     d2h = W * 4
 
+    # ---- the summed step (every worker on the head, only the sum wanted) and the evaluation pass, same inputs
+    gsum = torch.empty(ps.P_PAD, dtype=torch.float32, device="cuda")
+
+    def summed_tick():
+        t = tick_no[0]
+        x, y = bufs[t % N_BATCH_BUFFERS]
+        snaps = [srv.ps_pull_snapshot(w) for w in range(W)]
+        srv.workers_grad_step_summed(snaps, ids, x, y, DROP_SEED, t, grad_sum_dev=gsum, loss_dev=loss_dev, argmax_dev=am_dev)
+        srv.ps_apply_summed(gsum, W, LR)
+        tick_no[0] += 1
+
+    def timed(fn, n):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(srv.stream)
+        for _ in range(n):
+            fn()
+        e1.record(srv.stream)
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1)) / n
+
+    n_extra = max(3, min(args.steps, 50))
+    summed_ms = timed(summed_tick, n_extra)
+    srv.ps_profile(True)
+    for _ in range(5):
+        summed_tick()
+    prof_s = srv.ps_profile_read()
+    srv.ps_profile(False)
+    summed = {"ms_per_tick": summed_ms, "worker_samples_per_s": W * b * world / (summed_ms * 1e-3), "ticks": n_extra,
+              "kernels_ms": {k: ms / n for k, (ms, n) in prof_s.items() if n},
+              "note": "pull + workers_grad_step_summed + ps_apply_summed: one summed gradient vector instead of W; "
+                      "not the headline metric, which is the per-worker stale-weight step"}
+
+    def eval_pass():
+        x, y = bufs[0]
+        srv.workers_eval([srv.ps_pull_snapshot(w) for w in range(W)], x, y)
+
+    eval_ms = timed(eval_pass, n_extra)
+    evaluation = {"ms_per_pass": eval_ms, "samples_per_s": W * b * world / (eval_ms * 1e-3), "samples": W * b}
+
     # ---- the other configurations at their stated sizes, and the FP32 path at this one (a few ticks each)
     configs, fp32_path = None, None
     if rank == 0:
@@ -412,6 +454,30 @@ def main():
                                # (2.654663 GB over 816 gradients), scaled to this launch
                                "traffic": K_replay * REPLAY_TRAFFIC_PER_GRADIENT, "peak_source": peaks["source"]},
                   "all_ms": reps}
+    # ---- the same replay with clipping by global norm: one pass that takes the norms, one that sums
+    replay_clipped = None
+    if do_replay:
+        srv.ps_kill()
+        for _ in range(DOWN_TICKS):
+            tick(apply=False)
+        srv.ps_restore()
+        srv.ps_profile(True)
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        r0.record(srv.stream)
+        res = srv.ps_apply_stale(ps.REPLAY, LR, scale=1.0 / DOWN_TICKS, clip_norm=1.0)
+        r1.record(srv.stream)
+        barrier()
+        assert res["applied"] == K_replay
+        ms = max_over_ranks(r0.elapsed_time(r1))
+        prof_c = srv.ps_profile_read()
+        srv.ps_profile(False)
+        pass_bytes = K_replay * GRAD_BYTES
+        replay_clipped = {"queue_gradients": K_replay, "ms": ms, "clip_norm": 1.0,
+                          "norm_pass_ms": prof_c["sq_norm_partial"][0], "norm_pass_gb_per_s": pass_bytes / (prof_c["sq_norm_partial"][0] * 1e-3) / 1e9,
+                          "sum_pass_ms": prof_c["sum_partial"][0], "sum_pass_gb_per_s": pass_bytes / (prof_c["sum_partial"][0] * 1e-3) / 1e9,
+                          "frac_of_hbm_peak_per_pass": [pass_bytes / (prof_c["sq_norm_partial"][0] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                                        pass_bytes / (prof_c["sum_partial"][0] * 1e-3) / 1e9 / peaks["hbm_gbs"]]}
     stats = srv.ps_stats()
 
     if rank == 0:
@@ -470,6 +536,9 @@ def main():
             "kernels": kernels,
             "grad_step": grad_step,
             "replay": replay,
+            "replay_clipped": replay_clipped,
+            "summed_step": summed,
+            "evaluation": evaluation,
             "configs": configs,
             "fp32_path": fp32_path,
             "cpu_baseline": cpu,

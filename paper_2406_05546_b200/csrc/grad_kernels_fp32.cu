@@ -704,7 +704,7 @@ __global__ void __launch_bounds__(256) conv_grad_reduce(GradStepArgs a, WorkerTa
 constexpr int FUSED_W1_VEC = HID * FLAT / 4;                                 // 200,704 float4
 constexpr int FUSED_W1_BLOCKS = (FUSED_W1_VEC + 255) / 256;                  // 784
 constexpr int FUSED_SMALL = C2_GRAD + C1_GRAD + (NCLS * HID + HID + NCLS) + (P_PAD - P);
-constexpr int FUSED_SMALL_BLOCKS = (FUSED_SMALL + 255) / 256;
+constexpr int FUSED_SMALL_BLOCKS = (FUSED_SMALL + 7) / 8;                    // one warp per small output
 __global__ void __launch_bounds__(256) fused_finish(GradStepArgs a, WorkerTable wt, Workspace ws, const float* __restrict__ super_part,
                                                     int n_super, float* __restrict__ grad_sum, int n_chunks, int seg_len1,
                                                     int n_chunks2, int seg_len) {
@@ -720,44 +720,44 @@ __global__ void __launch_bounds__(256) fused_finish(GradStepArgs a, WorkerTable 
     reinterpret_cast<float4*>(grad_sum + OFF_F1W)[i] = t;
     return;
   }
-  int o = (blockIdx.x - FUSED_W1_BLOCKS) * 256 + threadIdx.x;
-  if (o < a.W) {      // the per-worker losses ride along (W <= 256 fits the first block of this part)
+  // A small output is summed by one warp: lane l adds the partial sums of workers l, l + 32, ... in order, then the
+  // lanes are combined by a butterfly, which is the same sequence of additions on every run.
+  const int lane = threadIdx.x & 31;
+  int o = (blockIdx.x - FUSED_W1_BLOCKS) * 8 + (threadIdx.x >> 5);
+  if (blockIdx.x == FUSED_W1_BLOCKS && threadIdx.x < a.W) {      // the per-worker losses ride along (W <= 256)
     float t = 0.f;
 #pragma unroll
-    for (int c = 0; c < FC2_SPLIT; ++c) t += ws.partf[((int64_t)o * FC2_SPLIT + c) * FC_PART + NCLS * HID + HID + NCLS];
-    a.loss[wt.src[o]] = t * (1.0f / (float)b);
+    for (int c = 0; c < FC2_SPLIT; ++c) t += ws.partf[((int64_t)threadIdx.x * FC2_SPLIT + c) * FC_PART + NCLS * HID + HID + NCLS];
+    a.loss[wt.src[threadIdx.x]] = t * (1.0f / (float)b);
   }
   if (o >= FUSED_SMALL) return;
   float t = 0.f;
+  float* dst;
   if (o < C2_GRAD) {
-    for (int s = 0; s < a.W; ++s) {
+    for (int s = lane; s < a.W; s += 32) {
       const int used2 = seg_len > 0 ? (s * b + b - 1) / seg_len - (s * b) / seg_len + 1 : n_chunks2;
       for (int c = 0; c < used2; ++c) t += ws.part2[((int64_t)s * n_chunks2 + c) * C2_GRAD + o];
     }
-    grad_sum[OFF_C2W + o] = t;
-    return;
-  }
-  o -= C2_GRAD;
-  if (o < C1_GRAD) {
-    for (int s = 0; s < a.W; ++s) {
+    dst = grad_sum + OFF_C2W + o;
+  } else if (o < C2_GRAD + C1_GRAD) {
+    const int oo = o - C2_GRAD;
+    for (int s = lane; s < a.W; s += 32) {
       const int used1 = seg_len1 > 0 ? 8 * ((s * b + b - 1) / seg_len1 - (s * b) / seg_len1 + 1) : n_chunks;
-      for (int c = 0; c < used1; ++c) t += ws.part1[((int64_t)s * n_chunks + c) * C1_GRAD + o];
+      for (int c = 0; c < used1; ++c) t += ws.part1[((int64_t)s * n_chunks + c) * C1_GRAD + oo];
     }
-    grad_sum[OFF_C1W + o] = t;
-    return;
-  }
-  o -= C1_GRAD;
-  if (o < NCLS * HID + HID + NCLS) {
-    for (int s = 0; s < a.W; ++s)
+    dst = grad_sum + OFF_C1W + oo;
+  } else if (o < C2_GRAD + C1_GRAD + NCLS * HID + HID + NCLS) {
+    const int oo = o - C2_GRAD - C1_GRAD;
+    for (int s = lane; s < a.W; s += 32)
 #pragma unroll
-      for (int c = 0; c < FC2_SPLIT; ++c) t += ws.partf[((int64_t)s * FC2_SPLIT + c) * FC_PART + o];
-    if (o < NCLS * HID) grad_sum[OFF_F2W + o] = t;
-    else if (o < NCLS * HID + HID) grad_sum[OFF_F1B + o - NCLS * HID] = t;
-    else grad_sum[OFF_F2B + o - NCLS * HID - HID] = t;
-    return;
+      for (int c = 0; c < FC2_SPLIT; ++c) t += ws.partf[((int64_t)s * FC2_SPLIT + c) * FC_PART + oo];
+    dst = oo < NCLS * HID ? grad_sum + OFF_F2W + oo : (oo < NCLS * HID + HID ? grad_sum + OFF_F1B + oo - NCLS * HID : grad_sum + OFF_F2B + oo - NCLS * HID - HID);
+  } else {
+    dst = grad_sum + P + (o - C2_GRAD - C1_GRAD - NCLS * HID - HID - NCLS);      // padding: zero
   }
-  o -= NCLS * HID + HID + NCLS;
-  grad_sum[P + o] = 0.f;
+#pragma unroll
+  for (int sh = 16; sh > 0; sh >>= 1) t += __shfl_xor_sync(0xffffffffu, t, sh);
+  if (lane == 0) *dst = t;
 }
 
 // ---- evaluation: per worker, the mean loss from the output-layer kernel's partial sums and the number of samples

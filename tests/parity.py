@@ -27,6 +27,24 @@ def assert_params_close(got, ref, tol, what=""):
     return errs
 
 
+def assert_sum_close(got, parts, tol, what=""):
+    """got [P] against the sum of parts [W, P] (one gradient per worker): each worker's gradient is allowed tol times its
+    own tensor's max-abs, so their sum is allowed the sum of those allowances (the workers' errors add at worst), which is
+    what is checked per tensor.  Returns the errors relative to the SUM's max-abs, for the record."""
+    parts = np.asarray(parts, dtype=np.float64)
+    ref = parts.sum(axis=0)
+    errs, bad = {}, {}
+    for name, off, shape in synth.layout():
+        n = int(np.prod(shape))
+        err = np.abs(np.asarray(got[off:off + n], dtype=np.float64) - ref[off:off + n]).max()
+        allowed = tol * np.abs(parts[:, off:off + n]).max(axis=1).sum()
+        errs[name] = err / max(np.abs(ref[off:off + n]).max(), 1e-300)
+        if not err <= allowed:
+            bad[name] = (err, allowed)
+    assert not bad, f"{what}: error above the summed allowance: {bad} (relative to the sum: {errs})"
+    return errs
+
+
 def assert_params_close_up_to_unit_flips(got, ref, tol, theta, diag, what=""):
     """As assert_params_close, except that a row of fc1.w (with its fc1.b entry) may differ from the reference by
     ReLU decisions of that hidden unit that came out the other way, under two conditions that are both checked:

@@ -4,7 +4,7 @@ import pytest
 
 from paper_2406_05546_b200 import synth
 from tests.parity import (TOL_FP32, TOL_TENSOR, assert_argmax_valid, assert_params_close,
-                          assert_params_close_up_to_unit_flips, tensor_rel_errors)
+                          assert_params_close_up_to_unit_flips, assert_sum_close, tensor_rel_errors)
 
 pytestmark = pytest.mark.gpu
 
@@ -365,7 +365,7 @@ def test_summed_step_equals_the_sum_of_the_workers_gradients_and_the_sync_update
     og, ol, oa, oz = cnn.workers_grad_step([theta0] * W, ids, x, y, SEED, 6, 0.25, precision=precision)
     got = gsum.cpu().numpy()
     assert (got[ps.P:] == 0).all()
-    assert_params_close(got[:ps.P], og.sum(axis=0), tol, "summed gradient")
+    assert_sum_close(got[:ps.P], og, tol, "summed gradient")
     np.testing.assert_allclose(loss.cpu().numpy(), ol, rtol=3e-3 if precision else 1e-5, atol=1e-6)
     assert_argmax_valid(am.cpu().numpy(), oz, tol)
     # the per-worker path gives the same sum (another order of additions)
