@@ -472,3 +472,33 @@ def test_staleness_scaled_learning_rate(mode_name):
         g.ps_apply_stale(getattr(ps, mode_name), 0.01, staleness_alpha=0.5)
     assert e.value.name == "PS_ERR_BAD_ARG"
     g2.close(); g.close()
+
+
+def test_two_failures_in_one_run():
+    """The schedule of the paper's second accuracy experiment, two server failures in one run, on both recovery
+    designs: checkpointing (each restore rolls back to the latest checkpoint, the updates since are lost and redone
+    with new gradients) and a chain of three (each failover moves to the next server, the second one to older weights)."""
+    ops, ps, o, g = _pair(queue_slots=4, ckpt_every=10, ckpt_slots=4)
+    _steps(o, g, ops, ps, 13, 1000)
+    o.kill(0); g.ps_kill(0)
+    assert o.restore() == g.ps_restore() == 10
+    _steps(o, g, ops, ps, 14, 1100)                     # 10 -> 24, checkpoint at 20
+    o.kill(0); g.ps_kill(0)
+    assert o.restore() == g.ps_restore() == 20
+    _steps(o, g, ops, ps, 3, 1200)
+    st = g.ps_stats()
+    assert st["version"] == o.version == 23 and st["last_ckpt_version"] == 20 and st["checkpoints"] == 2
+    assert [v for v, _ in o.ckpts] == [10, 20]
+    assert_params_close(g.ps_export_params()[0], o.head(), 1e-5, "after two rollbacks")
+    g.close()
+    ops, ps, o, g = _pair(queue_slots=4, chain_len=3, replicate_every=3)
+    _steps(o, g, ops, ps, 8, 1300)                      # events at 3 and 6: the servers hold 6 and 3
+    o.kill(0); g.ps_kill(0)
+    assert o.failover() == g.ps_failover() == 6
+    _steps(o, g, ops, ps, 2, 1400)                      # 7, 8: no event yet, the last server still holds 3
+    o.kill(0); g.ps_kill(0)
+    assert o.failover() == g.ps_failover() == 3
+    _steps(o, g, ops, ps, 2, 1500)
+    assert g.ps_stats()["version"] == o.version == 5 and g.ps_stats()["live_replicas"] == 0
+    assert_params_close(g.ps_export_params()[0], o.head(), 1e-5, "after two failovers")
+    g.close()
