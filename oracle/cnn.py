@@ -70,16 +70,17 @@ def dropout_keep(seed, worker, step, b, p):
 
 
 class _Diag(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("p1", "a2", "p2", "u", "dh", "code2", "on")]
+    _fields_ = [(n, C.c_void_p) for n in ("p1", "a2", "p2", "u", "dh", "code2", "on", "flip")]
 
 
-def grad_step_f64(theta, x, y, keep=None, drop_p=0.25, precision=0, diag=False):
+def grad_step_f64(theta, x, y, keep=None, drop_p=0.25, precision=0, diag=False, flips=None):
     """One worker, everything double.  Returns (grad[P], loss, argmax[b], logits[b,10]).
     precision 1: ReLU/pooling decisions are taken on a TF32-operand forward pass (values stay exact);
     precision 2: the same with BF16 operands in the second convolution (the 512-unit layer stays TF32).
     diag=True appends a dict of the exact pass's per-sample intermediates: p1 [b,16,14,14], a2 [b,32,14,14],
     p2 [b,1568], u [b,512] (pre-activations of the 512-unit layer), dh [b,512] (gradient w.r.t. that layer's
-    output after ReLU, dropout applied), code2 [b,1568] and on [b,512] (the decisions that were used)."""
+    output after ReLU, dropout applied), code2 [b,1568] and on [b,512] (the decisions that were used).
+    flips (needs diag=True): [(sample, unit), ...] whose ReLU decision is taken the other way."""
     theta = np.ascontiguousarray(theta, dtype=np.float64)
     x = np.ascontiguousarray(x, dtype=np.float64)
     y = np.ascontiguousarray(y, dtype=np.int32)
@@ -97,7 +98,10 @@ def grad_step_f64(theta, x, y, keep=None, drop_p=0.25, precision=0, diag=False):
         d = {"p1": np.zeros((b, 16, 14, 14)), "a2": np.zeros((b, 32, 14, 14)), "p2": np.zeros((b, 1568)),
              "u": np.zeros((b, HID)), "dh": np.zeros((b, HID)), "code2": np.zeros((b, 1568), dtype=np.int32),
              "on": np.zeros((b, HID), dtype=np.int32)}
-        dstruct = _Diag(*[d[n].ctypes.data for n, _ in _Diag._fields_])
+        flip = np.zeros((b, HID), dtype=np.uint8)
+        for i, j in (flips or []):
+            flip[int(i), int(j)] = 1
+        dstruct = _Diag(*[d[n].ctypes.data for n, _ in _Diag._fields_ if n != "flip"], flip.ctypes.data if flips else None)
     rc = lib().oracle_grad_step_f64_diag(_ptr(theta), _ptr(x), _ptr(y), b, _ptr(keep), float(drop_p), int(precision),
                                          _ptr(grad), _ptr(loss), _ptr(am), _ptr(logits),
                                          C.addressof(dstruct) if diag else None)
@@ -108,13 +112,14 @@ def grad_step_f64(theta, x, y, keep=None, drop_p=0.25, precision=0, diag=False):
     return grad, float(loss[0]), am, logits
 
 
-def worker_grad_step_diag(theta32, worker_id, x, y, seed, step, drop_p=0.25, precision=0):
+def worker_grad_step_diag(theta32, worker_id, x, y, seed, step, drop_p=0.25, precision=0, flips=None):
     """One worker of workers_grad_step (fp32 snapshot and images widened to double, Philox keep mask of
     (seed, worker_id, step)) with the intermediates of grad_step_f64(diag=True)."""
     y = np.ascontiguousarray(y, dtype=np.int32)
     keep = dropout_keep(seed, worker_id, step, y.shape[0], drop_p) if drop_p > 0 else None
     return grad_step_f64(np.asarray(theta32, dtype=np.float32).astype(np.float64),
-                         np.asarray(x, dtype=np.float32).astype(np.float64), y, keep, drop_p, precision, diag=True)
+                         np.asarray(x, dtype=np.float32).astype(np.float64), y, keep, drop_p, precision, diag=True,
+                         flips=flips)
 
 
 def workers_grad_step(thetas, worker_ids, x, y, seed, step, drop_p=0.25, precision=0):

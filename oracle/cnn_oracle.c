@@ -246,7 +246,8 @@ static void conv3x3_bwd_x(const double* dout, int cout, int hw, const double* w,
 
 /* Optional per-sample intermediates of the exact (double) pass, for tests that ask how far a decision
  * is from flipping.  Nothing here is new arithmetic: every array is a value the step computes anyway.
- * Any pointer may be NULL. */
+ * Any pointer may be NULL.  The one input, `flip`, overrides single ReLU decisions of the 512-unit layer (a unit that is
+ * switched on passes its pre-activation, whatever its sign, exactly as the backward pass then assumes). */
 typedef struct {
     double* p1;      /* [b][16][14][14] pooled output of the first convolution (the second one's input)        */
     double* a2;      /* [b][32][14][14] pre-activations of the second convolution                               */
@@ -256,6 +257,9 @@ typedef struct {
                      /*                 dropout applied: a unit that is on contributes dh * p2 to its row       */
     int32_t* code2;  /* [b][1568]       pooling decision of the second convolution that was used (0..3, 4 dead) */
     int32_t* on;     /* [b][512]        ReLU decision of the 512-unit layer that was used                       */
+    const uint8_t* flip; /* INPUT, [b][512] or NULL: 1 = take this unit's ReLU decision the other way.  For tests  */
+                     /*                 that ask what the exact gradient is under a different, equally valid choice */
+                     /*                 at a unit whose pre-activation is within rounding distance of zero           */
 } oracle_diag;
 
 /*
@@ -341,6 +345,7 @@ int32_t oracle_grad_step_f64_diag(const double* theta, const double* x, const in
                 for (int k = 0; k < FLAT; ++k) sq += round_operand(f1w[(size_t)j * FLAT + k], dense_rounding(precision)) * p2q[k];
                 on[j] = sq > 0.0;
             }
+            if (diag && diag->flip && diag->flip[(size_t)i * HID + j]) on[j] = !on[j];
             double h = on[j] ? s : 0.0;
             int kept = keep ? keep[(size_t)i * HID + j] : 1;
             d[j] = kept ? h * scale : 0.0;

@@ -45,15 +45,19 @@ def assert_sum_close(got, parts, tol, what=""):
     return errs
 
 
-def assert_params_close_up_to_unit_flips(got, ref, tol, theta, diag, what=""):
-    """As assert_params_close, except that a row of fc1.w (with its fc1.b entry) may differ from the reference by
-    ReLU decisions of that hidden unit that came out the other way, under two conditions that are both checked:
-    (1) only samples in which the unit's exact pre-activation lies within the operand-rounding bound of zero
-    (tests/margins.py) may have flipped, and (2) the difference of the row must equal, within the tolerance, the
-    signed sum of exactly those samples' contributions dh[i, j] * p2[i, :] (found by least squares over the
-    candidate samples, coefficients rounded to -1 / 0 / +1).  A row that is off for any other reason fails.
-    `theta` are the worker's weights and `diag` the oracle's intermediates of the same pass that produced `ref`.
-    Every other tensor must be within the tolerance.  Returns the list of (unit, [(sample, sign), ...])."""
+def assert_params_close_up_to_unit_flips(got, ref, tol, theta, diag, what="", recompute=None):
+    """As assert_params_close, except that ReLU decisions of the 512-unit layer that sit within rounding distance of
+    zero may have come out the other way.  What is admitted, and checked:
+    (1) a row of fc1.w (with its fc1.b entry) that is off must belong to a unit whose EXACT pre-activation lies within
+        the operand-rounding bound of zero (tests/margins.py) in some sample, and
+    (2) the row's difference must equal, within the tolerance, the signed sum of exactly such samples' contributions
+        dh[i, j] * p2[i, :] (least squares over the candidate samples, coefficients rounded to -1 / 0 / +1);
+    (3) with `recompute` (a function: list of (sample, unit) -> the oracle's gradient with those decisions taken the
+        other way), EVERY tensor must then be within the tolerance of that recomputed gradient: a flip also moves the
+        layers below through the back-propagated signal, visibly so at small batches.  Without `recompute` every other
+        tensor must be within the tolerance of `ref` as it stands.
+    `theta` are the worker's weights and `diag` the oracle's intermediates of the pass that produced `ref`.
+    Returns the list of (unit, [(sample, sign), ...])."""
     from tests import margins
     errs = tensor_rel_errors(got, ref)
     lay = {name: (off, shape) for name, off, shape in synth.layout()}
@@ -82,6 +86,10 @@ def assert_params_close_up_to_unit_flips(got, ref, tol, theta, diag, what=""):
             assert flips, (f"{what}: hidden unit {j} is off by {unit_err[j]:.2e} and no set of near-zero samples "
                            f"({cand.tolist()}) explains the difference of its row")
             explained.append((int(j), flips))
+    if explained and recompute is not None:
+        new_ref = recompute([(i, j) for j, fl in explained for i, _ in fl])
+        assert_params_close(got, new_ref, tol, what + ", against the gradient under the decisions it took")
+        return explained
     bad = {k: v for k, v in errs.items() if not v <= tol and k not in ("fc1.w", "fc1.b")}
     assert not bad, f"{what}: relative error above {tol}: {bad} (all: {errs})"
     return explained

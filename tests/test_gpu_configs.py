@@ -246,8 +246,9 @@ def _full_size_tick(n, precision, t, srv, o, lags=None):
         errs = tensor_rel_errors(gg[w, :ps.P], og[w])
         if precision and max(errs.values()) > tol:
             diag = cnn.worker_grad_step_diag(pulled[w][1], w, x[w], y[w], s.seed, t, s.dropout_p, precision)[4]
+            redo = lambda fl, w=w: cnn.worker_grad_step_diag(pulled[w][1], w, x[w], y[w], s.seed, t, s.dropout_p, precision, flips=fl)[0]
             n_flipped += len(assert_params_close_up_to_unit_flips(gg[w, :ps.P], og[w], tol, pulled[w][1], diag,
-                                                                  f"config {n} worker {w}"))
+                                                                  f"config {n} worker {w}", recompute=redo))
         else:
             assert_params_close(gg[w, :ps.P], og[w], tol, f"config {n} worker {w}")
     if n_flipped:

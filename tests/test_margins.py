@@ -94,3 +94,42 @@ def test_flip_explanation_accepts_real_flips_and_rejects_anything_else():
     other[160] += 1.0
     with pytest.raises(AssertionError, match="conv2.w"):
         assert_params_close_up_to_unit_flips(other, g, 2e-2, theta, d, "other tensor")
+
+
+def test_a_forced_decision_changes_exactly_what_a_flip_changes():
+    """The oracle's decision override (used to ask for the exact gradient under the other, equally valid choice at a
+    unit near zero): the unit's row of fc1.w moves by the sample's contribution dh * p2 and its fc1.b entry by dh, no
+    other row of the layer moves, the output layer's gradient moves only through the forward value (which a unit near
+    zero barely changes), overriding twice is the identity, and the result is what torch's autograd gives when the
+    unit's ReLU is replaced by the identity (switched on) or by zero (switched off)."""
+    import torch
+    theta, x, y = _case(4, 6)
+    g, loss, _, _, d = cnn.worker_grad_step_diag(theta, 0, x, y, 5, 7, 0.25, precision=0)
+    m = margins.decision_margins(theta, d)
+    i, j = [int(v) for v in np.unravel_index(np.argmax(np.where(m["relu_uncertain"], np.abs(d["dh"]), 0)), d["dh"].shape)]
+    g1, _, _, _, d1 = cnn.worker_grad_step_diag(theta, 0, x, y, 5, 7, 0.25, precision=0, flips=[(i, j)])
+    assert d1["on"][i, j] != d["on"][i, j] and (np.delete(d1["on"].ravel(), i * 512 + j) == np.delete(d["on"].ravel(), i * 512 + j)).all()
+    dw = (g1 - g)[OFF_F1W:OFF_F1B].reshape(512, 1568)
+    sign = -1.0 if d["on"][i, j] else 1.0
+    # the contribution that appears or disappears is the one of the pass in which the unit is on (the forward pass, and
+    # with it dh, differs between the two passes by what u[i, j], a value near zero, does to the logits)
+    dh_on = d["dh"][i, j] if d["on"][i, j] else d1["dh"][i, j]
+    assert np.abs(dw[j] - sign * dh_on * d["p2"][i]).max() <= 1e-9 * np.abs(dw[j]).max() + 1e-15
+    assert np.abs(np.delete(dw, j, axis=0)).max() <= 1e-2 * np.abs(dw[j]).max()
+    assert abs((g1 - g)[OFF_F1B + j] - sign * dh_on) <= 1e-9 * abs(dh_on) + 1e-15
+    g2 = cnn.worker_grad_step_diag(theta, 0, x, y, 5, 7, 0.25, precision=0, flips=[(i, j), (i, j)])[0]
+    assert np.array_equal(g2, g1)                   # the list marks units; marking one twice is marking it once
+    # torch: the same graph with that one unit's ReLU replaced
+    t = torch.tensor(theta.astype(np.float64), requires_grad=True)
+    seg = lambda name: t[cnn.TENSORS[name][0]:cnn.TENSORS[name][0] + int(np.prod(cnn.TENSORS[name][1]))].reshape(cnn.TENSORS[name][1])
+    F = torch.nn.functional
+    keep = torch.tensor(cnn.dropout_keep(5, 0, 7, 6, 0.25).astype(np.float64))
+    h = torch.tensor(x.astype(np.float64)).reshape(6, 1, 28, 28)
+    h = F.max_pool2d(F.relu(F.conv2d(h, seg("conv1.w"), seg("conv1.b"), padding=1)), 2)
+    h = F.max_pool2d(F.relu(F.conv2d(h, seg("conv2.w"), seg("conv2.b"), padding=1)), 2)
+    u = F.linear(h.flatten(1), seg("fc1.w"), seg("fc1.b"))
+    gate = (u > 0).to(u.dtype).detach()
+    gate[i, j] = 1.0 - gate[i, j]
+    z = F.linear(u * gate * keep / 0.75, seg("fc2.w"), seg("fc2.b"))
+    F.cross_entropy(z, torch.tensor(y.astype(np.int64))).backward()
+    assert np.abs(t.grad.numpy() - g1).max() <= 1e-11
