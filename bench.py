@@ -210,7 +210,7 @@ def run_small_case(args):
 
 
 GRAD_KERNELS_EXCLUDED = ("sum_apply_direct", "sum_partial", "sum_finish", "async_apply", "copy_rows", "dropout_mask",
-                         "norm_partial", "scaled_sum_apply")
+                         "sq_norm_partial", "clip_coef_finish", "eval_finish")      # server-side and auxiliary kernels
 
 
 def measure_config(n, precision, pool_x, pool_y, ticks=10, warmup=3):
