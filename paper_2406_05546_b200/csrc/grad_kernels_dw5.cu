@@ -10,16 +10,21 @@
 //
 //   D[(kx, ic)][(ky, oc)] += A[(kx, ic)][q] * B[(ky, oc)][q],   A[(kx, ic)][q] = p1pad[ic][q + kx],
 //                                                                B[(ky, oc)][q] = g2[oc][q - 16 ky]
+//                                                                (at the k-step of image row ks: row ks - ky of g2)
 //
 // i.e. M = 48 (+ one row of ones, whose products are the bias gradient; the tile is M = 64, the other rows
 // are never read), N = 96, K = 16: fourteen MMAs per sample (the input's two border rows contribute nothing),
 // accumulated over all samples of a worker.
 // The staging warps build both operands: A by transposing 8 x 8 blocks of the BF16 input planes (one
 // ldmatrix.trans + stmatrix pair per four blocks; the three kx copies differ in the rows addressed), B from the
-// pooled gradient and the pooling decisions, written three times, one image row apart, for the three ky.
+// pooled gradient and the pooling decisions.  B is stored ONCE: its three ky copies are the same rows of g2 one
+// image row apart, and with the image rows stored in descending order, 512 bytes apart, and the four channel octets
+// of a row 128 bytes apart, row group (ky, octet) of the operand is simply 128 (4 ky + octet) bytes after the start
+// address of the k-step: a uniform stride, which is all a shared-memory descriptor can express.
 // One CTA per SM walks over a contiguous range of rows (sorted worker, sample); where the range passes from one
 // worker to the next, and at its end, the accumulator is written out as a partial sum that a later kernel adds
-// in a fixed order.  Every mbarrier wait is bounded.
+// in a fixed order.  Two groups of staging warps take alternate samples; three operand stages are used in turn, so
+// that a group's next sample does not wait for the MMAs of its previous one.  Every mbarrier wait is bounded.
 #include "device_common.cuh"
 #include "kernels.h"
 #include "tc5_common.cuh"
@@ -30,19 +35,26 @@ namespace {
 
 constexpr int W5_LOAD_WARPS = 16;                       // two groups: group g stages samples n = g, g + 2, ...
 constexpr int W5_GW = W5_LOAD_WARPS / 2;                // warps per group
-constexpr int W5_THREADS = 32 * (1 + W5_LOAD_WARPS + 4);   // warp 0: MMA issue and tensor memory; the last four warps write out
+constexpr int W5_THREADS = 32 * (1 + W5_LOAD_WARPS + 4 + 1);   // warp 0: MMA issue and tensor memory; then the staging warps, four
+                                                               // write-out warps, and the warp that issues the loads
 constexpr int W5_CHUNKS = 32;                           // 8-position chunks of the 256 contraction indices of a sample
 constexpr int W5_GROUP_BYTES = W5_CHUNKS * 128;         // one group of 8 operand rows: 32 core matrices of 128 bytes
 constexpr int W5_A_GROUPS = 7;                          // (kx, channel octet) x 6, then the group whose first row is all ones
-constexpr int W5_B_GROUPS = 12;                         // (ky, channel octet)
 constexpr int W5_A_BYTES = W5_A_GROUPS * W5_GROUP_BYTES;     // 28,672
-constexpr int W5_STAGE_BYTES = W5_A_BYTES + W5_B_GROUPS * W5_GROUP_BYTES;   // 77,824; the A descriptor of M = 64 spans 8
-                                                        // groups from the stage's start (the eighth is B's first: rows never read)
+// B: [half of the image row (x / 8)][image row, descending: y = 14 .. -1][channel octet][8 channels x 8 positions];
+// rows y = 14 and y = -1 are never written (zeros): the k-steps next to the border read them
+constexpr int W5_B_ROW = 4 * 128, W5_B_HALF = 16 * W5_B_ROW;      // 512 bytes per image row, 8,192 per half
+constexpr int W5_B_BYTES = 2 * W5_B_HALF;               // 16,384
+constexpr int W5_STAGE_BYTES = W5_A_BYTES + W5_B_BYTES; // 45,056; the A descriptor of M = 64 spans 8 groups from the stage's
+                                                        // start (the eighth is B's first 4 KB: rows never read)
+constexpr int W5_NSTAGE = 3;                            // operand stages, used in turn (sample n -> stage n % 3)
 constexpr int W5_RAW_P1 = P1_PLANE_ELEMS * 4, W5_RAW_DP2 = FLAT * 4, W5_RAW_CODE = FLAT;
 constexpr int W5_RAW_BYTES = W5_RAW_P1 + W5_RAW_DP2 + W5_RAW_CODE;          // 16,032
 constexpr int W5_RAW_SLOT = (W5_RAW_BYTES + 127) / 128 * 128;
-constexpr int W5_NRAW = 4;                              // raw input slots: each group's copies run two of its samples ahead
-constexpr int W5_SMEM = 2 * W5_STAGE_BYTES + W5_NRAW * W5_RAW_SLOT + 256 + 128;
+constexpr int W5_NRAW = 6;                              // raw input slots (sample n -> slot n % 6): the copies, issued by a warp of their
+                                                        // own (issuing them costs a staging thread hundreds of cycles per sample, which
+                                                        // its whole group then waits for), run up to six samples ahead
+constexpr int W5_SMEM = W5_NSTAGE * W5_STAGE_BYTES + W5_NRAW * W5_RAW_SLOT + 256 + 128;
 constexpr int W5_NACC = 1;                              // accumulators used in turn and added up at write-out (measured: four instead of one
                                                         // change nothing, so consecutive MMAs into one accumulator do not wait for each other)
 constexpr int W5_TMEM_COLS = 128;                       // W5_NACC x 96 accumulator columns, rounded up to a power of two
@@ -63,7 +75,7 @@ __device__ __forceinline__ void stmatrix_x4(uint32_t addr, const uint32_t (&r)[4
 }
 
 struct W5Bars {
-  uint64_t op_full[2], op_empty[2], raw_full[W5_NRAW], raw_empty[W5_NRAW], acc_full, acc_empty;
+  uint64_t op_full[W5_NSTAGE], op_empty[W5_NSTAGE], raw_full[W5_NRAW], raw_empty[W5_NRAW], acc_full, acc_empty;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -72,7 +84,7 @@ struct W5Bars {
 // to part2[s][range index - first range of s].
 __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, WorkerTable wt, Workspace ws, int seg_len, int slots) {
   extern __shared__ __align__(1024) uint8_t sm[];
-  uint8_t* raw = sm + 2 * W5_STAGE_BYTES;
+  uint8_t* raw = sm + W5_NSTAGE * W5_STAGE_BYTES;
   W5Bars* bars = reinterpret_cast<W5Bars*>(raw + W5_NRAW * W5_RAW_SLOT);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int total = a.W * a.b;
@@ -80,13 +92,13 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
 
   // operand stages start as zeros (B: borders and rows that a ky copy never reaches); the ones row of A is
   // written once: row 0 of group 6, i.e. the first 16 bytes of each of its core matrices
-  for (int i = tid; i < 2 * W5_STAGE_BYTES / 16; i += W5_THREADS) reinterpret_cast<uint4*>(sm)[i] = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = tid; i < W5_NSTAGE * W5_STAGE_BYTES / 16; i += W5_THREADS) reinterpret_cast<uint4*>(sm)[i] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
-  for (int i = tid; i < 2 * W5_CHUNKS; i += W5_THREADS)
+  for (int i = tid; i < W5_NSTAGE * W5_CHUNKS; i += W5_THREADS)
     *reinterpret_cast<uint4*>(sm + (i / W5_CHUNKS) * W5_STAGE_BYTES + 6 * W5_GROUP_BYTES + (i % W5_CHUNKS) * 128) =
         make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->op_full[i], W5_LOAD_WARPS / 2); mbar_init(&bars->op_empty[i], 1); }
+    for (int i = 0; i < W5_NSTAGE; ++i) { mbar_init(&bars->op_full[i], W5_LOAD_WARPS / 2); mbar_init(&bars->op_empty[i], 1); }
     for (int i = 0; i < W5_NRAW; ++i) { mbar_init(&bars->raw_full[i], 1); mbar_init(&bars->raw_empty[i], W5_LOAD_WARPS / 2); }
     mbar_init(&bars->acc_full, 1);
     mbar_init(&bars->acc_empty, 4);
@@ -110,17 +122,18 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       int writes = 0;
       bool fresh = true;                       // the next MMA starts a new sum
       for (int n = 0; n < n_samples; ++n) {
-        const int st = n & 1;
-        if (!mbar_wait(&bars->op_full[st], (n >> 1) & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
+        const int st = n % W5_NSTAGE;
+        if (!mbar_wait(&bars->op_full[st], (n / W5_NSTAGE) & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
         tc_fence_after();
         const uint32_t a_lo = plain_desc_lo(smem_u32(sm) + st * W5_STAGE_BYTES, 128);
-        const uint32_t b_lo = plain_desc_lo(smem_u32(sm) + st * W5_STAGE_BYTES + W5_A_BYTES, 128);
+        // B at k-step ks starts at the stored row of y = ks (14 - ks rows in); its two k-chunks are the halves of a row
+        const uint32_t b_lo = plain_desc_lo(smem_u32(sm) + st * W5_STAGE_BYTES + W5_A_BYTES + 14 * W5_B_ROW, W5_B_HALF);
         // contraction indices 16 ks .. 16 ks + 15 (image row ks of the bordered input): two chunks of 128 bytes.
         // Rows 0 and 15 are the input's zero border, so their products vanish and are not issued.
 #pragma unroll
         for (int ks = 1; ks < 15; ++ks)
-          umma_f16_split(tmem + ((ks - 1) % W5_NACC) * 96, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo + ks * 16,
-                         plain_desc_hi(W5_GROUP_BYTES), idesc, (ks - 1 < W5_NACC && fresh) ? 0u : 1u);
+          umma_f16_split(tmem + ((ks - 1) % W5_NACC) * 96, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo - ks * (W5_B_ROW / 16),
+                         plain_desc_hi(128), idesc, (ks - 1 < W5_NACC && fresh) ? 0u : 1u);
         fresh = false;
         umma_commit(&bars->op_empty[st]);
         const int row = r0 + n;
@@ -135,27 +148,17 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       }
     }
   } else if (warp <= W5_LOAD_WARPS) {
-    // ---------------- staging: group g (W5_GW warps) builds the operands of samples n = g, g + 2, ... in stage g
-    const int grp = (warp - 1) / W5_GW, gw = (warp - 1) - grp * W5_GW, gt_ = gw * 32 + lane;      // thread index inside the group
-    auto issue = [&](int n) {            // one thread: the three input rows of sample r0 + n
-      const int64_t row = r0 + n;
-      uint8_t* dst = raw + (n & 3) * W5_RAW_SLOT;
-      uint64_t* bar = &bars->raw_full[n & 3];
-      mbar_expect_tx(bar, W5_RAW_BYTES);
-      bulk_load(dst, ws.p1 + row * P1_PLANE_ELEMS, W5_RAW_P1, bar);
-      bulk_load(dst + W5_RAW_P1, ws.dp2 + row * FLAT, W5_RAW_DP2, bar);
-      bulk_load(dst + W5_RAW_P1 + W5_RAW_DP2, ws.code2 + row * FLAT, W5_RAW_CODE, bar);
-    };
-    if (gt_ == 0) { if (grp < n_samples) issue(grp); if (grp + 2 < n_samples) issue(grp + 2); }
+    // ---------------- staging: group g (W5_GW warps) builds the operands of samples n = g, g + 2, ... in stage n % 3
+    const int grp = (warp - 1) / W5_GW, gw = (warp - 1) - grp * W5_GW;      // group, and warp inside the group
     for (int n = grp; n < n_samples; n += 2) {
-      const int slot = n & 3;
-      bool ok = mbar_wait(&bars->raw_full[slot], (n >> 2) & 1);
-      if (ok && n >= 2) ok = mbar_wait(&bars->op_empty[grp], ((n >> 1) - 1) & 1);
+      const int slot = n % W5_NRAW, st = n % W5_NSTAGE;
+      bool ok = mbar_wait(&bars->raw_full[slot], (n / W5_NRAW) & 1);
+      if (ok && n >= W5_NSTAGE) ok = mbar_wait(&bars->op_empty[st], ((n / W5_NSTAGE) - 1) & 1);      // the MMAs of sample n - 3 have read the stage
       if (!__all_sync(0xffffffffu, ok) || bars->abort_flag) { bars->abort_flag = 1; break; }
       const uint8_t* rp1 = raw + slot * W5_RAW_SLOT;
       const float* rdp2f = reinterpret_cast<const float*>(rp1 + W5_RAW_P1);
       const uint8_t* rcode8 = rp1 + W5_RAW_P1 + W5_RAW_DP2;
-      uint8_t* stage = sm + grp * W5_STAGE_BYTES;
+      uint8_t* stage = sm + st * W5_STAGE_BYTES;
       // A: 6 groups x 32 chunks = 192 blocks of 8 positions x 8 channels, transposed four at a time.  Operation o of
       // the 48 covers chunks 4 (o % 8) .. + 3 of group o / 8 = (kx, channel octet).  Lane l addresses row l % 8 of
       // block l / 8: on the way in the input plane's row of position 8 chunk + row + kx (plane rows keep even and
@@ -173,8 +176,8 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       // the octet and one pooled column of the four: its words then fall into 32 different banks.  Every pooled entry
       // owns the four positions of its window: shifted left by 16 bits per decision, the BF16 gradient lands in the
       // half-word of the winner (low word: image row 2py, high word: row 2py + 1; decision 4 shifts it out), the other
-      // three are cleared.  The pair of columns (2px, 2px + 1) is one word of a core-matrix row; the three ky copies
-      // lie one image row (two chunks) apart, image rows 2py and 2py + 1 likewise.
+      // three are cleared.  The pair of columns (2px, 2px + 1) is one word of a core-matrix row; image row y is stored
+      // 14 - y rows into its half.
 #pragma unroll
       for (int wi = gw; wi < 56; wi += W5_GW) {
         const int oct = wi / 14, rem = wi - oct * 14, py = rem >> 1, pxhi = rem & 1;
@@ -183,23 +186,30 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
           const int oc = 8 * oct + rr, e = ((oc >> 2) * 49 + py * 7 + px) * 4 + (oc & 3);
           const uint32_t code = rcode8[e];
           const unsigned long long slot64 = shl64_clamped(bf16_bits(rdp2f[e]), 16u * code);
-          uint32_t* d = reinterpret_cast<uint32_t*>(stage + W5_A_BYTES + oct * W5_GROUP_BYTES + (4 * py + pxhi) * 128 + rr * 16) + pl;
-#pragma unroll
-          for (int ky = 0; ky < 3; ++ky) {
-            uint32_t* dk = d + ky * ((4 * W5_GROUP_BYTES + 256) / 4);          // copy ky: four groups on, image row 2py + ky
-            dk[0] = (uint32_t)slot64;
-            dk[64] = (uint32_t)(slot64 >> 32);                               // image row 2py + 1 + ky
-          }
+          uint32_t* d = reinterpret_cast<uint32_t*>(stage + W5_A_BYTES + pxhi * W5_B_HALF + (14 - 2 * py) * W5_B_ROW + oct * 128 + rr * 16) + pl;
+          d[0] = (uint32_t)slot64;                               // image row 2py
+          d[-(W5_B_ROW / 4)] = (uint32_t)(slot64 >> 32);         // image row 2py + 1
         }
       }
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) { mbar_arrive(&bars->op_full[grp]); mbar_arrive(&bars->raw_empty[slot]); }
-      if (gt_ == 0 && n + 4 < n_samples) {
-        if (!mbar_wait(&bars->raw_empty[slot], (n >> 2) & 1)) { bars->abort_flag = 1; break; }
-        issue(n + 4);
-      }
+      if (lane == 0) { mbar_arrive(&bars->op_full[st]); mbar_arrive(&bars->raw_empty[slot]); }
     }
+  } else if (warp == W5_LOAD_WARPS + 5) {
+    // ---------------- loads: one thread issues every sample's three bulk copies into the raw slots in turn; before a
+    // slot's reuse it waits until the eight warps that staged the slot's previous sample have read it
+    if (lane == 0)
+      for (int n = 0; n < n_samples; ++n) {
+        const int slot = n % W5_NRAW, use = n / W5_NRAW;
+        if (use > 0 && (!mbar_wait(&bars->raw_empty[slot], (use - 1) & 1) || bars->abort_flag)) { bars->abort_flag = 1; break; }
+        const int64_t row = r0 + n;
+        uint8_t* dst = raw + slot * W5_RAW_SLOT;
+        uint64_t* bar = &bars->raw_full[slot];
+        mbar_expect_tx(bar, W5_RAW_BYTES);
+        bulk_load(dst, ws.p1 + row * P1_PLANE_ELEMS, W5_RAW_P1, bar);
+        bulk_load(dst + W5_RAW_P1, ws.dp2 + row * FLAT, W5_RAW_DP2, bar);
+        bulk_load(dst + W5_RAW_P1 + W5_RAW_DP2, ws.code2 + row * FLAT, W5_RAW_CODE, bar);
+      }
   } else {
     // ---------------- write-out: a warp reads the accumulator lanes 32 (warp % 4) .. + 31.  An accumulator of 64 rows
     // keeps rows 16 w .. 16 w + 15 in the first sixteen lanes of quarter w.
