@@ -79,14 +79,22 @@ __device__ __forceinline__ uint32_t win_flags(uint32_t onehot, int w) { return o
 
 // The rows [row, r1) of a CTA are taken in units of two consecutive samples of one worker, or of one sample where a
 // worker's (or the range's) last sample has no partner.  After a unit with `flush` the accumulator is written out.
-struct D1Unit { int row, n; bool flush; };
-__device__ __forceinline__ bool d1_next_unit(int& row, int r1, int b, D1Unit& u) {
-  if (row >= r1) return false;
-  const int wend = (row / b + 1) * b;            // first row of the next worker
-  u.row = row;
-  u.n = (row + 1 < r1 && row + 1 < wend) ? 2 : 1;
-  row += u.n;
-  u.flush = row == r1 || row == wend;
+// The walk carries the worker's index and the first row of the next worker along: every role's loop is a serial
+// instruction stream, in which an integer division per unit costs hundreds of cycles.
+struct D1Unit { int row, n, s; bool flush; };       // first row, rows, sorted worker of those rows
+struct D1Walk { int row, wend, s; };                // next row, first row of the next worker, worker of `row`
+__device__ __forceinline__ D1Walk d1_begin(int r0, int b) {
+  const int s = r0 / b;
+  return {r0, (s + 1) * b, s};
+}
+__device__ __forceinline__ bool d1_next_unit(D1Walk& w, int r1, int b, D1Unit& u) {
+  if (w.row >= r1) return false;
+  u.row = w.row;
+  u.s = w.s;
+  u.n = (w.row + 1 < r1 && w.row + 1 < w.wend) ? 2 : 1;
+  w.row += u.n;
+  u.flush = w.row == r1 || w.row == w.wend;
+  if (w.row == w.wend) { w.wend += b; ++w.s; }
   return true;
 }
 
@@ -125,10 +133,11 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(GradStepArgs a, Wo
     // ---------------- MMA issue
     if (lane == 0) {
       constexpr uint32_t idesc = d1_idesc(128, 48);
-      int writes = 0, row = r0;
+      int writes = 0;
+      D1Walk walk = d1_begin(r0, a.b);
       bool fresh = true;                       // the next MMA starts a new sum
       D1Unit un;
-      for (int u = 0; d1_next_unit(row, r1, a.b, un); ++u) {
+      for (int u = 0; d1_next_unit(walk, r1, a.b, un); ++u) {
         const int st = u & 1;
         if (!mbar_wait(&bars->op_full[st], (u >> 1) & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
         tc_fence_after();
@@ -178,13 +187,22 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(GradStepArgs a, Wo
         b_off[hh][j] = (p < 196 && iy >= 0 && iy < IMG && ix >= 0 && ix < IMG) ? D1_RAW_ZERO / 4 + iy * IMG + ix : 0;
       }
 
-    int row = r0, q0 = 0;                            // q0: samples of the range before this unit
+    // The range's q-th sample uses raw slot q % 5 for the (q / 5)-th time; slot0 / use0 are those of the unit's first
+    // sample, kept as counters.
+    D1Walk walk = d1_begin(r0, a.b);
+    int slot0 = 0;
+    uint32_t use0 = 0;
     D1Unit un;
-    for (int u = 0; d1_next_unit(row, r1, a.b, un); q0 += un.n, ++u) {
-      const int st = u & 1, q = q0 + h, slot = q % D1_NRAW;      // this group's sample is the range's q-th: the (q / 5)-th use of its slot
+    for (int u = 0; d1_next_unit(walk, r1, a.b, un); ++u) {
+      const int st = u & 1;
+      int slot = slot0 + h;                          // this group's sample is the unit's h-th
+      uint32_t use = use0;
+      if (slot >= D1_NRAW) { slot -= D1_NRAW; ++use; }
+      slot0 += un.n;
+      if (slot0 >= D1_NRAW) { slot0 -= D1_NRAW; ++use0; }
       const bool mine = h < un.n;                    // an odd last sample: group 1 only clears its shift block
       bool ok = true;
-      if (mine) ok = mbar_wait(&bars->raw_full[slot], (q / D1_NRAW) & 1);
+      if (mine) ok = mbar_wait(&bars->raw_full[slot], use & 1);
       if (ok && u >= 2) ok = mbar_wait(&bars->op_empty[st], ((u >> 1) - 1) & 1);      // the MMAs of unit u - 2 have read the stage
       if (!__all_sync(0xffffffffu, ok) || bars->abort_flag) { bars->abort_flag = 1; break; }
       const uint8_t* rslot = raw + slot * D1_RAW_SLOT;
@@ -239,20 +257,21 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(GradStepArgs a, Wo
     // ---------------- loads: one thread issues every sample's three bulk copies into the raw slots in turn; before a
     // slot's k-th reuse it waits until the eight warps that staged the slot's previous sample have read it
     if (lane == 0) {
-      int row = r0, q = 0;
+      D1Walk walk = d1_begin(r0, a.b);
+      int slot = 0, use = 0;
       D1Unit un;
       bool ok = true;
-      while (ok && d1_next_unit(row, r1, a.b, un))
-        for (int h = 0; h < un.n; ++h, ++q) {
-          const int slot = q % D1_NRAW, use = q / D1_NRAW;
+      while (ok && d1_next_unit(walk, r1, a.b, un))
+        for (int h = 0; h < un.n; ++h) {
           if (use > 0 && (!mbar_wait(&bars->raw_empty[slot], (use - 1) & 1) || bars->abort_flag)) { bars->abort_flag = 1; ok = false; break; }
-          const int r = un.row + h, s = r / a.b, i = r - s * a.b;
+          const int r = un.row + h, s = un.s, i = r - s * a.b;
           uint8_t* dst = raw + slot * D1_RAW_SLOT + D1_RAW_ZERO;
           uint64_t* bar = &bars->raw_full[slot];
           mbar_expect_tx(bar, D1_RAW_BYTES);
           bulk_load(dst, a.x + ((int64_t)wt.src[s] * a.b + i) * (IMG * IMG), D1_RAW_X, bar);
           bulk_load(dst + D1_RAW_X, reinterpret_cast<const uint8_t*>(ws.dp1) + (int64_t)r * (P1_ELEMS * 4), D1_RAW_G, bar);
           bulk_load(dst + D1_RAW_X + D1_RAW_G, ws.code1 + (int64_t)r * P1_ELEMS, D1_RAW_CODE, bar);
+          if (++slot == D1_NRAW) { slot = 0; ++use; }
         }
     }
   } else {
@@ -261,9 +280,10 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(GradStepArgs a, Wo
     // (sample, window element) writes its share of the 160 sums to a partial slot of its own (the final reduction adds
     // them in a fixed order), so the warps exchange nothing.
     const int quarter = warp & 3, half = quarter >> 1, my_w = 2 * (quarter & 1) + (lane >> 4), oc = lane & 15;
-    int writes = 0, row = r0;
+    int writes = 0;
+    D1Walk walk = d1_begin(r0, a.b);
     D1Unit un;
-    while (d1_next_unit(row, r1, a.b, un)) {
+    while (d1_next_unit(walk, r1, a.b, un)) {
       if (!un.flush) continue;
       if (!mbar_wait(&bars->acc_full, writes & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
       tc_fence_after();
@@ -274,7 +294,7 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(GradStepArgs a, Wo
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->acc_empty);
-      const int s = un.row / a.b;
+      const int s = un.s;
       float* part = ws.part1 + (((int64_t)s * slots + (blockIdx.x - (s * a.b) / seg_len)) * D1_SUBSLOTS + 4 * half + my_w) * C1_GRAD;
       // dW[oc][ky][kx] takes shift (wy + ky, wx + kx) of this window element
 #pragma unroll

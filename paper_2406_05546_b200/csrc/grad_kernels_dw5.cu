@@ -118,42 +118,52 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
   if (warp == 0) {
     // ---------------- MMA issue
     if (lane == 0) {
+      // This loop is one thread's serial instruction stream, with nothing to hide its latencies: an integer division
+      // or modulo here costs hundreds of cycles per sample, so stage, parity, descriptors and the next write-out row are
+      // all carried along as counters.
       constexpr uint32_t idesc = w5_idesc(64, 96);
-      int writes = 0;
+      constexpr uint32_t stage_step = W5_STAGE_BYTES / 16;
+      const uint32_t a_lo0 = plain_desc_lo(smem_u32(sm), 128);
+      // B at k-step ks starts at the stored row of y = ks (14 - ks rows in); its two k-chunks are the halves of a row
+      const uint32_t b_lo0 = plain_desc_lo(smem_u32(sm) + W5_A_BYTES + 14 * W5_B_ROW, W5_B_HALF);
+      const uint32_t full0 = smem_u32(&bars->op_full[0]), empty0 = smem_u32(&bars->op_empty[0]);
+      uint32_t a_lo = a_lo0, b_lo = b_lo0, full = full0, empty = empty0, parity = 0, writes = 0;
+      int st = 0;
+      int flush_at = min(r1, (r0 / a.b + 1) * a.b) - 1 - r0;     // index in the range of the next row that ends a worker or the range
       bool fresh = true;                       // the next MMA starts a new sum
       for (int n = 0; n < n_samples; ++n) {
-        const int st = n % W5_NSTAGE;
-        if (!mbar_wait(&bars->op_full[st], (n / W5_NSTAGE) & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
+        if (!mbar_wait_addr(full, parity) || bars->abort_flag) { bars->abort_flag = 1; break; }
         tc_fence_after();
-        const uint32_t a_lo = plain_desc_lo(smem_u32(sm) + st * W5_STAGE_BYTES, 128);
-        // B at k-step ks starts at the stored row of y = ks (14 - ks rows in); its two k-chunks are the halves of a row
-        const uint32_t b_lo = plain_desc_lo(smem_u32(sm) + st * W5_STAGE_BYTES + W5_A_BYTES + 14 * W5_B_ROW, W5_B_HALF);
         // contraction indices 16 ks .. 16 ks + 15 (image row ks of the bordered input): two chunks of 128 bytes.
         // Rows 0 and 15 are the input's zero border, so their products vanish and are not issued.
 #pragma unroll
         for (int ks = 1; ks < 15; ++ks)
-          umma_f16_split(tmem + ((ks - 1) % W5_NACC) * 96, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo - ks * (W5_B_ROW / 16),
-                         plain_desc_hi(128), idesc, (ks - 1 < W5_NACC && fresh) ? 0u : 1u);
+          umma_f16_split(tmem, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo - ks * (W5_B_ROW / 16), plain_desc_hi(128), idesc,
+                         (ks == 1 && fresh) ? 0u : 1u);
         fresh = false;
-        umma_commit(&bars->op_empty[st]);
-        const int row = r0 + n;
-        if (row + 1 == r1 || (row + 1) % a.b == 0) {
+        umma_commit_addr(empty);
+        if (n == flush_at) {
           // last row of the range or of a worker: hand the sum to the write-out warps and wait until they have read it
           umma_commit(&bars->acc_full);
           if (!mbar_wait(&bars->acc_empty, writes & 1)) { bars->abort_flag = 1; break; }
           tc_fence_after();
           ++writes;
           fresh = true;
+          flush_at = min(flush_at + a.b, n_samples - 1);
         }
+        if (++st == W5_NSTAGE) { st = 0; parity ^= 1; a_lo = a_lo0; b_lo = b_lo0; full = full0; empty = empty0; }
+        else { a_lo += stage_step; b_lo += stage_step; full += 8; empty += 8; }
       }
     }
   } else if (warp <= W5_LOAD_WARPS) {
     // ---------------- staging: group g (W5_GW warps) builds the operands of samples n = g, g + 2, ... in stage n % 3
     const int grp = (warp - 1) / W5_GW, gw = (warp - 1) - grp * W5_GW;      // group, and warp inside the group
+    // sample n uses raw slot n % 6 for the (n / 6)-th time and operand stage n % 3 for the (n / 3)-th: kept as counters
+    int slot = grp, st = grp;
+    uint32_t slot_use = 0, st_use = 0;
     for (int n = grp; n < n_samples; n += 2) {
-      const int slot = n % W5_NRAW, st = n % W5_NSTAGE;
-      bool ok = mbar_wait(&bars->raw_full[slot], (n / W5_NRAW) & 1);
-      if (ok && n >= W5_NSTAGE) ok = mbar_wait(&bars->op_empty[st], ((n / W5_NSTAGE) - 1) & 1);      // the MMAs of sample n - 3 have read the stage
+      bool ok = mbar_wait(&bars->raw_full[slot], slot_use & 1);
+      if (ok && st_use > 0) ok = mbar_wait(&bars->op_empty[st], (st_use - 1) & 1);      // the MMAs of sample n - 3 have read the stage
       if (!__all_sync(0xffffffffu, ok) || bars->abort_flag) { bars->abort_flag = 1; break; }
       const uint8_t* rp1 = raw + slot * W5_RAW_SLOT;
       const float* rdp2f = reinterpret_cast<const float*>(rp1 + W5_RAW_P1);
@@ -194,13 +204,17 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) { mbar_arrive(&bars->op_full[st]); mbar_arrive(&bars->raw_empty[slot]); }
+      slot += 2;
+      if (slot >= W5_NRAW) { slot -= W5_NRAW; ++slot_use; }
+      st += 2;
+      if (st >= W5_NSTAGE) { st -= W5_NSTAGE; ++st_use; }
     }
   } else if (warp == W5_LOAD_WARPS + 5) {
     // ---------------- loads: one thread issues every sample's three bulk copies into the raw slots in turn; before a
     // slot's reuse it waits until the eight warps that staged the slot's previous sample have read it
-    if (lane == 0)
+    if (lane == 0) {
+      int slot = 0, use = 0;
       for (int n = 0; n < n_samples; ++n) {
-        const int slot = n % W5_NRAW, use = n / W5_NRAW;
         if (use > 0 && (!mbar_wait(&bars->raw_empty[slot], (use - 1) & 1) || bars->abort_flag)) { bars->abort_flag = 1; break; }
         const int64_t row = r0 + n;
         uint8_t* dst = raw + slot * W5_RAW_SLOT;
@@ -209,17 +223,19 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
         bulk_load(dst, ws.p1 + row * P1_PLANE_ELEMS, W5_RAW_P1, bar);
         bulk_load(dst + W5_RAW_P1, ws.dp2 + row * FLAT, W5_RAW_DP2, bar);
         bulk_load(dst + W5_RAW_P1 + W5_RAW_DP2, ws.code2 + row * FLAT, W5_RAW_CODE, bar);
+        if (++slot == W5_NRAW) { slot = 0; ++use; }
       }
+    }
   } else {
     // ---------------- write-out: a warp reads the accumulator lanes 32 (warp % 4) .. + 31.  An accumulator of 64 rows
     // keeps rows 16 w .. 16 w + 15 in the first sixteen lanes of quarter w.
     const int quarter = warp & 3;
     int writes = 0;
-    for (int row = r0; row < r1; ++row) {
-      if (!(row + 1 == r1 || (row + 1) % a.b == 0)) continue;
+    int s = r0 / a.b;                                    // sorted worker of the rows being summed
+    // the rows after which the sum is written out: the last of every worker in the range, and the range's last
+    for (int row = min(r1, (s + 1) * a.b) - 1; row < r1; row = (row + 1 == r1) ? r1 : min(row + a.b, r1 - 1), ++s) {
       if (!mbar_wait(&bars->acc_full, writes & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
       tc_fence_after();
-      const int s = row / a.b;
       float* part = ws.part2 + ((int64_t)s * slots + (blockIdx.x - (s * a.b) / seg_len)) * C2_GRAD;
       const int rr = lane < 16 ? quarter * 16 + lane : 64;   // accumulator row: (kx, ic) for rr < 48, the ones row at 48
 #pragma unroll
