@@ -99,20 +99,34 @@ struct GemmArgs {
 // BN = tile columns: 256 for the 512-wide forward product, 224 = 1568/7 for the other two.
 struct TileCoord { int grp, m0, m_end, n0, z; };
 
+// A CTA's tiles are t = blockIdx.x, + gridDim.x, ...; their (column tile, row-tile index) pair is carried along by
+// additions: the role loops below are serial instruction streams in which a division per tile is dead time.
+struct TileWalk { int nt, rest, d_nt, d_rest; };
+__device__ __forceinline__ TileWalk tile_walk_begin(const GemmArgs& ga) {
+  TileWalk w;
+  w.nt = (int)blockIdx.x % ga.n_tiles_n;
+  w.rest = (int)blockIdx.x / ga.n_tiles_n;
+  w.d_nt = (int)gridDim.x % ga.n_tiles_n;
+  w.d_rest = (int)gridDim.x / ga.n_tiles_n;
+  return w;
+}
+__device__ __forceinline__ void tile_walk_next(TileWalk& w, const GemmArgs& ga) {
+  w.nt += w.d_nt;
+  w.rest += w.d_rest;
+  if (w.nt >= ga.n_tiles_n) { w.nt -= ga.n_tiles_n; ++w.rest; }
+}
 template <int BN>
-__device__ __forceinline__ bool decode_tile(int t, const GemmArgs& ga, const GroupTable& gt, int b, TileCoord& c) {
-  const int nt = t % ga.n_tiles_n;
-  const int rest = t / ga.n_tiles_n;
-  c.n0 = nt * BN;
+__device__ __forceinline__ bool decode_tile(const TileWalk& w, const GemmArgs& ga, const GroupTable& gt, int b, TileCoord& c) {
+  c.n0 = w.nt * BN;
   c.grp = 0;
   if (ga.per_worker) {
-    c.z = rest / (HID / BM);
-    c.m0 = (rest % (HID / BM)) * BM;
+    c.z = w.rest / (HID / BM);
+    c.m0 = (w.rest % (HID / BM)) * BM;
     c.m_end = HID;
     return true;
   }
   c.z = 0;
-  return locate_group_tile<BM>(gt, b, rest, c.grp, c.m0, c.m_end);
+  return locate_group_tile<BM>(gt, b, w.rest, c.grp, c.m0, c.m_end);
 }
 
 template <int EPI, int BN, bool MN = false>
@@ -155,9 +169,10 @@ __global__ void __launch_bounds__(gemm_threads(EPI), 1) tc5_gemm(const __grid_co
     if (lane == 0) {
       int it = 0;                            // k-blocks issued so far, over all tiles
       bool ok = true;
-      for (int t = blockIdx.x; t < ga.n_tiles && ok; t += gridDim.x) {
+      TileWalk tw = tile_walk_begin(ga);
+      for (int t = blockIdx.x; t < ga.n_tiles && ok; t += gridDim.x, tile_walk_next(tw, ga)) {
         TileCoord c;
-        if (!decode_tile<BN>(t, ga, gt, a.b, c)) continue;
+        if (!decode_tile<BN>(tw, ga, gt, a.b, c)) continue;
         const CUtensorMap* map_a = &maps.a;
         const CUtensorMap* map_b = &maps.b[c.grp];
         for (int kb = 0; kb < n_k; ++kb, ++it) {
@@ -181,9 +196,10 @@ __global__ void __launch_bounds__(gemm_threads(EPI), 1) tc5_gemm(const __grid_co
       const uint32_t desc_hi = (uint32_t)((MN ? smem_desc_mn_sw128(0, 0) : smem_desc_sw128(0)) >> 32);
       int it = 0, tile_i = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < ga.n_tiles && ok; t += gridDim.x) {
+      TileWalk tw = tile_walk_begin(ga);
+      for (int t = blockIdx.x; t < ga.n_tiles && ok; t += gridDim.x, tile_walk_next(tw, ga)) {
         TileCoord c;
-        if (!decode_tile<BN>(t, ga, gt, a.b, c)) continue;
+        if (!decode_tile<BN>(tw, ga, gt, a.b, c)) continue;
         const int ab = tile_i & 1;
         if (tile_i >= 2 && !mbar_wait(&acc_empty[ab], ((tile_i >> 1) - 1) & 1)) { *abort_flag = 1; break; }
         tc_fence_after();
@@ -212,9 +228,10 @@ __global__ void __launch_bounds__(gemm_threads(EPI), 1) tc5_gemm(const __grid_co
     int tile_i = 0;
     const float scale = 1.0f / (1.0f - a.drop_p);
     const uint2 key = make_uint2((uint32_t)a.seed, (uint32_t)(a.seed >> 32));
-    for (int t = blockIdx.x; t < ga.n_tiles; t += gridDim.x) {
+    TileWalk tw = tile_walk_begin(ga);
+    for (int t = blockIdx.x; t < ga.n_tiles; t += gridDim.x, tile_walk_next(tw, ga)) {
       TileCoord c;
-      if (!decode_tile<BN>(t, ga, gt, a.b, c)) continue;
+      if (!decode_tile<BN>(tw, ga, gt, a.b, c)) continue;
       const int ab = tile_i & 1;
       if (!mbar_wait(&acc_full[ab], (tile_i >> 1) & 1) || *abort_flag) {
         if (lane == 0) { *abort_flag = 1; atomicOr(ws.status, STATUS_WAIT_TIMEOUT); }
