@@ -250,7 +250,7 @@ constexpr int X_PLANE_ROWS = 256 + 51;                     // 34 rows of tap ove
 constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // staging stores of the four planes over all shared-memory banks)
 constexpr int X_BUF_BYTES = 4 * X_PLANE_BYTES;             // four planes of eight output channels
 constexpr int X_W_BYTES = 12 * 48 * 16;                    // [filter row ky][k chunk oc/8][column = kx*16 + ic][8 bf16]
-constexpr int X_RAW_BYTES = FLAT * 4 + FLAT;                // one sample's pooled gradients (fp32) and pooling decisions (bytes)
+constexpr int X_RAW_BYTES = FLAT * 2 + FLAT;                // one sample's pooled gradients (BF16) and pooling decisions (bytes)
 constexpr int X_RAW_SLOTS = 4;
 constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + X_RAW_SLOTS * X_RAW_BYTES + sizeof(Pipe) + 128;
 
@@ -319,8 +319,8 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
       const int64_t row = r_begin + t;
       uint8_t* slot = raw + (t & 3) * X_RAW_BYTES;
       mbar_expect_tx(&pipe->raw_full[t & 3], X_RAW_BYTES);
-      bulk_load(slot, ws.dp2 + row * FLAT, FLAT * 4, &pipe->raw_full[t & 3]);
-      bulk_load(slot + FLAT * 4, ws.code2 + row * FLAT, FLAT, &pipe->raw_full[t & 3]);
+      bulk_load(slot, ws.dp2 + row * FLAT, FLAT * 2, &pipe->raw_full[t & 3]);      // BF16 in the first half of the row
+      bulk_load(slot + FLAT * 2, ws.code2 + row * FLAT, FLAT, &pipe->raw_full[t & 3]);
     };
     if (lt == 0) { if (grp_w < n_tiles) fetch_raw(grp_w); if (grp_w + 2 < n_tiles) fetch_raw(grp_w + 2); }
     for (int t = grp_w; t < n_tiles; t += 2) {
@@ -330,11 +330,11 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
       if (ok && t >= 2) ok = mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1);
       if (!__all_sync(0xffffffffu, ok) || pipe->abort_flag) { pipe->abort_flag = 1; break; }
       uint16_t* dst = bufs + buf * (X_BUF_BYTES / 2);
-      const float* rg = reinterpret_cast<const float*>(raw + slot_i * X_RAW_BYTES);
-      const uint8_t* rc = raw + slot_i * X_RAW_BYTES + FLAT * 4;
+      const uint2* rg = reinterpret_cast<const uint2*>(raw + slot_i * X_RAW_BYTES);      // four BF16 channels of a position
+      const uint8_t* rc = raw + slot_i * X_RAW_BYTES + FLAT * 2;
       // Item e = lt + 128 k is (octet of output channels e / 49, pooled position e % 49).  The raw slot holds
-      // the gradients and the decisions as [channel quad][position][4 channels], so an item is two 16-byte and
-      // two 4-byte loads.  Its eight gradients become four BF16 pairs once; for each of the four positions of
+      // the gradients and the decisions as [channel quad][position][4 channels], so an item is two 8-byte and
+      // two 4-byte loads.  Its eight gradients arrive as four BF16 pairs; for each of the four positions of
       // the window the pairs are masked by "this position won" and stored as the position's 16-byte row, which
       // also clears the losers.
 #pragma unroll
@@ -342,9 +342,9 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
         const int e = lt + k * 128;
         if (e < 4 * 49) {
           const int o8 = e / 49, p = e - o8 * 49, py = p / 7, px = p - py * 7;
-          const float4 va = reinterpret_cast<const float4*>(rg)[(2 * o8) * 49 + p], vb = reinterpret_cast<const float4*>(rg)[(2 * o8 + 1) * 49 + p];
+          const uint2 va = rg[(2 * o8) * 49 + p], vb = rg[(2 * o8 + 1) * 49 + p];
           const uint32_t ca = reinterpret_cast<const uint32_t*>(rc)[(2 * o8) * 49 + p], cb = reinterpret_cast<const uint32_t*>(rc)[(2 * o8 + 1) * 49 + p];
-          const uint32_t h0 = bf16_pair(va.x, va.y), h1 = bf16_pair(va.z, va.w), h2 = bf16_pair(vb.x, vb.y), h3 = bf16_pair(vb.z, vb.w);
+          const uint32_t h0 = va.x, h1 = va.y, h2 = vb.x, h3 = vb.y;
           uint4* d = reinterpret_cast<uint4*>(dst) + o8 * (X_PLANE_BYTES / 16) + (2 * py + 1) * 16 + 2 * px + 1;
 #pragma unroll
           for (int j = 0; j < 4; ++j) {

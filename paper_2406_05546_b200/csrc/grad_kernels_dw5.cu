@@ -48,8 +48,8 @@ constexpr int W5_B_BYTES = 2 * W5_B_HALF;               // 16,384
 constexpr int W5_STAGE_BYTES = W5_A_BYTES + W5_B_BYTES; // 45,056; the A descriptor of M = 64 spans 8 groups from the stage's
                                                         // start (the eighth is B's first 4 KB: rows never read)
 constexpr int W5_NSTAGE = 3;                            // operand stages, used in turn (sample n -> stage n % 3)
-constexpr int W5_RAW_P1 = P1_PLANE_ELEMS * 4, W5_RAW_DP2 = FLAT * 4, W5_RAW_CODE = FLAT;
-constexpr int W5_RAW_BYTES = W5_RAW_P1 + W5_RAW_DP2 + W5_RAW_CODE;          // 16,032
+constexpr int W5_RAW_P1 = P1_PLANE_ELEMS * 4, W5_RAW_DP2 = FLAT * 2, W5_RAW_CODE = FLAT;      // dp2 arrives as BF16
+constexpr int W5_RAW_BYTES = W5_RAW_P1 + W5_RAW_DP2 + W5_RAW_CODE;          // 12,896
 constexpr int W5_RAW_SLOT = (W5_RAW_BYTES + 127) / 128 * 128;
 constexpr int W5_NRAW = 6;                              // raw input slots (sample n -> slot n % 6): the copies, issued by a warp of their
                                                         // own (issuing them costs a staging thread hundreds of cycles per sample, which
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       if (ok && st_use > 0) ok = mbar_wait(&bars->op_empty[st], (st_use - 1) & 1);      // the MMAs of sample n - 3 have read the stage
       if (!__all_sync(0xffffffffu, ok) || bars->abort_flag) { bars->abort_flag = 1; break; }
       const uint8_t* rp1 = raw + slot * W5_RAW_SLOT;
-      const float* rdp2f = reinterpret_cast<const float*>(rp1 + W5_RAW_P1);
+      const uint16_t* rdp2h = reinterpret_cast<const uint16_t*>(rp1 + W5_RAW_P1);
       const uint8_t* rcode8 = rp1 + W5_RAW_P1 + W5_RAW_DP2;
       uint8_t* stage = sm + st * W5_STAGE_BYTES;
       // A: 6 groups x 32 chunks = 192 blocks of 8 positions x 8 channels, transposed four at a time.  Operation o of
@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
         if (px < 7) {
           const int oc = 8 * oct + rr, e = ((oc >> 2) * 49 + py * 7 + px) * 4 + (oc & 3);
           const uint32_t code = rcode8[e];
-          const unsigned long long slot64 = shl64_clamped(bf16_bits(rdp2f[e]), 16u * code);
+          const unsigned long long slot64 = shl64_clamped(rdp2h[e], 16u * code);
           uint32_t* d = reinterpret_cast<uint32_t*>(stage + W5_A_BYTES + pxhi * W5_B_HALF + (14 - 2 * py) * W5_B_ROW + oct * 128 + rr * 16) + pl;
           d[0] = (uint32_t)slot64;                               // image row 2py
           d[-(W5_B_ROW / 4)] = (uint32_t)(slot64 >> 32);         // image row 2py + 1

@@ -75,11 +75,11 @@ struct GemmMaps {
   CUtensorMap b[MAX_GROUPS];
 };
 
-enum { EPI_FC1_FWD = 0, EPI_STORE = 1 };
+enum { EPI_FC1_FWD = 0, EPI_STORE = 1, EPI_STORE_BF16 = 2 };   // the last: the output rounded to BF16 (its readers multiply in BF16)
 // Epilogue warps: the plain-store products are bound by getting the accumulator out to global memory, so two warps
 // share each quarter of the accumulator rows and take alternate 32-column blocks; the forward product's epilogue
 // keeps one warp per quarter (its registers and shared memory leave no room for more).
-__host__ __device__ constexpr int epi_warps(int epi) { return epi == EPI_STORE ? 8 : 4; }
+__host__ __device__ constexpr int epi_warps(int epi) { return epi == EPI_FC1_FWD ? 4 : 8; }
 __host__ __device__ constexpr int gemm_threads(int epi) { return 64 + 32 * epi_warps(epi); }
 
 struct GemmArgs {
@@ -277,7 +277,13 @@ __global__ void __launch_bounds__(gemm_threads(EPI), 1) tc5_gemm(const __grid_co
           const int rr = i * 4 + (lane >> 3), cc = (lane & 7) * 4;
           const int m = c.m0 + quarter * 32 + rr;
           const uint4 v = *reinterpret_cast<const uint4*>(stage + rr * EPI_ROW_FLOATS + cc);
-          if (m < c.m_end) *reinterpret_cast<uint4*>(cbase + (int64_t)m * ga.ldc + n + cc) = v;
+          if (EPI == EPI_STORE_BF16) {     // ga.ldc counts BF16 elements here
+            if (m < c.m_end)
+              *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(cbase) + (int64_t)m * ga.ldc + n + cc) =
+                  make_uint2(bf16_pair(__uint_as_float(v.x), __uint_as_float(v.y)), bf16_pair(__uint_as_float(v.z), __uint_as_float(v.w)));
+          } else if (m < c.m_end) {
+            *reinterpret_cast<uint4*>(cbase + (int64_t)m * ga.ldc + n + cc) = v;
+          }
         }
       }
       // all of this warp's tensor-memory reads of the buffer are complete (tmem_ld32 waits): hand it back
@@ -382,7 +388,7 @@ int configure_tc5_kernels() {
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || g_sm_count <= 0) return -1;
   cudaError_t e = cudaFuncSetAttribute(tc5_gemm<EPI_FC1_FWD, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(256, MAX_STAGES, epi_warps(EPI_FC1_FWD)));
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES, epi_warps(EPI_STORE)));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE_BF16, 224>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES, epi_warps(EPI_STORE_BF16)));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(tc5_gemm<EPI_STORE, 224, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes(224, MAX_STAGES, epi_warps(EPI_STORE)));
   return e == cudaSuccess ? 0 : -1;
 }
@@ -416,9 +422,11 @@ int launch_fc1_dx_tc5(const GradStepArgs& a, const WorkerTable& wt, const GroupT
   for (int g = 0; g < gt.n_groups; ++g)
     if (!make_map(&maps.b[g], ws.w1tr + (int64_t)g * HID * FLAT, HID, FLAT, 1, HID, (uint64_t)HID * FLAT, 224)) return -1;
   const int mt = group_tiles(gt, a.b, BM);
-  GemmArgs ga{HID, FLAT, FLAT, 0, ws.dp2, FLAT / 224, (FLAT / 224) * mt};
+  // dp2 leaves as BF16, in the first half of each row of the fp32-sized buffer (row pitch 2 FLAT half-words): the
+  // convolution's two backward kernels multiply it in BF16, so rounding it here once changes no result
+  GemmArgs ga{HID, FLAT, 2 * FLAT, 0, ws.dp2, FLAT / 224, (FLAT / 224) * mt};
   const int grid = ga.n_tiles < g_sm_count ? ga.n_tiles : g_sm_count;
-  TIMED(K_FC1_DX, (tc5_gemm<EPI_STORE, 224><<<grid, gemm_threads(EPI_STORE), gemm_smem_bytes(224, MAX_STAGES, epi_warps(EPI_STORE)), st>>>(maps, ga, a, wt, gt, ws)));
+  TIMED(K_FC1_DX, (tc5_gemm<EPI_STORE_BF16, 224><<<grid, gemm_threads(EPI_STORE_BF16), gemm_smem_bytes(224, MAX_STAGES, epi_warps(EPI_STORE_BF16)), st>>>(maps, ga, a, wt, gt, ws)));
   return 1;
 }
 

@@ -104,7 +104,7 @@ struct Workspace {
   float* d;        // [rows][512]         fc1 -> ReLU -> dropout (scaled)
   float* da1;      // [rows][512]         gradient w.r.t. fc1 pre-activation
   float* dz;       // [rows][16]          gradient w.r.t. logits (10 used)
-  float* dp2;      // [rows][1568]        gradient w.r.t. p2
+  float* dp2;      // [rows][1568]        gradient w.r.t. p2 (tensor-core path: BF16 in the first half of each row)
   float* dp1;      // [rows][3136]        gradient w.r.t. p1; [16][196] fp32 (FP32 path) or [4 channel quads][196][4] BF16 in the first half of the row (tensor-core path)
   float* part2;    // [W][chunks][4640]   per-block partial conv2 weight/bias gradients
   float* part1;    // [W][8 chunks][160]  per-block partial conv1 weight/bias gradients (tensor-core path: eight per range, one per sample of a pair and window element)
