@@ -70,34 +70,38 @@ constexpr int F_BUF_BYTES = 2 * F_PLANE_BYTES;             // two planes of eigh
 // input plane shifted by (sy, sx) = (jy + ky, jx + kx), sixteen shifts in all, and a shift serves every (window
 // element, tap) pair that adds up to it: the products of one shifted plane with the filters of all those taps land
 // side by side in the accumulator columns [window element][channel] when the weight operand stacks the taps' filters
-// in that column order.  A shift whose window elements are not adjacent in the column order takes two MMAs, so a
-// tile costs 20 MMAs (N = 128, 64 or 32) instead of 36 of N = 32; an MMA of M = 128, K = 16 is bound by reading
-// its 4 KB position operand from shared memory whatever N is.  The host lists the MMAs (FoldTable).
-constexpr int F_OPS = 20;
-constexpr int F_W_BLOCKS = 36;                             // 32-row blocks of the stacked weight operand (1,152 rows)
+// in that column order.  Where a shift's two window elements are not neighbours in the column order, the 32 columns
+// between them get a block of zero filters, so a tile costs 16 MMAs (four each of N = 128, 96, 64 and 32) instead of
+// 36 of N = 32: the tensor core spends about as long on an MMA of M = 128, K = 16 with N = 32 as with N = 96.  The
+// host lists the MMAs (FoldTable).
+constexpr int F_OPS = 16;
+constexpr int F_W_BLOCKS = 40;                             // 32-row blocks of the stacked weight operand (1,280 rows)
 constexpr int F_W_ROWS = 32 * F_W_BLOCKS;
 constexpr int F_W_BYTES = 2 * F_W_ROWS * 16;               // [channel octet][row][8 bf16]
 constexpr int F_SMEM = F_NBUF * F_BUF_BYTES + F_W_BYTES + 32 * 4 + sizeof(Pipe) + 128;
 static_assert(2 * F_SMEM <= 227 * 1024, "two CTAs per SM");
 
+constexpr uint8_t F_ZERO_BLOCK = 255;
 struct FoldTable {
   int32_t a_off[F_OPS];        // start of the shifted plane, in 16-byte rows
   int32_t d_col[F_OPS];        // first accumulator column
   int32_t b_row[F_OPS];        // first row of the op's block of the weight operand
   uint32_t idesc[F_OPS];       // instruction descriptor (M = 128, the op's N)
-  uint8_t tap_of_block[F_W_BLOCKS];   // filter tap ky * 3 + kx whose 32 filters fill a 32-row block
+  uint8_t tap_of_block[F_W_BLOCKS];   // filter tap ky * 3 + kx whose 32 filters fill a 32-row block; F_ZERO_BLOCK: 32 rows of zeros
 };
 
 FoldTable make_fold_table() {
   FoldTable t;
   int n_ops = 0, row = 0;
-  auto add = [&](int sy, int sx, int jy0, int ny, int jx0, int nx) {       // window elements [jy0, jy0 + ny) x [jx0, jx0 + nx)
+  // one op: the plane shifted by (sy, sx) against the filters of the column blocks [first, first + n_blocks); block c
+  // belongs to window element c = 2 jy + jx, whose tap for this shift is (sy - jy, sx - jx), or is a block of zeros
+  auto add = [&](int sy, int sx, int first, int n_blocks, unsigned used) {
     t.a_off[n_ops] = sy * 16 + (sx & 1) * 8 + (sx >> 1);
-    t.d_col[n_ops] = (2 * jy0 + jx0) * 32;
+    t.d_col[n_ops] = first * 32;
     t.b_row[n_ops] = row;
-    t.idesc[n_ops] = idesc_bf16(128, 32 * ny * nx);
-    for (int jy = jy0; jy < jy0 + ny; ++jy)
-      for (int jx = jx0; jx < jx0 + nx; ++jx) { t.tap_of_block[row / 32] = (uint8_t)((sy - jy) * 3 + (sx - jx)); row += 32; }
+    t.idesc[n_ops] = idesc_bf16(128, 32 * n_blocks);
+    for (int c = first; c < first + n_blocks; ++c, row += 32)
+      t.tap_of_block[row / 32] = (used >> c) & 1u ? (uint8_t)((sy - (c >> 1)) * 3 + (sx - (c & 1))) : F_ZERO_BLOCK;
     ++n_ops;
   };
   for (int pass = 0; pass < 2; ++pass)          // the op that covers all 128 columns comes first: it starts the sums
@@ -106,10 +110,16 @@ FoldTable make_fold_table() {
         if ((pass == 0) != (sy == 1 && sx == 1)) continue;
         const int jy0 = sy == 3 ? 1 : 0, ny = (sy == 0 || sy == 3) ? 1 : 2;
         const int jx0 = sx == 3 ? 1 : 0, nx = (sx == 0 || sx == 3) ? 1 : 2;
-        if (nx == 2) add(sy, sx, jy0, ny, jx0, 2);                       // columns of consecutive window elements
-        else for (int jy = jy0; jy < jy0 + ny; ++jy) add(sy, sx, jy, 1, jx0, 1);
+        unsigned used = 0;
+        for (int jy = jy0; jy < jy0 + ny; ++jy)
+          for (int jx = jx0; jx < jx0 + nx; ++jx) used |= 1u << (2 * jy + jx);
+        // the window elements of a shift are the blocks from its first to its last one; where two of them are not
+        // neighbours (same column of the window, both rows) the block between them is zeros: one MMA of N = 96 costs
+        // less than two of N = 32
+        const int first = 2 * jy0 + jx0, last = 2 * (jy0 + ny - 1) + (jx0 + nx - 1);
+        add(sy, sx, first, last - first + 1, used);
       }
-  return t;      // n_ops == F_OPS and row == F_W_ROWS by construction (checked where the table is made)
+  return t;      // n_ops == F_OPS and row == F_W_ROWS by construction
 }
 
 __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, GroupTable gt, Workspace ws, int range_len, const __grid_constant__ FoldTable fold) {
@@ -133,7 +143,8 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Gr
   // row per output channel
   for (int idx = tid; idx < F_W_BLOCKS * 512; idx += F_THREADS) {
     const int rb = idx >> 9, oc = (idx >> 4) & 31, ic = idx & 15;
-    Wk[((ic >> 3) * F_W_ROWS + rb * 32 + oc) * 8 + (ic & 7)] = bf16_bits(wtmp[(oc * 16 + ic) * 9 + fold.tap_of_block[rb]]);
+    const uint32_t tap = fold.tap_of_block[rb];
+    Wk[((ic >> 3) * F_W_ROWS + rb * 32 + oc) * 8 + (ic & 7)] = tap == F_ZERO_BLOCK ? (uint16_t)0 : bf16_bits(wtmp[(oc * 16 + ic) * 9 + tap]);
   }
   __syncthreads();
   // rows never written by a copy (the overrun of the padding rows, a missing second sample) only feed
@@ -159,7 +170,7 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Gr
         if (t >= 2 && !mbar_wait(&pipe->acc_empty[ab], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
         if (pipe->abort_flag) break;
         tc_fence_after();
-        // 20 MMAs, one or two per input shift (K = 16 channels); every descriptor is a per-tile base plus a table entry
+        // 16 MMAs, one per input shift (K = 16 channels); every descriptor is a per-tile base plus a table entry
         const uint32_t a_lo = plain_desc_lo(smem_u32(smem) + buf * F_BUF_BYTES, F_PLANE_BYTES);
         const uint32_t d_tmem = tmem + ab * 128;
 #pragma unroll
