@@ -23,16 +23,17 @@ namespace psk {
 
 namespace {
 
-constexpr int THREADS = 416;           // input-gradient kernel: 1 MMA warp, 8 staging warps, 4 epilogue warps
+constexpr int THREADS = 448;           // input-gradient kernel: 1 MMA warp, 8 staging warps, 4 epilogue warps, 1 copy warp
 constexpr int LOADERS = 256;
 
 __host__ __device__ constexpr uint32_t idesc_bf16(int m, int n) {     // fp32 accumulate, BF16 x BF16, k-contiguous
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+constexpr int RAW_SLOTS = 8;          // raw input slots of the input-gradient kernel
 constexpr int F_NBUF = 4;             // shared-memory tile buffers of the forward kernel (copies run four tiles ahead)
 struct Pipe {
-  uint64_t a_full[F_NBUF], a_empty[F_NBUF], acc_full[2], acc_empty[2], raw_full[4], raw_empty[4];
+  uint64_t a_full[F_NBUF], a_empty[F_NBUF], acc_full[2], acc_empty[2], raw_full[RAW_SLOTS], raw_empty[RAW_SLOTS];
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
@@ -46,7 +47,7 @@ __device__ __forceinline__ void pipe_init(Pipe* p, int a_full_arrivals, int acc_
     mbar_init(&p->acc_full[i], 1);
     mbar_init(&p->acc_empty[i], acc_empty_arrivals);
   }
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < RAW_SLOTS; ++i) {
     mbar_init(&p->raw_full[i], 1);
     mbar_init(&p->raw_empty[i], LOADERS / 64);
   }
@@ -262,14 +263,14 @@ constexpr int X_PLANE_BYTES = X_PLANE_ROWS * 16;           // staging stores of 
 constexpr int X_BUF_BYTES = 4 * X_PLANE_BYTES;             // four planes of eight output channels
 constexpr int X_W_BYTES = 12 * 48 * 16;                    // [filter row ky][k chunk oc/8][column = kx*16 + ic][8 bf16]
 constexpr int X_RAW_BYTES = FLAT * 2 + FLAT;                // one sample's pooled gradients (BF16) and pooling decisions (bytes)
-constexpr int X_RAW_SLOTS = 4;
+constexpr int X_RAW_SLOTS = RAW_SLOTS;
 constexpr int X_SMEM = 2 * X_BUF_BYTES + X_W_BYTES + X_RAW_SLOTS * X_RAW_BYTES + sizeof(Pipe) + 128;
 
 __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, GroupTable gt, Workspace ws, int range_len) {
   extern __shared__ __align__(128) uint8_t smem[];
   uint16_t* bufs = reinterpret_cast<uint16_t*>(smem);
   uint16_t* Wk = reinterpret_cast<uint16_t*>(smem + 2 * X_BUF_BYTES);
-  uint8_t* raw = smem + 2 * X_BUF_BYTES + X_W_BYTES;        // two raw staging slots filled by bulk copies
+  uint8_t* raw = smem + 2 * X_BUF_BYTES + X_W_BYTES;        // raw slots filled by bulk copies
   Pipe* pipe = reinterpret_cast<Pipe*>(smem + 2 * X_BUF_BYTES + X_W_BYTES + X_RAW_SLOTS * X_RAW_BYTES);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int grp, r_begin, r_end;
@@ -323,21 +324,14 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
     // Two groups of four staging warps: group g builds the tiles t = g, g + 2, ... into plane buffer g, so two
     // tiles are being staged at any time (a tile's staging is a chain of dependent shared-memory accesses, bound
     // by latency rather than by throughput).  The pooled gradients and decisions of a sample arrive in one of
-    // four raw slots by two bulk copies issued by the group's first thread, two of the group's tiles ahead.
+    // eight raw slots by two bulk copies that a warp of its own issues (a staging thread that issued them held its
+    // whole group up for hundreds of cycles per tile).
     const int grp_w = (warp - 1) >> 2, lt = (tid - 32) & 127;
     constexpr int X_ITEMS = (4 * 49 + 127) / 128;                  // (channel octet, position) items per thread
-    auto fetch_raw = [&](int t) {
-      const int64_t row = r_begin + t;
-      uint8_t* slot = raw + (t & 3) * X_RAW_BYTES;
-      mbar_expect_tx(&pipe->raw_full[t & 3], X_RAW_BYTES);
-      bulk_load(slot, ws.dp2 + row * FLAT, FLAT * 2, &pipe->raw_full[t & 3]);      // BF16 in the first half of the row
-      bulk_load(slot + FLAT * 2, ws.code2 + row * FLAT, FLAT, &pipe->raw_full[t & 3]);
-    };
-    if (lt == 0) { if (grp_w < n_tiles) fetch_raw(grp_w); if (grp_w + 2 < n_tiles) fetch_raw(grp_w + 2); }
     for (int t = grp_w; t < n_tiles; t += 2) {
-      const int buf = t & 1, slot_i = t & 3;
+      const int buf = t & 1, slot_i = t & (X_RAW_SLOTS - 1);
       // every staging warp waits and reports on its own (no block-level barrier among them)
-      bool ok = mbar_wait(&pipe->raw_full[slot_i], (t >> 2) & 1);
+      bool ok = mbar_wait(&pipe->raw_full[slot_i], (t >> 3) & 1);
       if (ok && t >= 2) ok = mbar_wait(&pipe->a_empty[buf], ((t >> 1) - 1) & 1);
       if (!__all_sync(0xffffffffu, ok) || pipe->abort_flag) { pipe->abort_flag = 1; break; }
       uint16_t* dst = bufs + buf * (X_BUF_BYTES / 2);
@@ -371,12 +365,20 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) { mbar_arrive(&pipe->a_full[buf]); mbar_arrive(&pipe->raw_empty[slot_i]); }
-      // the raw slot is refilled once every warp of the group has read it
-      if (lt == 0 && t + 4 < n_tiles) {
-        if (!mbar_wait(&pipe->raw_empty[slot_i], (t >> 2) & 1)) { pipe->abort_flag = 1; break; }
-        fetch_raw(t + 4);
-      }
     }
+  } else if (warp == THREADS / 32 - 1) {
+    // ---------------- copies: one thread brings every sample's pooled gradients (BF16) and decisions into the raw slots
+    // in turn, up to eight samples ahead; a slot is refilled once the four warps that staged its last sample have read it
+    if (lane == 0)
+      for (int t = 0; t < n_tiles; ++t) {
+        const int slot_i = t & (X_RAW_SLOTS - 1);
+        if (t >= X_RAW_SLOTS && (!mbar_wait(&pipe->raw_empty[slot_i], ((t >> 3) - 1) & 1) || pipe->abort_flag)) { pipe->abort_flag = 1; break; }
+        const int64_t row = r_begin + t;
+        uint8_t* slot = raw + slot_i * X_RAW_BYTES;
+        mbar_expect_tx(&pipe->raw_full[slot_i], X_RAW_BYTES);
+        bulk_load(slot, ws.dp2 + row * FLAT, FLAT * 2, &pipe->raw_full[slot_i]);      // BF16 in the first half of the row
+        bulk_load(slot + FLAT * 2, ws.code2 + row * FLAT, FLAT, &pipe->raw_full[slot_i]);
+      }
   } else {
     const int quarter = warp & 3;
     for (int t = 0; t < n_tiles; ++t) {
