@@ -41,7 +41,7 @@ constexpr int W5_CHUNKS = 32;                           // 8-position chunks of 
 constexpr int W5_GROUP_BYTES = W5_CHUNKS * 128;         // one group of 8 operand rows: 32 core matrices of 128 bytes
 constexpr int W5_A_GROUPS = 7;                          // (kx, channel octet) x 6, then the group whose first row is all ones
 constexpr int W5_A_BYTES = W5_A_GROUPS * W5_GROUP_BYTES;     // 28,672
-// B: [half of the image row (x / 8)][image row, descending: y = 14 .. -1][channel octet][8 channels x 8 positions];
+// B: [column parity (x & 1)][image row, descending: y = 14 .. -1][channel octet][8 channels x 8 places (x / 2)];
 // rows y = 14 and y = -1 are never written (zeros): the k-steps next to the border read them
 constexpr int W5_B_ROW = 4 * 128, W5_B_HALF = 16 * W5_B_ROW;      // 512 bytes per image row, 8,192 per half
 constexpr int W5_B_BYTES = 2 * W5_B_HALF;               // 16,384
@@ -169,37 +169,41 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       const uint16_t* rdp2h = reinterpret_cast<const uint16_t*>(rp1 + W5_RAW_P1);
       const uint8_t* rcode8 = rp1 + W5_RAW_P1 + W5_RAW_DP2;
       uint8_t* stage = sm + st * W5_STAGE_BYTES;
+      // Inside an image row the sixteen positions are taken in the order of the input planes' rows, even columns then
+      // odd columns (contraction index 16 y + 8 (x & 1) + x / 2 for both operands: a sum does not care about its order),
+      // so that the eight positions of a chunk are eight CONSECUTIVE plane rows and a transposing load meets no bank twice.
       // A: 6 groups x 32 chunks = 192 blocks of 8 positions x 8 channels, transposed four at a time.  Operation o of
       // the 48 covers chunks 4 (o % 8) .. + 3 of group o / 8 = (kx, channel octet).  Lane l addresses row l % 8 of
-      // block l / 8: on the way in the input plane's row of position 8 chunk + row + kx (plane rows keep even and
-      // odd columns apart; positions past the end read the all-zero row 0), on the way out the core matrix's row.
+      // block l / 8: on the way in the plane row of the position kx columns to the right of the chunk's (l % 8)-th
+      // (positions past the end read the all-zero row 0), on the way out the core matrix's row.
 #pragma unroll
       for (int o = gw; o < 48; o += W5_GW) {
         const int g = o >> 3, kx = g >> 1, oct = g & 1, chunk = 4 * (o & 7) + (lane >> 3);
-        const int i = 8 * chunk + (lane & 7) + kx;
+        const int i = 16 * (chunk >> 1) + 2 * (lane & 7) + (chunk & 1) + kx;       // position y * 16 + x
         const int prow = i < 256 ? (i & ~15) + ((i & 1) << 3) + ((i & 15) >> 1) : 0;
         uint32_t r[4];
         ldmatrix_x4_trans(r, smem_u32(rp1 + oct * 4096 + prow * 16));
         stmatrix_x4(smem_u32(stage + g * W5_GROUP_BYTES + chunk * 128 + (lane & 7) * 16), r);
       }
-      // B: a warp takes (octet of output channels, pooled row py, half of the pooled columns) and a lane one channel of
-      // the octet and one pooled column of the four: its words then fall into 32 different banks.  Every pooled entry
-      // owns the four positions of its window: shifted left by 16 bits per decision, the BF16 gradient lands in the
-      // half-word of the winner (low word: image row 2py, high word: row 2py + 1; decision 4 shifts it out), the other
-      // three are cleared.  The pair of columns (2px, 2px + 1) is one word of a core-matrix row; image row y is stored
-      // 14 - y rows into its half.
-#pragma unroll
-      for (int wi = gw; wi < 56; wi += W5_GW) {
-        const int oct = wi / 14, rem = wi - oct * 14, py = rem >> 1, pxhi = rem & 1;
-        const int rr = lane >> 2, pl = lane & 3, px = 4 * pxhi + pl;
-        if (px < 7) {
-          const int oc = 8 * oct + rr, e = ((oc >> 2) * 49 + py * 7 + px) * 4 + (oc & 3);
-          const uint32_t code = rcode8[e];
-          const unsigned long long slot64 = shl64_clamped(rdp2h[e], 16u * code);
-          uint32_t* d = reinterpret_cast<uint32_t*>(stage + W5_A_BYTES + pxhi * W5_B_HALF + (14 - 2 * py) * W5_B_ROW + oct * 128 + rr * 16) + pl;
-          d[0] = (uint32_t)slot64;                               // image row 2py
-          d[-(W5_B_ROW / 4)] = (uint32_t)(slot64 >> 32);         // image row 2py + 1
-        }
+      // B: a warp takes (octet of output channels, pooled row py) and a lane one channel of the octet and the pooled
+      // columns 2j, 2j + 1: its words then fall into 32 different banks.  Every pooled entry owns the four positions of
+      // its window: shifted left by 16 bits per decision, the BF16 gradient lands in the half-word of the winner (low
+      // word: image row 2py, high word: row 2py + 1; in each, low half: column 2px, high half: column 2px + 1; decision
+      // 4 shifts it out), the other three are cleared.  Column x of an image row sits in chunk x & 1 at place x / 2, so
+      // the two entries' half-words of equal (row, column parity) make one word; image row y is stored 14 - y rows into
+      // its half.
+      for (int wi = gw; wi < 28; wi += W5_GW) {
+        const int oct = wi / 7, py = wi - oct * 7;
+        const int rr = lane >> 2, j = lane & 3, oc = 8 * oct + rr;
+        const int e = ((oc >> 2) * 49 + py * 7 + 2 * j) * 4 + (oc & 3);
+        const uint32_t code0 = rcode8[e], code1 = j < 3 ? rcode8[e + 4] : 4u;      // pooled column 7 does not exist
+        const unsigned long long s0 = shl64_clamped(rdp2h[e], 16u * code0), s1 = shl64_clamped(j < 3 ? rdp2h[e + 4] : (uint16_t)0, 16u * code1);
+        const uint32_t lo0 = (uint32_t)s0, hi0 = (uint32_t)(s0 >> 32), lo1 = (uint32_t)s1, hi1 = (uint32_t)(s1 >> 32);
+        uint32_t* d = reinterpret_cast<uint32_t*>(stage + W5_A_BYTES + (14 - 2 * py) * W5_B_ROW + oct * 128 + rr * 16) + j;
+        d[0] = prmt(lo0, lo1, 0x5410u);                                   // image row 2py, even columns
+        d[W5_B_HALF / 4] = prmt(lo0, lo1, 0x7632u);                       // image row 2py, odd columns
+        d[-(W5_B_ROW / 4)] = prmt(hi0, hi1, 0x5410u);                     // image row 2py + 1, even columns
+        d[W5_B_HALF / 4 - W5_B_ROW / 4] = prmt(hi0, hi1, 0x7632u);        // image row 2py + 1, odd columns
       }
       fence_proxy_async_smem();
       __syncwarp();
