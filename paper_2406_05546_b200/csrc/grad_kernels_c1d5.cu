@@ -137,26 +137,33 @@ __global__ void __launch_bounds__(D1_THREADS, 1) conv1_dw_tc5(GradStepArgs a, Wo
       D1Walk walk = d1_begin(r0, a.b);
       bool fresh = true;                       // the next MMA starts a new sum
       D1Unit un;
-      for (int u = 0; d1_next_unit(walk, r1, a.b, un); ++u) {
-        const int st = u & 1;
-        if (!mbar_wait(&bars->op_full[st], (u >> 1) & 1) || bars->abort_flag) { bars->abort_flag = 1; break; }
-        tc_fence_after();
-        const uint32_t a_lo = plain_desc_lo(smem_u32(sm) + st * D1_STAGE_BYTES, D1_CHUNK_PITCH);
-        const uint32_t b_lo = plain_desc_lo(smem_u32(sm) + st * D1_STAGE_BYTES + D1_A_BYTES, D1_CHUNK_PITCH);
-        // contraction indices 16 ks .. 16 ks + 15: two core matrices, 2 x 144 bytes further along every row group
+      // One pass of the outer loop takes the two stages in turn (unrolled: a stage's addresses are constants of its
+      // copy of the body, and the backward branch comes once per two units).
+      const uint32_t a_lo0 = plain_desc_lo(smem_u32(sm), D1_CHUNK_PITCH), b_lo0 = plain_desc_lo(smem_u32(sm) + D1_A_BYTES, D1_CHUNK_PITCH);
+      const uint32_t full0 = smem_u32(&bars->op_full[0]), empty0 = smem_u32(&bars->op_empty[0]);
+      bool go_on = true;
+      for (uint32_t parity = 0; go_on; parity ^= 1) {
 #pragma unroll
-        for (int ks = 0; ks < D1_KSTEPS; ++ks)
-          umma_f16_split(tmem, a_lo + ks * (2 * D1_CHUNK_PITCH / 16), plain_desc_hi(D1_GROUP_BYTES), b_lo + ks * (2 * D1_CHUNK_PITCH / 16),
-                         plain_desc_hi(D1_GROUP_BYTES), idesc, (ks == 0 && fresh) ? 0u : 1u);
-        fresh = false;
-        umma_commit(&bars->op_empty[st]);
-        if (un.flush) {
-          // last rows of the range or of a worker: hand the sums to the write-out warps and wait until they have read them
-          umma_commit(&bars->acc_full);
-          if (!mbar_wait(&bars->acc_empty, writes & 1)) { bars->abort_flag = 1; break; }
+        for (int st = 0; st < D1_NSTAGE; ++st) {
+          if (!d1_next_unit(walk, r1, a.b, un)) { go_on = false; break; }
+          if (!mbar_wait_addr(full0 + 8 * st, parity) || bars->abort_flag) { bars->abort_flag = 1; go_on = false; break; }
           tc_fence_after();
-          ++writes;
-          fresh = true;
+          const uint32_t a_lo = a_lo0 + st * (D1_STAGE_BYTES / 16), b_lo = b_lo0 + st * (D1_STAGE_BYTES / 16);
+          // contraction indices 16 ks .. 16 ks + 15: two core matrices, 2 x 144 bytes further along every row group
+#pragma unroll
+          for (int ks = 0; ks < D1_KSTEPS; ++ks)
+            umma_f16_split(tmem, a_lo + ks * (2 * D1_CHUNK_PITCH / 16), plain_desc_hi(D1_GROUP_BYTES), b_lo + ks * (2 * D1_CHUNK_PITCH / 16),
+                           plain_desc_hi(D1_GROUP_BYTES), idesc, (ks == 0 && fresh) ? 0u : 1u);
+          fresh = false;
+          umma_commit_addr(empty0 + 8 * st);
+          if (un.flush) {
+            // last rows of the range or of a worker: hand the sums to the write-out warps and wait until they have read them
+            umma_commit(&bars->acc_full);
+            if (!mbar_wait(&bars->acc_empty, writes & 1)) { bars->abort_flag = 1; go_on = false; break; }
+            tc_fence_after();
+            ++writes;
+            fresh = true;
+          }
         }
       }
     }

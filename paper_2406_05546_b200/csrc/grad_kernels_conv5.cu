@@ -165,21 +165,32 @@ __global__ void __launch_bounds__(F_THREADS, 2) conv2_fwd_tc5(GradStepArgs a, Gr
   if (warp == 0) {
     if (lane == 0) {
       const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), F_W_ROWS * 16);
-      for (int t = 0; t < n_tiles; ++t) {
-        const int buf = t % F_NBUF, ab = t & 1;
-        if (!mbar_wait(&pipe->a_full[buf], (t / F_NBUF) & 1)) { pipe->abort_flag = 1; break; }
-        if (t >= 2 && !mbar_wait(&pipe->acc_empty[ab], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
-        if (pipe->abort_flag) break;
-        tc_fence_after();
-        // 16 MMAs, one per input shift (K = 16 channels); every descriptor is a per-tile base plus a table entry
-        const uint32_t a_lo = plain_desc_lo(smem_u32(smem) + buf * F_BUF_BYTES, F_PLANE_BYTES);
-        const uint32_t d_tmem = tmem + ab * 128;
+      // one pass of the outer loop takes the four tile buffers in turn (unrolled: buffer, accumulator and the parity of
+      // the accumulator's barrier are constants of each copy of the body, and the backward branch comes once per four tiles)
+      static_assert(F_NBUF == 4, "the accumulator parities below assume four tile buffers");
+      const uint32_t a_lo0 = plain_desc_lo(smem_u32(smem), F_PLANE_BYTES);
+      bool go_on = true;
+      uint32_t parity = 0;
+      for (int t = 0; go_on && t < n_tiles; parity ^= 1) {
 #pragma unroll
-        for (int op = 0; op < F_OPS; ++op)
-          umma_f16_split(d_tmem + fold.d_col[op], a_lo + fold.a_off[op], plain_desc_hi(512), w_lo + fold.b_row[op],
-                         plain_desc_hi(128), fold.idesc[op], op ? 1u : 0u);
-        umma_commit(&pipe->a_empty[buf]);
-        umma_commit(&pipe->acc_full[ab]);
+        for (int buf = 0; buf < F_NBUF; ++buf, ++t) {
+          const int ab = buf & 1;
+          if (t >= n_tiles) { go_on = false; break; }
+          if (!mbar_wait(&pipe->a_full[buf], parity)) { pipe->abort_flag = 1; go_on = false; break; }
+          // tile t = 4 k + buf is the (2 k + buf / 2)-th user of its accumulator: it waits for the phase of the user before
+          if (t >= 2 && !mbar_wait(&pipe->acc_empty[ab], ((buf >> 1) ^ 1) & 1)) { pipe->abort_flag = 1; go_on = false; break; }
+          if (pipe->abort_flag) { go_on = false; break; }
+          tc_fence_after();
+          // 16 MMAs, one per input shift (K = 16 channels); every descriptor is a per-tile base plus a table entry
+          const uint32_t a_lo = a_lo0 + buf * (F_BUF_BYTES / 16);
+          const uint32_t d_tmem = tmem + ab * 128;
+#pragma unroll
+          for (int op = 0; op < F_OPS; ++op)
+            umma_f16_split(d_tmem + fold.d_col[op], a_lo + fold.a_off[op], plain_desc_hi(512), w_lo + fold.b_row[op],
+                           plain_desc_hi(128), fold.idesc[op], op ? 1u : 0u);
+          umma_commit(&pipe->a_empty[buf]);
+          umma_commit(&pipe->acc_full[ab]);
+        }
       }
     }
   } else if (warp == 1) {
@@ -298,26 +309,34 @@ __global__ void __launch_bounds__(THREADS, 2) conv2_dx_tc5(GradStepArgs a, Group
     if (lane == 0) {
       constexpr uint32_t idesc = idesc_bf16(128, 48);
       const uint32_t w_lo = plain_desc_lo(smem_u32(Wk), 48 * 16);
-      for (int t = 0; t < n_tiles; ++t) {
-        const int buf = t & 1;
-        if (!mbar_wait(&pipe->a_full[buf], (t >> 1) & 1)) { pipe->abort_flag = 1; break; }
-        if (t >= 2 && !mbar_wait(&pipe->acc_empty[buf], ((t >> 1) - 1) & 1)) { pipe->abort_flag = 1; break; }
-        if (pipe->abort_flag) break;
-        tc_fence_after();
-        const uint32_t a_lo = plain_desc_lo(smem_u32(smem) + buf * X_BUF_BYTES, X_PLANE_BYTES);
-        const uint32_t d_tmem = tmem + buf * 128;
-        // 12 MMAs: per block of 128 positions and filter row ky, the products with the three taps of that row sit
-        // side by side in the 48 accumulator columns (kx, ic); the rows read are shifted by the filter row only
+      // one pass of the outer loop takes the two plane buffers in turn (unrolled: the buffer's addresses are constants
+      // of its copy of the body, and the backward branch comes once per two tiles)
+      const uint32_t a_lo0 = plain_desc_lo(smem_u32(smem), X_PLANE_BYTES);
+      bool go_on = true;
+      uint32_t parity = 0;
+      for (int t = 0; go_on && t < n_tiles; parity ^= 1) {
 #pragma unroll
-        for (int ky = 0; ky < 3; ++ky)
+        for (int buf = 0; buf < 2; ++buf, ++t) {
+          if (t >= n_tiles) { go_on = false; break; }
+          if (!mbar_wait(&pipe->a_full[buf], parity)) { pipe->abort_flag = 1; go_on = false; break; }
+          if (t >= 2 && !mbar_wait(&pipe->acc_empty[buf], parity ^ 1)) { pipe->abort_flag = 1; go_on = false; break; }
+          if (pipe->abort_flag) { go_on = false; break; }
+          tc_fence_after();
+          const uint32_t a_lo = a_lo0 + buf * (X_BUF_BYTES / 16);
+          const uint32_t d_tmem = tmem + buf * 128;
+          // 12 MMAs: per block of 128 positions and filter row ky, the products with the three taps of that row sit
+          // side by side in the 48 accumulator columns (kx, ic); the rows read are shifted by the filter row only
 #pragma unroll
-          for (int q = 0; q < 2; ++q)                                        // 16 output channels per MMA
+          for (int ky = 0; ky < 3; ++ky)
 #pragma unroll
-            for (int m = 0; m < 2; ++m)
-              umma_f16_split(d_tmem + m * 48, a_lo + (2 * q) * (X_PLANE_BYTES / 16) + m * 128 + (2 - ky) * 16 + 1, plain_desc_hi(128),
-                             w_lo + ((ky * 4 + 2 * q) * 48), plain_desc_hi(128), idesc, (ky | q) ? 1u : 0u);
-        umma_commit(&pipe->a_empty[buf]);
-        umma_commit(&pipe->acc_full[buf]);
+            for (int q = 0; q < 2; ++q)                                        // 16 output channels per MMA
+#pragma unroll
+              for (int m = 0; m < 2; ++m)
+                umma_f16_split(d_tmem + m * 48, a_lo + (2 * q) * (X_PLANE_BYTES / 16) + m * 128 + (2 - ky) * 16 + 1, plain_desc_hi(128),
+                               w_lo + ((ky * 4 + 2 * q) * 48), plain_desc_hi(128), idesc, (ky | q) ? 1u : 0u);
+          umma_commit(&pipe->a_empty[buf]);
+          umma_commit(&pipe->acc_full[buf]);
+        }
       }
     }
   } else if (warp <= LOADERS / 32) {

@@ -127,32 +127,37 @@ __global__ void __launch_bounds__(W5_THREADS, 1) conv2_dw_tc5(GradStepArgs a, Wo
       // B at k-step ks starts at the stored row of y = ks (14 - ks rows in); its two k-chunks are the halves of a row
       const uint32_t b_lo0 = plain_desc_lo(smem_u32(sm) + W5_A_BYTES + 14 * W5_B_ROW, W5_B_HALF);
       const uint32_t full0 = smem_u32(&bars->op_full[0]), empty0 = smem_u32(&bars->op_empty[0]);
-      uint32_t a_lo = a_lo0, b_lo = b_lo0, full = full0, empty = empty0, parity = 0, writes = 0;
-      int st = 0;
+      uint32_t parity = 0, writes = 0;
       int flush_at = min(r1, (r0 / a.b + 1) * a.b) - 1 - r0;     // index in the range of the next row that ends a worker or the range
       bool fresh = true;                       // the next MMA starts a new sum
-      for (int n = 0; n < n_samples; ++n) {
-        if (!mbar_wait_addr(full, parity) || bars->abort_flag) { bars->abort_flag = 1; break; }
-        tc_fence_after();
-        // contraction indices 16 ks .. 16 ks + 15 (image row ks of the bordered input): two chunks of 128 bytes.
-        // Rows 0 and 15 are the input's zero border, so their products vanish and are not issued.
+      bool go_on = true;
+      // One pass of the outer loop takes the stages in turn (unrolled: a stage's addresses are constants of its copy
+      // of the body, and the backward branch, after which the instruction fetch starts afresh, comes once per three samples).
+      for (int n = 0; go_on && n < n_samples; parity ^= 1) {
 #pragma unroll
-        for (int ks = 1; ks < 15; ++ks)
-          umma_f16_split(tmem, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo - ks * (W5_B_ROW / 16), plain_desc_hi(128), idesc,
-                         (ks == 1 && fresh) ? 0u : 1u);
-        fresh = false;
-        umma_commit_addr(empty);
-        if (n == flush_at) {
-          // last row of the range or of a worker: hand the sum to the write-out warps and wait until they have read it
-          umma_commit(&bars->acc_full);
-          if (!mbar_wait(&bars->acc_empty, writes & 1)) { bars->abort_flag = 1; break; }
+        for (int st = 0; st < W5_NSTAGE; ++st, ++n) {
+          if (n >= n_samples) { go_on = false; break; }
+          const uint32_t a_lo = a_lo0 + st * stage_step, b_lo = b_lo0 + st * stage_step;
+          if (!mbar_wait_addr(full0 + 8 * st, parity) || bars->abort_flag) { bars->abort_flag = 1; go_on = false; break; }
           tc_fence_after();
-          ++writes;
-          fresh = true;
-          flush_at = min(flush_at + a.b, n_samples - 1);
+          // contraction indices 16 ks .. 16 ks + 15 (image row ks of the bordered input): two chunks of 128 bytes.
+          // Rows 0 and 15 are the input's zero border, so their products vanish and are not issued.
+#pragma unroll
+          for (int ks = 1; ks < 15; ++ks)
+            umma_f16_split(tmem, a_lo + ks * 16, plain_desc_hi(W5_GROUP_BYTES), b_lo - ks * (W5_B_ROW / 16), plain_desc_hi(128), idesc,
+                           (ks == 1 && fresh) ? 0u : 1u);
+          fresh = false;
+          umma_commit_addr(empty0 + 8 * st);
+          if (n == flush_at) {
+            // last row of the range or of a worker: hand the sum to the write-out warps and wait until they have read it
+            umma_commit(&bars->acc_full);
+            if (!mbar_wait(&bars->acc_empty, writes & 1)) { bars->abort_flag = 1; go_on = false; break; }
+            tc_fence_after();
+            ++writes;
+            fresh = true;
+            flush_at = min(flush_at + a.b, n_samples - 1);
+          }
         }
-        if (++st == W5_NSTAGE) { st = 0; parity ^= 1; a_lo = a_lo0; b_lo = b_lo0; full = full0; empty = empty0; }
-        else { a_lo += stage_step; b_lo += stage_step; full += 8; empty += 8; }
       }
     }
   } else if (warp <= W5_LOAD_WARPS) {
