@@ -36,8 +36,8 @@ N_BATCH_BUFFERS = 8
 REPLAY_TRAFFIC_PER_GRADIENT = 2.654663e9 / 816
 # dram bytes (read + written) per sample of the grad-step kernels, from one ncu capture of a reduced case
 # (W=128, b=64: 8,192 samples; traffic grows in proportion to the samples); None = not captured since the kernel changed
-KERNEL_TRAFFIC_PER_SAMPLE = {"conv2_dw": 16626, "conv1_fwd": 7434, "conv2_bwd": 9321, "fc1_dw": 51780, "conv2_fwd": 9822,
-                             "fc1_dx": 2757, "fc1_fwd": 6757, "fc2_fwd_bwd": 2060, "conv1_bwd": 13058}
+KERNEL_TRAFFIC_PER_SAMPLE = {"conv2_dw": 13406, "conv1_fwd": 7393, "conv2_bwd": 5515, "fc1_dw": 51641, "conv2_fwd": 10064,
+                             "fc1_dx": 2452, "fc1_fwd": 6745, "fc2_fwd_bwd": 2061, "conv1_bwd": 12972}
 
 
 def measured_peaks():
