@@ -35,7 +35,8 @@ GRAD_BYTES = 813258 * 4                 # algorithmic bytes per queued gradient
 N_BATCH_BUFFERS = 8
 REPLAY_TRAFFIC_PER_GRADIENT = 2.654663e9 / 816
 # dram bytes (read + written) per sample of the grad-step kernels, from one ncu capture of a reduced case
-# (W=128, b=64: 8,192 samples; traffic grows in proportion to the samples); None = not captured since the kernel changed
+# (W=128, b=64: 8,192 samples; traffic grows in proportion to the samples, except for fc1_dw, whose 3.2 MB of output per
+# worker do not depend on the batch: its figure holds at b = 64 only); None = not captured since the kernel changed
 KERNEL_TRAFFIC_PER_SAMPLE = {"conv2_dw": 13406, "conv1_fwd": 7393, "conv2_bwd": 5515, "fc1_dw": 51641, "conv2_fwd": 10064,
                              "fc1_dx": 2452, "fc1_fwd": 6745, "fc2_fwd_bwd": 2061, "conv1_bwd": 12972}
 
