@@ -41,6 +41,22 @@ KERNEL_TRAFFIC_PER_SAMPLE = {"conv2_dw": 13406, "conv1_fwd": 7393, "conv2_bwd": 
                              "fc1_dx": 2452, "fc1_fwd": 6745, "fc2_fwd_bwd": 2061, "conv1_bwd": 12972}
 
 
+# Algorithmic HBM bytes of the tensor-core path's grad-step kernels at (W, b): what each must read and write once
+# (images fp32, p1 as 8 KB BF16 planes, decisions as bytes, p2 / a1 / da1 fp32, dp2 and dp1 BF16, the per-worker fc1
+# weight gradient fp32; weights are small and stay in L2).
+ALGORITHMIC_BYTES = {
+    "conv1_fwd": lambda W, b: (3136 + 8192 + 3136) * W * b,
+    "conv2_fwd": lambda W, b: (8192 + 6272 + 1568) * W * b,
+    "fc1_fwd": lambda W, b: (6272 + 2048) * W * b,
+    "fc2_fwd_bwd": lambda W, b: (2048 + 2048) * W * b,
+    "fc1_dw": lambda W, b: (2048 + 6272) * W * b + 512 * 1568 * 4 * W,
+    "fc1_dx": lambda W, b: (2048 + 3136) * W * b,
+    "conv2_bwd": lambda W, b: (3136 + 1568 + 6272) * W * b,
+    "conv2_dw": lambda W, b: (8192 + 3136 + 1568) * W * b,
+    "conv1_bwd": lambda W, b: (3136 + 6272 + 3136) * W * b,
+}
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -501,6 +517,21 @@ def main():
             roofs = {k: kernel_roofline(k, 1.0, W, b, peaks, args.precision, sustained) for k in kernels}
             return sum(r["flops"] / (r["peak"] * 1e12) * 1e3 for r in roofs.values() if r["bound"] != "hbm")
         sol_ms, sol_ms_sustained = composite_ms(False), composite_ms(True)
+        # the same with every kernel bound by the larger of its compute time and the time the measured copy bandwidth
+        # needs for its algorithmic bytes (tensor-core path; None on the FP32 path, whose buffers differ)
+        def compute_or_hbm_ms():
+            if args.precision == "fp32":
+                return None, None
+            per = {}
+            for k in kernels:
+                if k in GRAD_KERNELS_EXCLUDED or k not in ALGORITHMIC_BYTES:
+                    continue
+                r = kernel_roofline(k, 1.0, W, b, peaks, args.precision)
+                t_c = r["flops"] / (r["peak"] * 1e12) * 1e3 if r["bound"] != "hbm" else 0.0
+                t_m = ALGORITHMIC_BYTES[k](W, b) / (peaks["hbm_gbs"] * 1e9) * 1e3
+                per[k] = max(t_c, t_m)
+            return sum(per.values()), per
+        bound_ms, bound_per_kernel = compute_or_hbm_ms()
         tflops = FLOP_PER_SAMPLE * W * b / (grad_ms * 1e-3) / 1e12
         grad_step = {"ms": grad_ms, "worker_samples_per_s": W * b / (grad_ms * 1e-3), "tflops": tflops,
                      "tensor_flop_share": tensor_flop / (FLOP_PER_SAMPLE * W * b),
@@ -508,6 +539,9 @@ def main():
                      "roofline_ms_sustained_peaks": sol_ms_sustained,
                      "frac_of_composite_roofline_sustained_peaks": sol_ms_sustained / grad_ms,
                      "frac_of_tf32_roofline": tflops / (peaks["bf16_tflops"] * (1.1 / 2.25)),
+                     "roofline_ms_compute_or_hbm": bound_ms,
+                     "frac_of_compute_or_hbm_roofline": bound_ms / grad_ms if bound_ms else None,
+                     "per_kernel_frac_compute_or_hbm": {k: v / kernels[k]["ms_per_launch"] for k, v in bound_per_kernel.items()} if bound_per_kernel else None,
                      "per_kernel_frac": {k: kernel_roofline(k, v["ms_per_launch"], W, b, peaks, args.precision)["frac"]
                                          for k, v in kernels.items() if k not in GRAD_KERNELS_EXCLUDED and k not in ("conv_grad_reduce", "prep_w1")},
                      "note": "ms = sum of the per-kernel times measured one kernel at a time (in the timed region "
@@ -515,7 +549,9 @@ def main():
                              "sum over products of flop / peak of the unit and type each uses, with the measured "
                              "burst bf16 GEMM rate (kernels timed alone at the full SM clock); the _sustained_peaks "
                              "figures use the sustained rate instead; "
-                             "frac_of_tf32_roofline = all flop / ms against the TF32 dense peak alone"}
+                             "frac_of_tf32_roofline = all flop / ms against the TF32 dense peak alone; "
+                             "roofline_ms_compute_or_hbm = sum over kernels of max(flop / peak, algorithmic bytes / "
+                             "measured copy bandwidth)"}
         # the whole grad step next to the dominant kernel
         roof["grad_step"] = {"ms": grad_ms, "roofline_ms": sol_ms, "frac": sol_ms / grad_ms, "bound": "composite compute",
                              "peaks": "burst"}
